@@ -1,0 +1,130 @@
+/*
+ * CPU oracle for the best-matching-unit (BMU) search on sparse binary documents.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the arbiter the CUDA library is
+ * checked against; it is never a fallback for it.  It shares no code, header,
+ * table or helper with the CUDA path and is only ever called from the tests,
+ * from the smoke check and from the CPU-baseline leg of the benchmark.
+ *
+ * What it computes (the exact result the paper's kernel reaches faster;
+ * Section 3: the search finds, for each article, the neuron whose weight
+ * vector is closest, and an exact-argmin BMU does not depend on how the
+ * codebook is stored):
+ *
+ *     d_ij = |x_i| + ||w_j||^2 - 2 * sum_{f in x_i} W[f][j]
+ *
+ * for document i (a set x_i of active feature ids, binary values) and neuron j
+ * of a feature-major codebook W[f*M + j] (Section 3, "W[v.M+i]").  For binary x
+ * this equals the squared Euclidean distance ||x_i - w_j||^2.  The BMU is the
+ * lowest j that attains min_j d_ij.
+ *
+ * All arithmetic is IEEE double on the float inputs, in the plainest order:
+ * one accumulator per neuron, features added in the order the row lists them,
+ * neurons scanned in ascending order with a strict "<".  No blocking, no
+ * fusion, no reordering.  Threads (OpenMP) split the documents only.
+ *
+ * Parity status: pinned (dense brute force, closed forms, invariants, a
+ * library matmul and a hand-worked fixture; see tests/test_oracle_pins.py).
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <math.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* n_j = sum_f W[f][j]^2, the "norms" step of the epoch (Table 4). */
+void oracle_norms(const float *W, int64_t D, int64_t M, double *norms)
+{
+    for (int64_t j = 0; j < M; ++j)
+        norms[j] = 0.0;
+    for (int64_t f = 0; f < D; ++f) {
+        const float *row = W + f * M;
+        for (int64_t j = 0; j < M; ++j) {
+            double w = (double)row[j];
+            norms[j] += w * w;
+        }
+    }
+}
+
+/* Distance of one (document, neuron) pair, by the definition above. */
+double oracle_eval(const float *W, int64_t D, int64_t M, const double *norms,
+                   const int32_t *rowptr, const int32_t *colidx, int64_t i, int64_t j)
+{
+    (void)D;
+    double s = 0.0;
+    for (int32_t e = rowptr[i]; e < rowptr[i + 1]; ++e)
+        s += (double)W[(int64_t)colidx[e] * M + j];
+    double nx = (double)(rowptr[i + 1] - rowptr[i]);
+    return nx + norms[j] - 2.0 * s;
+}
+
+/*
+ * BMU of every document.  Outputs per document i:
+ *   bmu[i]  lowest index attaining the minimum distance
+ *   d1[i]   the minimum distance
+ *   d2[i]   the second-smallest distance (over j != bmu[i]; +inf when M == 1)
+ * d2 exists only so that a comparison can tell a near-tie from a wrong answer.
+ * Returns 0, or -1 if scratch memory could not be allocated.
+ */
+int oracle_bmu(const float *W, int64_t D, int64_t M, const double *norms,
+               const int32_t *rowptr, const int32_t *colidx, int64_t N,
+               int32_t *bmu, double *d1, double *d2, int nthreads)
+{
+    (void)D;
+    int failed = 0;
+#ifdef _OPENMP
+    if (nthreads > 0)
+        omp_set_num_threads(nthreads);
+#else
+    (void)nthreads;
+#endif
+#pragma omp parallel
+    {
+        double *acc = (double *)malloc((size_t)(M > 0 ? M : 1) * sizeof(double));
+        if (!acc) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t i = 0; i < N; ++i) {
+            if (!acc)
+                continue;
+            for (int64_t j = 0; j < M; ++j)
+                acc[j] = 0.0;
+            for (int32_t e = rowptr[i]; e < rowptr[i + 1]; ++e) {
+                const float *row = W + (int64_t)colidx[e] * M;
+                for (int64_t j = 0; j < M; ++j)
+                    acc[j] += (double)row[j];
+            }
+            double nx = (double)(rowptr[i + 1] - rowptr[i]);
+            double best = INFINITY, second = INFINITY;
+            int32_t arg = -1;
+            for (int64_t j = 0; j < M; ++j) {
+                double d = nx + norms[j] - 2.0 * acc[j];
+                if (arg < 0 || d < best) {
+                    second = (arg < 0) ? INFINITY : best;
+                    best = d;
+                    arg = (int32_t)j;
+                } else if (d < second) {
+                    second = d;
+                }
+            }
+            bmu[i] = arg;
+            d1[i] = best;
+            d2[i] = second;
+        }
+        free(acc);
+    }
+    return failed ? -1 : 0;
+}
+
+/* Number of threads an oracle_bmu call with nthreads <= 0 would use. */
+int oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
