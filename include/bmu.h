@@ -1,0 +1,158 @@
+/*
+ * bmu.h -- C ABI of the B200 (sm_100a) best-matching-unit search library.
+ *
+ * The operation (paper Section 3: "finding, for each article, the neuron whose
+ * weight vector is closest to it"; the kernel "fuses the argmin into the
+ * product, so the score block is never materialised"): for every document i of
+ * a sparse binary corpus and every neuron j of an M-neuron codebook
+ *
+ *     d_ij = |x_i| + ||w_j||^2 - 2 * sum_{f in x_i} W[f*M + j]
+ *
+ * and the library returns, per document, the lowest j attaining min_j d_ij and
+ * that minimum (the SQUARED distance, not clamped, not rooted).
+ *
+ * Layouts (all arrays are DEVICE memory unless the name says "host"; the
+ * caller owns every buffer it passes and keeps it alive until the stream has
+ * finished the call):
+ *   W       float32 [D][M], feature-major: the M weights of feature f are
+ *           contiguous at W + f*M (Section 3, "W[v.M+i]").  The fast path needs
+ *           W 16-byte aligned and M % 4 == 0; any other M takes a scalar path.
+ *   rowptr  int32 [N+1], rowptr[0] == 0, non-decreasing; row i is
+ *           colidx[rowptr[i] .. rowptr[i+1])            (CSR of the binary corpus)
+ *   colidx  int32 [nnz], feature ids in [0, D); distinct inside a row (a
+ *           repeated id is simply added twice and counted twice in |x_i|);
+ *           any order inside a row.
+ *   norms   float32 [M], ||w_j||^2.
+ *   out_bmu int32 [N], out_dist float32 [N], in the caller's document order.
+ * Limits: M < 2^30; N, D < 2^31; nnz < 2^31 per call (int32 rowptr).  Ids out of
+ * range and non-finite weights are preconditions that the hot path does not
+ * check (bmu_validate_csr checks the former).  An empty row is legal: its
+ * distances are the norms.  N == 0 is legal and does nothing.
+ *
+ * Every call is asynchronous on `stream` (a cudaStream_t passed as void*, NULL =
+ * the legacy default stream) unless stated otherwise, and returns a bmu_status;
+ * errors detected at launch time are returned, nothing throws or aborts.
+ * bmu_last_error() gives a thread-local detail string for the last failure.
+ * There is no CPU fallback: without a CUDA device every compute call returns
+ * BMU_ERR_CUDA.
+ */
+#ifndef BMU_H
+#define BMU_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define BMU_API __attribute__((visibility("default")))
+#else
+#define BMU_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BMU_OK = 0,
+    BMU_ERR_INVALID_ARG = 1,   /* null pointer, negative size, bad option */
+    BMU_ERR_UNSUPPORTED = 2,   /* size beyond a stated limit */
+    BMU_ERR_WORKSPACE = 3,     /* workspace missing, misaligned or too small */
+    BMU_ERR_CUDA = 4,          /* a CUDA runtime call failed (see bmu_last_error) */
+    BMU_ERR_TIMEOUT = 5        /* a bounded device-side wait ran out */
+} bmu_status;
+
+/*
+ * Tunables of the search (the paper's levers, Section 4: tile size, tile
+ * membership, neuron-axis chunking, vector width).  0 in any field = choose
+ * automatically.  Unknown combinations return BMU_ERR_INVALID_ARG.
+ */
+typedef struct bmu_opts {
+    int32_t kernel;         /* 0 auto, 1 direct (rows read through L1/L2), 2 staged
+                               (rows staged through shared memory by bulk copies) */
+    int32_t chunk_neurons;  /* neurons per L2-resident chunk of the codebook (Section 4.2,
+                               "neuron-axis chunking"); rounded to the slab width */
+    int32_t vec;            /* floats per lane per row segment: 4 or 8 */
+    int32_t docs_per_warp;  /* documents a warp carries through one slab pass */
+    int32_t warps;          /* warps per thread block */
+    int32_t cluster;        /* staged kernel: 0 keep corpus order, 1 order documents by
+                               their rarest features before tiling (Section 4.2, "tile
+                               membership") */
+    int32_t stage_rows;     /* staged kernel: codebook rows per pipeline stage */
+    int32_t stages;         /* staged kernel: pipeline depth */
+    int32_t reserved[8];    /* must be 0 */
+} bmu_opts;
+
+BMU_API const char *bmu_status_string(int status);
+BMU_API const char *bmu_last_error(void);
+
+/* Library version as major*10000 + minor*100 + patch. */
+BMU_API int bmu_version(void);
+
+/*
+ * Codebook norms, the "norms" step of an epoch (Table 4): norms[j] = sum_f
+ * W[f*M+j]^2.  Products and the running sum are taken in fp64 and rounded to
+ * fp32 once.  Deterministic.  Uses no scratch memory.
+ */
+BMU_API int bmu_codebook_norms(const float *W, int64_t D, int64_t M, float *norms, void *stream);
+
+/*
+ * Scratch bytes bmu_search_ws needs for a problem of this size (norms, the
+ * per-document running minimum merged across neuron chunks, and the tiling
+ * plan when the staged kernel is selected).  `nnz` is the length of colidx.
+ */
+BMU_API size_t bmu_search_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,
+                                  const bmu_opts *opts);
+
+/*
+ * The whole search (norms -> tiling -> gather-accumulate sweep over neuron
+ * chunks with the argmin fused in -> outputs in document order; Section 3 and
+ * Section 4) with caller-supplied scratch.  `norms` may be NULL (computed into
+ * the workspace) or a device array from bmu_codebook_norms.  `workspace` must be
+ * 256-byte aligned device memory of at least bmu_search_workspace_bytes(...)
+ * bytes; its contents are undefined afterwards.  Allocates nothing.  Calls that
+ * share a workspace must not overlap on the GPU.
+ */
+BMU_API int bmu_search_ws(const float *W, int64_t D, int64_t M, const float *norms,
+                  const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
+                  int32_t *out_bmu, float *out_dist, const bmu_opts *opts,
+                  void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * One-shot form.  Same as bmu_search_ws with norms == NULL and default options,
+ * but the scratch is a library-owned buffer per device that only ever grows
+ * (cudaMalloc on first use or growth; freed by bmu_release_scratch or at
+ * process exit).  Reads rowptr[N] back to size the scratch, so the call
+ * synchronises the stream once before the kernels are queued.  Calls on
+ * different streams of one device share the scratch and must not overlap.
+ */
+BMU_API int bmu_search(const float *W, int64_t D, int64_t M, const int32_t *rowptr,
+               const int32_t *colidx, int64_t N, int32_t *out_bmu, float *out_dist,
+               void *stream);
+
+/*
+ * End-to-end form for a corpus batch that lives in HOST memory (pinned for
+ * full copy speed): copies rowptr_host[N+1] and colidx_host[nnz] to the device,
+ * runs bmu_search against the device-resident codebook W, and copies the N
+ * results back into out_bmu_host / out_dist_host.  Synchronous: returns when
+ * the results are in host memory.  Device staging buffers come from the same
+ * grow-only library scratch as bmu_search.
+ */
+BMU_API int bmu_search_host(const float *W, int64_t D, int64_t M, const int32_t *rowptr_host,
+                    const int32_t *colidx_host, int64_t N, int32_t *out_bmu_host,
+                    float *out_dist_host, void *stream);
+
+/* Frees the library-owned scratch of the current device (synchronises it). */
+BMU_API int bmu_release_scratch(void);
+
+/*
+ * Checks the CSR preconditions on the device: rowptr[0] == 0, rowptr
+ * non-decreasing, rowptr[N] == nnz, 0 <= colidx < D.  Synchronises the stream.
+ * Returns BMU_ERR_INVALID_ARG (detail in bmu_last_error) when one fails.
+ */
+BMU_API int bmu_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
+                     int64_t D, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BMU_H */

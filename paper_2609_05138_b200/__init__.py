@@ -1,0 +1,12 @@
+"""B200-native best-matching-unit search for sparse binary corpora.
+
+The product is the C-ABI CUDA library `libbmu.so` (include/bmu.h, csrc/); this
+package is its thin Python binding.  Nothing here computes on the CPU.
+"""
+from .binding import (BmuError, Opts, bmu_codebook_norms, bmu_release_scratch, bmu_search,
+                      bmu_search_host, bmu_search_workspace_bytes, bmu_search_ws,
+                      bmu_validate_csr, bmu_version, load)
+
+__all__ = ["BmuError", "Opts", "bmu_codebook_norms", "bmu_release_scratch", "bmu_search",
+           "bmu_search_host", "bmu_search_workspace_bytes", "bmu_search_ws",
+           "bmu_validate_csr", "bmu_version", "load"]

@@ -1,0 +1,199 @@
+"""ctypes binding of libbmu.so: argument marshalling only.
+
+Every function takes torch tensors (device memory, or pinned host memory where
+the name says host), checks dtype/contiguity/device, and passes raw pointers,
+sizes and the current CUDA stream to the C entry point of the same name
+(include/bmu.h).  No arithmetic happens here and there is no fallback: if the
+library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbmu.so")
+_lib = None
+
+STATUS_OK = 0
+
+
+class BmuError(RuntimeError):
+    def __init__(self, status: int, detail: str):
+        super().__init__("bmu status %d (%s)" % (status, detail))
+        self.status = status
+
+
+class Opts(ctypes.Structure):
+    """Mirror of `bmu_opts` (include/bmu.h); 0 = automatic."""
+    _fields_ = [("kernel", ctypes.c_int32), ("chunk_neurons", ctypes.c_int32),
+                ("vec", ctypes.c_int32), ("docs_per_warp", ctypes.c_int32),
+                ("warps", ctypes.c_int32), ("cluster", ctypes.c_int32),
+                ("stage_rows", ctypes.c_int32), ("stages", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 8)]
+
+
+EXPORTS = {
+    # name: (restype, argtypes)
+    "bmu_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+    "bmu_last_error": (ctypes.c_char_p, []),
+    "bmu_version": (ctypes.c_int, []),
+    "bmu_codebook_norms": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                          ctypes.c_void_p, ctypes.c_void_p]),
+    "bmu_search_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int64, ctypes.c_int64,
+                                                     ctypes.c_int64, ctypes.c_int64,
+                                                     ctypes.c_void_p]),
+    "bmu_search_ws": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                     ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
+                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                     ctypes.c_size_t, ctypes.c_void_p]),
+    "bmu_search": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "bmu_search_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                       ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                                       ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "bmu_release_scratch": (ctypes.c_int, []),
+    "bmu_validate_csr": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                                        ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
+}
+
+
+def load():
+    """Loads libbmu.so (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                "libbmu.so is not built: run `python -m paper_2609_05138_b200.build` "
+                "(there is no CPU fallback)")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in EXPORTS.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def _check(status: int):
+    if status != STATUS_OK:
+        lib = load()
+        detail = lib.bmu_last_error().decode() or lib.bmu_status_string(status).decode()
+        raise BmuError(status, detail)
+
+
+def _dev(t: torch.Tensor, dtype, name: str):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError("%s must be a contiguous CUDA tensor of dtype %s" % (name, dtype))
+    return t.data_ptr()
+
+
+def _host(t: torch.Tensor, dtype, name: str):
+    if not (isinstance(t, torch.Tensor) and not t.is_cuda and t.dtype == dtype
+            and t.is_contiguous()):
+        raise TypeError("%s must be a contiguous host tensor of dtype %s" % (name, dtype))
+    return t.data_ptr()
+
+
+def _stream(t: torch.Tensor) -> int:
+    return torch.cuda.current_stream(t.device).cuda_stream
+
+
+def _codebook(W: torch.Tensor):
+    if W.dim() != 2:
+        raise TypeError("W must be [D, M] (feature-major)")
+    return _dev(W, torch.float32, "W"), W.shape[0], W.shape[1]
+
+
+def bmu_version() -> int:
+    return load().bmu_version()
+
+
+def bmu_codebook_norms(W: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    wp, D, M = _codebook(W)
+    if out is None:
+        out = torch.empty(M, dtype=torch.float32, device=W.device)
+    with torch.cuda.device(W.device):
+        _check(load().bmu_codebook_norms(wp, D, M, _dev(out, torch.float32, "norms"),
+                                         _stream(W)))
+    return out
+
+
+def bmu_search_workspace_bytes(D: int, M: int, N: int, nnz: int, opts: Opts | None = None) -> int:
+    return int(load().bmu_search_workspace_bytes(D, M, N, nnz,
+                                                 ctypes.byref(opts) if opts else None))
+
+
+def bmu_search_ws(W, rowptr, colidx, norms=None, opts: Opts | None = None, workspace=None,
+                  out_bmu=None, out_dist=None):
+    """Search with caller-owned scratch.  Returns (out_bmu int32 [N], out_dist float32 [N])."""
+    wp, D, M = _codebook(W)
+    N = rowptr.numel() - 1
+    nnz = colidx.numel()
+    if out_bmu is None:
+        out_bmu = torch.empty(N, dtype=torch.int32, device=W.device)
+    if out_dist is None:
+        out_dist = torch.empty(N, dtype=torch.float32, device=W.device)
+    need = bmu_search_workspace_bytes(D, M, N, nnz, opts)
+    if workspace is None:
+        workspace = torch.empty(need + 256, dtype=torch.uint8, device=W.device)
+    ws_ptr = (workspace.data_ptr() + 255) // 256 * 256
+    ws_bytes = workspace.numel() * workspace.element_size() - (ws_ptr - workspace.data_ptr())
+    with torch.cuda.device(W.device):
+        _check(load().bmu_search_ws(
+            wp, D, M, _dev(norms, torch.float32, "norms") if norms is not None else None,
+            _dev(rowptr, torch.int32, "rowptr"),
+            _dev(colidx, torch.int32, "colidx") if nnz else None, N, nnz,
+            _dev(out_bmu, torch.int32, "out_bmu"), _dev(out_dist, torch.float32, "out_dist"),
+            ctypes.byref(opts) if opts else None, ws_ptr, ws_bytes, _stream(W)))
+    return out_bmu, out_dist
+
+
+def bmu_search(W, rowptr, colidx, out_bmu=None, out_dist=None):
+    """One-shot search (library-owned scratch).  Returns (out_bmu, out_dist)."""
+    wp, D, M = _codebook(W)
+    N = rowptr.numel() - 1
+    if out_bmu is None:
+        out_bmu = torch.empty(N, dtype=torch.int32, device=W.device)
+    if out_dist is None:
+        out_dist = torch.empty(N, dtype=torch.float32, device=W.device)
+    with torch.cuda.device(W.device):
+        _check(load().bmu_search(
+            wp, D, M, _dev(rowptr, torch.int32, "rowptr"),
+            _dev(colidx, torch.int32, "colidx") if colidx.numel() else None, N,
+            _dev(out_bmu, torch.int32, "out_bmu"), _dev(out_dist, torch.float32, "out_dist"),
+            _stream(W)))
+    return out_bmu, out_dist
+
+
+def bmu_search_host(W, rowptr_host, colidx_host, out_bmu_host=None, out_dist_host=None):
+    """End-to-end search of a host-resident CSR batch against a device codebook."""
+    wp, D, M = _codebook(W)
+    N = rowptr_host.numel() - 1
+    if out_bmu_host is None:
+        out_bmu_host = torch.empty(N, dtype=torch.int32).pin_memory()
+    if out_dist_host is None:
+        out_dist_host = torch.empty(N, dtype=torch.float32).pin_memory()
+    with torch.cuda.device(W.device):
+        _check(load().bmu_search_host(
+            wp, D, M, _host(rowptr_host, torch.int32, "rowptr_host"),
+            _host(colidx_host, torch.int32, "colidx_host") if colidx_host.numel() else None, N,
+            _host(out_bmu_host, torch.int32, "out_bmu_host"),
+            _host(out_dist_host, torch.float32, "out_dist_host"), _stream(W)))
+    return out_bmu_host, out_dist_host
+
+
+def bmu_release_scratch():
+    _check(load().bmu_release_scratch())
+
+
+def bmu_validate_csr(rowptr, colidx, D: int):
+    N = rowptr.numel() - 1
+    with torch.cuda.device(rowptr.device):
+        _check(load().bmu_validate_csr(
+            _dev(rowptr, torch.int32, "rowptr"),
+            _dev(colidx, torch.int32, "colidx") if colidx.numel() else None, N, colidx.numel(),
+            D, _stream(rowptr)))

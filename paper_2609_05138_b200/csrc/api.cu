@@ -1,0 +1,338 @@
+// Host side of the C ABI: argument checks, workspace layout, neuron-axis
+// chunking (Section 4.2) and the order in which the kernels are queued.
+#include "common.cuh"
+
+#include <stdarg.h>
+#include <string.h>
+
+#include <mutex>
+
+namespace bmu {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
+int cuda_fail(cudaError_t e, const char *what)
+{
+    set_error("%s: %s", what, cudaGetErrorString(e));
+    return BMU_ERR_CUDA;
+}
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static const int64_t MAX_M = (int64_t)1 << 30;   // row pitch M*4 must fit 32 bits
+static const int64_t MAX_I32 = 0x7fffffff;
+
+// ---- workspace layout -----------------------------------------------------
+struct Layout {
+    size_t norms_off, state_off, total;
+};
+
+static Layout layout_for(int64_t M, int64_t N)
+{
+    Layout l;
+    size_t off = 0;
+    l.norms_off = off; off = align_up(off + (size_t)M * sizeof(float), 256);
+    l.state_off = off; off = align_up(off + (size_t)N * sizeof(u64), 256);
+    l.total = off;
+    return l;
+}
+
+static int check_sizes(int64_t D, int64_t M, int64_t N, int64_t nnz)
+{
+    if (D < 0 || M < 0 || N < 0 || nnz < 0) {
+        set_error("negative size (D=%lld M=%lld N=%lld nnz=%lld)", (long long)D, (long long)M,
+                  (long long)N, (long long)nnz);
+        return BMU_ERR_INVALID_ARG;
+    }
+    if (M >= MAX_M || D > MAX_I32 || N >= MAX_I32 || nnz > MAX_I32) {
+        set_error("size beyond the limits (M < 2^30; D, N, nnz < 2^31)");
+        return BMU_ERR_UNSUPPORTED;
+    }
+    return BMU_OK;
+}
+
+static int check_opts(const bmu_opts &o)
+{
+    for (int i = 0; i < 8; ++i)
+        if (o.reserved[i] != 0) { set_error("bmu_opts.reserved must be zero"); return BMU_ERR_INVALID_ARG; }
+    if (o.kernel < 0 || o.kernel > 2) { set_error("bmu_opts.kernel must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
+    if (o.chunk_neurons < 0) { set_error("bmu_opts.chunk_neurons < 0"); return BMU_ERR_INVALID_ARG; }
+    if (o.vec != 0 && o.vec != 4 && o.vec != 8) { set_error("bmu_opts.vec must be 0, 4 or 8"); return BMU_ERR_INVALID_ARG; }
+    return BMU_OK;
+}
+
+// Neurons per L2-resident chunk: the chunk's share of the codebook,
+// D * chunk * 4 bytes, is kept to about half of L2 so that the rows of one
+// chunk stay cached while every document passes over them.
+static int64_t auto_chunk(int64_t D, int64_t M, int slab)
+{
+    int dev = 0, l2 = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess || l2 <= 0)
+        l2 = 64 << 20;
+    int64_t c = D > 0 ? ((int64_t)l2 / 2) / (D * 4) : M;
+    c = c / slab * slab;
+    if (c < slab) c = slab;
+    if (c > M) c = (M + slab - 1) / slab * slab;
+    return c;
+}
+
+static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
+                       const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
+                       int32_t *out_bmu, float *out_dist, const bmu_opts *opts_in, void *ws,
+                       size_t ws_bytes, cudaStream_t s)
+{
+    int rc = check_sizes(D, M, N, nnz);
+    if (rc) return rc;
+    bmu_opts o;
+    memset(&o, 0, sizeof(o));
+    if (opts_in) o = *opts_in;
+    if ((rc = check_opts(o))) return rc;
+    if (N == 0) return BMU_OK;
+    if (!W || !rowptr || !out_bmu || !out_dist || (nnz > 0 && !colidx)) {
+        set_error("null pointer argument");
+        return BMU_ERR_INVALID_ARG;
+    }
+    if (M == 0 || D == 0) {
+        set_error("empty codebook (D=%lld, M=%lld): no neuron to return", (long long)D, (long long)M);
+        return BMU_ERR_INVALID_ARG;
+    }
+    const Layout l = layout_for(M, N);
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < l.total) {
+        set_error("workspace missing, not 256-byte aligned, or smaller than %zu bytes", l.total);
+        return BMU_ERR_WORKSPACE;
+    }
+    char *base = static_cast<char *>(ws);
+    u64 *state = reinterpret_cast<u64 *>(base + l.state_off);
+    if (!norms) {
+        float *n = reinterpret_cast<float *>(base + l.norms_off);
+        if ((rc = launch_norms(W, D, M, n, s))) return rc;
+        norms = n;
+    }
+    if (o.kernel == 2) {
+        set_error("staged kernel not available in this build");
+        return BMU_ERR_UNSUPPORTED;
+    }
+    const int V = o.vec ? o.vec : 4;
+    const int slab = 32 * V;
+    int64_t chunk = o.chunk_neurons ? (o.chunk_neurons + slab - 1) / slab * slab
+                                    : auto_chunk(D, M, slab);
+    SweepArgs a;
+    a.W = W; a.D = D; a.M = M; a.norms = norms; a.rowptr = rowptr; a.colidx = colidx;
+    a.N = N; a.state = state;
+    for (int64_t j = 0; j < M; j += chunk) {
+        a.j_lo = (int32_t)j;
+        a.j_hi = (int32_t)(j + chunk < M ? j + chunk : M);
+        a.first = j == 0;
+        if ((rc = launch_sweep_direct(a, o, s))) return rc;
+    }
+    return launch_finalize(state, rowptr, N, out_bmu, out_dist, s);
+}
+
+// ---- library-owned grow-only scratch (one per device) ----------------------
+struct Scratch { void *p; size_t bytes; };
+static Scratch g_scratch[64];
+static std::mutex g_mu;
+
+static int scratch_get(size_t bytes, void **out)
+{
+    int dev = 0;
+    BMU_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) { set_error("device ordinal %d out of range", dev); return BMU_ERR_UNSUPPORTED; }
+    std::lock_guard<std::mutex> g(g_mu);
+    Scratch &sc = g_scratch[dev];
+    if (sc.bytes < bytes) {
+        if (sc.p) {
+            BMU_CUDA(cudaDeviceSynchronize());
+            BMU_CUDA(cudaFree(sc.p));
+            sc.p = nullptr; sc.bytes = 0;
+        }
+        const size_t want = align_up(bytes + bytes / 8, (size_t)1 << 20);
+        BMU_CUDA(cudaMalloc(&sc.p, want));
+        sc.bytes = want;
+    }
+    *out = sc.p;
+    return BMU_OK;
+}
+
+// ---- CSR validation ---------------------------------------------------------
+__global__ void validate_kernel(const int32_t *__restrict__ rowptr,
+                                const int32_t *__restrict__ colidx, int64_t N, int64_t nnz,
+                                int64_t D, int32_t *__restrict__ flags)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    if (t == 0) {
+        if (rowptr[0] != 0) atomicOr(flags, 1);
+        if ((int64_t)rowptr[N] != nnz) atomicOr(flags, 2);
+    }
+    for (int64_t i = t; i < N; i += stride)
+        if (rowptr[i + 1] < rowptr[i]) atomicOr(flags, 4);
+    for (int64_t e = t; e < nnz; e += stride) {
+        const int32_t f = colidx[e];
+        if (f < 0 || (int64_t)f >= D) atomicOr(flags, 8);
+    }
+}
+
+int launch_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
+                        int64_t D, int32_t *flags, cudaStream_t s)
+{
+    BMU_CUDA(cudaMemsetAsync(flags, 0, sizeof(int32_t), s));
+    validate_kernel<<<296, 256, 0, s>>>(rowptr, colidx, N, nnz, D, flags);
+    BMU_CUDA(cudaGetLastError());
+    return BMU_OK;
+}
+
+}  // namespace bmu
+
+using namespace bmu;
+
+extern "C" {
+
+const char *bmu_status_string(int status)
+{
+    switch (status) {
+    case BMU_OK: return "ok";
+    case BMU_ERR_INVALID_ARG: return "invalid argument";
+    case BMU_ERR_UNSUPPORTED: return "unsupported size or option";
+    case BMU_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case BMU_ERR_CUDA: return "CUDA runtime error";
+    case BMU_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+    }
+}
+
+const char *bmu_last_error(void) { return g_err; }
+
+int bmu_version(void) { return 100; }
+
+int bmu_codebook_norms(const float *W, int64_t D, int64_t M, float *norms, void *stream)
+{
+    int rc = check_sizes(D, M, 0, 0);
+    if (rc) return rc;
+    if (M == 0) return BMU_OK;
+    if (!norms || (D > 0 && !W)) { set_error("null pointer argument"); return BMU_ERR_INVALID_ARG; }
+    return launch_norms(W, D, M, norms, static_cast<cudaStream_t>(stream));
+}
+
+size_t bmu_search_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,
+                                  const bmu_opts *opts)
+{
+    (void)D; (void)nnz; (void)opts;
+    if (M < 0 || N < 0) return 0;
+    return layout_for(M, N).total;
+}
+
+int bmu_search_ws(const float *W, int64_t D, int64_t M, const float *norms,
+                  const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
+                  int32_t *out_bmu, float *out_dist, const bmu_opts *opts, void *workspace,
+                  size_t workspace_bytes, void *stream)
+{
+    return search_impl(W, D, M, norms, rowptr, colidx, N, nnz, out_bmu, out_dist, opts,
+                       workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int bmu_search(const float *W, int64_t D, int64_t M, const int32_t *rowptr,
+               const int32_t *colidx, int64_t N, int32_t *out_bmu, float *out_dist,
+               void *stream)
+{
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int rc = check_sizes(D, M, N, 0);
+    if (rc) return rc;
+    if (N == 0) return BMU_OK;
+    if (!rowptr) { set_error("null pointer argument"); return BMU_ERR_INVALID_ARG; }
+    int32_t nnz = 0;
+    BMU_CUDA(cudaMemcpyAsync(&nnz, rowptr + N, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    BMU_CUDA(cudaStreamSynchronize(s));
+    const size_t need = bmu_search_workspace_bytes(D, M, N, nnz, nullptr);
+    void *ws = nullptr;
+    if ((rc = scratch_get(need, &ws))) return rc;
+    return search_impl(W, D, M, nullptr, rowptr, colidx, N, nnz, out_bmu, out_dist, nullptr, ws,
+                       need, s);
+}
+
+int bmu_search_host(const float *W, int64_t D, int64_t M, const int32_t *rowptr_host,
+                    const int32_t *colidx_host, int64_t N, int32_t *out_bmu_host,
+                    float *out_dist_host, void *stream)
+{
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int rc = check_sizes(D, M, N, 0);
+    if (rc) return rc;
+    if (N == 0) return BMU_OK;
+    if (!rowptr_host || !out_bmu_host || !out_dist_host) {
+        set_error("null pointer argument");
+        return BMU_ERR_INVALID_ARG;
+    }
+    const int64_t nnz = rowptr_host[N];
+    if (nnz < 0 || (nnz > 0 && !colidx_host)) { set_error("bad rowptr[N] or null colidx"); return BMU_ERR_INVALID_ARG; }
+    const size_t ws_need = bmu_search_workspace_bytes(D, M, N, nnz, nullptr);
+    const size_t rp_off = align_up(ws_need, 256);
+    const size_t ci_off = align_up(rp_off + (size_t)(N + 1) * 4, 256);
+    const size_t ob_off = align_up(ci_off + (size_t)nnz * 4, 256);
+    const size_t od_off = align_up(ob_off + (size_t)N * 4, 256);
+    const size_t total = align_up(od_off + (size_t)N * 4, 256);
+    void *p = nullptr;
+    if ((rc = scratch_get(total, &p))) return rc;
+    char *b = static_cast<char *>(p);
+    int32_t *rp = reinterpret_cast<int32_t *>(b + rp_off);
+    int32_t *ci = reinterpret_cast<int32_t *>(b + ci_off);
+    int32_t *ob = reinterpret_cast<int32_t *>(b + ob_off);
+    float *od = reinterpret_cast<float *>(b + od_off);
+    BMU_CUDA(cudaMemcpyAsync(rp, rowptr_host, (size_t)(N + 1) * 4, cudaMemcpyHostToDevice, s));
+    if (nnz)
+        BMU_CUDA(cudaMemcpyAsync(ci, colidx_host, (size_t)nnz * 4, cudaMemcpyHostToDevice, s));
+    if ((rc = search_impl(W, D, M, nullptr, rp, ci, N, nnz, ob, od, nullptr, b, ws_need, s)))
+        return rc;
+    BMU_CUDA(cudaMemcpyAsync(out_bmu_host, ob, (size_t)N * 4, cudaMemcpyDeviceToHost, s));
+    BMU_CUDA(cudaMemcpyAsync(out_dist_host, od, (size_t)N * 4, cudaMemcpyDeviceToHost, s));
+    BMU_CUDA(cudaStreamSynchronize(s));
+    return BMU_OK;
+}
+
+int bmu_release_scratch(void)
+{
+    int dev = 0;
+    BMU_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return BMU_OK;
+    std::lock_guard<std::mutex> g(g_mu);
+    Scratch &sc = g_scratch[dev];
+    if (sc.p) {
+        BMU_CUDA(cudaDeviceSynchronize());
+        BMU_CUDA(cudaFree(sc.p));
+        sc.p = nullptr; sc.bytes = 0;
+    }
+    return BMU_OK;
+}
+
+int bmu_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
+                     int64_t D, void *stream)
+{
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int rc = check_sizes(D, 0, N, nnz);
+    if (rc) return rc;
+    if (!rowptr || (nnz > 0 && !colidx)) { set_error("null pointer argument"); return BMU_ERR_INVALID_ARG; }
+    void *p = nullptr;
+    if ((rc = scratch_get(256, &p))) return rc;
+    int32_t *flags = static_cast<int32_t *>(p);
+    if ((rc = launch_validate_csr(rowptr, colidx, N, nnz, D, flags, s))) return rc;
+    int32_t h = 0;
+    BMU_CUDA(cudaMemcpyAsync(&h, flags, sizeof(h), cudaMemcpyDeviceToHost, s));
+    BMU_CUDA(cudaStreamSynchronize(s));
+    if (h) {
+        set_error("invalid CSR:%s%s%s%s", (h & 1) ? " rowptr[0] != 0;" : "",
+                  (h & 2) ? " rowptr[N] != nnz;" : "", (h & 4) ? " rowptr decreases;" : "",
+                  (h & 8) ? " colidx outside [0, D);" : "");
+        return BMU_ERR_INVALID_ARG;
+    }
+    return BMU_OK;
+}
+
+}  // extern "C"

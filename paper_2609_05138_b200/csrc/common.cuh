@@ -1,0 +1,97 @@
+// Shared device/host helpers of the BMU library (CUDA path only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "bmu.h"
+
+namespace bmu {
+
+typedef unsigned long long u64;
+
+// ---- error plumbing -------------------------------------------------------
+void set_error(const char *fmt, ...);
+int cuda_fail(cudaError_t e, const char *what);
+
+#define BMU_CUDA(call)                                       \
+    do {                                                     \
+        cudaError_t e__ = (call);                            \
+        if (e__ != cudaSuccess) return bmu::cuda_fail(e__, #call); \
+    } while (0)
+
+// ---- (distance, index) keys ----------------------------------------------
+// A 64-bit key whose unsigned order is the lexicographic order of (distance,
+// neuron index): the smallest key is the smallest distance and, among equal
+// distances, the lowest index -- the tie rule of the search.  The float is
+// mapped to an unsigned int that sorts like the float does.
+__host__ __device__ __forceinline__ uint32_t float_to_ordered(float x)
+{
+#ifdef __CUDA_ARCH__
+    uint32_t b = __float_as_uint(x);
+#else
+    union { float f; uint32_t u; } c; c.f = x; uint32_t b = c.u;
+#endif
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+__host__ __device__ __forceinline__ float ordered_to_float(uint32_t o)
+{
+    uint32_t b = (o & 0x80000000u) ? (o & 0x7fffffffu) : ~o;
+#ifdef __CUDA_ARCH__
+    return __uint_as_float(b);
+#else
+    union { float f; uint32_t u; } c; c.u = b; return c.f;
+#endif
+}
+
+__host__ __device__ __forceinline__ u64 make_key(float d, int32_t j)
+{
+    return ((u64)float_to_ordered(d) << 32) | (uint32_t)j;
+}
+
+static const u64 KEY_WORST = ~0ull;
+
+#ifdef __CUDACC__
+// lexicographic (d, j) minimum across the warp; every lane gets the result
+__device__ __forceinline__ void warp_argmin(float &d, int &j)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        float od = __shfl_xor_sync(0xffffffffu, d, off);
+        int oj = __shfl_xor_sync(0xffffffffu, j, off);
+        if (od < d || (od == d && oj < j)) { d = od; j = oj; }
+    }
+}
+
+// packed fp32 pair add: two IEEE round-to-nearest adds in one issue slot (sm_100a)
+__device__ __forceinline__ void add2(u64 &acc, u64 w)
+{
+    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(acc) : "l"(w));
+}
+__device__ __forceinline__ float lo_f(u64 p) { return __uint_as_float((uint32_t)p); }
+__device__ __forceinline__ float hi_f(u64 p) { return __uint_as_float((uint32_t)(p >> 32)); }
+#endif
+
+// ---- kernels' host launchers (one per .cu file) ---------------------------
+int launch_norms(const float *W, int64_t D, int64_t M, float *norms, cudaStream_t s);
+
+struct SweepArgs {
+    const float *W;
+    int64_t D, M;
+    const float *norms;
+    const int32_t *rowptr;
+    const int32_t *colidx;
+    int64_t N;
+    u64 *state;           // per-document running (distance, index) key
+    int32_t j_lo, j_hi;   // neuron chunk [j_lo, j_hi)
+    int32_t first;        // 1: this chunk initialises the state, 0: merges into it
+};
+int launch_sweep_direct(const SweepArgs &a, const bmu_opts &o, cudaStream_t s);
+int launch_finalize(const u64 *state, const int32_t *rowptr, int64_t N, int32_t *out_bmu,
+                    float *out_dist, cudaStream_t s);
+int launch_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
+                        int64_t D, int32_t *flags, cudaStream_t s);
+
+}  // namespace bmu

@@ -1,0 +1,89 @@
+// Codebook norms: norms[j] = sum_f W[f*M + j]^2   (the "norms" step, Table 4).
+//
+// A pure HBM stream over the D x M codebook.  One thread block owns a band of
+// columns; its warps take the feature rows round-robin, square and sum in fp64,
+// and the per-warp partials are added in a fixed order in shared memory, so
+// the result does not depend on scheduling.  No scratch memory.
+#include "common.cuh"
+
+namespace bmu {
+
+static const int NORM_WARPS = 16;
+
+// VEC: a lane owns 4 consecutive columns (one 16-byte load per row);
+// otherwise a lane owns one column.
+template <bool VEC>
+__global__ void __launch_bounds__(NORM_WARPS * 32)
+norms_kernel(const float *__restrict__ W, int64_t D, int64_t M, float *__restrict__ norms)
+{
+    constexpr int C = VEC ? 4 : 1;
+    __shared__ double part[NORM_WARPS][32 * C];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t col = (int64_t)blockIdx.x * (32 * C) + lane * C;
+    const bool act = col < M;
+    double a[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) a[c] = 0.0;
+
+    if (act) {
+        const float *p = W + col;
+        int64_t f = warp;
+        // four rows in flight per thread
+        for (; f + 3 * NORM_WARPS < D; f += 4 * NORM_WARPS) {
+            float v[4][C];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float *q = p + (f + (int64_t)u * NORM_WARPS) * M;
+                if constexpr (VEC) {
+                    float4 t = __ldcs(reinterpret_cast<const float4 *>(q));
+                    v[u][0] = t.x; v[u][1] = t.y; v[u][2] = t.z; v[u][3] = t.w;
+                } else {
+                    v[u][0] = __ldcs(q);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int c = 0; c < C; ++c) {
+                    double w = (double)v[u][c];
+                    a[c] = fma(w, w, a[c]);
+                }
+        }
+        for (; f < D; f += NORM_WARPS) {
+            const float *q = p + f * M;
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                double w = (double)q[c];
+                a[c] = fma(w, w, a[c]);
+            }
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < C; ++c) part[warp][lane * C + c] = a[c];
+    __syncthreads();
+    if (threadIdx.x < 32 * C) {
+        const int64_t j = (int64_t)blockIdx.x * (32 * C) + threadIdx.x;
+        if (j < M) {
+            double s = 0.0;
+#pragma unroll
+            for (int w = 0; w < NORM_WARPS; ++w) s += part[w][threadIdx.x];
+            norms[j] = (float)s;
+        }
+    }
+}
+
+int launch_norms(const float *W, int64_t D, int64_t M, float *norms, cudaStream_t s)
+{
+    if (M == 0) return BMU_OK;
+    const bool vec = (M % 4 == 0) && ((reinterpret_cast<uintptr_t>(W) & 15) == 0);
+    const int cols = vec ? 128 : 32;
+    const int64_t blocks = (M + cols - 1) / cols;
+    if (vec)
+        norms_kernel<true><<<(unsigned)blocks, NORM_WARPS * 32, 0, s>>>(W, D, M, norms);
+    else
+        norms_kernel<false><<<(unsigned)blocks, NORM_WARPS * 32, 0, s>>>(W, D, M, norms);
+    BMU_CUDA(cudaGetLastError());
+    return BMU_OK;
+}
+
+}  // namespace bmu

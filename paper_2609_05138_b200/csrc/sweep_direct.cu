@@ -1,0 +1,220 @@
+// Direct gather-accumulate sweep with the argmin fused in (Section 3; levers of
+// Section 4: vector loads, neuron-axis chunking).
+//
+// One warp carries K documents through the neuron chunk [j_lo, j_hi) slab by
+// slab.  A slab is 32*V consecutive neurons: every lane owns V of them and adds,
+// for each active feature f of the document, its piece of the codebook row
+// W[f*M + slab] -- a 128-bit load per lane, 512 contiguous bytes per warp --
+// into fp32 accumulators (x is binary, so there is no multiply).  The rows come
+// through L1/L2: all warps of a block walk the slabs in the same order, so the
+// rows of frequent features are shared in L1, and the host keeps one chunk of
+// the codebook (D * chunk * 4 bytes) resident in L2 by launching chunk by chunk.
+// After the last feature each lane turns its sums into distances
+// n_j - 2 s_ij (|x_i| is added once at the end), keeps a running minimum with
+// a strict "<" over ascending j, and after the last slab the warp reduces
+// (distance, index) lexicographically by shuffles and merges it into the
+// per-document state that persists across chunks.
+#include "common.cuh"
+
+#include <math_constants.h>
+
+namespace bmu {
+
+template <int V, int K, int NW, bool VEC>
+__global__ void __launch_bounds__(NW * 32)
+sweep_direct_kernel(const SweepArgs a)
+{
+    static_assert(!VEC || V % 4 == 0, "vector path owns whole float4s");
+    constexpr int H = VEC ? V / 4 : V;            // loads per lane per row
+    constexpr int STEP = VEC ? 4 : 1;             // floats per load
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t doc0 = ((int64_t)blockIdx.x * NW + warp) * K;
+    if (doc0 >= a.N) return;
+
+    int beg[K], end[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const int64_t i = doc0 + k;
+        beg[k] = i < a.N ? __ldg(a.rowptr + i) : 0;
+        end[k] = i < a.N ? __ldg(a.rowptr + i + 1) : 0;
+    }
+    float best[K];
+    int bidx[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) { best[k] = CUDART_INF_F; bidx[k] = 0x7fffffff; }
+
+    const uint32_t rowbytes = (uint32_t)(a.M * 4);
+
+    for (int j0 = a.j_lo; j0 < a.j_hi; j0 += 32 * V) {
+        // this lane's columns of the slab
+        int col[H];
+        bool act[H];
+        const char *base[H];
+#pragma unroll
+        for (int h = 0; h < H; ++h) {
+            col[h] = VEC ? j0 + h * 128 + lane * 4 : j0 + h * 32 + lane;
+            act[h] = col[h] < a.j_hi;
+            base[h] = reinterpret_cast<const char *>(a.W + (act[h] ? col[h] : a.j_lo));
+        }
+        float nrm[H][STEP];
+#pragma unroll
+        for (int h = 0; h < H; ++h)
+#pragma unroll
+            for (int c = 0; c < STEP; ++c)
+                nrm[h][c] = act[h] ? __ldg(a.norms + col[h] + c) : CUDART_INF_F;
+
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            if (doc0 + k >= a.N) continue;             // warp-uniform
+            float s[H][STEP];
+            if constexpr (VEC) {
+                u64 acc[H][2];
+#pragma unroll
+                for (int h = 0; h < H; ++h) acc[h][0] = acc[h][1] = 0ull;
+                for (int eb = beg[k]; eb < end[k]; eb += 32) {
+                    const int myf = (eb + lane < end[k]) ? __ldg(a.colidx + eb + lane) : 0;
+                    const int c = min(32, end[k] - eb);
+                    int q = 0;
+                    for (; q + 4 <= c; q += 4) {
+                        ulonglong2 w[4][H];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const uint32_t f = (uint32_t)__shfl_sync(0xffffffffu, myf, q + u);
+                            const u64 off = (u64)f * rowbytes;
+#pragma unroll
+                            for (int h = 0; h < H; ++h)
+                                w[u][h] = act[h]
+                                    ? __ldg(reinterpret_cast<const ulonglong2 *>(base[h] + off))
+                                    : make_ulonglong2(0ull, 0ull);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+#pragma unroll
+                            for (int h = 0; h < H; ++h) {
+                                add2(acc[h][0], w[u][h].x);
+                                add2(acc[h][1], w[u][h].y);
+                            }
+                    }
+                    for (; q < c; ++q) {
+                        const uint32_t f = (uint32_t)__shfl_sync(0xffffffffu, myf, q);
+                        const u64 off = (u64)f * rowbytes;
+#pragma unroll
+                        for (int h = 0; h < H; ++h) {
+                            const ulonglong2 w = act[h]
+                                ? __ldg(reinterpret_cast<const ulonglong2 *>(base[h] + off))
+                                : make_ulonglong2(0ull, 0ull);
+                            add2(acc[h][0], w.x);
+                            add2(acc[h][1], w.y);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int h = 0; h < H; ++h) {
+                    s[h][0] = lo_f(acc[h][0]); s[h][1] = hi_f(acc[h][0]);
+                    s[h][2] = lo_f(acc[h][1]); s[h][3] = hi_f(acc[h][1]);
+                }
+            } else {
+#pragma unroll
+                for (int h = 0; h < H; ++h) s[h][0] = 0.f;
+                for (int eb = beg[k]; eb < end[k]; eb += 32) {
+                    const int myf = (eb + lane < end[k]) ? __ldg(a.colidx + eb + lane) : 0;
+                    const int c = min(32, end[k] - eb);
+                    for (int q = 0; q < c; ++q) {
+                        const uint32_t f = (uint32_t)__shfl_sync(0xffffffffu, myf, q);
+                        const u64 off = (u64)f * rowbytes;
+#pragma unroll
+                        for (int h = 0; h < H; ++h)
+                            if (act[h])
+                                s[h][0] += __ldg(reinterpret_cast<const float *>(base[h] + off));
+                    }
+                }
+            }
+            // distances of this slab, running minimum over ascending neuron index
+#pragma unroll
+            for (int h = 0; h < H; ++h)
+#pragma unroll
+                for (int c = 0; c < STEP; ++c) {
+                    const float d = fmaf(-2.f, s[h][c], nrm[h][c]);
+                    if (d < best[k]) { best[k] = d; bidx[k] = col[h] + c; }
+                }
+        }
+    }
+
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        if (doc0 + k >= a.N) continue;
+        float d = best[k];
+        int j = bidx[k];
+        warp_argmin(d, j);
+        if (lane == 0) {
+            u64 key = make_key(d, j);
+            if (!a.first) {
+                const u64 old = a.state[doc0 + k];
+                if (old < key) key = old;
+            }
+            a.state[doc0 + k] = key;
+        }
+    }
+}
+
+// state -> outputs: out_dist = |x_i| + min_j (n_j - 2 s_ij)
+__global__ void finalize_kernel(const u64 *__restrict__ state, const int32_t *__restrict__ rowptr,
+                                int64_t N, int32_t *__restrict__ out_bmu,
+                                float *__restrict__ out_dist)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    const u64 key = state[i];
+    const float nx = (float)(rowptr[i + 1] - rowptr[i]);
+    out_bmu[i] = (int32_t)(uint32_t)key;
+    out_dist[i] = nx + ordered_to_float((uint32_t)(key >> 32));
+}
+
+int launch_finalize(const u64 *state, const int32_t *rowptr, int64_t N, int32_t *out_bmu,
+                    float *out_dist, cudaStream_t s)
+{
+    if (N == 0) return BMU_OK;
+    finalize_kernel<<<(unsigned)((N + 255) / 256), 256, 0, s>>>(state, rowptr, N, out_bmu,
+                                                                out_dist);
+    BMU_CUDA(cudaGetLastError());
+    return BMU_OK;
+}
+
+template <int V, int K, int NW, bool VEC>
+static int launch_one(const SweepArgs &a, cudaStream_t s)
+{
+    const int64_t per_block = (int64_t)NW * K;
+    const int64_t blocks = (a.N + per_block - 1) / per_block;
+    sweep_direct_kernel<V, K, NW, VEC><<<(unsigned)blocks, NW * 32, 0, s>>>(a);
+    BMU_CUDA(cudaGetLastError());
+    return BMU_OK;
+}
+
+template <int V, bool VEC>
+static int launch_vk(const SweepArgs &a, int K, int NW, cudaStream_t s)
+{
+#define BMU_CASE(k, nw) if (K == k && NW == nw) return launch_one<V, k, nw, VEC>(a, s);
+    BMU_CASE(1, 8) BMU_CASE(1, 16) BMU_CASE(1, 32)
+    BMU_CASE(2, 8) BMU_CASE(2, 16) BMU_CASE(2, 32)
+    BMU_CASE(4, 8) BMU_CASE(4, 16) BMU_CASE(4, 32)
+#undef BMU_CASE
+    set_error("direct kernel: docs_per_warp must be 1, 2 or 4 and warps 8, 16 or 32");
+    return BMU_ERR_INVALID_ARG;
+}
+
+int launch_sweep_direct(const SweepArgs &a, const bmu_opts &o, cudaStream_t s)
+{
+    if (a.N == 0 || a.j_lo >= a.j_hi) return BMU_OK;
+    const int K = o.docs_per_warp ? o.docs_per_warp : 4;
+    const int NW = o.warps ? o.warps : 16;
+    const bool vec = (a.M % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.W) & 15) == 0) &&
+                     (a.j_lo % 4 == 0);
+    if (!vec) return launch_vk<4, false>(a, K, NW, s);
+    const int V = o.vec ? o.vec : 4;
+    if (V == 4) return launch_vk<4, true>(a, K, NW, s);
+    if (V == 8) return launch_vk<8, true>(a, K, NW, s);
+    set_error("vec must be 4 or 8");
+    return BMU_ERR_INVALID_ARG;
+}
+
+}  // namespace bmu

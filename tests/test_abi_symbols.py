@@ -1,0 +1,69 @@
+"""The C-ABI library loads and exports every entry point include/bmu.h declares,
+and its host-side argument checks answer without touching a GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2609_05138_b200 import build, binding
+    build.build_library()
+    return binding.load()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "bmu.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"BMU_API\s+[\w\s\*]+?\b(bmu_\w+)\s*\(", text)))
+
+
+def test_header_and_binding_agree(lib):
+    from paper_2609_05138_b200 import binding
+    names = declared_functions()
+    assert len(names) >= 10
+    assert sorted(binding.EXPORTS) == names
+    for n in names:
+        assert getattr(lib, n) is not None           # dlsym succeeds
+
+
+def test_only_the_api_is_exported():
+    import subprocess
+    from paper_2609_05138_b200 import binding
+    out = subprocess.check_output(["nm", "-D", "--defined-only", binding.LIB_PATH], text=True)
+    syms = [l.split()[-1] for l in out.splitlines() if " T " in l]
+    assert sorted(syms) == declared_functions()
+
+
+def test_status_strings_and_version(lib):
+    assert lib.bmu_status_string(0) == b"ok"
+    assert b"workspace" in lib.bmu_status_string(3)
+    assert lib.bmu_version() >= 100
+
+
+def test_workspace_size_is_monotone(lib):
+    f = lib.bmu_search_workspace_bytes
+    a = f(4096, 1024, 10_000, 640_000, None)
+    b = f(16384, 262144, 2_000_000, 160_000_000, None)
+    assert 0 < a < b
+    assert a % 256 == 0 and b >= 262144 * 4 + 2_000_000 * 8
+
+
+def test_argument_checks_need_no_gpu(lib):
+    # sizes are checked before any CUDA call is made
+    assert lib.bmu_codebook_norms(None, -1, 4, None, None) == 1
+    assert lib.bmu_search(None, 4, 1 << 30, None, None, 1, None, None, None) == 2
+    assert b"limits" in lib.bmu_last_error()
+    assert lib.bmu_search_ws(None, 4, 4, None, None, None, 0, 0, None, None, None, None, 0,
+                             None) == 0           # N == 0: nothing to do
+    assert lib.bmu_search_ws(None, 4, 4, None, None, None, 3, 0, None, None, None, None, 0,
+                             None) == 1           # null pointers
+    from paper_2609_05138_b200 import Opts
+    o = Opts()
+    o.vec = 3
+    assert lib.bmu_search_ws(None, 4, 4, None, None, None, 3, 0, None, None,
+                             ctypes.byref(o), None, 0, None) == 1

@@ -1,0 +1,203 @@
+"""Parity of the CUDA path against the fp64 oracle, through the C ABI.
+
+Same seeded arrays on both sides; the rule is tests/parity.py (indices equal
+except inside a 1e-5 near-tie, distances within 1e-5 relative).
+"""
+import numpy as np
+import pytest
+import torch
+
+from inputs import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def bmu():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_05138_b200 as lib
+    lib.load()
+    return lib
+
+
+def dev(*arrays):
+    return [a.cuda() if isinstance(a, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(a)).cuda()
+            for a in arrays]
+
+
+def run_and_check(bmu, W, rowptr, colidx, opts=None, cancel_floor=False, one_shot=False):
+    Wd, rp, ci = dev(W, rowptr, colidx)
+    if one_shot:
+        ob, od = bmu.bmu_search(Wd, rp, ci)
+    else:
+        ob, od = bmu.bmu_search_ws(Wd, rp, ci, opts=opts)
+    torch.cuda.synchronize()
+    return parity.compare(ob.cpu().numpy(), od.cpu().numpy(), W.numpy(), rowptr.numpy(),
+                          colidx.numpy(), cancel_floor=cancel_floor)
+
+
+def make_opts(bmu, **kw):
+    o = bmu.Opts()
+    for k, v in kw.items():
+        setattr(o, k, v)
+    return o
+
+
+# ------------------------------------------------------------------ norms
+@pytest.mark.parametrize("D,M,kind", [(4096, 1024, "uniform"), (16384, 4096, "uniform"),
+                                      (513, 1000, "signed"), (77, 37, "uniform"),
+                                      (1, 5, "uniform"), (300, 130, "scaled")])
+def test_norms_match_oracle(bmu, D, M, kind):
+    import oracle
+    W = synth.make_codebook(D, M, 5, kind=kind)
+    got = bmu.bmu_codebook_norms(W.cuda()).cpu().numpy().astype(np.float64)
+    ref = oracle.norms(W.numpy())
+    # fp64 accumulation rounded once to fp32: half an ulp
+    np.testing.assert_allclose(got, ref, rtol=6e-8, atol=0)
+
+
+# ------------------------------------------------------------------ benchmark shapes
+def test_cfg1_full(bmu):
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg)
+    W = synth.make_codebook(cfg.D, cfg.M, synth.codebook_seed(cfg))
+    res = run_and_check(bmu, W, rowptr, colidx, one_shot=True)
+    assert res["docs"] == cfg.N and res["exact"] > 0.98 * cfg.N
+
+
+@pytest.mark.parametrize("name,n_docs,M", [("cfg2", 3000, 4096), ("cfg3", 600, 16384),
+                                           ("cfg5", 600, 16384)])
+def test_reduced_benchmark_shapes(bmu, name, n_docs, M):
+    cfg = synth.CONFIGS[name]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=n_docs)
+    W = synth.make_codebook(cfg.D, M, synth.codebook_seed(cfg))
+    run_and_check(bmu, W, rowptr, colidx)
+
+
+# ------------------------------------------------------------------ codebooks where the sum decides
+@pytest.mark.parametrize("kind,floor", [("scaled", False), ("sparse", False), ("signed", False),
+                                        ("dupes", False), ("const", False),
+                                        ("prototype", True)])
+def test_codebook_kinds(bmu, kind, floor):
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=1500)
+    W = synth.make_codebook(cfg.D, 640, 77, kind=kind, docs=(rowptr, colidx))
+    res = run_and_check(bmu, W, rowptr, colidx, cancel_floor=floor)
+    if kind == "dupes":
+        Wd, rp, ci = dev(W, rowptr, colidx)
+        ob, _ = bmu.bmu_search_ws(Wd, rp, ci)
+        assert int((ob % 2).sum()) == 0            # equal columns: the lower index wins
+    if kind == "const":
+        Wd, rp, ci = dev(W, rowptr, colidx)
+        ob, _ = bmu.bmu_search_ws(Wd, rp, ci)
+        assert int(ob.abs().sum()) == 0            # every neuron ties: index 0
+    assert res["failed"] == 0
+
+
+# ------------------------------------------------------------------ ragged sizes and chunking
+@pytest.mark.parametrize("N,D,M,chunk", [
+    (1, 1, 1, 0), (3, 9, 4, 0), (257, 300, 1000, 0), (130, 64, 1028, 256), (515, 128, 37, 0),
+    (99, 2048, 2500, 512), (1000, 512, 4100, 1024), (64, 100, 131, 0), (200, 50, 6, 0),
+])
+def test_ragged_shapes(bmu, N, D, M, chunk):
+    r = np.random.default_rng(N * 7 + M)
+    rows = [np.sort(r.choice(D, size=int(r.integers(0, min(D, 40) + 1)), replace=False))
+            for _ in range(N)]
+    rowptr = np.zeros(N + 1, dtype=np.int32)
+    rowptr[1:] = np.cumsum([len(x) for x in rows])
+    colidx = np.concatenate(rows).astype(np.int32) if rowptr[-1] else np.zeros(0, np.int32)
+    W = synth.make_codebook(D, M, 3 + M, kind="scaled")
+    opts = make_opts(bmu, chunk_neurons=chunk) if chunk else None
+    run_and_check(bmu, W, torch.from_numpy(rowptr), torch.from_numpy(colidx), opts=opts)
+
+
+def test_long_and_empty_rows(bmu):
+    D, M = 16384, 1536
+    nnz = torch.tensor([400, 0, 1, 33, 0, 400, 97, 64, 32, 31, 0])
+    rowptr, colidx = synth.draw_corpus(nnz.numel(), D, 1.1, nnz, seed=4)
+    assert rowptr[-1] == nnz.sum()
+    W = synth.make_codebook(D, M, 8)
+    run_and_check(bmu, W, rowptr, colidx)
+
+
+def test_unsorted_rows(bmu):
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=300)
+    ci = colidx.numpy().copy()
+    r = np.random.default_rng(0)
+    rp = rowptr.numpy()
+    for i in range(300):
+        r.shuffle(ci[rp[i]:rp[i + 1]])
+    W = synth.make_codebook(cfg.D, 512, 9, kind="scaled")
+    run_and_check(bmu, W, rowptr, torch.from_numpy(ci))
+
+
+# ------------------------------------------------------------------ every lever gives the same answer
+@pytest.mark.parametrize("vec", [4, 8])
+@pytest.mark.parametrize("docs_per_warp", [1, 2, 4])
+@pytest.mark.parametrize("warps", [8, 32])
+def test_direct_kernel_options(bmu, vec, docs_per_warp, warps):
+    cfg = synth.CONFIGS["cfg2"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=777)
+    W = synth.make_codebook(cfg.D, 2048 + 128, 13, kind="scaled")
+    opts = make_opts(bmu, kernel=1, vec=vec, docs_per_warp=docs_per_warp, warps=warps,
+                     chunk_neurons=768)
+    run_and_check(bmu, W, rowptr, colidx, opts=opts)
+
+
+def test_chunk_count_does_not_change_result(bmu):
+    """Merging the per-chunk minima gives the single-pass BMU (Section 4.2)."""
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=2000)
+    W = synth.make_codebook(cfg.D, 4096, 21, kind="scaled")
+    Wd, rp, ci = dev(W, rowptr, colidx)
+    base = None
+    for chunk in (4096, 2048, 512, 128):
+        ob, od = bmu.bmu_search_ws(Wd, rp, ci, opts=make_opts(bmu, chunk_neurons=chunk))
+        if base is None:
+            base = (ob.clone(), od.clone())
+        assert torch.equal(ob, base[0]) and torch.equal(od, base[1])
+
+
+def test_deterministic_and_norms_reuse(bmu):
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=3000)
+    W = synth.make_codebook(cfg.D, cfg.M, 2)
+    Wd, rp, ci = dev(W, rowptr, colidx)
+    a = bmu.bmu_search_ws(Wd, rp, ci)
+    b = bmu.bmu_search(Wd, rp, ci)
+    n = bmu.bmu_codebook_norms(Wd)
+    c = bmu.bmu_search_ws(Wd, rp, ci, norms=n)
+    for x in (b, c):
+        assert torch.equal(a[0], x[0]) and torch.equal(a[1], x[1])
+
+
+def test_host_entry_point_matches_device_one(bmu):
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=2500)
+    W = synth.make_codebook(cfg.D, cfg.M, 2)
+    Wd, rp, ci = dev(W, rowptr, colidx)
+    a = bmu.bmu_search(Wd, rp, ci)
+    hb, hd = bmu.bmu_search_host(Wd, rowptr.pin_memory(), colidx.pin_memory())
+    assert torch.equal(a[0].cpu(), hb) and torch.equal(a[1].cpu(), hd)
+
+
+def test_validate_csr(bmu):
+    rp = torch.tensor([0, 2, 3], dtype=torch.int32).cuda()
+    ci = torch.tensor([0, 5, 2], dtype=torch.int32).cuda()
+    bmu.bmu_validate_csr(rp, ci, 6)
+    with pytest.raises(bmu.BmuError, match="outside"):
+        bmu.bmu_validate_csr(rp, ci, 5)
+    with pytest.raises(bmu.BmuError, match="decreases"):
+        bmu.bmu_validate_csr(torch.tensor([0, 3, 2, 3], dtype=torch.int32).cuda(), ci, 6)
+
+
+def test_workspace_errors(bmu):
+    W = torch.zeros(8, 8, device="cuda")
+    rp = torch.tensor([0, 1], dtype=torch.int32).cuda()
+    ci = torch.tensor([0], dtype=torch.int32).cuda()
+    with pytest.raises(bmu.BmuError) as e:
+        bmu.bmu_search_ws(W, rp, ci, workspace=torch.empty(300, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 3
