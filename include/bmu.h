@@ -152,6 +152,24 @@ BMU_API int bmu_release_scratch(void);
 BMU_API int bmu_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                      int64_t D, void *stream);
 
+/*
+ * Measures one on-chip ceiling of the current device with a microbenchmark, so
+ * that achieved throughput can be quoted against the roof that binds (the paper
+ * quotes its kernel against the L2 roof of its card, Section 6 / Table 3).
+ *   which 0  L2 -> SM read bandwidth, 128-bit loads bypassing L1      [bytes/s]
+ *         1  L2 -> shared memory by bulk asynchronous copies of `piece` bytes
+ *            (multiple of 16, <= 24576)                                [bytes/s]
+ *         2  shared memory -> registers, conflict-free 128-bit loads   [bytes/s]
+ *         3  L1-resident global loads -> registers, 128-bit            [bytes/s]
+ *         4  fp32 adds, scalar instructions                            [adds/s]
+ *         5  fp32 adds, packed two-wide instructions                   [adds/s]
+ * `buffer` is 256-byte aligned device memory the benchmark may overwrite; for
+ * 0 and 1 its size is the footprint that is swept (keep it well inside L2), for
+ * 3 it must hold 64 KiB per SM.  Synchronous; the result goes to *out_value.
+ */
+BMU_API int bmu_measure_roof(int which, void *buffer, size_t buffer_bytes, int piece,
+                             double *out_value, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -59,6 +59,9 @@ EXPORTS = {
     "bmu_release_scratch": (ctypes.c_int, []),
     "bmu_validate_csr": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                         ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
+    "bmu_measure_roof": (ctypes.c_int, [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t,
+                                        ctypes.c_int, ctypes.POINTER(ctypes.c_double),
+                                        ctypes.c_void_p]),
 }
 
 
@@ -197,3 +200,20 @@ def bmu_validate_csr(rowptr, colidx, D: int):
             _dev(rowptr, torch.int32, "rowptr"),
             _dev(colidx, torch.int32, "colidx") if colidx.numel() else None, N, colidx.numel(),
             D, _stream(rowptr)))
+
+
+ROOFS = {"l2_ldg": 0, "l2_bulk": 1, "smem": 2, "l1": 3, "fadd": 4, "fadd2": 5}
+
+
+def bmu_measure_roof(which: str, footprint_bytes: int = 32 << 20, piece: int = 2048,
+                     device=None) -> float:
+    """One on-chip ceiling of the device, measured now (bytes/s or adds/s)."""
+    device = torch.device("cuda" if device is None else device)
+    buf = torch.empty(footprint_bytes + 512, dtype=torch.uint8, device=device)
+    ptr = (buf.data_ptr() + 255) // 256 * 256
+    out = ctypes.c_double(0.0)
+    with torch.cuda.device(device):
+        _check(load().bmu_measure_roof(ROOFS[which], ptr, footprint_bytes, piece,
+                                       ctypes.byref(out),
+                                       torch.cuda.current_stream(device).cuda_stream))
+    return out.value
