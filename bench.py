@@ -1,0 +1,382 @@
+"""Benchmark of the BMU search hot path on B200.
+
+A step is one pass of the whole hot path -- codebook norms, the neuron-chunked
+gather-accumulate sweep with the fused argmin, outputs in document order --
+over one synthetic corpus batch.  Default workload: the 512x512 map
+(M=262144, D=16384, 17 GB fp32 codebook) against 2,000,000 documents.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg4] [--impl reference]
+
+With N > 1 (under torchrun) every rank holds a replica of the codebook and its
+own batch of documents (documents are independent: no collective on the data
+path, weak scaling); the time is the maximum over ranks.
+Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from inputs import synth  # noqa: E402
+
+METRIC = "bmu_search_docs_per_s"
+UNIT = "docs/s"
+
+
+# ----------------------------------------------------------------------------- helpers
+def dist_env():
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")),
+            int(os.environ.get("WORLD_SIZE", "1")))
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device):
+        self.uuid = None
+        try:
+            u = str(torch.cuda.get_device_properties(device).uuid)
+            self.uuid = u if u.startswith("GPU-") else "GPU-" + u
+        except Exception:
+            pass
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+
+    def start(self):
+        cmd = ["nvidia-smi", "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+               "-lms", "200"]
+        if self.uuid:
+            cmd += ["-i", self.uuid]
+        try:
+            self.proc = subprocess.Popen(cmd, stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx),
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def union_rows_per_block(rowptr, colidx, D, docs_per_block):
+    """Sum over blocks of consecutive documents of the number of distinct features the
+    block touches: the rows an SM has to fetch at least once per slab when `docs_per_block`
+    documents share its L1 (the design's own grouping)."""
+    N = rowptr.numel() - 1
+    lens = (rowptr[1:] - rowptr[:-1]).to(torch.int64)
+    doc = torch.repeat_interleave(torch.arange(N, device=rowptr.device), lens)
+    key = (doc // docs_per_block) * D + colidx.to(torch.int64)
+    del doc
+    key = torch.sort(key).values
+    return int((key[1:] != key[:-1]).sum().item()) + (1 if key.numel() else 0)
+
+
+# ----------------------------------------------------------------------------- reference arm
+def run_reference(args, cfg):
+    """The CPU oracle, as it stands, on the host cores: the reference arm and the
+    cpu_baseline leg.  A step = full norms + BMU search of a bounded sample of documents;
+    the value extrapolates that to the whole batch (documents are independent)."""
+    import numpy as np
+    import oracle
+
+    n_docs = args.docs or synth.batch_size(cfg)
+    gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
+    W = synth.make_codebook(cfg.D, cfg.M, synth.codebook_seed(cfg), device=gen_dev).cpu().numpy()
+    sample = min(n_docs, args.ref_sample)
+    rowptr, colidx = synth.make_corpus(cfg, device=gen_dev, n_docs=sample)
+    rowptr, colidx = rowptr.cpu().numpy(), colidx.cpu().numpy()
+    cores = oracle.max_threads()
+    times = []
+    for it in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        nrm = oracle.norms(W)
+        t1 = time.perf_counter()
+        oracle.bmu(W, rowptr, colidx, nrm)
+        t2 = time.perf_counter()
+        if it >= args.warmup:
+            times.append(((t1 - t0), (t2 - t1)))
+    t_norm = statistics.mean(t[0] for t in times)
+    t_bmu = statistics.mean(t[1] for t in times)
+    step_s = t_norm + t_bmu * (n_docs / sample)
+    value = n_docs / step_s
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": workload_config(cfg, n_docs, 1),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": "norms of the full codebook (%.2f s, one thread) + BMU of the "
+                                   "first %d documents (%.2f s, %d threads), extrapolated to %d "
+                                   "documents" % (t_norm, sample, t_bmu, cores, n_docs)},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    return line
+
+
+def cpu_baseline(cfg, W_dev, rowptr, colidx, n_docs, budget_s=15.0):
+    """Oracle timed on a bounded sample of this run's own arrays (rank 0, N=1)."""
+    import oracle
+    W = W_dev.cpu().numpy()
+    cores = oracle.max_threads()
+    t0 = time.perf_counter()
+    nrm = oracle.norms(W)
+    t_norm = time.perf_counter() - t0
+    rp = rowptr.cpu().numpy()
+
+    def run(k):
+        ci = colidx[: int(rp[k])].cpu().numpy()
+        t = time.perf_counter()
+        oracle.bmu(W, rp[: k + 1], ci, nrm)
+        return time.perf_counter() - t
+
+    probe = min(n_docs, 4 * cores)
+    t_probe = run(probe)
+    sample = int(max(probe, min(n_docs, probe * budget_s / max(t_probe, 1e-6))))
+    t_bmu = run(sample)
+    step_s = t_norm + t_bmu * (n_docs / sample)
+    return {"value": n_docs / step_s, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "norms of the full codebook (%.2f s, one thread) + BMU of the first %d "
+                      "documents (%.2f s, %d threads), extrapolated to %d documents"
+                      % (t_norm, sample, t_bmu, cores, n_docs)}
+
+
+def workload_config(cfg, n_docs, world):
+    return {
+        "workload": "%s: %dx%d map (M=%d), D=%d, fp32 feature-major codebook U[0,1), "
+                    "N=%d docs per GPU, nnz/doc %s, Zipf(s=%.1f) ids without replacement"
+                    % (cfg.name, cfg.edge, cfg.edge, cfg.M, cfg.D, n_docs,
+                       "Poisson(%g)>=1" % cfg.nnz_param if cfg.nnz_kind == "poisson"
+                       else "lognormal(median %g, sigma 0.5) in [1,400]" % cfg.nnz_param,
+                       cfg.zipf_s),
+        "docs_per_gpu": n_docs, "global_docs": n_docs * world,
+        "parallelism": "docs sharded over %d GPU(s), codebook replicated, no collective" % world,
+        "l2_policy": "inputs larger than L2 (codebook %.1f GB); no flush between steps"
+                     % (cfg.D * cfg.M * 4 / 1e9),
+    }
+
+
+# ----------------------------------------------------------------------------- our arm
+def run_ours(args, cfg, rank, local_rank, world):
+    import paper_2609_05138_b200 as bmu
+    bmu.load()                                    # fails loudly if the CUDA library is missing
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    n_docs = args.docs or synth.batch_size(cfg)
+    W = synth.make_codebook(cfg.D, cfg.M, synth.codebook_seed(cfg), device=dev)
+    rowptr, colidx = synth.make_corpus(cfg, batch=rank % synth.num_batches(cfg), device=dev,
+                                       n_docs=n_docs,
+                                       seed=synth.corpus_seed(cfg, rank))
+    N, nnz = rowptr.numel() - 1, colidx.numel()
+    opts = bmu.Opts()
+    for kv in args.opt:
+        k, v = kv.split("=")
+        setattr(opts, k, int(v))
+    ws = torch.empty(bmu.bmu_search_workspace_bytes(cfg.D, cfg.M, N, nnz, opts) + 256,
+                     dtype=torch.uint8, device=dev)
+    norms = torch.empty(cfg.M, dtype=torch.float32, device=dev)
+    out_bmu = torch.empty(N, dtype=torch.int32, device=dev)
+    out_dist = torch.empty(N, dtype=torch.float32, device=dev)
+
+    # launch geometry of the sweep (mirrors the library's defaults; reported, not used by it)
+    vec = opts.vec or 4
+    slab = 32 * vec
+    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
+    chunk = opts.chunk_neurons or max(slab, (l2_bytes // 2) // (cfg.D * 4) // slab * slab)
+    chunk = min((chunk + slab - 1) // slab * slab, (cfg.M + slab - 1) // slab * slab)
+    n_chunks = (cfg.M + chunk - 1) // chunk
+    docs_per_block = (opts.warps or 16) * (opts.docs_per_warp or 4)
+
+    def step(e0=None, e1=None, e2=None):
+        if e0 is not None:
+            e0.record()
+        bmu.bmu_codebook_norms(W, norms)
+        if e1 is not None:
+            e1.record()
+        bmu.bmu_search_ws(W, rowptr, colidx, norms=norms, opts=opts, workspace=ws,
+                          out_bmu=out_bmu, out_dist=out_dist)
+        if e2 is not None:
+            e2.record()
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(args.warmup):
+        step()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    barrier()
+    sampler = ClockSampler(dev)
+    sampler.start()
+    for k in range(args.steps):
+        step(*ev[k])
+    barrier()
+    clocks = sampler.stop()
+    total_ms = ev[0][0].elapsed_time(ev[-1][2])
+    sweep_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
+    norms_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
+    t = torch.tensor([total_ms, sweep_ms, norms_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, sweep_ms, norms_ms = t.tolist()
+    ms_per_step = total_ms / args.steps
+    value = n_docs * world / (ms_per_step * 1e-3)
+
+    # ---- end to end through the host entry point (pinned CSR in, results out)
+    rp_h, ci_h = rowptr.cpu().pin_memory(), colidx.cpu().pin_memory()
+    ob_h = torch.empty(N, dtype=torch.int32).pin_memory()
+    od_h = torch.empty(N, dtype=torch.float32).pin_memory()
+    bmu.bmu_search_host(W, rp_h, ci_h, ob_h, od_h)          # warm-up (grows the scratch)
+    e2e_steps = max(1, min(args.steps, 2))
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        bmu.bmu_search_host(W, rp_h, ci_h, ob_h, od_h)
+    torch.cuda.synchronize(dev)
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_s = te.item()
+    same = bool(torch.equal(ob_h, out_bmu.cpu()))
+
+    if rank != 0:
+        return None
+
+    # ---- roofline of the dominant kernel (the sweep): algorithmic units per launch / time
+    peaks, peaks_kind = measured_peaks()
+    roofs = {k: bmu.bmu_measure_roof(k, device=dev) for k in ("l2_ldg", "smem", "fadd2")}
+    launch_s = sweep_ms * 1e-3 / n_chunks
+    adds = float(nnz) * chunk                                   # one fp32 add per (nnz, neuron)
+    union_rows = union_rows_per_block(rowptr, colidx, cfg.D, docs_per_block)
+    alg = {
+        "alu": (adds / launch_s, roofs["fadd2"], "add/s"),
+        "l1": (4.0 * adds / launch_s, roofs["smem"], "B/s"),           # one 4-byte operand per add
+        "l2": (4.0 * union_rows * chunk / launch_s, roofs["l2_ldg"], "B/s"),
+        "hbm": ((4.0 * cfg.D * chunk + 4.0 * nnz + 24.0 * N) / launch_s,
+                peaks["hbm_gbs"] * 1e9, "B/s"),
+    }
+    bound = max(alg, key=lambda k: alg[k][0] / alg[k][1])
+    ach, peak, unit = alg[bound]
+    scale = 1e9
+    roofline = {
+        "kernel": "sweep_direct_kernel", "bound": bound,
+        "achieved": ach / scale, "peak": peak / scale,
+        "unit": "GB/s" if unit == "B/s" else "Gadd/s", "frac": ach / peak,
+        "traffic": None,
+        "launch_ms": launch_s * 1e3, "launches_per_step": n_chunks,
+        "units_per_launch": {"adds": adds, "union_rows_x_chunk": float(union_rows) * chunk},
+        "fractions": {k: v[0] / v[1] for k, v in alg.items()},
+        "peaks": {"hbm_GBs": peaks["hbm_gbs"], "hbm_source": "MEASURED_PEAKS.json (%s)" % peaks_kind,
+                  "l2_GBs": roofs["l2_ldg"] / 1e9, "l1_smem_GBs": roofs["smem"] / 1e9,
+                  "fp32_Gadds": roofs["fadd2"] / 1e9,
+                  "on_chip_source": "bmu_measure_roof, this run"},
+    }
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_config(cfg, n_docs, world),
+        "updates_per_s": float(nnz) * cfg.M * world / (ms_per_step * 1e-3),
+        "phases_ms": {"norms": norms_ms, "sweep_and_output": sweep_ms},
+        "clocks": clocks,
+        "e2e": {"value": n_docs * world / e2e_s, "unit": UNIT,
+                "h2d_bytes_per_step": int((N + 1 + nnz) * 4), "d2h_bytes_per_step": int(N * 8),
+                "api": "bmu_search_host (codebook resident in HBM; CSR batch from pinned host "
+                       "memory; results back to host)", "matches_device_path": same},
+        "gpu_launches": args.steps * (1 + n_chunks + 1),
+        "roofline": roofline,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(cfg, W, rowptr, colidx, n_docs)
+    return line
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="cfg4", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--docs", type=int, default=0, help="documents per GPU (0 = the config's batch)")
+    ap.add_argument("--opt", action="append", default=[], help="bmu_opts field=value")
+    ap.add_argument("--ref-sample", type=int, default=4000)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = synth.CONFIGS[args.config]
+    rank, local_rank, world = dist_env()
+    if args.warmup < 3 and args.impl == "ours" and rank == 0:
+        print("note: fewer than 3 warm-up steps", file=sys.stderr)
+
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args, cfg)))
+        return
+    line = run_ours(args, cfg, rank, local_rank, world)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    if line is not None:
+        print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    main()
