@@ -29,7 +29,9 @@ sweep_direct_kernel(const SweepArgs a)
     constexpr int STEP = VEC ? 4 : 1;             // floats per load
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t doc0 = ((int64_t)blockIdx.x * NW + warp) * K;
+#ifndef BMU_SLAB_SYNC
     if (doc0 >= a.N) return;
+#endif
 
     int beg[K], end[K];
 #pragma unroll
@@ -46,6 +48,9 @@ sweep_direct_kernel(const SweepArgs a)
     const uint32_t rowbytes = (uint32_t)(a.M * 4);
 
     for (int j0 = a.j_lo; j0 < a.j_hi; j0 += 32 * V) {
+#ifdef BMU_SLAB_SYNC
+        __syncthreads();
+#endif
         // this lane's columns of the slab
         int col[H];
         bool act[H];
