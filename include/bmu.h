@@ -67,18 +67,20 @@ typedef enum {
  * automatically.  Unknown combinations return BMU_ERR_INVALID_ARG.
  */
 typedef struct bmu_opts {
-    int32_t kernel;         /* 0 auto, 1 direct (rows read through L1/L2), 2 staged
-                               (rows staged through shared memory by bulk copies) */
+    int32_t kernel;         /* 0 auto, 1 direct (a warp per document, rows read through
+                               L1/L2), 2 staged (a lane per document, rows streamed through
+                               shared memory by tensor (TMA) box copies; needs M % 4 == 0,
+                               M >= 32, 256 <= D <= 65024) */
     int32_t chunk_neurons;  /* neurons per L2-resident chunk of the codebook (Section 4.2,
                                "neuron-axis chunking"); rounded to the slab width */
-    int32_t vec;            /* floats per lane per row segment: 4 or 8 */
-    int32_t docs_per_warp;  /* documents a warp carries through one slab pass */
-    int32_t warps;          /* warps per thread block */
-    int32_t cluster;        /* staged kernel: 0 keep corpus order, 1 order documents by
-                               their rarest features before tiling (Section 4.2, "tile
-                               membership") */
-    int32_t stage_rows;     /* staged kernel: codebook rows per pipeline stage */
-    int32_t stages;         /* staged kernel: pipeline depth */
+    int32_t vec;            /* direct kernel: floats per lane per row segment, 4 or 8 */
+    int32_t docs_per_warp;  /* direct kernel: documents a warp carries through one slab */
+    int32_t warps;          /* direct kernel: warps per thread block */
+    int32_t cluster;        /* staged kernel, tile membership (Section 4.2): 0/1 order the
+                               documents by length before cutting tiles, so that the lanes
+                               of a warp carry similar rows; 2 keep the corpus order */
+    int32_t stage_rows;     /* staged kernel: codebook rows per pipeline stage (256) */
+    int32_t stages;         /* staged kernel: pipeline depth, a power of two (4) */
     int32_t reserved[8];    /* must be 0 */
 } bmu_opts;
 
@@ -109,8 +111,10 @@ BMU_API size_t bmu_search_workspace_bytes(int64_t D, int64_t M, int64_t N, int64
  * Section 4) with caller-supplied scratch.  `norms` may be NULL (computed into
  * the workspace) or a device array from bmu_codebook_norms.  `workspace` must be
  * 256-byte aligned device memory of at least bmu_search_workspace_bytes(...)
- * bytes; its contents are undefined afterwards.  Allocates nothing.  Calls that
- * share a workspace must not overlap on the GPU.
+ * bytes; its contents are undefined afterwards, except that its first 32-bit
+ * word is a status word: 0 after a clean run, non-zero if a bounded device-side
+ * wait of the staged kernel ran out (results are then invalid).  Allocates
+ * nothing.  Calls that share a workspace must not overlap on the GPU.
  */
 BMU_API int bmu_search_ws(const float *W, int64_t D, int64_t M, const float *norms,
                   const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,

@@ -32,15 +32,28 @@ static const int64_t MAX_I32 = 0x7fffffff;
 
 // ---- workspace layout -----------------------------------------------------
 struct Layout {
-    size_t norms_off, state_off, total;
+    size_t status_off, norms_off, state_off, plan_off, total;
+    PlanLayout plan;
 };
 
-static Layout layout_for(int64_t M, int64_t N)
+// The staged kernel needs 16-bit feature ids, whole 16-byte row segments and
+// boxes that fit inside the codebook; everything else takes the direct kernel.
+static bool staged_possible(const float *W, int64_t D, int64_t M)
+{
+    return M % 4 == 0 && M >= 32 && D >= 256 && D <= LANES_MAX_D &&
+           (reinterpret_cast<uintptr_t>(W) & 15) == 0;
+}
+
+static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kernel)
 {
     Layout l;
     size_t off = 0;
+    l.status_off = off; off = 256;
     l.norms_off = off; off = align_up(off + (size_t)M * sizeof(float), 256);
     l.state_off = off; off = align_up(off + (size_t)N * sizeof(u64), 256);
+    l.plan_off = off;
+    memset(&l.plan, 0, sizeof(l.plan));
+    if (kernel != 1 && D <= LANES_MAX_D) off += plan_bytes(N, nnz, &l.plan);
     l.total = off;
     return l;
 }
@@ -64,6 +77,7 @@ static int check_opts(const bmu_opts &o)
     for (int i = 0; i < 8; ++i)
         if (o.reserved[i] != 0) { set_error("bmu_opts.reserved must be zero"); return BMU_ERR_INVALID_ARG; }
     if (o.kernel < 0 || o.kernel > 2) { set_error("bmu_opts.kernel must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
+    if (o.cluster < 0 || o.cluster > 2) { set_error("bmu_opts.cluster must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
     if (o.chunk_neurons < 0) { set_error("bmu_opts.chunk_neurons < 0"); return BMU_ERR_INVALID_ARG; }
     if (o.vec != 0 && o.vec != 4 && o.vec != 8) { set_error("bmu_opts.vec must be 0, 4 or 8"); return BMU_ERR_INVALID_ARG; }
     return BMU_OK;
@@ -105,7 +119,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         set_error("empty codebook (D=%lld, M=%lld): no neuron to return", (long long)D, (long long)M);
         return BMU_ERR_INVALID_ARG;
     }
-    const Layout l = layout_for(M, N);
+    const Layout l = layout_for(D, M, N, nnz, o.kernel);
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < l.total) {
         set_error("workspace missing, not 256-byte aligned, or smaller than %zu bytes", l.total);
         return BMU_ERR_WORKSPACE;
@@ -117,9 +131,36 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         if ((rc = launch_norms(W, D, M, n, s))) return rc;
         norms = n;
     }
-    if (o.kernel == 2) {
-        set_error("staged kernel not available in this build");
+    uint32_t *status = reinterpret_cast<uint32_t *>(base + l.status_off);
+    BMU_CUDA(cudaMemsetAsync(status, 0, 256, s));
+    // the staged kernel pays off once every SM has at least a couple of full tiles
+    const bool staged = staged_possible(W, D, M) &&
+                        (o.kernel == 2 || (o.kernel == 0 && N >= 992 * 148 * 2));
+    if (o.kernel == 2 && !staged) {
+        set_error("staged kernel needs M %% 4 == 0, M >= 32, 256 <= D <= %d and W 16-byte aligned",
+                  LANES_MAX_D);
         return BMU_ERR_UNSUPPORTED;
+    }
+    if (staged) {
+        char *pw = base + l.plan_off;
+        if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, pw, l.plan, s))) return rc;
+        alignas(64) unsigned char tmap[128];
+        if ((rc = make_codebook_tensor_map(W, D, M, o.stage_rows ? o.stage_rows : 256, tmap)))
+            return rc;
+        LanesArgs a;
+        a.norms = norms;
+        a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
+        a.doc_off = reinterpret_cast<const uint32_t *>(pw + l.plan.docoff_off);
+        a.ids = reinterpret_cast<const uint4 *>(pw + l.plan.ids_off);
+        a.N = N; a.M = M; a.D = (int32_t)D; a.state = state; a.status = status;
+        int64_t chunk = o.chunk_neurons ? (o.chunk_neurons + 31) / 32 * 32 : auto_chunk(D, M, 32);
+        for (int64_t j = 0; j < M; j += chunk) {
+            a.j_lo = (int32_t)j;
+            a.j_hi = (int32_t)(j + chunk < M ? j + chunk : M);
+            a.first = j == 0;
+            if ((rc = launch_sweep_lanes(tmap, a, o, s))) return rc;
+        }
+        return launch_finalize(state, rowptr, N, out_bmu, out_dist, s);
     }
     const int V = o.vec ? o.vec : 4;
     const int slab = 32 * V;
@@ -226,9 +267,8 @@ int bmu_codebook_norms(const float *W, int64_t D, int64_t M, float *norms, void 
 size_t bmu_search_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,
                                   const bmu_opts *opts)
 {
-    (void)D; (void)nnz; (void)opts;
-    if (M < 0 || N < 0) return 0;
-    return layout_for(M, N).total;
+    if (D < 0 || M < 0 || N < 0 || nnz < 0) return 0;
+    return layout_for(D, M, N, nnz, opts ? opts->kernel : 0).total;
 }
 
 int bmu_search_ws(const float *W, int64_t D, int64_t M, const float *norms,

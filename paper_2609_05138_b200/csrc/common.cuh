@@ -91,6 +91,33 @@ struct SweepArgs {
 int launch_sweep_direct(const SweepArgs &a, const bmu_opts &o, cudaStream_t s);
 int launch_finalize(const u64 *state, const int32_t *rowptr, int64_t N, int32_t *out_bmu,
                     float *out_dist, cudaStream_t s);
+// ---- tiling plan (plan.cu) and staged sweep (sweep_lanes.cu) ---------------
+struct PlanLayout {
+    size_t perm_off, docoff_off, ngroups_off, bins_off, ids_off, scan_off, scan_bytes, total;
+};
+size_t plan_bytes(int64_t N, int64_t nnz, PlanLayout *l);
+int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
+                int order_by_length, char *ws, const PlanLayout &l, cudaStream_t s);
+
+static const int LANES_MAX_D = 65024;    // 16-bit ids with 0xFFFF as the end marker
+
+struct LanesArgs {
+    const float *norms;
+    const int32_t *perm;       // planned position -> document
+    const uint32_t *doc_off;   // planned position -> first 8-id group of its list (minus one)
+    const uint4 *ids;          // 8 ascending 16-bit ids per uint4, 0xFFFF = end
+    int64_t N, M;
+    int32_t D;
+    u64 *state;
+    uint32_t *status;          // set non-zero if a bounded wait ran out
+    int32_t j_lo, j_hi, first;
+};
+// `tensor_map` is a host copy of the CUtensorMap describing W as a [D][M] fp32 tensor
+int make_codebook_tensor_map(const float *W, int64_t D, int64_t M, int rows_per_stage,
+                             void *tensor_map_out);
+int launch_sweep_lanes(const void *tensor_map, const LanesArgs &a, const bmu_opts &o,
+                       cudaStream_t s);
+
 int launch_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                         int64_t D, int32_t *flags, cudaStream_t s);
 
