@@ -67,15 +67,17 @@ typedef enum {
  * automatically.  Unknown combinations return BMU_ERR_INVALID_ARG.
  */
 typedef struct bmu_opts {
-    int32_t kernel;         /* 0 auto, 1 direct (a warp per document, rows read through
-                               L1/L2), 2 staged (a lane per document, rows streamed through
-                               shared memory by tensor (TMA) box copies; needs M % 4 == 0,
-                               M >= 32, 256 <= D <= 65024) */
+    int32_t kernel;         /* 0 auto; 1 generic (a warp per document, ids straight from the
+                               CSR, any D and M); 3 planned (a warp per document, ids from
+                               the tiling pass; needs M % 4 == 0, M >= 128, D <= 65024);
+                               2 staged (a lane per document, rows streamed through shared
+                               memory by tensor (TMA) box copies; needs M % 4 == 0, M >= 32,
+                               256 <= D <= 65024) */
     int32_t chunk_neurons;  /* neurons per L2-resident chunk of the codebook (Section 4.2,
                                "neuron-axis chunking"); rounded to the slab width */
-    int32_t vec;            /* direct kernel: floats per lane per row segment, 4 or 8 */
-    int32_t docs_per_warp;  /* direct kernel: documents a warp carries through one slab */
-    int32_t warps;          /* direct kernel: warps per thread block */
+    int32_t vec;            /* warp-per-document kernels: floats per lane per row, 4 or 8 */
+    int32_t docs_per_warp;  /* generic kernel: documents a warp carries through one slab */
+    int32_t warps;          /* warp-per-document kernels: warps per thread block */
     int32_t cluster;        /* staged kernel, tile membership (Section 4.2): 0/1 order the
                                documents by length before cutting tiles, so that the lanes
                                of a warp carry similar rows; 2 keep the corpus order */

@@ -76,7 +76,7 @@ static int check_opts(const bmu_opts &o)
 {
     for (int i = 0; i < 8; ++i)
         if (o.reserved[i] != 0) { set_error("bmu_opts.reserved must be zero"); return BMU_ERR_INVALID_ARG; }
-    if (o.kernel < 0 || o.kernel > 2) { set_error("bmu_opts.kernel must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
+    if (o.kernel < 0 || o.kernel > 3) { set_error("bmu_opts.kernel must be 0, 1, 2 or 3"); return BMU_ERR_INVALID_ARG; }
     if (o.cluster < 0 || o.cluster > 2) { set_error("bmu_opts.cluster must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
     if (o.chunk_neurons < 0) { set_error("bmu_opts.chunk_neurons < 0"); return BMU_ERR_INVALID_ARG; }
     if (o.vec != 0 && o.vec != 4 && o.vec != 8) { set_error("bmu_opts.vec must be 0, 4 or 8"); return BMU_ERR_INVALID_ARG; }
@@ -133,17 +133,52 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     }
     uint32_t *status = reinterpret_cast<uint32_t *>(base + l.status_off);
     BMU_CUDA(cudaMemsetAsync(status, 0, 256, s));
-    // the staged kernel pays off once every SM has at least a couple of full tiles
-    const bool staged = staged_possible(W, D, M) &&
-                        (o.kernel == 2 || (o.kernel == 0 && N >= 992 * 148 * 2));
-    if (o.kernel == 2 && !staged) {
+    const bool staged = o.kernel == 2;
+    if (staged && !staged_possible(W, D, M)) {
         set_error("staged kernel needs M %% 4 == 0, M >= 32, 256 <= D <= %d and W 16-byte aligned",
                   LANES_MAX_D);
         return BMU_ERR_UNSUPPORTED;
     }
-    if (staged) {
-        char *pw = base + l.plan_off;
+    // the planned warp-per-document kernel needs 16-bit ids and whole 16-byte row pieces
+    const bool planned_ok = D <= LANES_MAX_D && M % 4 == 0 && M >= 128 &&
+                            (reinterpret_cast<uintptr_t>(W) & 15) == 0;
+    if (o.kernel == 3 && !planned_ok) {
+        set_error("planned kernel needs M %% 4 == 0, M >= 128, D <= %d and W 16-byte aligned",
+                  LANES_MAX_D);
+        return BMU_ERR_UNSUPPORTED;
+    }
+    const bool planned = o.kernel == 3 || (o.kernel == 0 && planned_ok);
+    char *pw = base + l.plan_off;
+    if (staged || planned)
         if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, pw, l.plan, s))) return rc;
+    if (planned) {
+        const int slab = rows_slab_width(o);
+        RowsArgs a;
+        a.W = W; a.M = M; a.N = N; a.norms = norms; a.rowptr = rowptr;
+        a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
+        a.doc_off = reinterpret_cast<const uint32_t *>(pw + l.plan.docoff_off);
+        a.ids = reinterpret_cast<const uint4 *>(pw + l.plan.ids_off);
+        a.state = state;
+        const int64_t chunk = o.chunk_neurons ? (o.chunk_neurons + slab - 1) / slab * slab
+                                              : auto_chunk(D, M, slab);
+        const int64_t m_full = M / slab * slab;
+        for (int64_t j = 0; j < m_full; j += chunk) {
+            a.j_lo = (int32_t)j;
+            a.j_hi = (int32_t)(j + chunk < m_full ? j + chunk : m_full);
+            a.first = j == 0;
+            if ((rc = launch_sweep_rows(a, o, s))) return rc;
+        }
+        if (m_full < M) {                      // ragged last slab: generic kernel, merged in
+            SweepArgs g;
+            g.W = W; g.D = D; g.M = M; g.norms = norms; g.rowptr = rowptr; g.colidx = colidx;
+            g.N = N; g.state = state; g.j_lo = (int32_t)m_full; g.j_hi = (int32_t)M; g.first = 0;
+            bmu_opts go;
+            memset(&go, 0, sizeof(go));
+            if ((rc = launch_sweep_direct(g, go, s))) return rc;
+        }
+        return launch_finalize(state, rowptr, N, out_bmu, out_dist, s);
+    }
+    if (staged) {
         alignas(64) unsigned char tmap[128];
         if ((rc = make_codebook_tensor_map(W, D, M, o.stage_rows ? o.stage_rows : 256, tmap)))
             return rc;

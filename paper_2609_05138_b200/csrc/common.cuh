@@ -118,6 +118,21 @@ int make_codebook_tensor_map(const float *W, int64_t D, int64_t M, int rows_per_
 int launch_sweep_lanes(const void *tensor_map, const LanesArgs &a, const bmu_opts &o,
                        cudaStream_t s);
 
+// planned warp-per-document sweep (sweep_direct.cu): whole slabs of [j_lo, j_hi) only
+struct RowsArgs {
+    const float *W;
+    int64_t M, N;
+    const float *norms;
+    const int32_t *rowptr;
+    const int32_t *perm;
+    const uint32_t *doc_off;
+    const uint4 *ids;
+    u64 *state;
+    int32_t j_lo, j_hi, first;
+};
+int rows_slab_width(const bmu_opts &o);
+int launch_sweep_rows(const RowsArgs &a, const bmu_opts &o, cudaStream_t s);
+
 int launch_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                         int64_t D, int32_t *flags, cudaStream_t s);
 

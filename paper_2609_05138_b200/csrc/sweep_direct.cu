@@ -162,6 +162,123 @@ sweep_direct_kernel(const SweepArgs a)
     }
 }
 
+// ---------------------------------------------------------------------------
+// Planned variant of the same sweep: a warp per document, but the feature ids
+// come from the tiling pass (ascending 16-bit ids, eight per aligned 128-bit
+// word, see plan.cu).  All lanes read the same word, so one broadcast load
+// yields eight ids, no shuffle is needed, and the row address is one
+// multiply-add.  Only whole slabs are handled here (no per-lane guards in the
+// loop); a ragged last slab goes through the generic kernel above.
+template <int V, int NW>
+__global__ void __launch_bounds__(NW * 32)
+sweep_rows_kernel(const RowsArgs a)
+{
+    constexpr int H = V / 4;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t p = (int64_t)blockIdx.x * NW + warp;
+    if (p >= a.N) return;
+    const int32_t orig = __ldg(a.perm + p);
+    const int len = __ldg(a.rowptr + orig + 1) - __ldg(a.rowptr + orig);
+    const uint4 *gp = a.ids + (size_t)__ldg(a.doc_off + p) + 1;
+    const int full = len >> 3, rem = len & 7;
+    const uint32_t rowbytes = (uint32_t)(a.M * 4);
+    float best = CUDART_INF_F;
+    int bidx = 0x7fffffff;
+
+    for (int j0 = a.j_lo; j0 < a.j_hi; j0 += 32 * V) {
+        const char *base = reinterpret_cast<const char *>(a.W + j0 + lane * 4);
+        u64 acc[H][2];
+#pragma unroll
+        for (int h = 0; h < H; ++h) acc[h][0] = acc[h][1] = 0ull;
+
+        for (int g = 0; g < full; ++g) {
+            const uint4 t = __ldg(gp + g);
+            const uint32_t f[8] = {t.x & 0xffffu, t.x >> 16, t.y & 0xffffu, t.y >> 16,
+                                   t.z & 0xffffu, t.z >> 16, t.w & 0xffffu, t.w >> 16};
+            ulonglong2 w[8][H];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+#pragma unroll
+                for (int h = 0; h < H; ++h)
+                    w[u][h] = __ldg(reinterpret_cast<const ulonglong2 *>(
+                        base + (u64)f[u] * rowbytes + h * 512));
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+#pragma unroll
+                for (int h = 0; h < H; ++h) {
+                    add2(acc[h][0], w[u][h].x);
+                    add2(acc[h][1], w[u][h].y);
+                }
+        }
+        if (rem) {
+            const uint4 t = __ldg(gp + full);
+            const uint32_t f[8] = {t.x & 0xffffu, t.x >> 16, t.y & 0xffffu, t.y >> 16,
+                                   t.z & 0xffffu, t.z >> 16, t.w & 0xffffu, t.w >> 16};
+#pragma unroll
+            for (int u = 0; u < 7; ++u)
+                if (u < rem) {
+#pragma unroll
+                    for (int h = 0; h < H; ++h) {
+                        const ulonglong2 w = __ldg(reinterpret_cast<const ulonglong2 *>(
+                            base + (u64)f[u] * rowbytes + h * 512));
+                        add2(acc[h][0], w.x);
+                        add2(acc[h][1], w.y);
+                    }
+                }
+        }
+#pragma unroll
+        for (int h = 0; h < H; ++h) {
+            const int col = j0 + h * 128 + lane * 4;
+            const float4 n = __ldg(reinterpret_cast<const float4 *>(a.norms + col));
+            const float s4[4] = {lo_f(acc[h][0]), hi_f(acc[h][0]), lo_f(acc[h][1]), hi_f(acc[h][1])};
+            const float n4[4] = {n.x, n.y, n.z, n.w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const float d = fmaf(-2.f, s4[c], n4[c]);
+                if (d < best) { best = d; bidx = col + c; }
+            }
+        }
+    }
+    warp_argmin(best, bidx);
+    if (lane == 0) {
+        u64 key = make_key(best, bidx);
+        if (!a.first) {
+            const u64 old = a.state[orig];
+            if (old < key) key = old;
+        }
+        a.state[orig] = key;
+    }
+}
+
+template <int V>
+static int launch_rows_v(const RowsArgs &a, int NW, cudaStream_t s)
+{
+#define BMU_CASE(nw)                                                                   \
+    if (NW == nw) {                                                                    \
+        sweep_rows_kernel<V, nw><<<(unsigned)((a.N + nw - 1) / nw), nw * 32, 0, s>>>(a); \
+        BMU_CUDA(cudaGetLastError());                                                  \
+        return BMU_OK;                                                                 \
+    }
+    BMU_CASE(4) BMU_CASE(8) BMU_CASE(16) BMU_CASE(32)
+#undef BMU_CASE
+    set_error("planned kernel: warps must be 4, 8, 16 or 32");
+    return BMU_ERR_INVALID_ARG;
+}
+
+int rows_slab_width(const bmu_opts &o) { return 32 * (o.vec ? o.vec : 4); }
+
+int launch_sweep_rows(const RowsArgs &a, const bmu_opts &o, cudaStream_t s)
+{
+    if (a.N == 0 || a.j_lo >= a.j_hi) return BMU_OK;
+    const int NW = o.warps ? o.warps : 8;
+    const int V = o.vec ? o.vec : 4;
+    if ((a.j_hi - a.j_lo) % (32 * V) != 0) {
+        set_error("planned kernel handles whole slabs only");
+        return BMU_ERR_INVALID_ARG;
+    }
+    return V == 8 ? launch_rows_v<8>(a, NW, s) : launch_rows_v<4>(a, NW, s);
+}
+
 // state -> outputs: out_dist = |x_i| + min_j (n_j - 2 s_ij)
 __global__ void finalize_kernel(const u64 *__restrict__ state, const int32_t *__restrict__ rowptr,
                                 int64_t N, int32_t *__restrict__ out_bmu,

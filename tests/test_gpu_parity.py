@@ -289,3 +289,32 @@ def test_staged_refuses_what_it_cannot_do(bmu):
     with pytest.raises(bmu.BmuError) as e:
         bmu.bmu_search_ws(W, rp, ci, opts=make_opts(bmu, kernel=2))
     assert e.value.status == 2
+
+
+# ------------------------------------------------------------------ planned warp-per-document kernel
+@pytest.mark.parametrize("vec", [4, 8])
+@pytest.mark.parametrize("warps", [4, 8, 32])
+def test_planned_kernel_matches_generic_bitwise(bmu, vec, warps):
+    cfg = synth.CONFIGS["cfg2"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=1500)
+    W = synth.make_codebook(cfg.D, 2048 + 36, 15, kind="scaled")   # ragged last slab
+    Wd, rp, ci = dev(W, rowptr, colidx)
+    a = bmu.bmu_search_ws(Wd, rp, ci, opts=make_opts(bmu, kernel=3, vec=vec, warps=warps,
+                                                     chunk_neurons=512))
+    g = bmu.bmu_search_ws(Wd, rp, ci, opts=make_opts(bmu, kernel=1))
+    assert torch.equal(a[0], g[0]) and torch.equal(a[1], g[1])
+    parity.compare(a[0].cpu().numpy(), a[1].cpu().numpy(), W.numpy(), rowptr.numpy(),
+                   colidx.numpy())
+
+
+def test_planned_kernel_long_empty_unsorted_rows(bmu):
+    D, M = 16384, 384
+    nnz = torch.tensor([400, 0, 1, 33, 0, 400, 97, 64, 32, 31, 0, 8, 16, 7, 9, 1500] * 9)
+    rowptr, colidx = synth.draw_corpus(nnz.numel(), D, 1.1, nnz, seed=6)
+    ci = colidx.numpy().copy()
+    rp = rowptr.numpy()
+    r = np.random.default_rng(2)
+    for i in range(0, nnz.numel(), 2):
+        r.shuffle(ci[rp[i]:rp[i + 1]])
+    W = synth.make_codebook(D, M, 10, kind="scaled")
+    run_and_check(bmu, W, rowptr, torch.from_numpy(ci), opts=make_opts(bmu, kernel=3))
