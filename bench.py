@@ -231,13 +231,23 @@ def run_ours(args, cfg, rank, local_rank, world):
     out_dist = torch.empty(N, dtype=torch.float32, device=dev)
 
     # launch geometry of the sweep (mirrors the library's defaults; reported, not used by it)
-    vec = opts.vec or 4
+    vec = opts.vec or (4 if opts.kernel == 1 else 8)
     slab = 32 * vec
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
     chunk = opts.chunk_neurons or max(slab, (l2_bytes // 2) // (cfg.D * 4) // slab * slab)
     chunk = min((chunk + slab - 1) // slab * slab, (cfg.M + slab - 1) // slab * slab)
     n_chunks = (cfg.M + chunk - 1) // chunk
-    docs_per_block = (opts.warps or 16) * (opts.docs_per_warp or 4)
+    # documents that share one SM's L1 at a time: resident warps x documents per warp
+    kernel_name = {0: "sweep_rows_kernel", 3: "sweep_rows_kernel", 1: "sweep_direct_kernel",
+                   2: "sweep_lanes_kernel"}[opts.kernel]
+    if opts.kernel == 2:
+        docs_per_block, chunk = 992, (opts.chunk_neurons or
+                                      max(32, (l2_bytes // 2) // (cfg.D * 4) // 32 * 32))
+        n_chunks = (cfg.M + chunk - 1) // chunk
+    elif opts.kernel == 1:
+        docs_per_block = (opts.warps or 16) * (opts.docs_per_warp or 4) * 2
+    else:
+        docs_per_block = 48
 
     def step(e0=None, e1=None, e2=None):
         if e0 is not None:
@@ -317,7 +327,7 @@ def run_ours(args, cfg, rank, local_rank, world):
     ach, peak, unit = alg[bound]
     scale = 1e9
     roofline = {
-        "kernel": "sweep_direct_kernel", "bound": bound,
+        "kernel": kernel_name, "bound": bound,
         "achieved": ach / scale, "peak": peak / scale,
         "unit": "GB/s" if unit == "B/s" else "Gadd/s", "frac": ach / peak,
         "traffic": None,
@@ -341,7 +351,7 @@ def run_ours(args, cfg, rank, local_rank, world):
                 "h2d_bytes_per_step": int((N + 1 + nnz) * 4), "d2h_bytes_per_step": int(N * 8),
                 "api": "bmu_search_host (codebook resident in HBM; CSR batch from pinned host "
                        "memory; results back to host)", "matches_device_path": same},
-        "gpu_launches": args.steps * (1 + n_chunks + 1),
+        "gpu_launches": args.steps * (1 + (0 if opts.kernel == 1 else 6) + n_chunks + 1),
         "roofline": roofline,
     }
     if world == 1 and not args.no_cpu_baseline:

@@ -69,7 +69,7 @@ typedef enum {
 typedef struct bmu_opts {
     int32_t kernel;         /* 0 auto; 1 generic (a warp per document, ids straight from the
                                CSR, any D and M); 3 planned (a warp per document, ids from
-                               the tiling pass; needs M % 4 == 0, M >= 128, D <= 65024);
+                               the tiling pass; needs M % 4 == 0, M >= 32 * vec, D <= 65024);
                                2 staged (a lane per document, rows streamed through shared
                                memory by tensor (TMA) box copies; needs M % 4 == 0, M >= 32,
                                256 <= D <= 65024) */

@@ -140,7 +140,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         return BMU_ERR_UNSUPPORTED;
     }
     // the planned warp-per-document kernel needs 16-bit ids and whole 16-byte row pieces
-    const bool planned_ok = D <= LANES_MAX_D && M % 4 == 0 && M >= 128 &&
+    const bool planned_ok = D <= LANES_MAX_D && M % 4 == 0 && M >= rows_slab_width(o) &&
                             (reinterpret_cast<uintptr_t>(W) & 15) == 0;
     if (o.kernel == 3 && !planned_ok) {
         set_error("planned kernel needs M %% 4 == 0, M >= 128, D <= %d and W 16-byte aligned",
@@ -199,6 +199,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     }
     const int V = o.vec ? o.vec : 4;
     const int slab = 32 * V;
+    if (o.warps == 4) { set_error("generic kernel: warps must be 8, 16 or 32"); return BMU_ERR_INVALID_ARG; }
     int64_t chunk = o.chunk_neurons ? (o.chunk_neurons + slab - 1) / slab * slab
                                     : auto_chunk(D, M, slab);
     SweepArgs a;

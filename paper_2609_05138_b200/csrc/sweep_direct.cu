@@ -265,13 +265,14 @@ static int launch_rows_v(const RowsArgs &a, int NW, cudaStream_t s)
     return BMU_ERR_INVALID_ARG;
 }
 
-int rows_slab_width(const bmu_opts &o) { return 32 * (o.vec ? o.vec : 4); }
+// defaults measured on B200: two 128-bit loads per lane and row, 16 warps per block
+int rows_slab_width(const bmu_opts &o) { return 32 * (o.vec ? o.vec : 8); }
 
 int launch_sweep_rows(const RowsArgs &a, const bmu_opts &o, cudaStream_t s)
 {
     if (a.N == 0 || a.j_lo >= a.j_hi) return BMU_OK;
-    const int NW = o.warps ? o.warps : 8;
-    const int V = o.vec ? o.vec : 4;
+    const int NW = o.warps ? o.warps : 16;
+    const int V = o.vec ? o.vec : 8;
     if ((a.j_hi - a.j_lo) % (32 * V) != 0) {
         set_error("planned kernel handles whole slabs only");
         return BMU_ERR_INVALID_ARG;

@@ -1,0 +1,106 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The oracle cannot sweep 2,000,000 documents against 262,144 neurons in test
+time, so the full-size run is checked (a) on a seeded sample of documents the
+oracle computes one by one, (b) by properties that hold for every document,
+and (c), on the 64x64 configuration, against an independent full-N
+computation by a library sparse-dense product (test-only code).
+"""
+import numpy as np
+import pytest
+import torch
+
+from inputs import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def bmu():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_05138_b200 as lib
+    lib.load()
+    return lib
+
+
+def check_sample(W_dev, rowptr, colidx, ob, od, n_sample, seed):
+    g = torch.Generator().manual_seed(seed)
+    N = rowptr.numel() - 1
+    docs = torch.sort(torch.randperm(N, generator=g)[:n_sample]).values.numpy()
+    res = parity.compare(ob.cpu().numpy(), od.cpu().numpy(), W_dev.cpu().numpy(),
+                         rowptr.cpu().numpy(), colidx.cpu().numpy(), docs=docs)
+    assert res["docs"] == n_sample and res["failed"] == 0
+    return res
+
+
+def check_properties(W_dev, norms, rowptr, colidx, ob, od, M):
+    N = rowptr.numel() - 1
+    assert int(ob.min()) >= 0 and int(ob.max()) < M
+    assert bool(torch.isfinite(od).all())
+    # the returned distance is the distance of the returned neuron (recomputed for every
+    # document with plain torch gathers, fp64)
+    lens = (rowptr[1:] - rowptr[:-1]).to(torch.int64)
+    doc = torch.repeat_interleave(torch.arange(N, device=rowptr.device), lens)
+    w = W_dev[colidx.to(torch.int64), ob.to(torch.int64)[doc]].double()
+    s = torch.zeros(N, dtype=torch.float64, device=rowptr.device).index_add_(0, doc, w)
+    d = lens.double() + norms.double()[ob.to(torch.int64)] - 2.0 * s
+    assert bool(((od.double() - d).abs() <= 1e-5 * d.abs()).all())
+
+
+def test_cfg4_full_size_sampled(bmu):
+    cfg = synth.CONFIGS["cfg4"]
+    dev = torch.device("cuda")
+    W = synth.make_codebook(cfg.D, cfg.M, synth.codebook_seed(cfg), device=dev)
+    rowptr, colidx = synth.make_corpus(cfg, device=dev)
+    assert rowptr.numel() - 1 == cfg.N
+    norms = bmu.bmu_codebook_norms(W)
+    ob, od = bmu.bmu_search_ws(W, rowptr, colidx, norms=norms)     # bench.py's call and options
+    torch.cuda.synchronize()
+    check_properties(W, norms, rowptr, colidx, ob, od, cfg.M)
+    check_sample(W, rowptr, colidx, ob, od, 256, seed=4)
+
+
+def test_cfg5_one_streamed_batch_sampled(bmu):
+    cfg = synth.CONFIGS["cfg5"]
+    dev = torch.device("cuda")
+    W = synth.make_codebook(cfg.D, cfg.M, synth.codebook_seed(cfg), device=dev)
+    norms = bmu.bmu_codebook_norms(W)
+    for batch in (0, 26):                                            # a full and the short batch
+        rowptr, colidx = synth.make_corpus(cfg, batch=batch, device=dev)
+        assert rowptr.numel() - 1 == (1_000_000 if batch == 0 else 900_000)
+        ob, od = bmu.bmu_search_ws(W, rowptr, colidx, norms=norms)
+        torch.cuda.synchronize()
+        check_properties(W, norms, rowptr, colidx, ob, od, cfg.M)
+        check_sample(W, rowptr, colidx, ob, od, 1500, seed=5 + batch)
+
+
+def test_cfg2_full_size_against_library_product(bmu):
+    cfg = synth.CONFIGS["cfg2"]
+    dev = torch.device("cuda")
+    W = synth.make_codebook(cfg.D, cfg.M, synth.codebook_seed(cfg), device=dev)
+    rowptr, colidx = synth.make_corpus(cfg, device=dev)
+    N = cfg.N
+    ob, od = bmu.bmu_search(W, rowptr, colidx)
+    torch.cuda.synchronize()
+    check_sample(W, rowptr, colidx, ob, od, 3000, seed=2)
+    norms = (W.double() ** 2).sum(0)
+    bad_d = bad_j = 0
+    step = 50_000
+    for lo in range(0, N, step):
+        hi = min(N, lo + step)
+        rp = (rowptr[lo:hi + 1] - rowptr[lo]).to(torch.int64)
+        ci = colidx[int(rowptr[lo]):int(rowptr[hi])].to(torch.int64)
+        X = torch.sparse_csr_tensor(rp, ci, torch.ones(ci.numel(), device=dev),
+                                    size=(hi - lo, cfg.D))
+        S = (X @ W).double()                                         # library sparse-dense product
+        d = (rp[1:] - rp[:-1]).double()[:, None] + norms[None, :] - 2.0 * S
+        dmin, jmin = d.min(dim=1)
+        got_d = od[lo:hi].double()
+        got_j = ob[lo:hi].to(torch.int64)
+        tol = 1e-5 * dmin.abs()
+        bad_d += int(((got_d - dmin).abs() > tol).sum())
+        d_at = d.gather(1, got_j[:, None])[:, 0]
+        bad_j += int(((got_j != jmin) & (d_at > dmin + tol)).sum())
+    assert bad_d == 0 and bad_j == 0
