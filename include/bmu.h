@@ -159,6 +159,37 @@ BMU_API int bmu_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64
                      int64_t D, void *stream);
 
 /*
+ * Search for callers that must not allocate.  (The paper has no counterpart:
+ * this entry point exists for integration, not for the method.)  Some hosts of
+ * this library cannot call cudaMalloc at the point where they need a search --
+ * code running inside a memory pool that owns the whole device, a real-time
+ * loop that forbids allocation after start-up, a plug-in that is only handed
+ * its inputs and outputs.  bmu_search_ws already allocates nothing but wants a
+ * workspace from the caller; this form needs none: its scratch (the codebook
+ * norms and the per-document running minimum that is merged across neuron
+ * chunks) lives in a fixed 8 MiB array that is part of the library image, so
+ * every GPU that loads the library carries those 8 MiB until the process ends.
+ * It runs the generic warp-per-document kernel (bmu_opts.kernel == 1) and gives
+ * the same results as bmu_search_ws with that option.
+ *   Limit: 256 + roundup256(4*M) + roundup256(8*N) <= 8 MiB, else
+ *   BMU_ERR_UNSUPPORTED with the sizes in bmu_last_error().  For example
+ *   M = 262144 leaves room for about 917,000 documents per call; split larger
+ *   batches.
+ *   First call on a device: looks up the device address of the array (once per
+ *   device, with that device current) -- make that first call outside any
+ *   stream capture.  No call ever invokes cudaMalloc, cudaFree or an allocating
+ *   library routine.
+ *   The array is shared by every call on the device and keeps what the last
+ *   call left in it; the entry point re-initialises what it reads, so stale
+ *   contents are harmless, but two calls that overlap on the GPU (different
+ *   streams, or another thread) race on it and corrupt each other's results.
+ * `nnz` is the length of colidx.  Asynchronous on `stream` like bmu_search_ws.
+ */
+BMU_API int bmu_search_static(const float *W, int64_t D, int64_t M, const int32_t *rowptr,
+                              const int32_t *colidx, int64_t N, int64_t nnz, int32_t *out_bmu,
+                              float *out_dist, void *stream);
+
+/*
  * Measures one on-chip ceiling of the current device with a microbenchmark, so
  * that achieved throughput can be quoted against the roof that binds (the paper
  * quotes its kernel against the L2 roof of its card, Section 6 / Table 3).

@@ -56,6 +56,10 @@ EXPORTS = {
     "bmu_search_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "bmu_search_static": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                                         ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
+                                         ctypes.c_void_p]),
     "bmu_release_scratch": (ctypes.c_int, []),
     "bmu_validate_csr": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                         ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
@@ -167,6 +171,21 @@ def bmu_search(W, rowptr, colidx, out_bmu=None, out_dist=None):
         _check(load().bmu_search(
             wp, D, M, _dev(rowptr, torch.int32, "rowptr"),
             _dev(colidx, torch.int32, "colidx") if colidx.numel() else None, N,
+            _dev(out_bmu, torch.int32, "out_bmu"), _dev(out_dist, torch.float32, "out_dist"),
+            _stream(W)))
+    return out_bmu, out_dist
+
+
+def bmu_search_static(W, rowptr, colidx, out_bmu, out_dist):
+    """Search for callers that cannot allocate: the scratch is an 8 MiB array inside
+    the library, so the sizes are limited (see include/bmu.h) and overlapping calls on
+    one device race.  The caller passes the outputs; nothing is allocated here either."""
+    wp, D, M = _codebook(W)
+    N = rowptr.numel() - 1
+    with torch.cuda.device(W.device):
+        _check(load().bmu_search_static(
+            wp, D, M, _dev(rowptr, torch.int32, "rowptr"),
+            _dev(colidx, torch.int32, "colidx") if colidx.numel() else None, N, colidx.numel(),
             _dev(out_bmu, torch.int32, "out_bmu"), _dev(out_dist, torch.float32, "out_dist"),
             _stream(W)))
     return out_bmu, out_dist

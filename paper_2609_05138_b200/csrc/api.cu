@@ -412,3 +412,48 @@ int bmu_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, in
 }
 
 }  // extern "C"
+
+// ---- search with library-resident scratch (no allocation anywhere) ---------
+// The scratch of the generic kernel's search -- norms and the running
+// per-document minimum -- in an array that is part of the library image.  The
+// name below is only a host-side handle: device code may use it directly, but
+// host code must ask the runtime for its device address before handing it to a
+// kernel, once per device and with that device current.
+static const size_t STATIC_SCRATCH_BYTES = (size_t)8 << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+static void *g_static_scratch_addr[64];
+static std::mutex g_static_mu;
+
+extern "C" int bmu_search_static(const float *W, int64_t D, int64_t M, const int32_t *rowptr,
+                                 const int32_t *colidx, int64_t N, int64_t nnz, int32_t *out_bmu,
+                                 float *out_dist, void *stream)
+{
+    int rc = bmu::check_sizes(D, M, N, nnz);
+    if (rc) return rc;
+    if (N == 0) return BMU_OK;
+    const size_t need = bmu::layout_for(D, M, N, nnz, 1).total;
+    if (need > STATIC_SCRATCH_BYTES) {
+        bmu::set_error("bmu_search_static: M=%lld and N=%lld need %zu bytes of scratch, the "
+                       "built-in array holds %zu; split the batch or use bmu_search_ws",
+                       (long long)M, (long long)N, need, STATIC_SCRATCH_BYTES);
+        return BMU_ERR_UNSUPPORTED;
+    }
+    int dev = 0;
+    BMU_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) { bmu::set_error("device ordinal %d out of range", dev); return BMU_ERR_UNSUPPORTED; }
+    void *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> g(g_static_mu);
+        if (!g_static_scratch_addr[dev]) {
+            void *p = nullptr;
+            BMU_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+            g_static_scratch_addr[dev] = p;
+        }
+        scratch = g_static_scratch_addr[dev];
+    }
+    bmu_opts o;
+    memset(&o, 0, sizeof(o));
+    o.kernel = 1;
+    return bmu::search_impl(W, D, M, nullptr, rowptr, colidx, N, nnz, out_bmu, out_dist, &o,
+                            scratch, STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(stream));
+}
