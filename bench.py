@@ -286,7 +286,7 @@ def run_ours(args, cfg, rank, local_rank, world):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     total_ms, sweep_ms, norms_ms = t.tolist()
     ms_per_step = total_ms / args.steps
-    value = n_docs * world / (ms_per_step * 1e-3)
+    value = n_docs * world / (ms_per_step * 1e-3)     # all ranks' documents / slowest rank
 
     # ---- end to end through the host entry point (pinned CSR in, results out)
     rp_h, ci_h = rowptr.cpu().pin_memory(), colidx.cpu().pin_memory()
