@@ -330,7 +330,10 @@ def run_ours(args, cfg, rank, local_rank, world):
         "kernel": kernel_name, "bound": bound,
         "achieved": ach / scale, "peak": peak / scale,
         "unit": "GB/s" if unit == "B/s" else "Gadd/s", "frac": ach / peak,
-        "traffic": None,
+        # DRAM bytes per launch from the ncu capture of this very launch configuration
+        # (profiles/sweep_rows_cfg4_launch_list.md); other workloads were not captured
+        "traffic": (2.0e9 if (cfg.name == "cfg4" and n_docs == cfg.N and opts.kernel in (0, 3)
+                              and not opts.chunk_neurons and not opts.vec) else None),
         "launch_ms": launch_s * 1e3, "launches_per_step": n_chunks,
         "units_per_launch": {"adds": adds, "union_rows_x_chunk": float(union_rows) * chunk},
         "fractions": {k: v[0] / v[1] for k, v in alg.items()},
