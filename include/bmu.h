@@ -124,6 +124,22 @@ BMU_API int bmu_search_ws(const float *W, int64_t D, int64_t M, const float *nor
                   void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same search that also returns the second-best unit, which the paper's
+ * kernel tracks because topographic error -- gated on by its stopping rules --
+ * needs it (Table 5, "bmu1-only").  out_bmu2[i] is the lowest index j !=
+ * out_bmu[i] attaining the second-smallest distance, out_dist2[i] that distance
+ * (-1 and +inf when M == 1).  Same tie rule, same options (the staged kernel
+ * does not support it), workspace of bmu_search_top2_workspace_bytes(...).
+ */
+BMU_API size_t bmu_search_top2_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,
+                                               const bmu_opts *opts);
+BMU_API int bmu_search_top2_ws(const float *W, int64_t D, int64_t M, const float *norms,
+                               const int32_t *rowptr, const int32_t *colidx, int64_t N,
+                               int64_t nnz, int32_t *out_bmu, float *out_dist,
+                               int32_t *out_bmu2, float *out_dist2, const bmu_opts *opts,
+                               void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * One-shot form.  Same as bmu_search_ws with norms == NULL and default options,
  * but the scratch is a library-owned buffer per device that only ever grows
  * (cudaMalloc on first use or growth; freed by bmu_release_scratch or at

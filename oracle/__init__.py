@@ -42,6 +42,8 @@ def _load():
         lib.oracle_eval.restype = ctypes.c_double
         lib.oracle_bmu.argtypes = [vp, i64, i64, vp, vp, vp, i64, vp, vp, vp, ci]
         lib.oracle_bmu.restype = ci
+        lib.oracle_bmu2.argtypes = [vp, i64, i64, vp, vp, vp, i64, vp, vp, vp, vp, ci]
+        lib.oracle_bmu2.restype = ci
         lib.oracle_max_threads.argtypes = []
         lib.oracle_max_threads.restype = ci
         _lib = lib
@@ -88,6 +90,24 @@ def bmu(W, rowptr, colidx, norms_=None, threads: int = 0):
     if rc != 0:
         raise MemoryError("oracle_bmu could not allocate its accumulators")
     return out_b, d1, d2
+
+
+def bmu2(W, rowptr, colidx, norms_=None, threads: int = 0):
+    """(bmu, d1, bmu2, d2): best and second-best unit of every document."""
+    W = _f32(W)
+    rowptr, colidx = _i32(rowptr), _i32(colidx)
+    D, M = W.shape
+    N = rowptr.shape[0] - 1
+    n = norms(W) if norms_ is None else np.ascontiguousarray(norms_, dtype=np.float64)
+    b1 = np.empty(N, dtype=np.int32)
+    b2 = np.empty(N, dtype=np.int32)
+    d1 = np.empty(N, dtype=np.float64)
+    d2 = np.empty(N, dtype=np.float64)
+    rc = _load().oracle_bmu2(_p(W), D, M, _p(n), _p(rowptr), _p(colidx), N,
+                             _p(b1), _p(d1), _p(d2), _p(b2), int(threads))
+    if rc != 0:
+        raise MemoryError("oracle_bmu2 could not allocate its accumulators")
+    return b1, d1, b2, d2
 
 
 def eval_pair(W, rowptr, colidx, norms_, i: int, j: int) -> float:

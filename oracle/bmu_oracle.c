@@ -64,12 +64,26 @@ double oracle_eval(const float *W, int64_t D, int64_t M, const double *norms,
  *   bmu[i]  lowest index attaining the minimum distance
  *   d1[i]   the minimum distance
  *   d2[i]   the second-smallest distance (over j != bmu[i]; +inf when M == 1)
- * d2 exists only so that a comparison can tell a near-tie from a wrong answer.
+ *   bmu2[i] (optional, may be NULL) the lowest index j != bmu[i] attaining d2[i],
+ *           -1 when M == 1: the second-best unit the paper's kernel tracks for
+ *           topographic error (Table 5, "bmu1-only")
+ * d2 also lets a comparison tell a near-tie from a wrong answer.
  * Returns 0, or -1 if scratch memory could not be allocated.
  */
+int oracle_bmu2(const float *W, int64_t D, int64_t M, const double *norms,
+                const int32_t *rowptr, const int32_t *colidx, int64_t N,
+                int32_t *bmu, double *d1, double *d2, int32_t *bmu2, int nthreads);
+
 int oracle_bmu(const float *W, int64_t D, int64_t M, const double *norms,
                const int32_t *rowptr, const int32_t *colidx, int64_t N,
                int32_t *bmu, double *d1, double *d2, int nthreads)
+{
+    return oracle_bmu2(W, D, M, norms, rowptr, colidx, N, bmu, d1, d2, (int32_t *)0, nthreads);
+}
+
+int oracle_bmu2(const float *W, int64_t D, int64_t M, const double *norms,
+                const int32_t *rowptr, const int32_t *colidx, int64_t N,
+                int32_t *bmu, double *d1, double *d2, int32_t *bmu2, int nthreads)
 {
     (void)D;
     int failed = 0;
@@ -99,20 +113,24 @@ int oracle_bmu(const float *W, int64_t D, int64_t M, const double *norms,
             }
             double nx = (double)(rowptr[i + 1] - rowptr[i]);
             double best = INFINITY, second = INFINITY;
-            int32_t arg = -1;
+            int32_t arg = -1, arg2 = -1;
             for (int64_t j = 0; j < M; ++j) {
                 double d = nx + norms[j] - 2.0 * acc[j];
                 if (arg < 0 || d < best) {
                     second = (arg < 0) ? INFINITY : best;
+                    arg2 = arg;
                     best = d;
                     arg = (int32_t)j;
-                } else if (d < second) {
+                } else if (arg2 < 0 || d < second) {
                     second = d;
+                    arg2 = (int32_t)j;
                 }
             }
             bmu[i] = arg;
             d1[i] = best;
             d2[i] = second;
+            if (bmu2)
+                bmu2[i] = arg2;
         }
         free(acc);
     }

@@ -50,6 +50,15 @@ EXPORTS = {
                                      ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
                                      ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                      ctypes.c_size_t, ctypes.c_void_p]),
+    "bmu_search_top2_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int64, ctypes.c_int64,
+                                                          ctypes.c_int64, ctypes.c_int64,
+                                                          ctypes.c_void_p]),
+    "bmu_search_top2_ws": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                          ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
+                                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
+                                          ctypes.c_void_p]),
     "bmu_search": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
@@ -157,6 +166,29 @@ def bmu_search_ws(W, rowptr, colidx, norms=None, opts: Opts | None = None, works
             _dev(out_bmu, torch.int32, "out_bmu"), _dev(out_dist, torch.float32, "out_dist"),
             ctypes.byref(opts) if opts else None, ws_ptr, ws_bytes, _stream(W)))
     return out_bmu, out_dist
+
+
+def bmu_search_top2_ws(W, rowptr, colidx, norms=None, opts: Opts | None = None):
+    """Best and second-best unit.  Returns (out_bmu, out_dist, out_bmu2, out_dist2)."""
+    wp, D, M = _codebook(W)
+    N = rowptr.numel() - 1
+    nnz = colidx.numel()
+    ob = torch.empty(N, dtype=torch.int32, device=W.device)
+    od = torch.empty(N, dtype=torch.float32, device=W.device)
+    ob2 = torch.empty(N, dtype=torch.int32, device=W.device)
+    od2 = torch.empty(N, dtype=torch.float32, device=W.device)
+    need = int(load().bmu_search_top2_workspace_bytes(D, M, N, nnz,
+                                                      ctypes.byref(opts) if opts else None))
+    ws = torch.empty(need + 256, dtype=torch.uint8, device=W.device)
+    ws_ptr = (ws.data_ptr() + 255) // 256 * 256
+    with torch.cuda.device(W.device):
+        _check(load().bmu_search_top2_ws(
+            wp, D, M, _dev(norms, torch.float32, "norms") if norms is not None else None,
+            _dev(rowptr, torch.int32, "rowptr"),
+            _dev(colidx, torch.int32, "colidx") if nnz else None, N, nnz,
+            ob.data_ptr(), od.data_ptr(), ob2.data_ptr(), od2.data_ptr(),
+            ctypes.byref(opts) if opts else None, ws_ptr, need, _stream(W)))
+    return ob, od, ob2, od2
 
 
 def bmu_search(W, rowptr, colidx, out_bmu=None, out_dist=None):

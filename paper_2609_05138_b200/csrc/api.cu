@@ -32,7 +32,7 @@ static const int64_t MAX_I32 = 0x7fffffff;
 
 // ---- workspace layout -----------------------------------------------------
 struct Layout {
-    size_t status_off, norms_off, state_off, plan_off, total;
+    size_t status_off, norms_off, state_off, state2_off, plan_off, total;
     PlanLayout plan;
 };
 
@@ -44,13 +44,16 @@ static bool staged_possible(const float *W, int64_t D, int64_t M)
            (reinterpret_cast<uintptr_t>(W) & 15) == 0;
 }
 
-static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kernel)
+static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kernel,
+                         bool top2 = false)
 {
     Layout l;
     size_t off = 0;
     l.status_off = off; off = 256;
     l.norms_off = off; off = align_up(off + (size_t)M * sizeof(float), 256);
     l.state_off = off; off = align_up(off + (size_t)N * sizeof(u64), 256);
+    l.state2_off = off;
+    if (top2) off = align_up(off + (size_t)N * sizeof(u64), 256);
     l.plan_off = off;
     memset(&l.plan, 0, sizeof(l.plan));
     if (kernel != 1 && D <= LANES_MAX_D) off += plan_bytes(N, nnz, &l.plan);
@@ -102,8 +105,10 @@ static int64_t auto_chunk(int64_t D, int64_t M, int slab)
 static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
                        const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                        int32_t *out_bmu, float *out_dist, const bmu_opts *opts_in, void *ws,
-                       size_t ws_bytes, cudaStream_t s)
+                       size_t ws_bytes, cudaStream_t s, int32_t *out_bmu2 = nullptr,
+                       float *out_dist2 = nullptr)
 {
+    const bool top2 = out_bmu2 != nullptr || out_dist2 != nullptr;
     int rc = check_sizes(D, M, N, nnz);
     if (rc) return rc;
     bmu_opts o;
@@ -111,7 +116,8 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     if (opts_in) o = *opts_in;
     if ((rc = check_opts(o))) return rc;
     if (N == 0) return BMU_OK;
-    if (!W || !rowptr || !out_bmu || !out_dist || (nnz > 0 && !colidx)) {
+    if (!W || !rowptr || !out_bmu || !out_dist || (nnz > 0 && !colidx) ||
+        (top2 && (!out_bmu2 || !out_dist2))) {
         set_error("null pointer argument");
         return BMU_ERR_INVALID_ARG;
     }
@@ -119,13 +125,14 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         set_error("empty codebook (D=%lld, M=%lld): no neuron to return", (long long)D, (long long)M);
         return BMU_ERR_INVALID_ARG;
     }
-    const Layout l = layout_for(D, M, N, nnz, o.kernel);
+    const Layout l = layout_for(D, M, N, nnz, o.kernel, top2);
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < l.total) {
         set_error("workspace missing, not 256-byte aligned, or smaller than %zu bytes", l.total);
         return BMU_ERR_WORKSPACE;
     }
     char *base = static_cast<char *>(ws);
     u64 *state = reinterpret_cast<u64 *>(base + l.state_off);
+    u64 *state2 = top2 ? reinterpret_cast<u64 *>(base + l.state2_off) : nullptr;
     if (!norms) {
         float *n = reinterpret_cast<float *>(base + l.norms_off);
         if ((rc = launch_norms(W, D, M, n, s))) return rc;
@@ -134,6 +141,10 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     uint32_t *status = reinterpret_cast<uint32_t *>(base + l.status_off);
     BMU_CUDA(cudaMemsetAsync(status, 0, 256, s));
     const bool staged = o.kernel == 2;
+    if (staged && top2) {
+        set_error("the staged kernel does not track the second-best unit");
+        return BMU_ERR_UNSUPPORTED;
+    }
     if (staged && !staged_possible(W, D, M)) {
         set_error("staged kernel needs M %% 4 == 0, M >= 32, 256 <= D <= %d and W 16-byte aligned",
                   LANES_MAX_D);
@@ -158,7 +169,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
         a.doc_off = reinterpret_cast<const uint32_t *>(pw + l.plan.docoff_off);
         a.ids = reinterpret_cast<const uint4 *>(pw + l.plan.ids_off);
-        a.state = state;
+        a.state = state; a.state2 = state2;
         const int64_t chunk = o.chunk_neurons ? (o.chunk_neurons + slab - 1) / slab * slab
                                               : auto_chunk(D, M, slab);
         const int64_t m_full = M / slab * slab;
@@ -171,12 +182,12 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         if (m_full < M) {                      // ragged last slab: generic kernel, merged in
             SweepArgs g;
             g.W = W; g.D = D; g.M = M; g.norms = norms; g.rowptr = rowptr; g.colidx = colidx;
-            g.N = N; g.state = state; g.j_lo = (int32_t)m_full; g.j_hi = (int32_t)M; g.first = 0;
+            g.N = N; g.state = state; g.state2 = state2; g.j_lo = (int32_t)m_full; g.j_hi = (int32_t)M; g.first = 0;
             bmu_opts go;
             memset(&go, 0, sizeof(go));
             if ((rc = launch_sweep_direct(g, go, s))) return rc;
         }
-        return launch_finalize(state, rowptr, N, out_bmu, out_dist, s);
+        return launch_finalize(state, state2, rowptr, N, out_bmu, out_dist, out_bmu2, out_dist2, s);
     }
     if (staged) {
         alignas(64) unsigned char tmap[128];
@@ -195,7 +206,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
             a.first = j == 0;
             if ((rc = launch_sweep_lanes(tmap, a, o, s))) return rc;
         }
-        return launch_finalize(state, rowptr, N, out_bmu, out_dist, s);
+        return launch_finalize(state, nullptr, rowptr, N, out_bmu, out_dist, nullptr, nullptr, s);
     }
     const int V = o.vec ? o.vec : 4;
     const int slab = 32 * V;
@@ -204,14 +215,14 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
                                     : auto_chunk(D, M, slab);
     SweepArgs a;
     a.W = W; a.D = D; a.M = M; a.norms = norms; a.rowptr = rowptr; a.colidx = colidx;
-    a.N = N; a.state = state;
+    a.N = N; a.state = state; a.state2 = state2;
     for (int64_t j = 0; j < M; j += chunk) {
         a.j_lo = (int32_t)j;
         a.j_hi = (int32_t)(j + chunk < M ? j + chunk : M);
         a.first = j == 0;
         if ((rc = launch_sweep_direct(a, o, s))) return rc;
     }
-    return launch_finalize(state, rowptr, N, out_bmu, out_dist, s);
+    return launch_finalize(state, state2, rowptr, N, out_bmu, out_dist, out_bmu2, out_dist2, s);
 }
 
 // ---- library-owned grow-only scratch (one per device) ----------------------
@@ -314,6 +325,27 @@ int bmu_search_ws(const float *W, int64_t D, int64_t M, const float *norms,
 {
     return search_impl(W, D, M, norms, rowptr, colidx, N, nnz, out_bmu, out_dist, opts,
                        workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+size_t bmu_search_top2_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,
+                                       const bmu_opts *opts)
+{
+    if (D < 0 || M < 0 || N < 0 || nnz < 0) return 0;
+    return layout_for(D, M, N, nnz, opts ? opts->kernel : 0, true).total;
+}
+
+int bmu_search_top2_ws(const float *W, int64_t D, int64_t M, const float *norms,
+                       const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
+                       int32_t *out_bmu, float *out_dist, int32_t *out_bmu2, float *out_dist2,
+                       const bmu_opts *opts, void *workspace, size_t workspace_bytes,
+                       void *stream)
+{
+    if (N > 0 && (!out_bmu2 || !out_dist2)) {
+        set_error("null pointer argument");
+        return BMU_ERR_INVALID_ARG;
+    }
+    return search_impl(W, D, M, norms, rowptr, colidx, N, nnz, out_bmu, out_dist, opts, workspace,
+                       workspace_bytes, static_cast<cudaStream_t>(stream), out_bmu2, out_dist2);
 }
 
 int bmu_search(const float *W, int64_t D, int64_t M, const int32_t *rowptr,

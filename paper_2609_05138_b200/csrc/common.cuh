@@ -65,6 +65,74 @@ __device__ __forceinline__ void warp_argmin(float &d, int &j)
     }
 }
 
+// Running minimum of one lane / warp / document: the best unit, and with TOP2 also
+// the second-best unit (Table 5: the paper's kernel tracks it for topographic
+// error).  push() must see a lane's neurons in ascending index order; ties then
+// keep the lower index.  Across lanes and chunks the 64-bit keys decide.
+template <bool TOP2>
+struct Best {
+    float d1, d2;
+    int j1, j2;
+    __device__ __forceinline__ void init()
+    {
+        d1 = d2 = __int_as_float(0x7f800000);
+        j1 = j2 = 0x7fffffff;
+    }
+    __device__ __forceinline__ void push(float d, int j)
+    {
+        if (d < d1) {
+            if (TOP2) { d2 = d1; j2 = j1; }
+            d1 = d; j1 = j;
+        } else if (TOP2 && d < d2) {
+            d2 = d; j2 = j;
+        }
+    }
+    // any order of j (staged kernel): full lexicographic test
+    __device__ __forceinline__ void push_any(float d, int j)
+    {
+        if (d < d1 || (d == d1 && j < j1)) {
+            if (TOP2) { d2 = d1; j2 = j1; }
+            d1 = d; j1 = j;
+        } else if (TOP2 && (d < d2 || (d == d2 && j < j2))) {
+            d2 = d; j2 = j;
+        }
+    }
+    static __device__ __forceinline__ void merge(u64 &a1, u64 &a2, u64 b1, u64 b2)
+    {
+        const u64 lo = a1 < b1 ? a1 : b1, mid = a1 < b1 ? b1 : a1;
+        const u64 rest = a2 < b2 ? a2 : b2;
+        a1 = lo;
+        a2 = mid < rest ? mid : rest;
+    }
+    // warp-wide result into (k1, k2) on every lane
+    __device__ __forceinline__ void warp_keys(u64 &k1, u64 &k2) const
+    {
+        k1 = make_key(d1, j1);
+        k2 = TOP2 ? make_key(d2, j2) : KEY_WORST;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const u64 o1 = __shfl_xor_sync(0xffffffffu, k1, off);
+            if (TOP2) {
+                const u64 o2 = __shfl_xor_sync(0xffffffffu, k2, off);
+                merge(k1, k2, o1, o2);
+            } else {
+                k1 = o1 < k1 ? o1 : k1;
+            }
+        }
+    }
+    // merge the warp's result into the per-document state (one owner per document)
+    static __device__ __forceinline__ void commit(u64 k1, u64 k2, u64 *state, u64 *state2,
+                                                  int64_t doc, bool first)
+    {
+        if (!first) {
+            if (TOP2) merge(k1, k2, state[doc], state2[doc]);
+            else { const u64 old = state[doc]; k1 = old < k1 ? old : k1; }
+        }
+        state[doc] = k1;
+        if (TOP2) state2[doc] = k2;
+    }
+};
+
 // packed fp32 pair add: two IEEE round-to-nearest adds in one issue slot (sm_100a)
 __device__ __forceinline__ void add2(u64 &acc, u64 w)
 {
@@ -85,12 +153,14 @@ struct SweepArgs {
     const int32_t *colidx;
     int64_t N;
     u64 *state;           // per-document running (distance, index) key
+    u64 *state2;          // same for the second-best unit (NULL unless it is wanted)
     int32_t j_lo, j_hi;   // neuron chunk [j_lo, j_hi)
     int32_t first;        // 1: this chunk initialises the state, 0: merges into it
 };
 int launch_sweep_direct(const SweepArgs &a, const bmu_opts &o, cudaStream_t s);
-int launch_finalize(const u64 *state, const int32_t *rowptr, int64_t N, int32_t *out_bmu,
-                    float *out_dist, cudaStream_t s);
+int launch_finalize(const u64 *state, const u64 *state2, const int32_t *rowptr, int64_t N,
+                    int32_t *out_bmu, float *out_dist, int32_t *out_bmu2, float *out_dist2,
+                    cudaStream_t s);
 // ---- tiling plan (plan.cu) and staged sweep (sweep_lanes.cu) ---------------
 struct PlanLayout {
     size_t perm_off, docoff_off, ngroups_off, bins_off, ids_off, scan_off, scan_bytes, total;
@@ -128,6 +198,7 @@ struct RowsArgs {
     const uint32_t *doc_off;
     const uint4 *ids;
     u64 *state;
+    u64 *state2;          // NULL unless the second-best unit is wanted
     int32_t j_lo, j_hi, first;
 };
 int rows_slab_width(const bmu_opts &o);

@@ -20,7 +20,7 @@
 
 namespace bmu {
 
-template <int V, int K, int NW, bool VEC>
+template <int V, int K, int NW, bool VEC, bool TOP2>
 __global__ void __launch_bounds__(NW * 32)
 sweep_direct_kernel(const SweepArgs a)
 {
@@ -40,10 +40,9 @@ sweep_direct_kernel(const SweepArgs a)
         beg[k] = i < a.N ? __ldg(a.rowptr + i) : 0;
         end[k] = i < a.N ? __ldg(a.rowptr + i + 1) : 0;
     }
-    float best[K];
-    int bidx[K];
+    Best<TOP2> best[K];
 #pragma unroll
-    for (int k = 0; k < K; ++k) { best[k] = CUDART_INF_F; bidx[k] = 0x7fffffff; }
+    for (int k = 0; k < K; ++k) best[k].init();
 
     const uint32_t rowbytes = (uint32_t)(a.M * 4);
 
@@ -139,8 +138,7 @@ sweep_direct_kernel(const SweepArgs a)
             for (int h = 0; h < H; ++h)
 #pragma unroll
                 for (int c = 0; c < STEP; ++c) {
-                    const float d = fmaf(-2.f, s[h][c], nrm[h][c]);
-                    if (d < best[k]) { best[k] = d; bidx[k] = col[h] + c; }
+                    best[k].push(fmaf(-2.f, s[h][c], nrm[h][c]), col[h] + c);
                 }
         }
     }
@@ -148,17 +146,9 @@ sweep_direct_kernel(const SweepArgs a)
 #pragma unroll
     for (int k = 0; k < K; ++k) {
         if (doc0 + k >= a.N) continue;
-        float d = best[k];
-        int j = bidx[k];
-        warp_argmin(d, j);
-        if (lane == 0) {
-            u64 key = make_key(d, j);
-            if (!a.first) {
-                const u64 old = a.state[doc0 + k];
-                if (old < key) key = old;
-            }
-            a.state[doc0 + k] = key;
-        }
+        u64 k1, k2;
+        best[k].warp_keys(k1, k2);
+        if (lane == 0) Best<TOP2>::commit(k1, k2, a.state, a.state2, doc0 + k, a.first);
     }
 }
 
@@ -169,7 +159,7 @@ sweep_direct_kernel(const SweepArgs a)
 // yields eight ids, no shuffle is needed, and the row address is one
 // multiply-add.  Only whole slabs are handled here (no per-lane guards in the
 // loop); a ragged last slab goes through the generic kernel above.
-template <int V, int NW>
+template <int V, int NW, bool TOP2>
 __global__ void __launch_bounds__(NW * 32)
 sweep_rows_kernel(const RowsArgs a)
 {
@@ -182,8 +172,8 @@ sweep_rows_kernel(const RowsArgs a)
     const uint4 *gp = a.ids + (size_t)__ldg(a.doc_off + p) + 1;
     const int full = len >> 3, rem = len & 7;
     const uint32_t rowbytes = (uint32_t)(a.M * 4);
-    float best = CUDART_INF_F;
-    int bidx = 0x7fffffff;
+    Best<TOP2> best;
+    best.init();
 
     for (int j0 = a.j_lo; j0 < a.j_hi; j0 += 32 * V) {
         const char *base = reinterpret_cast<const char *>(a.W + j0 + lane * 4);
@@ -233,21 +223,12 @@ sweep_rows_kernel(const RowsArgs a)
             const float s4[4] = {lo_f(acc[h][0]), hi_f(acc[h][0]), lo_f(acc[h][1]), hi_f(acc[h][1])};
             const float n4[4] = {n.x, n.y, n.z, n.w};
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const float d = fmaf(-2.f, s4[c], n4[c]);
-                if (d < best) { best = d; bidx = col + c; }
-            }
+            for (int c = 0; c < 4; ++c) best.push(fmaf(-2.f, s4[c], n4[c]), col + c);
         }
     }
-    warp_argmin(best, bidx);
-    if (lane == 0) {
-        u64 key = make_key(best, bidx);
-        if (!a.first) {
-            const u64 old = a.state[orig];
-            if (old < key) key = old;
-        }
-        a.state[orig] = key;
-    }
+    u64 k1, k2;
+    best.warp_keys(k1, k2);
+    if (lane == 0) Best<TOP2>::commit(k1, k2, a.state, a.state2, orig, a.first);
 }
 
 template <int V>
@@ -255,7 +236,9 @@ static int launch_rows_v(const RowsArgs &a, int NW, cudaStream_t s)
 {
 #define BMU_CASE(nw)                                                                   \
     if (NW == nw) {                                                                    \
-        sweep_rows_kernel<V, nw><<<(unsigned)((a.N + nw - 1) / nw), nw * 32, 0, s>>>(a); \
+        const unsigned blocks = (unsigned)((a.N + nw - 1) / nw);                       \
+        if (a.state2) sweep_rows_kernel<V, nw, true><<<blocks, nw * 32, 0, s>>>(a);    \
+        else sweep_rows_kernel<V, nw, false><<<blocks, nw * 32, 0, s>>>(a);            \
         BMU_CUDA(cudaGetLastError());                                                  \
         return BMU_OK;                                                                 \
     }
@@ -281,9 +264,11 @@ int launch_sweep_rows(const RowsArgs &a, const bmu_opts &o, cudaStream_t s)
 }
 
 // state -> outputs: out_dist = |x_i| + min_j (n_j - 2 s_ij)
-__global__ void finalize_kernel(const u64 *__restrict__ state, const int32_t *__restrict__ rowptr,
-                                int64_t N, int32_t *__restrict__ out_bmu,
-                                float *__restrict__ out_dist)
+// (a second-best unit that does not exist, M == 1, comes out as index -1 at distance +inf)
+__global__ void finalize_kernel(const u64 *__restrict__ state, const u64 *__restrict__ state2,
+                                const int32_t *__restrict__ rowptr, int64_t N,
+                                int32_t *__restrict__ out_bmu, float *__restrict__ out_dist,
+                                int32_t *__restrict__ out_bmu2, float *__restrict__ out_dist2)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
@@ -291,14 +276,21 @@ __global__ void finalize_kernel(const u64 *__restrict__ state, const int32_t *__
     const float nx = (float)(rowptr[i + 1] - rowptr[i]);
     out_bmu[i] = (int32_t)(uint32_t)key;
     out_dist[i] = nx + ordered_to_float((uint32_t)(key >> 32));
+    if (state2) {
+        const u64 k2 = state2[i];
+        const bool none = (uint32_t)k2 == 0x7fffffffu;
+        out_bmu2[i] = none ? -1 : (int32_t)(uint32_t)k2;
+        out_dist2[i] = none ? CUDART_INF_F : nx + ordered_to_float((uint32_t)(k2 >> 32));
+    }
 }
 
-int launch_finalize(const u64 *state, const int32_t *rowptr, int64_t N, int32_t *out_bmu,
-                    float *out_dist, cudaStream_t s)
+int launch_finalize(const u64 *state, const u64 *state2, const int32_t *rowptr, int64_t N,
+                    int32_t *out_bmu, float *out_dist, int32_t *out_bmu2, float *out_dist2,
+                    cudaStream_t s)
 {
     if (N == 0) return BMU_OK;
-    finalize_kernel<<<(unsigned)((N + 255) / 256), 256, 0, s>>>(state, rowptr, N, out_bmu,
-                                                                out_dist);
+    finalize_kernel<<<(unsigned)((N + 255) / 256), 256, 0, s>>>(state, state2, rowptr, N, out_bmu,
+                                                                out_dist, out_bmu2, out_dist2);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
@@ -308,7 +300,10 @@ static int launch_one(const SweepArgs &a, cudaStream_t s)
 {
     const int64_t per_block = (int64_t)NW * K;
     const int64_t blocks = (a.N + per_block - 1) / per_block;
-    sweep_direct_kernel<V, K, NW, VEC><<<(unsigned)blocks, NW * 32, 0, s>>>(a);
+    if (a.state2)
+        sweep_direct_kernel<V, K, NW, VEC, true><<<(unsigned)blocks, NW * 32, 0, s>>>(a);
+    else
+        sweep_direct_kernel<V, K, NW, VEC, false><<<(unsigned)blocks, NW * 32, 0, s>>>(a);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

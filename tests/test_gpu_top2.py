@@ -1,0 +1,80 @@
+"""Second-best unit (the paper's kernel tracks it for topographic error, Table 5):
+best and runner-up from the CUDA path against the oracle's."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from inputs import synth
+
+pytestmark = pytest.mark.gpu
+REL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def bmu():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_05138_b200 as lib
+    lib.load()
+    return lib
+
+
+def check(bmu, W, rowptr, colidx, **kw):
+    o = bmu.Opts()
+    for k, v in kw.items():
+        setattr(o, k, v)
+    b1, d1, b2, d2 = bmu.bmu_search_top2_ws(W.cuda(), rowptr.cuda(), colidx.cuda(), opts=o)
+    torch.cuda.synchronize()
+    b1, d1, b2, d2 = (t.cpu().numpy() for t in (b1, d1, b2, d2))
+    Wn, rp, ci = W.numpy(), rowptr.numpy(), colidx.numpy()
+    nrm = oracle.norms(Wn)
+    e1, f1, e2, f2 = oracle.bmu2(Wn, rp, ci, nrm)
+    M = Wn.shape[1]
+    # best unit: same answer as the plain search
+    pb, pd = bmu.bmu_search_ws(W.cuda(), rowptr.cuda(), colidx.cuda(), opts=o)
+    assert np.array_equal(pb.cpu().numpy(), b1) and np.array_equal(pd.cpu().numpy(), d1)
+    if M == 1:
+        assert np.all(b2 == -1) and np.all(np.isinf(d2))
+        return
+    assert np.all(b2 != b1) and np.all((b2 >= 0) & (b2 < M))
+    margin = REL * np.abs(f1)
+    assert np.all(np.abs(d1 - f1) <= margin) and np.all(np.abs(d2 - f2) <= REL * np.abs(f2))
+    # indices: equal, or the oracle's distances at the returned units sit inside the margin
+    for i in np.nonzero((b1 != e1) | (b2 != e2))[0]:
+        g1 = oracle.eval_pair(Wn, rp, ci, nrm, int(i), int(b1[i]))
+        g2 = oracle.eval_pair(Wn, rp, ci, nrm, int(i), int(b2[i]))
+        assert g1 <= f1[i] + margin[i] and g2 <= f2[i] + REL * abs(f2[i]), (i, b1[i], b2[i])
+    return b1, b2
+
+
+@pytest.mark.parametrize("kernel", [1, 3])
+@pytest.mark.parametrize("kind", ["uniform", "scaled", "signed"])
+def test_top2_against_oracle(bmu, kernel, kind):
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=1700)
+    W = synth.make_codebook(cfg.D, 1024 + 72, 40, kind=kind)     # ragged last slab
+    check(bmu, W, rowptr, colidx, kernel=kernel, chunk_neurons=256)
+
+
+@pytest.mark.parametrize("kernel", [1, 3])
+def test_top2_ties_take_lower_indices(bmu, kernel):
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=600)
+    W = synth.make_codebook(cfg.D, 512, 41, kind="dupes")
+    b1, b2 = check(bmu, W, rowptr, colidx, kernel=kernel, chunk_neurons=256)
+    assert np.array_equal(b2, b1 + 1)                            # the copy is the runner-up
+    Z = synth.make_codebook(cfg.D, 512, 1, kind="const")
+    b1, b2 = check(bmu, Z, rowptr, colidx, kernel=kernel)
+    assert np.all(b1 == 0) and np.all(b2 == 1)
+
+
+def test_top2_small_maps(bmu):
+    r = np.random.default_rng(3)
+    for M in (1, 2, 5):
+        rows = [np.sort(r.choice(50, size=int(r.integers(0, 9)), replace=False)) for _ in range(40)]
+        rp = np.zeros(41, dtype=np.int32)
+        rp[1:] = np.cumsum([len(x) for x in rows])
+        ci = np.concatenate(rows).astype(np.int32)
+        W = synth.make_codebook(50, M, 7 + M, kind="scaled")
+        check(bmu, W, torch.from_numpy(rp), torch.from_numpy(ci))

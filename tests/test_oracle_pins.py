@@ -311,3 +311,34 @@ def test_unsorted_rows_give_same_result(small_problem):
     b2, e1, _ = oracle.bmu(W, rowptr, shuffled)
     np.testing.assert_array_equal(b2, bmu)
     np.testing.assert_allclose(e1, d1, rtol=1e-12)
+
+
+# ---------------------------------------------------------------- second-best unit
+@pytest.mark.parametrize("seed,N,D,M", [(0, 80, 23, 11), (1, 50, 40, 2), (2, 30, 9, 1)])
+def test_second_best_unit_matches_brute_force(seed, N, D, M):
+    r = rng(seed)
+    rowptr, colidx = random_csr(r, N, D, D)
+    W = synth.make_codebook(D, M, 200 + seed, kind="signed").numpy()
+    d = brute_force(densify(rowptr, colidx, D), W)
+    b1, d1, b2, d2 = oracle.bmu2(W, rowptr, colidx)
+    order = np.argsort(d, axis=1, kind="stable")          # ties -> lower index first
+    np.testing.assert_array_equal(b1, order[:, 0])
+    if M == 1:
+        assert np.all(b2 == -1) and np.all(np.isinf(d2))
+        return
+    e2 = d[np.arange(N), order[:, 1]]
+    np.testing.assert_allclose(d2, e2, rtol=1e-12, atol=1e-12)
+    clear = np.ones(N, bool) if M == 2 else (d[np.arange(N), order[:, 2]] - e2) > 1e-9
+    np.testing.assert_array_equal(b2[clear], order[:, 1][clear])
+    assert np.all(b2 != b1)
+
+
+def test_second_best_unit_ties_take_the_lower_index():
+    W = synth.make_codebook(40, 16, 3, kind="dupes").numpy()   # neuron 2k+1 copies neuron 2k
+    rowptr, colidx = random_csr(rng(17), 100, 40, 10)
+    b1, d1, b2, d2 = oracle.bmu2(W, rowptr, colidx)
+    np.testing.assert_array_equal(b2, b1 + 1)                    # the copy is the runner-up
+    np.testing.assert_array_equal(d1, d2)
+    Z = np.zeros((5, 4), dtype=np.float32)                       # every neuron ties
+    b1, d1, b2, d2 = oracle.bmu2(Z, np.array([0, 2], np.int32), np.array([1, 3], np.int32))
+    assert (b1[0], b2[0], d1[0], d2[0]) == (0, 1, 2.0, 2.0)
