@@ -140,6 +140,23 @@ BMU_API int bmu_search_top2_ws(const float *W, int64_t D, int64_t M, const float
                                void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Half-precision codebook, the paper's own storage (Section 4.2: "two bytes per
+ * half-precision weight"; Section 4.3: __half2 loads).  W16 is IEEE fp16
+ * [D][M], feature-major, 16-byte aligned; sums and distances are still fp32
+ * (norms: fp64 accumulate).  Needs M % 256 == 0 (M % 8 == 0 for the norms
+ * alone) and D <= 65024.  out_bmu2 / out_dist2 may both be NULL, or both given
+ * to get the second-best unit as in bmu_search_top2_ws.  Workspace:
+ * bmu_search_top2_workspace_bytes(...) covers either case.
+ */
+BMU_API int bmu_codebook_norms_f16(const void *W16, int64_t D, int64_t M, float *norms,
+                                   void *stream);
+BMU_API int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
+                              const int32_t *rowptr, const int32_t *colidx, int64_t N,
+                              int64_t nnz, int32_t *out_bmu, float *out_dist, int32_t *out_bmu2,
+                              float *out_dist2, const bmu_opts *opts, void *workspace,
+                              size_t workspace_bytes, void *stream);
+
+/*
  * One-shot form.  Same as bmu_search_ws with norms == NULL and default options,
  * but the scratch is a library-owned buffer per device that only ever grows
  * (cudaMalloc on first use or growth; freed by bmu_release_scratch or at

@@ -59,6 +59,14 @@ EXPORTS = {
                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
                                           ctypes.c_void_p]),
+    "bmu_codebook_norms_f16": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                              ctypes.c_void_p, ctypes.c_void_p]),
+    "bmu_search_f16_ws": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                         ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
+                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
+                                         ctypes.c_void_p]),
     "bmu_search": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
@@ -189,6 +197,43 @@ def bmu_search_top2_ws(W, rowptr, colidx, norms=None, opts: Opts | None = None):
             ob.data_ptr(), od.data_ptr(), ob2.data_ptr(), od2.data_ptr(),
             ctypes.byref(opts) if opts else None, ws_ptr, need, _stream(W)))
     return ob, od, ob2, od2
+
+
+def bmu_codebook_norms_f16(W16: torch.Tensor) -> torch.Tensor:
+    D, M = W16.shape
+    out = torch.empty(M, dtype=torch.float32, device=W16.device)
+    with torch.cuda.device(W16.device):
+        _check(load().bmu_codebook_norms_f16(_dev(W16, torch.float16, "W16"), D, M,
+                                             out.data_ptr(), _stream(W16)))
+    return out
+
+
+def bmu_search_f16_ws(W16, rowptr, colidx, norms=None, opts: Opts | None = None, top2=False,
+                      workspace=None):
+    """Search against an fp16 codebook [D, M].  Returns (bmu, dist) or, with top2,
+    (bmu, dist, bmu2, dist2)."""
+    D, M = W16.shape
+    N = rowptr.numel() - 1
+    nnz = colidx.numel()
+    dev = W16.device
+    ob = torch.empty(N, dtype=torch.int32, device=dev)
+    od = torch.empty(N, dtype=torch.float32, device=dev)
+    ob2 = torch.empty(N, dtype=torch.int32, device=dev) if top2 else None
+    od2 = torch.empty(N, dtype=torch.float32, device=dev) if top2 else None
+    need = int(load().bmu_search_top2_workspace_bytes(D, M, N, nnz, None))
+    ws = workspace if workspace is not None else torch.empty(need + 256, dtype=torch.uint8,
+                                                             device=dev)
+    ws_ptr = (ws.data_ptr() + 255) // 256 * 256
+    with torch.cuda.device(dev):
+        _check(load().bmu_search_f16_ws(
+            _dev(W16, torch.float16, "W16"), D, M,
+            _dev(norms, torch.float32, "norms") if norms is not None else None,
+            _dev(rowptr, torch.int32, "rowptr"),
+            _dev(colidx, torch.int32, "colidx") if nnz else None, N, nnz,
+            ob.data_ptr(), od.data_ptr(), ob2.data_ptr() if top2 else None,
+            od2.data_ptr() if top2 else None, ctypes.byref(opts) if opts else None,
+            ws_ptr, ws.numel() - (ws_ptr - ws.data_ptr()), _stream(W16)))
+    return (ob, od, ob2, od2) if top2 else (ob, od)
 
 
 def bmu_search(W, rowptr, colidx, out_bmu=None, out_dist=None):

@@ -348,6 +348,78 @@ int bmu_search_top2_ws(const float *W, int64_t D, int64_t M, const float *norms,
                        workspace_bytes, static_cast<cudaStream_t>(stream), out_bmu2, out_dist2);
 }
 
+int bmu_codebook_norms_f16(const void *W16, int64_t D, int64_t M, float *norms, void *stream)
+{
+    int rc = check_sizes(D, M, 0, 0);
+    if (rc) return rc;
+    if (M == 0) return BMU_OK;
+    if (!norms || (D > 0 && !W16)) { set_error("null pointer argument"); return BMU_ERR_INVALID_ARG; }
+    if (M % 8 != 0 || (reinterpret_cast<uintptr_t>(W16) & 15) != 0) {
+        set_error("half-precision codebook needs M %% 8 == 0 and 16-byte alignment");
+        return BMU_ERR_UNSUPPORTED;
+    }
+    return launch_norms_f16(W16, D, M, norms, static_cast<cudaStream_t>(stream));
+}
+
+int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
+                      const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
+                      int32_t *out_bmu, float *out_dist, int32_t *out_bmu2, float *out_dist2,
+                      const bmu_opts *opts, void *ws, size_t ws_bytes, void *stream)
+{
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int rc = check_sizes(D, M, N, nnz);
+    if (rc) return rc;
+    bmu_opts o;
+    memset(&o, 0, sizeof(o));
+    if (opts) o = *opts;
+    if ((rc = check_opts(o))) return rc;
+    if (N == 0) return BMU_OK;
+    const bool top2 = out_bmu2 != nullptr || out_dist2 != nullptr;
+    if (!W16 || !rowptr || !out_bmu || !out_dist || (nnz > 0 && !colidx) ||
+        (top2 && (!out_bmu2 || !out_dist2))) {
+        set_error("null pointer argument");
+        return BMU_ERR_INVALID_ARG;
+    }
+    if (M % 256 != 0 || D < 1 || D > LANES_MAX_D || (reinterpret_cast<uintptr_t>(W16) & 15) != 0 ||
+        (o.kernel != 0 && o.kernel != 3)) {
+        set_error("half-precision search needs M %% 256 == 0, 1 <= D <= %d, 16-byte alignment and "
+                  "the planned kernel", LANES_MAX_D);
+        return BMU_ERR_UNSUPPORTED;
+    }
+    const Layout l = layout_for(D, M, N, nnz, 3, top2);
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < l.total) {
+        set_error("workspace missing, not 256-byte aligned, or smaller than %zu bytes", l.total);
+        return BMU_ERR_WORKSPACE;
+    }
+    char *base = static_cast<char *>(ws);
+    u64 *state = reinterpret_cast<u64 *>(base + l.state_off);
+    u64 *state2 = top2 ? reinterpret_cast<u64 *>(base + l.state2_off) : nullptr;
+    if (!norms) {
+        float *n = reinterpret_cast<float *>(base + l.norms_off);
+        if ((rc = launch_norms_f16(W16, D, M, n, s))) return rc;
+        norms = n;
+    }
+    BMU_CUDA(cudaMemsetAsync(base + l.status_off, 0, 256, s));
+    char *pw = base + l.plan_off;
+    if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, pw, l.plan, s))) return rc;
+    RowsArgs a;
+    a.W = static_cast<const float *>(W16); a.M = M; a.N = N; a.norms = norms; a.rowptr = rowptr;
+    a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
+    a.doc_off = reinterpret_cast<const uint32_t *>(pw + l.plan.docoff_off);
+    a.ids = reinterpret_cast<const uint4 *>(pw + l.plan.ids_off);
+    a.state = state; a.state2 = state2;
+    // twice the neurons per L2-resident chunk: the rows are half as wide
+    const int64_t chunk = o.chunk_neurons ? (o.chunk_neurons + 255) / 256 * 256
+                                          : auto_chunk(D, M, 256) * 2;
+    for (int64_t j = 0; j < M; j += chunk) {
+        a.j_lo = (int32_t)j;
+        a.j_hi = (int32_t)(j + chunk < M ? j + chunk : M);
+        a.first = j == 0;
+        if ((rc = launch_sweep_rows_f16(a, o, s))) return rc;
+    }
+    return launch_finalize(state, state2, rowptr, N, out_bmu, out_dist, out_bmu2, out_dist2, s);
+}
+
 int bmu_search(const float *W, int64_t D, int64_t M, const int32_t *rowptr,
                const int32_t *colidx, int64_t N, int32_t *out_bmu, float *out_dist,
                void *stream)

@@ -144,6 +144,7 @@ __device__ __forceinline__ float hi_f(u64 p) { return __uint_as_float((uint32_t)
 
 // ---- kernels' host launchers (one per .cu file) ---------------------------
 int launch_norms(const float *W, int64_t D, int64_t M, float *norms, cudaStream_t s);
+int launch_norms_f16(const void *W16, int64_t D, int64_t M, float *norms, cudaStream_t s);
 
 struct SweepArgs {
     const float *W;
@@ -203,6 +204,8 @@ struct RowsArgs {
 };
 int rows_slab_width(const bmu_opts &o);
 int launch_sweep_rows(const RowsArgs &a, const bmu_opts &o, cudaStream_t s);
+// same with W pointing at an fp16 codebook (row pitch 2*M bytes), 256-neuron slabs
+int launch_sweep_rows_f16(const RowsArgs &a, const bmu_opts &o, cudaStream_t s);
 
 int launch_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                         int64_t D, int32_t *flags, cudaStream_t s);

@@ -6,6 +6,8 @@
 // the result does not depend on scheduling.  No scratch memory.
 #include "common.cuh"
 
+#include <cuda_fp16.h>
+
 namespace bmu {
 
 static const int NORM_WARPS = 16;
@@ -70,6 +72,51 @@ norms_kernel(const float *__restrict__ W, int64_t D, int64_t M, float *__restric
             norms[j] = (float)s;
         }
     }
+}
+
+// fp16 codebook: a lane owns 8 consecutive columns (one 16-byte load per row)
+__global__ void __launch_bounds__(NORM_WARPS * 32)
+norms_f16_kernel(const __half *__restrict__ W, int64_t D, int64_t M, float *__restrict__ norms)
+{
+    __shared__ double part[NORM_WARPS][256];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t col = (int64_t)blockIdx.x * 256 + lane * 8;
+    double a[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) a[c] = 0.0;
+    if (col < M) {
+        for (int64_t f = warp; f < D; f += NORM_WARPS) {
+            const uint4 t = __ldcs(reinterpret_cast<const uint4 *>(W + f * M + col));
+            const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 v = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
+                a[2 * i] = fma((double)v.x, (double)v.x, a[2 * i]);
+                a[2 * i + 1] = fma((double)v.y, (double)v.y, a[2 * i + 1]);
+            }
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < 8; ++c) part[warp][lane * 8 + c] = a[c];
+    __syncthreads();
+    if (threadIdx.x < 256) {
+        const int64_t j = (int64_t)blockIdx.x * 256 + threadIdx.x;
+        if (j < M) {
+            double s = 0.0;
+#pragma unroll
+            for (int w = 0; w < NORM_WARPS; ++w) s += part[w][threadIdx.x];
+            norms[j] = (float)s;
+        }
+    }
+}
+
+int launch_norms_f16(const void *W16, int64_t D, int64_t M, float *norms, cudaStream_t s)
+{
+    if (M == 0) return BMU_OK;
+    norms_f16_kernel<<<(unsigned)((M + 255) / 256), NORM_WARPS * 32, 0, s>>>(
+        static_cast<const __half *>(W16), D, M, norms);
+    BMU_CUDA(cudaGetLastError());
+    return BMU_OK;
 }
 
 int launch_norms(const float *W, int64_t D, int64_t M, float *norms, cudaStream_t s)

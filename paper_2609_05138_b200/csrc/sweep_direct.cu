@@ -16,6 +16,7 @@
 // per-document state that persists across chunks.
 #include "common.cuh"
 
+#include <cuda_fp16.h>
 #include <math_constants.h>
 
 namespace bmu {
@@ -229,6 +230,94 @@ sweep_rows_kernel(const RowsArgs a)
     u64 k1, k2;
     best.warp_keys(k1, k2);
     if (lane == 0) Best<TOP2>::commit(k1, k2, a.state, a.state2, orig, a.first);
+}
+
+// ---------------------------------------------------------------------------
+// Half-precision codebook (the paper's own storage, Section 4.2/4.3: "two bytes
+// per half-precision weight", __half2 loads): the planned kernel with rows of
+// fp16, eight neurons per 128-bit load, widened to fp32 in registers and
+// accumulated in fp32.  Slab = 256 neurons.
+template <int NW, bool TOP2>
+__global__ void __launch_bounds__(NW * 32)
+sweep_rows_f16_kernel(const RowsArgs a)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t p = (int64_t)blockIdx.x * NW + warp;
+    if (p >= a.N) return;
+    const int32_t orig = __ldg(a.perm + p);
+    const int len = __ldg(a.rowptr + orig + 1) - __ldg(a.rowptr + orig);
+    const uint4 *gp = a.ids + (size_t)__ldg(a.doc_off + p) + 1;
+    const int full = len >> 3, rem = len & 7;
+    const uint32_t rowbytes = (uint32_t)(a.M * 2);
+    const __half *W16 = reinterpret_cast<const __half *>(a.W);
+    Best<TOP2> best;
+    best.init();
+
+    for (int j0 = a.j_lo; j0 < a.j_hi; j0 += 256) {
+        const char *base = reinterpret_cast<const char *>(W16 + j0 + lane * 8);
+        u64 acc[4] = {0ull, 0ull, 0ull, 0ull};
+        auto add_row = [&](const uint4 h) {
+            const uint32_t w[4] = {h.x, h.y, h.z, h.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f2 = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
+                const u64 pk = ((u64)__float_as_uint(f2.y) << 32) | __float_as_uint(f2.x);
+                add2(acc[i], pk);
+            }
+        };
+        for (int g = 0; g < full; ++g) {
+            const uint4 t = __ldg(gp + g);
+            const uint32_t f[8] = {t.x & 0xffffu, t.x >> 16, t.y & 0xffffu, t.y >> 16,
+                                   t.z & 0xffffu, t.z >> 16, t.w & 0xffffu, t.w >> 16};
+            uint4 w[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                w[u] = __ldg(reinterpret_cast<const uint4 *>(base + (u64)f[u] * rowbytes));
+#pragma unroll
+            for (int u = 0; u < 8; ++u) add_row(w[u]);
+        }
+        if (rem) {
+            const uint4 t = __ldg(gp + full);
+            const uint32_t f[8] = {t.x & 0xffffu, t.x >> 16, t.y & 0xffffu, t.y >> 16,
+                                   t.z & 0xffffu, t.z >> 16, t.w & 0xffffu, t.w >> 16};
+#pragma unroll
+            for (int u = 0; u < 7; ++u)
+                if (u < rem)
+                    add_row(__ldg(reinterpret_cast<const uint4 *>(base + (u64)f[u] * rowbytes)));
+        }
+        const int col = j0 + lane * 8;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 n = __ldg(reinterpret_cast<const float2 *>(a.norms + col + 2 * i));
+            best.push(fmaf(-2.f, lo_f(acc[i]), n.x), col + 2 * i);
+            best.push(fmaf(-2.f, hi_f(acc[i]), n.y), col + 2 * i + 1);
+        }
+    }
+    u64 k1, k2;
+    best.warp_keys(k1, k2);
+    if (lane == 0) Best<TOP2>::commit(k1, k2, a.state, a.state2, orig, a.first);
+}
+
+int launch_sweep_rows_f16(const RowsArgs &a, const bmu_opts &o, cudaStream_t s)
+{
+    if (a.N == 0 || a.j_lo >= a.j_hi) return BMU_OK;
+    if ((a.j_hi - a.j_lo) % 256 != 0) {
+        set_error("half-precision kernel handles whole 256-neuron slabs only");
+        return BMU_ERR_INVALID_ARG;
+    }
+    const int NW = o.warps ? o.warps : 8;
+#define BMU_CASE(nw)                                                                      \
+    if (NW == nw) {                                                                       \
+        const unsigned blocks = (unsigned)((a.N + nw - 1) / nw);                          \
+        if (a.state2) sweep_rows_f16_kernel<nw, true><<<blocks, nw * 32, 0, s>>>(a);      \
+        else sweep_rows_f16_kernel<nw, false><<<blocks, nw * 32, 0, s>>>(a);              \
+        BMU_CUDA(cudaGetLastError());                                                     \
+        return BMU_OK;                                                                    \
+    }
+    BMU_CASE(8) BMU_CASE(16) BMU_CASE(32)
+#undef BMU_CASE
+    set_error("half-precision kernel: warps must be 8, 16 or 32");
+    return BMU_ERR_INVALID_ARG;
 }
 
 template <int V>

@@ -1,0 +1,60 @@
+"""Half-precision codebook (the paper's storage, Section 4.2 / 4.3): the fp16
+weights are exact in fp32, so the oracle simply runs on their fp32 copies."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from inputs import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def bmu():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_05138_b200 as lib
+    lib.load()
+    return lib
+
+
+@pytest.mark.parametrize("name,n_docs,M,kind", [("cfg1", 4000, 1024, "uniform"),
+                                                ("cfg2", 1500, 4096, "uniform"),
+                                                ("cfg5", 700, 2048, "scaled"),
+                                                ("cfg1", 900, 512, "signed"),
+                                                ("cfg1", 900, 256, "dupes")])
+def test_f16_search_matches_oracle(bmu, name, n_docs, M, kind):
+    cfg = synth.CONFIGS[name]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=n_docs)
+    W16 = synth.make_codebook(cfg.D, M, 50, kind=kind).half()
+    W32 = W16.float()                                   # exact widening: what the kernel sees
+    norms = bmu.bmu_codebook_norms_f16(W16.cuda())
+    ref = oracle.norms(W32.numpy())
+    np.testing.assert_allclose(norms.cpu().numpy().astype(np.float64), ref, rtol=6e-8)
+    o = bmu.Opts()
+    o.chunk_neurons = 512
+    ob, od = bmu.bmu_search_f16_ws(W16.cuda(), rowptr.cuda(), colidx.cuda(), opts=o)
+    torch.cuda.synchronize()
+    parity.compare(ob.cpu().numpy(), od.cpu().numpy(), W32.numpy(), rowptr.numpy(),
+                   colidx.numpy())
+    # the fp32 kernels on the widened codebook add the same fp32 values in the same order
+    fb, fd = bmu.bmu_search_ws(W32.cuda(), rowptr.cuda(), colidx.cuda())
+    assert torch.equal(ob, fb) and torch.equal(od, fd)
+    if kind == "dupes":
+        assert int((ob % 2).sum()) == 0
+
+
+def test_f16_top2_and_limits(bmu):
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=800)
+    W16 = synth.make_codebook(cfg.D, 768, 51, kind="scaled").half()
+    b1, d1, b2, d2 = bmu.bmu_search_f16_ws(W16.cuda(), rowptr.cuda(), colidx.cuda(), top2=True)
+    e1, f1, e2, f2 = oracle.bmu2(W16.float().numpy(), rowptr.numpy(), colidx.numpy())
+    clear = (f2 - f1) > 1e-4 * np.abs(f1)
+    assert np.array_equal(b1.cpu().numpy()[clear], e1[clear])
+    np.testing.assert_allclose(d2.cpu().numpy(), f2, rtol=1e-5)
+    with pytest.raises(bmu.BmuError) as e:
+        bmu.bmu_search_f16_ws(W16[:, :100].contiguous().cuda(), rowptr.cuda(), colidx.cuda())
+    assert e.value.status == 2
