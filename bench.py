@@ -214,21 +214,31 @@ def run_ours(args, cfg, rank, local_rank, world):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    n_docs = args.docs or synth.batch_size(cfg)
+    # one batch per step for the single-batch configs; config 5 streams its batches
+    n_batches = min(synth.num_batches(cfg), args.batches) if args.batches else synth.num_batches(cfg)
     W = synth.make_codebook(cfg.D, cfg.M, synth.codebook_seed(cfg), device=dev)
-    rowptr, colidx = synth.make_corpus(cfg, batch=rank % synth.num_batches(cfg), device=dev,
-                                       n_docs=n_docs,
-                                       seed=synth.corpus_seed(cfg, rank))
-    N, nnz = rowptr.numel() - 1, colidx.numel()
     opts = bmu.Opts()
     for kv in args.opt:
         k, v = kv.split("=")
         setattr(opts, k, int(v))
-    ws = torch.empty(bmu.bmu_search_workspace_bytes(cfg.D, cfg.M, N, nnz, opts) + 256,
+    batches = []
+    for b in range(n_batches):
+        bsz = min(synth.batch_size(cfg), cfg.N - b * synth.batch_size(cfg))
+        rp_b, ci_b = synth.make_corpus(cfg, batch=b, device=dev,
+                                       n_docs=min(bsz, args.docs) if args.docs else bsz,
+                                       seed=synth.corpus_seed(cfg, b) + 1000 * rank)
+        batches.append((rp_b, ci_b))
+    n_docs = sum(rp_b.numel() - 1 for rp_b, _ in batches)
+    rowptr, colidx = batches[0]
+    N, nnz = rowptr.numel() - 1, colidx.numel()
+    total_nnz = sum(ci_b.numel() for _, ci_b in batches)
+    max_n = max(rp_b.numel() - 1 for rp_b, _ in batches)
+    max_nnz = max(ci_b.numel() for _, ci_b in batches)
+    ws = torch.empty(bmu.bmu_search_workspace_bytes(cfg.D, cfg.M, max_n, max_nnz, opts) + 256,
                      dtype=torch.uint8, device=dev)
     norms = torch.empty(cfg.M, dtype=torch.float32, device=dev)
-    out_bmu = torch.empty(N, dtype=torch.int32, device=dev)
-    out_dist = torch.empty(N, dtype=torch.float32, device=dev)
+    out_bmu = torch.empty(max_n, dtype=torch.int32, device=dev)
+    out_dist = torch.empty(max_n, dtype=torch.float32, device=dev)
 
     # launch geometry of the sweep (mirrors the library's defaults; reported, not used by it)
     vec = opts.vec or (4 if opts.kernel == 1 else 8)
@@ -255,8 +265,10 @@ def run_ours(args, cfg, rank, local_rank, world):
         bmu.bmu_codebook_norms(W, norms)
         if e1 is not None:
             e1.record()
-        bmu.bmu_search_ws(W, rowptr, colidx, norms=norms, opts=opts, workspace=ws,
-                          out_bmu=out_bmu, out_dist=out_dist)
+        for rp_b, ci_b in batches:
+            nb = rp_b.numel() - 1
+            bmu.bmu_search_ws(W, rp_b, ci_b, norms=norms, opts=opts, workspace=ws,
+                              out_bmu=out_bmu[:nb], out_dist=out_dist[:nb])
         if e2 is not None:
             e2.record()
 
@@ -289,15 +301,24 @@ def run_ours(args, cfg, rank, local_rank, world):
     value = n_docs * world / (ms_per_step * 1e-3)     # all ranks' documents / slowest rank
 
     # ---- end to end through the host entry point (pinned CSR in, results out)
-    rp_h, ci_h = rowptr.cpu().pin_memory(), colidx.cpu().pin_memory()
-    ob_h = torch.empty(N, dtype=torch.int32).pin_memory()
-    od_h = torch.empty(N, dtype=torch.float32).pin_memory()
-    bmu.bmu_search_host(W, rp_h, ci_h, ob_h, od_h)          # warm-up (grows the scratch)
+    host = [(rp_b.cpu().pin_memory(), ci_b.cpu().pin_memory()) for rp_b, ci_b in batches]
+    outs = [(torch.empty(rp_b.numel() - 1, dtype=torch.int32).pin_memory(),
+             torch.empty(rp_b.numel() - 1, dtype=torch.float32).pin_memory()) for rp_b, _ in host]
+    rp_h, ci_h = host[0]
+    ob_h, od_h = outs[0]
+
+    def e2e_step():
+        if len(host) == 1:
+            bmu.bmu_search_host(W, rp_h, ci_h, ob_h, od_h)
+        else:
+            bmu.bmu_search_batches_host(W, host, outs)
+
+    e2e_step()                                              # warm-up (grows the scratch)
     e2e_steps = max(1, min(args.steps, 2))
     barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
-        bmu.bmu_search_host(W, rp_h, ci_h, ob_h, od_h)
+        e2e_step()
     torch.cuda.synchronize(dev)
     e2e_s = (time.perf_counter() - t0) / e2e_steps
     te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
@@ -305,7 +326,9 @@ def run_ours(args, cfg, rank, local_rank, world):
         import torch.distributed as dist
         dist.all_reduce(te, op=dist.ReduceOp.MAX)
     e2e_s = te.item()
-    same = bool(torch.equal(ob_h, out_bmu.cpu()))
+    bmu.bmu_search_ws(W, rowptr, colidx, norms=norms, opts=opts, workspace=ws,
+                      out_bmu=out_bmu[:N], out_dist=out_dist[:N])
+    same = bool(torch.equal(ob_h, out_bmu[:N].cpu()))
 
     if rank != 0:
         return None
@@ -313,9 +336,12 @@ def run_ours(args, cfg, rank, local_rank, world):
     # ---- roofline of the dominant kernel (the sweep): algorithmic units per launch / time
     peaks, peaks_kind = measured_peaks()
     roofs = {k: bmu.bmu_measure_roof(k, device=dev) for k in ("l2_ldg", "smem", "fadd2")}
-    launch_s = sweep_ms * 1e-3 / n_chunks
+    launch_s = sweep_ms * 1e-3 / (n_chunks * len(batches))
+    nnz = total_nnz / len(batches)                              # mean batch
+    N = n_docs / len(batches)
     adds = float(nnz) * chunk                                   # one fp32 add per (nnz, neuron)
-    union_rows = union_rows_per_block(rowptr, colidx, cfg.D, docs_per_block)
+    union_rows = union_rows_per_block(rowptr, colidx, cfg.D, docs_per_block) * (
+        nnz / max(1, colidx.numel()))
     alg = {
         "alu": (adds / launch_s, roofs["fadd2"], "add/s"),
         "l1": (4.0 * adds / launch_s, roofs["smem"], "B/s"),           # one 4-byte operand per add
@@ -347,18 +373,23 @@ def run_ours(args, cfg, rank, local_rank, world):
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": workload_config(cfg, n_docs, world),
-        "updates_per_s": float(nnz) * cfg.M * world / (ms_per_step * 1e-3),
+        "updates_per_s": float(total_nnz) * cfg.M * world / (ms_per_step * 1e-3),
         "phases_ms": {"norms": norms_ms, "sweep_and_output": sweep_ms},
         "clocks": clocks,
         "e2e": {"value": n_docs * world / e2e_s, "unit": UNIT,
-                "h2d_bytes_per_step": int((N + 1 + nnz) * 4), "d2h_bytes_per_step": int(N * 8),
-                "api": "bmu_search_host (codebook resident in HBM; CSR batch from pinned host "
-                       "memory; results back to host)", "matches_device_path": same},
-        "gpu_launches": args.steps * (1 + (0 if opts.kernel == 1 else 6) + n_chunks + 1),
+                "h2d_bytes_per_step": int((n_docs + len(batches) + total_nnz) * 4),
+                "d2h_bytes_per_step": int(n_docs * 8),
+                "api": ("bmu_search_host" if len(batches) == 1 else
+                        "bmu_search_batches_host (%d batches, upload of the next batch overlapped "
+                        "with the search of the current one)" % len(batches)) +
+                       " (codebook resident in HBM; CSR from pinned host memory; results back "
+                       "to host)", "matches_device_path": same},
+        "gpu_launches": args.steps * (1 + len(batches) * ((0 if opts.kernel == 1 else 6)
+                                                           + n_chunks + 1)),
         "roofline": roofline,
     }
     if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(cfg, W, rowptr, colidx, n_docs)
+        line["cpu_baseline"] = cpu_baseline(cfg, W, rowptr, colidx, rowptr.numel() - 1)
     return line
 
 
@@ -369,7 +400,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="cfg4", choices=sorted(synth.CONFIGS))
-    ap.add_argument("--docs", type=int, default=0, help="documents per GPU (0 = the config's batch)")
+    ap.add_argument("--docs", type=int, default=0, help="documents per batch (0 = the config's)")
+    ap.add_argument("--batches", type=int, default=0, help="batches per step (0 = the config's)")
     ap.add_argument("--opt", action="append", default=[], help="bmu_opts field=value")
     ap.add_argument("--ref-sample", type=int, default=4000)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -180,6 +180,23 @@ BMU_API int bmu_search_host(const float *W, int64_t D, int64_t M, const int32_t 
                     const int32_t *colidx_host, int64_t N, int32_t *out_bmu_host,
                     float *out_dist_host, void *stream);
 
+/*
+ * A corpus streamed in batches from HOST memory against one device-resident
+ * codebook (the corpus-scale epoch is fed this way: one CSR per batch, because a
+ * whole corpus exceeds the int32 row pointers).  The norms are computed once;
+ * two device staging buffers let a copy stream upload batch k+1 and download the
+ * results of batch k-1 while `stream` searches batch k.  Arrays of n_batches
+ * host pointers: rowptr_host[k] has N[k]+1 entries, colidx_host[k] has
+ * rowptr_host[k][N[k]], out_*_host[k] have N[k]; pinned memory lets the copies
+ * overlap.  Synchronous: returns when every result is in host memory.  Staging
+ * comes from the grow-only library scratch (sized for the largest batch).
+ */
+BMU_API int bmu_search_batches_host(const float *W, int64_t D, int64_t M, int32_t n_batches,
+                                    const int32_t *const *rowptr_host,
+                                    const int32_t *const *colidx_host, const int64_t *N,
+                                    int32_t *const *out_bmu_host, float *const *out_dist_host,
+                                    void *stream);
+
 /* Frees the library-owned scratch of the current device (synchronises it). */
 BMU_API int bmu_release_scratch(void);
 

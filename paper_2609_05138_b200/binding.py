@@ -77,6 +77,10 @@ EXPORTS = {
                                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                          ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
                                          ctypes.c_void_p]),
+    "bmu_search_batches_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                               ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                               ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                               ctypes.c_void_p]),
     "bmu_release_scratch": (ctypes.c_int, []),
     "bmu_validate_csr": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                         ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
@@ -283,6 +287,27 @@ def bmu_search_host(W, rowptr_host, colidx_host, out_bmu_host=None, out_dist_hos
             _host(out_bmu_host, torch.int32, "out_bmu_host"),
             _host(out_dist_host, torch.float32, "out_dist_host"), _stream(W)))
     return out_bmu_host, out_dist_host
+
+
+def bmu_search_batches_host(W, batches, outs=None):
+    """Streams host-resident CSR batches [(rowptr_host, colidx_host), ...] through the
+    search with copy/compute overlap.  Returns [(out_bmu_host, out_dist_host), ...]."""
+    wp, D, M = _codebook(W)
+    nb = len(batches)
+    if outs is None:
+        outs = [(torch.empty(rp.numel() - 1, dtype=torch.int32).pin_memory(),
+                 torch.empty(rp.numel() - 1, dtype=torch.float32).pin_memory())
+                for rp, _ in batches]
+    PtrArr = ctypes.c_void_p * nb
+    rps = PtrArr(*[_host(rp, torch.int32, "rowptr_host") for rp, _ in batches])
+    cis = PtrArr(*[_host(ci, torch.int32, "colidx_host") if ci.numel() else None
+                   for _, ci in batches])
+    obs = PtrArr(*[_host(ob, torch.int32, "out_bmu_host") for ob, _ in outs])
+    ods = PtrArr(*[_host(od, torch.float32, "out_dist_host") for _, od in outs])
+    ns = (ctypes.c_int64 * nb)(*[rp.numel() - 1 for rp, _ in batches])
+    with torch.cuda.device(W.device):
+        _check(load().bmu_search_batches_host(wp, D, M, nb, rps, cis, ns, obs, ods, _stream(W)))
+    return outs
 
 
 def bmu_release_scratch():

@@ -477,6 +477,101 @@ int bmu_search_host(const float *W, int64_t D, int64_t M, const int32_t *rowptr_
     return BMU_OK;
 }
 
+// ---- streamed batches from host memory (config 5: a corpus fed in batches) ----
+// Two staging buffers; the copy stream uploads batch k+1 and downloads the results
+// of batch k-1 while the caller's stream searches batch k.
+struct StreamCtx { cudaStream_t copy; cudaEvent_t h2d[2], done[2], d2h[2]; bool ready; };
+static StreamCtx g_stream_ctx[64];
+
+static int stream_ctx_get(int dev, StreamCtx **out)
+{
+    StreamCtx &c = g_stream_ctx[dev];
+    if (!c.ready) {
+        BMU_CUDA(cudaStreamCreateWithFlags(&c.copy, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; ++i) {
+            BMU_CUDA(cudaEventCreateWithFlags(&c.h2d[i], cudaEventDisableTiming));
+            BMU_CUDA(cudaEventCreateWithFlags(&c.done[i], cudaEventDisableTiming));
+            BMU_CUDA(cudaEventCreateWithFlags(&c.d2h[i], cudaEventDisableTiming));
+        }
+        c.ready = true;
+    }
+    *out = &c;
+    return BMU_OK;
+}
+
+int bmu_search_batches_host(const float *W, int64_t D, int64_t M, int32_t n_batches,
+                            const int32_t *const *rowptr_host, const int32_t *const *colidx_host,
+                            const int64_t *N, int32_t *const *out_bmu_host,
+                            float *const *out_dist_host, void *stream)
+{
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (n_batches < 0 || (n_batches > 0 && (!rowptr_host || !colidx_host || !N || !out_bmu_host ||
+                                            !out_dist_host))) {
+        set_error("null pointer argument or negative batch count");
+        return BMU_ERR_INVALID_ARG;
+    }
+    int rc;
+    int64_t max_n = 0, max_nnz = 0;
+    for (int k = 0; k < n_batches; ++k) {
+        if (N[k] < 0 || (N[k] > 0 && (!rowptr_host[k] || !out_bmu_host[k] || !out_dist_host[k]))) {
+            set_error("batch %d: null pointer or negative size", k);
+            return BMU_ERR_INVALID_ARG;
+        }
+        const int64_t nnz = N[k] > 0 ? rowptr_host[k][N[k]] : 0;
+        if ((rc = check_sizes(D, M, N[k], nnz))) return rc;
+        if (nnz > 0 && !colidx_host[k]) { set_error("batch %d: null colidx", k); return BMU_ERR_INVALID_ARG; }
+        if (N[k] > max_n) max_n = N[k];
+        if (nnz > max_nnz) max_nnz = nnz;
+    }
+    if (max_n == 0) return BMU_OK;
+    // layout: shared norms | per buffer: workspace, rowptr, colidx, out_bmu, out_dist
+    const size_t ws_need = layout_for(D, M, max_n, max_nnz, 0).total;
+    const size_t norms_bytes = align_up((size_t)M * 4, 256);
+    const size_t rp_off = align_up(ws_need, 256);
+    const size_t ci_off = align_up(rp_off + (size_t)(max_n + 1) * 4, 256);
+    const size_t ob_off = align_up(ci_off + (size_t)max_nnz * 4, 256);
+    const size_t od_off = align_up(ob_off + (size_t)max_n * 4, 256);
+    const size_t per_buf = align_up(od_off + (size_t)max_n * 4, 256);
+    void *p = nullptr;
+    if ((rc = scratch_get(norms_bytes + 2 * per_buf, &p))) return rc;
+    int dev = 0;
+    BMU_CUDA(cudaGetDevice(&dev));
+    StreamCtx *c = nullptr;
+    if ((rc = stream_ctx_get(dev, &c))) return rc;
+    char *b = static_cast<char *>(p);
+    float *norms = reinterpret_cast<float *>(b);
+    if ((rc = launch_norms(W, D, M, norms, s))) return rc;
+    for (int k = 0; k < n_batches; ++k) {
+        if (N[k] == 0) continue;
+        const int i = k & 1;
+        char *buf = b + norms_bytes + (size_t)i * per_buf;
+        const int64_t n = N[k], nnz = rowptr_host[k][n];
+        int32_t *rp = reinterpret_cast<int32_t *>(buf + rp_off);
+        int32_t *ci = reinterpret_cast<int32_t *>(buf + ci_off);
+        int32_t *ob = reinterpret_cast<int32_t *>(buf + ob_off);
+        float *od = reinterpret_cast<float *>(buf + od_off);
+        // upload: the buffer is free once the results of its previous batch are out
+        if (k >= 2) BMU_CUDA(cudaStreamWaitEvent(c->copy, c->d2h[i], 0));
+        BMU_CUDA(cudaMemcpyAsync(rp, rowptr_host[k], (size_t)(n + 1) * 4, cudaMemcpyHostToDevice, c->copy));
+        if (nnz)
+            BMU_CUDA(cudaMemcpyAsync(ci, colidx_host[k], (size_t)nnz * 4, cudaMemcpyHostToDevice, c->copy));
+        BMU_CUDA(cudaEventRecord(c->h2d[i], c->copy));
+        // search on the caller's stream
+        BMU_CUDA(cudaStreamWaitEvent(s, c->h2d[i], 0));
+        if ((rc = search_impl(W, D, M, norms, rp, ci, n, nnz, ob, od, nullptr, buf, ws_need, s)))
+            return rc;
+        BMU_CUDA(cudaEventRecord(c->done[i], s));
+        // download on the copy stream
+        BMU_CUDA(cudaStreamWaitEvent(c->copy, c->done[i], 0));
+        BMU_CUDA(cudaMemcpyAsync(out_bmu_host[k], ob, (size_t)n * 4, cudaMemcpyDeviceToHost, c->copy));
+        BMU_CUDA(cudaMemcpyAsync(out_dist_host[k], od, (size_t)n * 4, cudaMemcpyDeviceToHost, c->copy));
+        BMU_CUDA(cudaEventRecord(c->d2h[i], c->copy));
+    }
+    BMU_CUDA(cudaStreamSynchronize(s));
+    BMU_CUDA(cudaStreamSynchronize(c->copy));
+    return BMU_OK;
+}
+
 int bmu_release_scratch(void)
 {
     int dev = 0;

@@ -318,3 +318,19 @@ def test_planned_kernel_long_empty_unsorted_rows(bmu):
         r.shuffle(ci[rp[i]:rp[i + 1]])
     W = synth.make_codebook(D, M, 10, kind="scaled")
     run_and_check(bmu, W, rowptr, torch.from_numpy(ci), opts=make_opts(bmu, kernel=3))
+
+
+def test_streamed_batches_match_single_calls(bmu):
+    cfg = synth.CONFIGS["cfg5"]
+    W = synth.make_codebook(cfg.D, 1024, 3).cuda()
+    batches = []
+    for k, n in enumerate((3000, 0, 4100, 1, 2500)):
+        rp, ci = synth.make_corpus(cfg, batch=k, n_docs=n) if n else (
+            torch.zeros(1, dtype=torch.int32), torch.zeros(0, dtype=torch.int32))
+        batches.append((rp.pin_memory(), ci.pin_memory()))
+    outs = bmu.bmu_search_batches_host(W, batches)
+    for (rp, ci), (ob, od) in zip(batches, outs):
+        if rp.numel() == 1:
+            continue
+        rb, rd = bmu.bmu_search(W, rp.cuda(), ci.cuda())
+        assert torch.equal(rb.cpu(), ob) and torch.equal(rd.cpu(), od)
