@@ -197,6 +197,17 @@ BMU_API int bmu_search_batches_host(const float *W, int64_t D, int64_t M, int32_
                                     int32_t *const *out_bmu_host, float *const *out_dist_host,
                                     void *stream);
 
+/*
+ * Self-test of the failure path of device-side waits.  The staged kernel's
+ * producer and consumers wait on shared-memory barriers; every such wait has an
+ * iteration limit, after which the kernel records a status word and returns
+ * instead of trapping or spinning forever.  This call runs a one-block kernel
+ * that waits (limit: 4096 polls) on a barrier nothing ever arrives on and hands
+ * the outcome back the way bmu_search_host does: it returns BMU_ERR_TIMEOUT, and
+ * the CUDA context stays usable.  Synchronises the stream.
+ */
+BMU_API int bmu_selftest_wait_timeout(void *stream);
+
 /* Frees the library-owned scratch of the current device (synchronises it). */
 BMU_API int bmu_release_scratch(void);
 

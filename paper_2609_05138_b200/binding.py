@@ -81,6 +81,7 @@ EXPORTS = {
                                                ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
                                                ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                                ctypes.c_void_p]),
+    "bmu_selftest_wait_timeout": (ctypes.c_int, [ctypes.c_void_p]),
     "bmu_release_scratch": (ctypes.c_int, []),
     "bmu_validate_csr": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                         ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
@@ -308,6 +309,13 @@ def bmu_search_batches_host(W, batches, outs=None):
     with torch.cuda.device(W.device):
         _check(load().bmu_search_batches_host(wp, D, M, nb, rps, cis, ns, obs, ods, _stream(W)))
     return outs
+
+
+def bmu_selftest_wait_timeout(device=None) -> int:
+    """Runs the bounded-wait self-test; returns the status (5 = BMU_ERR_TIMEOUT expected)."""
+    device = torch.device("cuda" if device is None else device)
+    with torch.cuda.device(device):
+        return int(load().bmu_selftest_wait_timeout(torch.cuda.current_stream(device).cuda_stream))
 
 
 def bmu_release_scratch():

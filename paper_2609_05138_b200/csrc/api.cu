@@ -473,7 +473,13 @@ int bmu_search_host(const float *W, int64_t D, int64_t M, const int32_t *rowptr_
         return rc;
     BMU_CUDA(cudaMemcpyAsync(out_bmu_host, ob, (size_t)N * 4, cudaMemcpyDeviceToHost, s));
     BMU_CUDA(cudaMemcpyAsync(out_dist_host, od, (size_t)N * 4, cudaMemcpyDeviceToHost, s));
+    uint32_t status = 0;                               // first word of the workspace
+    BMU_CUDA(cudaMemcpyAsync(&status, b, sizeof(status), cudaMemcpyDeviceToHost, s));
     BMU_CUDA(cudaStreamSynchronize(s));
+    if (status) {
+        set_error("a bounded device-side wait ran out (status word %u); results are invalid", status);
+        return BMU_ERR_TIMEOUT;
+    }
     return BMU_OK;
 }
 
@@ -569,6 +575,25 @@ int bmu_search_batches_host(const float *W, int64_t D, int64_t M, int32_t n_batc
     }
     BMU_CUDA(cudaStreamSynchronize(s));
     BMU_CUDA(cudaStreamSynchronize(c->copy));
+    return BMU_OK;
+}
+
+int bmu_selftest_wait_timeout(void *stream)
+{
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    void *p = nullptr;
+    int rc = scratch_get(256, &p);
+    if (rc) return rc;
+    uint32_t *status = static_cast<uint32_t *>(p);
+    BMU_CUDA(cudaMemsetAsync(status, 0, 256, s));
+    if ((rc = launch_wait_timeout_selftest(status, s))) return rc;
+    uint32_t h = 0;
+    BMU_CUDA(cudaMemcpyAsync(&h, status, sizeof(h), cudaMemcpyDeviceToHost, s));
+    BMU_CUDA(cudaStreamSynchronize(s));
+    if (h) {
+        set_error("a bounded device-side wait ran out (status word %u)", h);
+        return BMU_ERR_TIMEOUT;
+    }
     return BMU_OK;
 }
 

@@ -54,17 +54,6 @@ __host__ __device__ __forceinline__ u64 make_key(float d, int32_t j)
 static const u64 KEY_WORST = ~0ull;
 
 #ifdef __CUDACC__
-// lexicographic (d, j) minimum across the warp; every lane gets the result
-__device__ __forceinline__ void warp_argmin(float &d, int &j)
-{
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        float od = __shfl_xor_sync(0xffffffffu, d, off);
-        int oj = __shfl_xor_sync(0xffffffffu, j, off);
-        if (od < d || (od == d && oj < j)) { d = od; j = oj; }
-    }
-}
-
 // Running minimum of one lane / warp / document: the best unit, and with TOP2 also
 // the second-best unit (Table 5: the paper's kernel tracks it for topographic
 // error).  push() must see a lane's neurons in ascending index order; ties then
@@ -188,6 +177,7 @@ int make_codebook_tensor_map(const float *W, int64_t D, int64_t M, int rows_per_
                              void *tensor_map_out);
 int launch_sweep_lanes(const void *tensor_map, const LanesArgs &a, const bmu_opts &o,
                        cudaStream_t s);
+int launch_wait_timeout_selftest(uint32_t *status, cudaStream_t s);
 
 // planned warp-per-document sweep (sweep_direct.cu): whole slabs of [j_lo, j_hi) only
 struct RowsArgs {

@@ -206,6 +206,35 @@ sweep_lanes_kernel(const __grid_constant__ CUtensorMap tm, const LanesArgs a, co
     }
 }
 
+// A wait that cannot succeed: one mbarrier that nothing ever arrives on.  It shows
+// that a wait which runs out leaves the kernel through the status word and the
+// context usable (no trap, no endless loop); the limit here is short on purpose.
+__global__ void wait_timeout_selftest_kernel(uint32_t *status)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_addr(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    bool ok = false;
+    for (uint32_t spin = 0; spin < 4096u && !ok; ++spin) {
+        uint32_t r;
+        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; "
+                     "selp.u32 %0, 1, 0, p; }"
+                     : "=r"(r) : "r"(smem_addr(&bar)), "r"(0u) : "memory");
+        ok = r != 0;
+    }
+    if (!ok && threadIdx.x == 0) atomicOr(status, 2u);
+}
+
+int launch_wait_timeout_selftest(uint32_t *status, cudaStream_t s)
+{
+    wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(status);
+    BMU_CUDA(cudaGetLastError());
+    return BMU_OK;
+}
+
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
                                   const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
@@ -259,7 +288,7 @@ static int launch_rn(const CUtensorMap &tm, const LanesArgs &a, int n_groups, in
     return BMU_OK;
 }
 
-int lanes_rows_per_stage(const bmu_opts &o) { return o.stage_rows ? o.stage_rows : 256; }
+static int lanes_rows_per_stage(const bmu_opts &o) { return o.stage_rows ? o.stage_rows : 256; }
 
 int launch_sweep_lanes(const void *tensor_map, const LanesArgs &a, const bmu_opts &o,
                        cudaStream_t s)

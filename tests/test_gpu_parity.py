@@ -334,3 +334,13 @@ def test_streamed_batches_match_single_calls(bmu):
             continue
         rb, rd = bmu.bmu_search(W, rp.cuda(), ci.cuda())
         assert torch.equal(rb.cpu(), ob) and torch.equal(rd.cpu(), od)
+
+
+def test_bounded_wait_reports_timeout_and_context_survives(bmu):
+    """A device-side wait that cannot succeed ends through the status word, not a hang."""
+    assert bmu.bmu_selftest_wait_timeout() == 5            # BMU_ERR_TIMEOUT
+    assert b"wait ran out" in bmu.load().bmu_last_error()
+    cfg = synth.CONFIGS["cfg1"]                            # the context still works
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=200)
+    W = synth.make_codebook(cfg.D, 256, 5)
+    run_and_check(bmu, W, rowptr, colidx)
