@@ -70,9 +70,12 @@ typedef struct bmu_opts {
     int32_t kernel;         /* 0 auto; 1 generic (a warp per document, ids straight from the
                                CSR, any D and M); 3 planned (a warp per document, ids from
                                the tiling pass; needs M % 4 == 0, M >= 32 * vec, D <= 65024);
-                               2 staged (a lane per document, rows streamed through shared
-                               memory by tensor (TMA) box copies; needs M % 4 == 0, M >= 32,
-                               256 <= D <= 65024) */
+                               4 tiled (a warp carries 8 documents; frequent rows loaded once
+                               per tile; the warps of a block walk the feature axis in step
+                               so that L1 serves the rows they share; needs what 3 needs and
+                               length-ordered documents); 2 staged (a lane per document, rows
+                               streamed through shared memory by tensor (TMA) box copies;
+                               needs M % 4 == 0, M >= 32, 256 <= D <= 65024) */
     int32_t chunk_neurons;  /* neurons per L2-resident chunk of the codebook (Section 4.2,
                                "neuron-axis chunking"); rounded to the slab width */
     int32_t vec;            /* warp-per-document kernels: floats per lane per row, 4 or 8 */
@@ -83,7 +86,11 @@ typedef struct bmu_opts {
                                of a warp carry similar rows; 2 keep the corpus order */
     int32_t stage_rows;     /* staged kernel: codebook rows per pipeline stage (256) */
     int32_t stages;         /* staged kernel: pipeline depth, a power of two (4) */
-    int32_t reserved[8];    /* must be 0 */
+    int32_t tile_order;     /* tiled kernel: 0 deal the rows of a tile alternately from the
+                               frequent and the rare half of the lists, 1 ascending ids */
+    int32_t tile_head;      /* tiled kernel: 0 sweep the 32 most frequent features (ids < 32)
+                               densely, one load per tile, 1 treat them like all other ids */
+    int32_t reserved[6];    /* must be 0 */
 } bmu_opts;
 
 BMU_API const char *bmu_status_string(int status);

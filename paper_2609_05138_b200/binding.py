@@ -32,7 +32,8 @@ class Opts(ctypes.Structure):
                 ("vec", ctypes.c_int32), ("docs_per_warp", ctypes.c_int32),
                 ("warps", ctypes.c_int32), ("cluster", ctypes.c_int32),
                 ("stage_rows", ctypes.c_int32), ("stages", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 8)]
+                ("tile_order", ctypes.c_int32), ("tile_head", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 6)]
 
 
 EXPORTS = {

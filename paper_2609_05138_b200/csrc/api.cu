@@ -77,9 +77,11 @@ static int check_sizes(int64_t D, int64_t M, int64_t N, int64_t nnz)
 
 static int check_opts(const bmu_opts &o)
 {
-    for (int i = 0; i < 8; ++i)
+    if (o.tile_order < 0 || o.tile_order > 1) { set_error("bmu_opts.tile_order must be 0 or 1"); return BMU_ERR_INVALID_ARG; }
+    if (o.tile_head < 0 || o.tile_head > 1) { set_error("bmu_opts.tile_head must be 0 or 1"); return BMU_ERR_INVALID_ARG; }
+    for (int i = 0; i < 6; ++i)
         if (o.reserved[i] != 0) { set_error("bmu_opts.reserved must be zero"); return BMU_ERR_INVALID_ARG; }
-    if (o.kernel < 0 || o.kernel > 3) { set_error("bmu_opts.kernel must be 0, 1, 2 or 3"); return BMU_ERR_INVALID_ARG; }
+    if (o.kernel < 0 || o.kernel > 4) { set_error("bmu_opts.kernel must be 0 .. 4"); return BMU_ERR_INVALID_ARG; }
     if (o.cluster < 0 || o.cluster > 2) { set_error("bmu_opts.cluster must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
     if (o.chunk_neurons < 0) { set_error("bmu_opts.chunk_neurons < 0"); return BMU_ERR_INVALID_ARG; }
     if (o.vec != 0 && o.vec != 4 && o.vec != 8) { set_error("bmu_opts.vec must be 0, 4 or 8"); return BMU_ERR_INVALID_ARG; }
@@ -158,10 +160,48 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
                   LANES_MAX_D);
         return BMU_ERR_UNSUPPORTED;
     }
+    const bool tiled = o.kernel == 4;
+    if (tiled && (!planned_ok || M < 128 || o.cluster == 2)) {
+        set_error("tiled kernel needs M %% 4 == 0, M >= 128, D <= %d, W 16-byte aligned and "
+                  "length-ordered documents (cluster != 2)", LANES_MAX_D);
+        return BMU_ERR_UNSUPPORTED;
+    }
     const bool planned = o.kernel == 3 || (o.kernel == 0 && planned_ok);
     char *pw = base + l.plan_off;
-    if (staged || planned)
+    if (staged || planned || tiled)
         if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, pw, l.plan, s))) return rc;
+    if (tiled) {
+        const int head = (o.tile_head == 1 || D < TILE_HEAD_ROWS) ? 0 : TILE_HEAD_ROWS;
+        if ((rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, pw, l.plan, s))) return rc;
+        TileArgs a;
+        a.W = W; a.M = M; a.N = N; a.n_tiles = (N + 7) / 8; a.norms = norms;
+        a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
+        a.tile_len = reinterpret_cast<const uint32_t *>(pw + l.plan.tilelen_off);
+        a.tile_off = reinterpret_cast<const uint32_t *>(pw + l.plan.tileoff_off);
+        a.tile_ids = reinterpret_cast<const uint4 *>(pw + l.plan.tileids_off);
+        a.tile_head = reinterpret_cast<const uint32_t *>(pw + l.plan.tilehead_off);
+        a.head_rows = head;
+        a.state = state; a.state2 = state2;
+        const int64_t chunk = o.chunk_neurons ? (o.chunk_neurons + 127) / 128 * 128
+                                              : auto_chunk(D, M, 128);
+        const int64_t m_full = M / 128 * 128;
+        for (int64_t j = 0; j < m_full; j += chunk) {
+            a.j_lo = (int32_t)j;
+            a.j_hi = (int32_t)(j + chunk < m_full ? j + chunk : m_full);
+            a.first = j == 0;
+            if ((rc = launch_sweep_tiles(a, o, s))) return rc;
+        }
+        if (m_full < M) {                      // ragged last slab: generic kernel, merged in
+            SweepArgs g;
+            g.W = W; g.D = D; g.M = M; g.norms = norms; g.rowptr = rowptr; g.colidx = colidx;
+            g.N = N; g.state = state; g.state2 = state2; g.j_lo = (int32_t)m_full;
+            g.j_hi = (int32_t)M; g.first = 0;
+            bmu_opts go;
+            memset(&go, 0, sizeof(go));
+            if ((rc = launch_sweep_direct(g, go, s))) return rc;
+        }
+        return launch_finalize(state, state2, rowptr, N, out_bmu, out_dist, out_bmu2, out_dist2, s);
+    }
     if (planned) {
         const int slab = rows_slab_width(o);
         RowsArgs a;

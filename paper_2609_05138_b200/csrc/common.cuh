@@ -154,7 +154,28 @@ int launch_finalize(const u64 *state, const u64 *state2, const int32_t *rowptr, 
 // ---- tiling plan (plan.cu) and staged sweep (sweep_lanes.cu) ---------------
 struct PlanLayout {
     size_t perm_off, docoff_off, ngroups_off, bins_off, ids_off, scan_off, scan_bytes, total;
+    size_t tilelen_off, tilerows_off, tileoff_off, tilehead_off, tileids_off, tile_rows_cap;
 };
+static const int TILE_HEAD_ROWS = 32;    // ids below this are swept densely, once per tile
+int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head, char *ws,
+                      const PlanLayout &l, cudaStream_t s);
+
+// tiled sweep (sweep_tiles.cu): a warp carries 8 documents, 128-neuron slabs
+struct TileArgs {
+    const float *W;
+    int64_t M, N, n_tiles;
+    const float *norms;
+    const int32_t *perm;
+    const uint32_t *tile_len;   // longest | shortest << 16 row of the tile
+    const uint32_t *tile_off;   // first row of the tile's id matrix
+    const uint4 *tile_ids;      // row r: the r-th id (behind the head) of each of the 8 documents
+    const uint32_t *tile_head;  // 8 masks per tile: which of the ids < head_rows a document has
+    int32_t head_rows;          // 0 or TILE_HEAD_ROWS
+    u64 *state;
+    u64 *state2;
+    int32_t j_lo, j_hi, first;
+};
+int launch_sweep_tiles(const TileArgs &a, const bmu_opts &o, cudaStream_t s);
 size_t plan_bytes(int64_t N, int64_t nnz, PlanLayout *l);
 int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                 int order_by_length, char *ws, const PlanLayout &l, cudaStream_t s);

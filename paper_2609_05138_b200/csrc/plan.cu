@@ -11,15 +11,20 @@
 //      (8 ids), padded with the sentinel 0xFFFF and closed by one all-sentinel
 //      group, so a lane fetches eight ids with one aligned 128-bit load and
 //      stops by itself at the end of its row.
+//   3. (tiled sweep only) cuts the length-ordered documents into tiles of 8 and
+//      writes, per tile, an id matrix: row b holds the b-th id of each of the
+//      tile's 8 documents (0xFFFF where a document has run out), so one aligned
+//      128-bit load hands a warp the next row of all eight documents.
 // Integer work only; the order of documents never changes any result because
-// every document is reduced by one lane on its own.
+// every document is reduced on its own.
 #include "common.cuh"
 
 #include <cub/device/device_scan.cuh>
 
 namespace bmu {
 
-static const int PLAN_BINS = 1024;
+static const int PLAN_BINS = 65536;      // one bin per row length: documents end up exactly
+                                         // length-ordered (ids are 16-bit, so rows are shorter)
 
 __global__ void plan_hist_kernel(const int32_t *__restrict__ rowptr, int64_t N,
                                  uint32_t *__restrict__ hist)
@@ -31,20 +36,28 @@ __global__ void plan_hist_kernel(const int32_t *__restrict__ rowptr, int64_t N,
     atomicAdd(hist + bin, 1u);
 }
 
-// exclusive scan of the PLAN_BINS counters (one block)
-__global__ void plan_scan_bins_kernel(uint32_t *__restrict__ hist, uint32_t *__restrict__ cursor)
+// exclusive scan of the PLAN_BINS counters (one block of 1024 threads, 64 bins each)
+__global__ void __launch_bounds__(1024)
+plan_scan_bins_kernel(const uint32_t *__restrict__ hist, uint32_t *__restrict__ cursor)
 {
-    __shared__ uint32_t s[PLAN_BINS];
+    constexpr int PER = PLAN_BINS / 1024;
+    __shared__ uint32_t s[1024];
     const int t = threadIdx.x;
-    s[t] = hist[t];
+    uint32_t sum = 0;
+    for (int i = 0; i < PER; ++i) sum += hist[t * PER + i];
+    s[t] = sum;
     __syncthreads();
-    for (int off = 1; off < PLAN_BINS; off <<= 1) {
+    for (int off = 1; off < 1024; off <<= 1) {
         const uint32_t v = t >= off ? s[t - off] : 0u;
         __syncthreads();
         s[t] += v;
         __syncthreads();
     }
-    cursor[t] = s[t] - hist[t];
+    uint32_t run = s[t] - sum;
+    for (int i = 0; i < PER; ++i) {
+        cursor[t * PER + i] = run;
+        run += hist[t * PER + i];
+    }
 }
 
 __global__ void plan_scatter_kernel(const int32_t *__restrict__ rowptr, int64_t N,
@@ -114,6 +127,93 @@ plan_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__
     if (p == N - 1 && lane < 16) dst[padded + lane] = 0xFFFFu;      // two groups of slack at the end
 }
 
+// ---- tiles of 8 documents -------------------------------------------------
+// The ids below `head` at the front of a document's ascending list, as a bit mask, and
+// how many list entries that covers.  A list that repeats one of them keeps multiset
+// semantics by opting out (mask 0, nothing skipped): its ids all stay in the list.
+__device__ __forceinline__ void head_of_doc(const uint16_t *ids, uint32_t len, uint32_t head,
+                                            uint32_t &mask, uint32_t &skip)
+{
+    mask = 0;
+    skip = 0;
+    for (uint32_t e = 0; e < len && e <= head; ++e) {
+        const uint32_t f = ids[e];
+        if (f >= head) break;
+        mask |= 1u << f;
+        ++skip;
+    }
+    if (skip != (uint32_t)__popc(mask)) { mask = 0; skip = 0; }
+}
+
+// per tile: longest and shortest list behind the head (max | min << 16), and the 8 head masks
+__global__ void plan_tile_len_kernel(const int32_t *__restrict__ rowptr,
+                                     const int32_t *__restrict__ perm,
+                                     const uint32_t *__restrict__ doc_off,
+                                     const uint16_t *__restrict__ ids16, int64_t N, int64_t n_tiles,
+                                     uint32_t head, uint32_t *__restrict__ tile_rows,
+                                     uint32_t *__restrict__ tile_len, uint32_t *__restrict__ tile_head)
+{
+    const int64_t tile = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (tile >= n_tiles) return;
+    uint32_t mx = 0, mn = 0xffffu;
+    for (int t = 0; t < 8; ++t) {
+        const int64_t p = tile * 8 + t;
+        uint32_t len = 0, mask = 0, skip = 0;
+        if (p < N) {
+            const int32_t i = perm[p];
+            len = (uint32_t)min(rowptr[i + 1] - rowptr[i], 65535);
+            if (head) head_of_doc(ids16 + ((size_t)doc_off[p] + 1) * 8, len, head, mask, skip);
+        }
+        tile_head[tile * 8 + t] = mask;
+        mx = max(mx, len - skip);
+        mn = min(mn, len - skip);
+    }
+    tile_rows[tile] = mx;
+    tile_len[tile] = mx | (mn << 16);
+}
+
+// One warp per tile: row r of the matrix = the r-th id, in visiting order, of each of its
+// 8 documents behind the head.  Visiting order: ascending, or (interleave) dealt alternately
+// from the frequent and the rare half of the document's own list, so that at any moment a
+// warp mixes loads that hit L1 with loads that go to L2.  The order depends on the document
+// alone, never on its tile mates, so results do not depend on how tiles were cut.
+__global__ void __launch_bounds__(256)
+plan_tile_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ perm,
+                      const uint32_t *__restrict__ doc_off, const uint16_t *__restrict__ ids16,
+                      const uint32_t *__restrict__ tile_len, const uint32_t *__restrict__ tile_off,
+                      const uint32_t *__restrict__ tile_head, int64_t N, int64_t n_tiles,
+                      int interleave, uint4 *__restrict__ tile_ids)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t tile = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (tile >= n_tiles) return;
+    const uint32_t rows = tile_len[tile] & 0xffffu;
+    const uint16_t *src[8];
+    uint32_t len[8];
+    for (int t = 0; t < 8; ++t) {
+        const int64_t p = tile * 8 + t;
+        len[t] = 0;
+        src[t] = ids16;
+        if (p < N) {
+            const int32_t i = perm[p];
+            const uint32_t skip = (uint32_t)__popc(tile_head[tile * 8 + t]);
+            len[t] = (uint32_t)min(rowptr[i + 1] - rowptr[i], 65535) - skip;
+            src[t] = ids16 + ((size_t)doc_off[p] + 1) * 8 + skip;
+        }
+    }
+    uint4 *dst = tile_ids + tile_off[tile];
+    for (uint32_t r = lane; r < rows; r += 32) {
+        uint32_t f[8];
+        for (int t = 0; t < 8; ++t) {
+            uint32_t e = r;
+            if (interleave) e = (r & 1u) ? (len[t] + 1) / 2 + r / 2 : r / 2;
+            f[t] = r < len[t] ? src[t][e] : 0xffffu;
+        }
+        dst[r] = make_uint4(f[0] | (f[1] << 16), f[2] | (f[3] << 16), f[4] | (f[5] << 16),
+                            f[6] | (f[7] << 16));
+    }
+}
+
 size_t plan_bytes(int64_t N, int64_t nnz, PlanLayout *l)
 {
     auto up = [](size_t x) { return (x + 255) / 256 * 256; };
@@ -129,6 +229,15 @@ size_t plan_bytes(int64_t N, int64_t nnz, PlanLayout *l)
     cub::DeviceScan::ExclusiveSum(nullptr, scan_tmp, (uint32_t *)nullptr, (uint32_t *)nullptr,
                                   (int)(N + 1));
     t.scan_off = off; t.scan_bytes = scan_tmp; off = up(off + scan_tmp);
+    // tiles: with documents exactly length-ordered, the sum over tiles of the longest row
+    // is at most nnz / 8 plus the spread of lengths (< 65536)
+    const size_t n_tiles = ((size_t)N + 7) / 8;
+    t.tilelen_off = off; off = up(off + (n_tiles + 1) * 4);
+    t.tilerows_off = off; off = up(off + (n_tiles + 1) * 4);
+    t.tileoff_off = off; off = up(off + (n_tiles + 1) * 4);
+    t.tilehead_off = off; off = up(off + n_tiles * 8 * 4);
+    t.tile_rows_cap = (size_t)nnz / 8 + 65536 + n_tiles;
+    t.tileids_off = off; off = up(off + t.tile_rows_cap * 16);
     t.total = off;
     if (l) *l = t;
     return off;
@@ -148,7 +257,7 @@ int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t
     if (order_by_length) {
         BMU_CUDA(cudaMemsetAsync(hist, 0, PLAN_BINS * 4, s));
         plan_hist_kernel<<<blocks, 256, 0, s>>>(rowptr, N, hist);
-        plan_scan_bins_kernel<<<1, PLAN_BINS, 0, s>>>(hist, cursor);
+        plan_scan_bins_kernel<<<1, 1024, 0, s>>>(hist, cursor);
         plan_scatter_kernel<<<blocks, 256, 0, s>>>(rowptr, N, cursor, perm);
     } else {
         plan_identity_kernel<<<blocks, 256, 0, s>>>(N, perm);
@@ -159,6 +268,31 @@ int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t
     BMU_CUDA(cub::DeviceScan::ExclusiveSum(ws + l.scan_off, tmp, ngroups, doc_off, (int)(N + 1), s));
     plan_fill_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(rowptr, colidx, perm,
                                                                        doc_off, N, ids16);
+    BMU_CUDA(cudaGetLastError());
+    return BMU_OK;
+}
+
+int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head, char *ws,
+                      const PlanLayout &l, cudaStream_t s)
+{
+    const int64_t n_tiles = (N + 7) / 8;
+    const int32_t *perm = reinterpret_cast<const int32_t *>(ws + l.perm_off);
+    const uint32_t *doc_off = reinterpret_cast<const uint32_t *>(ws + l.docoff_off);
+    const uint16_t *ids16 = reinterpret_cast<const uint16_t *>(ws + l.ids_off);
+    uint32_t *tile_len = reinterpret_cast<uint32_t *>(ws + l.tilelen_off);
+    uint32_t *tile_rows = reinterpret_cast<uint32_t *>(ws + l.tilerows_off);
+    uint32_t *tile_off = reinterpret_cast<uint32_t *>(ws + l.tileoff_off);
+    uint4 *tile_ids = reinterpret_cast<uint4 *>(ws + l.tileids_off);
+    uint32_t *tile_head = reinterpret_cast<uint32_t *>(ws + l.tilehead_off);
+    plan_tile_len_kernel<<<(unsigned)((n_tiles + 255) / 256), 256, 0, s>>>(
+        rowptr, perm, doc_off, ids16, N, n_tiles, (uint32_t)head, tile_rows, tile_len, tile_head);
+    BMU_CUDA(cudaMemsetAsync(tile_rows + n_tiles, 0, 4, s));
+    size_t tmp = l.scan_bytes;
+    BMU_CUDA(cub::DeviceScan::ExclusiveSum(ws + l.scan_off, tmp, tile_rows, tile_off,
+                                           (int)(n_tiles + 1), s));
+    plan_tile_fill_kernel<<<(unsigned)((n_tiles * 32 + 255) / 256), 256, 0, s>>>(
+        rowptr, perm, doc_off, ids16, tile_len, tile_off, tile_head, N, n_tiles, interleave,
+        tile_ids);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

@@ -344,3 +344,55 @@ def test_bounded_wait_reports_timeout_and_context_survives(bmu):
     rowptr, colidx = synth.make_corpus(cfg, n_docs=200)
     W = synth.make_codebook(cfg.D, 256, 5)
     run_and_check(bmu, W, rowptr, colidx)
+
+
+# ------------------------------------------------------------------ tiled kernel (8 documents per warp)
+@pytest.mark.parametrize("tile_order,tile_head", [(0, 0), (1, 0), (0, 1), (1, 1)])
+@pytest.mark.parametrize("name,n_docs,M", [("cfg1", 4001, 1024 + 36), ("cfg5", 1203, 2048)])
+def test_tiled_kernel_matches_oracle(bmu, name, n_docs, M, tile_order, tile_head):
+    cfg = synth.CONFIGS[name]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=n_docs)
+    W = synth.make_codebook(cfg.D, M, 16, kind="scaled")
+    opts = make_opts(bmu, kernel=4, tile_order=tile_order, tile_head=tile_head, chunk_neurons=512)
+    run_and_check(bmu, W, rowptr, colidx, opts=opts)
+    Wd, rp, ci = dev(W, rowptr, colidx)
+    a = bmu.bmu_search_ws(Wd, rp, ci, opts=opts)
+    b = bmu.bmu_search_ws(Wd, rp, ci, opts=opts)      # tiles are cut differently run to run
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    if tile_order == 1:                                # ascending sums: the planned kernel's bits
+        p = bmu.bmu_search_ws(Wd, rp, ci, opts=make_opts(bmu, kernel=3))
+        assert torch.equal(a[0], p[0]) and torch.equal(a[1], p[1])
+
+
+@pytest.mark.parametrize("kind,floor", [("dupes", False), ("const", False), ("sparse", False),
+                                        ("signed", False), ("prototype", True)])
+def test_tiled_kernel_codebook_kinds(bmu, kind, floor):
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=1500)
+    W = synth.make_codebook(cfg.D, 640, 79, kind=kind, docs=(rowptr, colidx))
+    run_and_check(bmu, W, rowptr, colidx, opts=make_opts(bmu, kernel=4), cancel_floor=floor)
+
+
+def test_tiled_kernel_long_empty_unsorted_and_repeated_rows(bmu):
+    D, M = 16384, 384
+    nnz = torch.tensor([400, 0, 1, 33, 0, 400, 97, 64, 32, 31, 0, 8, 16, 7, 9, 1500, 40] * 9)
+    rowptr, colidx = synth.draw_corpus(nnz.numel(), D, 1.1, nnz, seed=8)
+    ci = colidx.numpy().copy()
+    rp = rowptr.numpy()
+    r = np.random.default_rng(3)
+    for i in range(0, nnz.numel(), 2):
+        r.shuffle(ci[rp[i]:rp[i + 1]])
+    # a row that lists a frequent id twice keeps multiset semantics (added twice, counted twice)
+    ci[rp[3]:rp[3] + 2] = 5
+    W = synth.make_codebook(D, M, 11, kind="scaled")
+    run_and_check(bmu, W, rowptr, torch.from_numpy(ci), opts=make_opts(bmu, kernel=4))
+    run_and_check(bmu, W, rowptr, torch.from_numpy(ci), opts=make_opts(bmu, kernel=3))
+
+
+def test_tiled_kernel_refuses_unordered_tiles(bmu):
+    W = torch.zeros(300, 256, device="cuda")
+    rp = torch.tensor([0, 1], dtype=torch.int32).cuda()
+    ci = torch.tensor([0], dtype=torch.int32).cuda()
+    with pytest.raises(bmu.BmuError) as e:
+        bmu.bmu_search_ws(W, rp, ci, opts=make_opts(bmu, kernel=4, cluster=2))
+    assert e.value.status == 2

@@ -78,3 +78,13 @@ def test_top2_small_maps(bmu):
         ci = np.concatenate(rows).astype(np.int32)
         W = synth.make_codebook(50, M, 7 + M, kind="scaled")
         check(bmu, W, torch.from_numpy(rp), torch.from_numpy(ci))
+
+
+def test_top2_tiled_kernel(bmu):
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=1300)
+    W = synth.make_codebook(cfg.D, 768 + 40, 42, kind="scaled")
+    check(bmu, W, rowptr, colidx, kernel=4, chunk_neurons=256)
+    W = synth.make_codebook(cfg.D, 512, 43, kind="dupes")
+    b1, b2 = check(bmu, W, rowptr, colidx, kernel=4)
+    assert np.array_equal(b2, b1 + 1)
