@@ -31,6 +31,9 @@ if ROOT not in sys.path:
 
 from inputs import synth  # noqa: E402
 
+# DRAM bytes per sweep launch of the default config-4 run, from ncu (profiles/)
+TRAFFIC_CFG4 = {3: 2.0e9}
+
 METRIC = "bmu_search_docs_per_s"
 UNIT = "docs/s"
 
@@ -241,20 +244,30 @@ def run_ours(args, cfg, rank, local_rank, world):
     out_dist = torch.empty(max_n, dtype=torch.float32, device=dev)
 
     # launch geometry of the sweep (mirrors the library's defaults; reported, not used by it)
-    vec = opts.vec or (4 if opts.kernel == 1 else 8)
+    kernel = opts.kernel
+    if kernel == 0:                     # the library's automatic choice
+        kernel = 4 if (float(max_nnz) * cfg.M >= 2e10 and cfg.M >= 128) else 3
+    vec = opts.vec or (4 if kernel == 1 else 8)
     slab = 32 * vec
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
     chunk = opts.chunk_neurons or max(slab, (l2_bytes // 2) // (cfg.D * 4) // slab * slab)
     chunk = min((chunk + slab - 1) // slab * slab, (cfg.M + slab - 1) // slab * slab)
     n_chunks = (cfg.M + chunk - 1) // chunk
     # documents that share one SM's L1 at a time: resident warps x documents per warp
-    kernel_name = {0: "sweep_rows_kernel", 3: "sweep_rows_kernel", 1: "sweep_direct_kernel",
-                   2: "sweep_lanes_kernel"}[opts.kernel]
-    if opts.kernel == 2:
+    kernel_name = {3: "sweep_rows_kernel", 1: "sweep_direct_kernel", 2: "sweep_lanes_kernel",
+                   4: "sweep_tiles_kernel"}[kernel]
+    if kernel == 4:
+        vec, slab = 4, 128
+        chunk = opts.chunk_neurons or max(slab, (l2_bytes // 2) // (cfg.D * 4) // slab * slab)
+        chunk = min((chunk + slab - 1) // slab * slab, (cfg.M + slab - 1) // slab * slab)
+        n_chunks = (cfg.M + chunk - 1) // chunk
+    if kernel == 2:
         docs_per_block, chunk = 992, (opts.chunk_neurons or
                                       max(32, (l2_bytes // 2) // (cfg.D * 4) // 32 * 32))
         n_chunks = (cfg.M + chunk - 1) // chunk
-    elif opts.kernel == 1:
+    elif kernel == 4:
+        docs_per_block = 8 * (opts.warps or 4) * 5
+    elif kernel == 1:
         docs_per_block = (opts.warps or 16) * (opts.docs_per_warp or 4) * 2
     else:
         docs_per_block = 48
@@ -358,8 +371,9 @@ def run_ours(args, cfg, rank, local_rank, world):
         "unit": "GB/s" if unit == "B/s" else "Gadd/s", "frac": ach / peak,
         # DRAM bytes per launch from the ncu capture of this very launch configuration
         # (profiles/sweep_rows_cfg4_launch_list.md); other workloads were not captured
-        "traffic": (2.0e9 if (cfg.name == "cfg4" and n_docs == cfg.N and opts.kernel in (0, 3)
-                              and not opts.chunk_neurons and not opts.vec) else None),
+        "traffic": (TRAFFIC_CFG4.get(kernel) if (cfg.name == "cfg4" and n_docs == cfg.N
+                                                 and not opts.chunk_neurons and not opts.vec
+                                                 and not opts.warps) else None),
         "launch_ms": launch_s * 1e3, "launches_per_step": n_chunks,
         "units_per_launch": {"adds": adds, "union_rows_x_chunk": float(union_rows) * chunk},
         "fractions": {k: v[0] / v[1] for k, v in alg.items()},
@@ -384,7 +398,7 @@ def run_ours(args, cfg, rank, local_rank, world):
                         "with the search of the current one)" % len(batches)) +
                        " (codebook resident in HBM; CSR from pinned host memory; results back "
                        "to host)", "matches_device_path": same},
-        "gpu_launches": args.steps * (1 + len(batches) * ((0 if opts.kernel == 1 else 6)
+        "gpu_launches": args.steps * (1 + len(batches) * ({1: 0, 2: 6, 3: 6, 4: 8}[kernel]
                                                            + n_chunks + 1)),
         "roofline": roofline,
     }

@@ -160,13 +160,17 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
                   LANES_MAX_D);
         return BMU_ERR_UNSUPPORTED;
     }
-    const bool tiled = o.kernel == 4;
-    if (tiled && (!planned_ok || M < 128 || o.cluster == 2)) {
+    // automatic choice: the tiled kernel once the sweep is large enough to repay its extra
+    // tiling work (a few more small kernels), the planned kernel below that
+    const bool tiled_ok = planned_ok && M >= 128 && o.cluster != 2;
+    const bool tiled = o.kernel == 4 ||
+                       (o.kernel == 0 && tiled_ok && (double)nnz * (double)M >= 2e10);
+    if (tiled && !tiled_ok) {
         set_error("tiled kernel needs M %% 4 == 0, M >= 128, D <= %d, W 16-byte aligned and "
                   "length-ordered documents (cluster != 2)", LANES_MAX_D);
         return BMU_ERR_UNSUPPORTED;
     }
-    const bool planned = o.kernel == 3 || (o.kernel == 0 && planned_ok);
+    const bool planned = !tiled && (o.kernel == 3 || (o.kernel == 0 && planned_ok));
     char *pw = base + l.plan_off;
     if (staged || planned || tiled)
         if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, pw, l.plan, s))) return rc;

@@ -15,25 +15,26 @@ __device__ __forceinline__ uint32_t smem_u32(const void *p)
 
 // Every block sweeps the whole buffer (far larger than L1, resident in L2) with
 // 128-bit loads that bypass L1, `rounds` times, each block starting at its own
-// offset so that the blocks do not march in step.
-__global__ void __launch_bounds__(1024)
+// offset so that the blocks do not march in step.  Four blocks of 512 threads per
+// SM with eight loads in flight per thread keep 256 KB per SM on the wing.
+__global__ void __launch_bounds__(512, 4)
 roof_l2_ldg_kernel(const uint4 *__restrict__ buf, size_t n_vec, int rounds, uint32_t *sink)
 {
     uint4 acc = make_uint4(0, 0, 0, 0);
-    const size_t start = ((size_t)blockIdx.x * 7919u * 1024u) % n_vec;
+    const size_t start = ((size_t)blockIdx.x * 7919u * 512u) % n_vec;
     for (int r = 0; r < rounds; ++r) {
-        for (size_t i = threadIdx.x; i < n_vec; i += 4 * 1024) {
-            size_t a = start + i;
-            uint4 v[4];
+        for (size_t i = threadIdx.x; i < n_vec; i += 8 * 512) {
+            const size_t a = start + i;
+            uint4 v[8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                size_t idx = a + (size_t)u * 1024;
+            for (int u = 0; u < 8; ++u) {
+                size_t idx = a + (size_t)u * 512;
                 if (idx >= n_vec) idx -= n_vec;
                 if (idx >= n_vec) idx -= n_vec;
                 v[u] = __ldcg(buf + idx);
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) { acc.x ^= v[u].x; acc.y ^= v[u].y; acc.z ^= v[u].z; acc.w ^= v[u].w; }
+            for (int u = 0; u < 8; ++u) { acc.x ^= v[u].x; acc.y ^= v[u].y; acc.z ^= v[u].z; acc.w ^= v[u].w; }
         }
     }
     if ((acc.x ^ acc.y ^ acc.z ^ acc.w) == 0x12345677u) sink[0] = acc.x;
@@ -176,7 +177,7 @@ static void do_launch(void *p)
 {
     Ctx &c = *static_cast<Ctx *>(p);
     switch (c.kind) {
-    case 0: roof_l2_ldg_kernel<<<c.sms, 1024, 0, c.s>>>(reinterpret_cast<const uint4 *>(c.buf), c.bytes / 16, c.rounds, c.sink); break;
+    case 0: roof_l2_ldg_kernel<<<c.sms * 4, 512, 0, c.s>>>(reinterpret_cast<const uint4 *>(c.buf), c.bytes / 16, c.rounds, c.sink); break;
     case 1: roof_l2_bulk_kernel<8><<<c.sms * 4, 32, 8 * c.piece, c.s>>>(c.buf, c.bytes, c.piece, c.rounds, c.sink); break;
     case 2: roof_smem_kernel<<<c.sms, 1024, 0, c.s>>>(c.iters, c.sink); break;
     case 3: roof_l1_kernel<<<c.sms, 1024, 0, c.s>>>(reinterpret_cast<const uint4 *>(c.buf), c.iters, c.sink); break;
@@ -214,9 +215,8 @@ extern "C" BMU_API int bmu_measure_roof(int which, void *buffer, size_t buffer_b
             BMU_CUDA(cudaFuncSetAttribute(roof_l2_bulk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * piece));
         }
         c.bytes = usable; c.piece = piece;
-        c.rounds = (int)(((size_t)2 << 30) / usable) + 1;   // about 2 GiB per block
-        if (which == 1) c.rounds = c.rounds / 4 + 1;
-        work = (double)usable * c.rounds * (which == 0 ? sms : sms * 4);
+        c.rounds = (int)(((size_t)2 << 30) / usable) / 4 + 1;   // about 0.5 GiB per block
+        work = (double)usable * c.rounds * sms * 4;
     } else if (which == 2 || which == 3) {
         if (which == 3 && buffer_bytes < 256 + (size_t)sms * 65536) { set_error("buffer too small"); return BMU_ERR_WORKSPACE; }
         c.iters = 20000;

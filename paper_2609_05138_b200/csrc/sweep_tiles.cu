@@ -61,10 +61,13 @@ __device__ __forceinline__ int doc_of_lane(int lane)
     return ((lane & 1) << 2) | (lane & 2) | ((lane & 4) >> 2);
 }
 
-// up to 128 registers per thread (the 32 sums, eight 128-bit loads in flight, masks):
-// 16 warps per SM
+// 640 resident threads per SM: 96 registers per thread (the 32 sums, eight 128-bit loads in
+// flight, no spill) and 20 warps -- the best trade between loads in flight per warp and warps
+#ifndef BMU_TILE_THREADS
+#define BMU_TILE_THREADS 640
+#endif
 template <int NW, bool TOP2>
-__global__ void __launch_bounds__(NW * 32, 512 / (NW * 32) > 0 ? 512 / (NW * 32) : 1)
+__global__ void __launch_bounds__(NW * 32, BMU_TILE_THREADS / (NW * 32) > 0 ? BMU_TILE_THREADS / (NW * 32) : 1)
 sweep_tiles_kernel(const TileArgs a)
 {
     constexpr int T = TILE_DOCS;
@@ -86,13 +89,14 @@ sweep_tiles_kernel(const TileArgs a)
     Keys<TOP2> run;
     run.k1 = run.k2 = KEY_WORST;
     const uint32_t rowbytes = (uint32_t)(a.M * 4);
-    // which of the frequent ids (< head_rows) each document has; `any`: their union
-    uint32_t hm[T], any = 0;
+    // which of the frequent ids (< head_rows) each document has (kept in shared memory: the
+    // registers are needed for loads in flight); `any`: their union
+    __shared__ uint32_t s_hm[NW][T];
+    uint32_t any = 0;
+    if (lane < T) s_hm[warp][lane] = (active && a.head_rows) ? __ldg(a.tile_head + tile * T + lane) : 0u;
+    __syncwarp();
 #pragma unroll
-    for (int t = 0; t < T; ++t) {
-        hm[t] = (active && a.head_rows) ? __ldg(a.tile_head + tile * T + t) : 0u;
-        any |= hm[t];
-    }
+    for (int t = 0; t < T; ++t) any |= s_hm[warp][t];
 
     for (int j0 = a.j_lo; j0 < a.j_hi; j0 += 128) {
         __syncthreads();                              // the block's warps start each slab together
@@ -114,10 +118,12 @@ sweep_tiles_kernel(const TileArgs a)
                     w[u] = __ldg(reinterpret_cast<const ulonglong2 *>(
                         base + (u64)(f0 + u) * rowbytes));
 #pragma unroll
-                for (int u = 0; u < 8; ++u)
+                for (int t = 0; t < T; ++t) {
+                    const uint32_t m = s_hm[warp][t];
 #pragma unroll
-                    for (int t = 0; t < T; ++t)
-                        add2_if(acc[t][0], acc[t][1], w[u].x, w[u].y, hm[t], 1u << (f0 + u));
+                    for (int u = 0; u < 8; ++u)
+                        add2_if(acc[t][0], acc[t][1], w[u].x, w[u].y, m, 1u << (f0 + u));
+                }
             }
         }
         uint32_t b = 0;
@@ -210,9 +216,9 @@ int launch_sweep_tiles(const TileArgs &a, const bmu_opts &o, cudaStream_t s)
         BMU_CUDA(cudaGetLastError());                                                       \
         return BMU_OK;                                                                      \
     }
-    BMU_CASE(4) BMU_CASE(8) BMU_CASE(16) BMU_CASE(32)
+    BMU_CASE(2) BMU_CASE(4) BMU_CASE(8) BMU_CASE(16) BMU_CASE(32)
 #undef BMU_CASE
-    set_error("tiled kernel: warps must be 4, 8, 16 or 32");
+    set_error("tiled kernel: warps must be 2, 4, 8, 16 or 32");
     return BMU_ERR_INVALID_ARG;
 }
 

@@ -40,7 +40,9 @@ def test_f16_search_matches_oracle(bmu, name, n_docs, M, kind):
     parity.compare(ob.cpu().numpy(), od.cpu().numpy(), W32.numpy(), rowptr.numpy(),
                    colidx.numpy())
     # the fp32 kernels on the widened codebook add the same fp32 values in the same order
-    fb, fd = bmu.bmu_search_ws(W32.cuda(), rowptr.cuda(), colidx.cuda())
+    o3 = bmu.Opts()
+    o3.kernel = 3
+    fb, fd = bmu.bmu_search_ws(W32.cuda(), rowptr.cuda(), colidx.cuda(), opts=o3)
     assert torch.equal(ob, fb) and torch.equal(od, fd)
     if kind == "dupes":
         assert int((ob % 2).sum()) == 0
