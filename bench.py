@@ -32,7 +32,7 @@ if ROOT not in sys.path:
 from inputs import synth  # noqa: E402
 
 # DRAM bytes per sweep launch of the default config-4 run, from ncu (profiles/)
-TRAFFIC_CFG4 = {3: 2.0e9}
+TRAFFIC_CFG4 = {3: 2.0e9, 4: 2.9e9}
 
 METRIC = "bmu_search_docs_per_s"
 UNIT = "docs/s"
