@@ -32,7 +32,7 @@ static const int64_t MAX_I32 = 0x7fffffff;
 
 // ---- workspace layout -----------------------------------------------------
 struct Layout {
-    size_t status_off, norms_off, state_off, state2_off, plan_off, total;
+    size_t status_off, norms_off, state_off, state2_off, head_off, plan_off, total;
     PlanLayout plan;
 };
 
@@ -54,6 +54,10 @@ static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kerne
     l.state_off = off; off = align_up(off + (size_t)N * sizeof(u64), 256);
     l.state2_off = off;
     if (top2) off = align_up(off + (size_t)N * sizeof(u64), 256);
+    // split image of the frequent rows for the tensor-core sweep (it may be the automatic choice)
+    l.head_off = off;
+    if ((kernel == 0 || kernel == 5) && !top2 && D >= MMA_HEAD && D <= LANES_MAX_D && M >= MMA_SLAB)
+        off = align_up(off + head_image_bytes(M), 256);
     l.plan_off = off;
     memset(&l.plan, 0, sizeof(l.plan));
     if (kernel != 1 && D <= LANES_MAX_D) off += plan_bytes(N, nnz, &l.plan);
@@ -81,7 +85,7 @@ static int check_opts(const bmu_opts &o)
     if (o.tile_head < 0 || o.tile_head > 1) { set_error("bmu_opts.tile_head must be 0 or 1"); return BMU_ERR_INVALID_ARG; }
     for (int i = 0; i < 6; ++i)
         if (o.reserved[i] != 0) { set_error("bmu_opts.reserved must be zero"); return BMU_ERR_INVALID_ARG; }
-    if (o.kernel < 0 || o.kernel > 4) { set_error("bmu_opts.kernel must be 0 .. 4"); return BMU_ERR_INVALID_ARG; }
+    if (o.kernel < 0 || o.kernel > 5) { set_error("bmu_opts.kernel must be 0 .. 5"); return BMU_ERR_INVALID_ARG; }
     if (o.cluster < 0 || o.cluster > 2) { set_error("bmu_opts.cluster must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
     if (o.chunk_neurons < 0) { set_error("bmu_opts.chunk_neurons < 0"); return BMU_ERR_INVALID_ARG; }
     if (o.vec != 0 && o.vec != 4 && o.vec != 8) { set_error("bmu_opts.vec must be 0, 4 or 8"); return BMU_ERR_INVALID_ARG; }
@@ -163,17 +167,60 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     // automatic choice: the tiled kernel once the sweep is large enough to repay its extra
     // tiling work (a few more small kernels), the planned kernel below that
     const bool tiled_ok = planned_ok && M >= 128 && o.cluster != 2;
-    const bool tiled = o.kernel == 4 ||
-                       (o.kernel == 0 && tiled_ok && (double)nnz * (double)M >= 2e10);
+    // tensor-core head: additionally whole 512-neuron slabs, at least 256 features, best unit only
+    const bool mma_ok = tiled_ok && !top2 && D >= MMA_HEAD && M >= MMA_SLAB;
+    if (o.kernel == 5 && !mma_ok) {
+        set_error("tensor-core sweep needs what the tiled kernel needs, D >= %d, M >= %d and no "
+                  "second-best unit", MMA_HEAD, MMA_SLAB);
+        return BMU_ERR_UNSUPPORTED;
+    }
+    const bool mma = o.kernel == 5;
+    const bool tiled = !mma && (o.kernel == 4 ||
+                       (o.kernel == 0 && tiled_ok && (double)nnz * (double)M >= 2e10));
     if (tiled && !tiled_ok) {
         set_error("tiled kernel needs M %% 4 == 0, M >= 128, D <= %d, W 16-byte aligned and "
                   "length-ordered documents (cluster != 2)", LANES_MAX_D);
         return BMU_ERR_UNSUPPORTED;
     }
-    const bool planned = !tiled && (o.kernel == 3 || (o.kernel == 0 && planned_ok));
+    const bool planned = !tiled && !mma && (o.kernel == 3 || (o.kernel == 0 && planned_ok));
     char *pw = base + l.plan_off;
-    if (staged || planned || tiled)
+    if (staged || planned || tiled || mma)
         if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, pw, l.plan, s))) return rc;
+    if (mma) {
+        const int64_t m_full = M / MMA_SLAB * MMA_SLAB;
+        uint32_t *head_max = status + 16;
+        unsigned char *img = reinterpret_cast<unsigned char *>(base + l.head_off);
+        if ((rc = launch_head_split(W, M, m_full, head_max, img, s))) return rc;
+        if ((rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, MMA_HEAD, pw, l.plan, s))) return rc;
+        MmaArgs a;
+        a.W = W; a.M = M; a.N = N; a.n_tiles = (N + 7) / 8; a.norms = norms;
+        a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
+        a.tile_len = reinterpret_cast<const uint32_t *>(pw + l.plan.tilelen_off);
+        a.tile_off = reinterpret_cast<const uint32_t *>(pw + l.plan.tileoff_off);
+        a.tile_ids = reinterpret_cast<const uint4 *>(pw + l.plan.tileids_off);
+        a.tile_head = reinterpret_cast<const uint32_t *>(pw + l.plan.tilehead_off);
+        a.head_max = head_max;
+        a.state = state; a.status = status;
+        const int64_t chunk = o.chunk_neurons ? (o.chunk_neurons + MMA_SLAB - 1) / MMA_SLAB * MMA_SLAB
+                                              : auto_chunk(D, M, MMA_SLAB);
+        for (int64_t j = 0; j < m_full; j += chunk) {
+            a.j_lo = (int32_t)j;
+            a.j_hi = (int32_t)(j + chunk < m_full ? j + chunk : m_full);
+            a.first = j == 0;
+            a.head_img = img + (size_t)(j / MMA_SLAB) * MMA_STAGES_PER_SLAB * MMA_STAGE_BYTES;
+            if ((rc = launch_sweep_mma(a, o, s))) return rc;
+        }
+        if (m_full < M) {                      // ragged last slab: generic kernel, merged in
+            SweepArgs g;
+            g.W = W; g.D = D; g.M = M; g.norms = norms; g.rowptr = rowptr; g.colidx = colidx;
+            g.N = N; g.state = state; g.state2 = nullptr; g.j_lo = (int32_t)m_full;
+            g.j_hi = (int32_t)M; g.first = 0;
+            bmu_opts go;
+            memset(&go, 0, sizeof(go));
+            if ((rc = launch_sweep_direct(g, go, s))) return rc;
+        }
+        return launch_finalize(state, nullptr, rowptr, N, out_bmu, out_dist, nullptr, nullptr, s);
+    }
     if (tiled) {
         const int head = (o.tile_head == 1 || D < TILE_HEAD_ROWS) ? 0 : TILE_HEAD_ROWS;
         if ((rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, pw, l.plan, s))) return rc;

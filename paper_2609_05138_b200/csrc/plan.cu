@@ -128,24 +128,36 @@ plan_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__
 }
 
 // ---- tiles of 8 documents -------------------------------------------------
-// The ids below `head` at the front of a document's ascending list, as a bit mask, and
-// how many list entries that covers.  A list that repeats one of them keeps multiset
-// semantics by opting out (mask 0, nothing skipped): its ids all stay in the list.
+// The ids below `head` (a multiple of 32, at most 256) at the front of a document's
+// ascending list, as a bit mask of head / 32 words, and how many list entries that
+// covers.  A list that repeats one of them keeps multiset semantics by opting out
+// (mask 0, nothing skipped): its ids all stay in the list.
 __device__ __forceinline__ void head_of_doc(const uint16_t *ids, uint32_t len, uint32_t head,
-                                            uint32_t &mask, uint32_t &skip)
+                                            uint32_t mask[8], uint32_t &skip)
 {
-    mask = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) mask[w] = 0;
     skip = 0;
     for (uint32_t e = 0; e < len && e <= head; ++e) {
         const uint32_t f = ids[e];
         if (f >= head) break;
-        mask |= 1u << f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w)
+            if ((f >> 5) == (uint32_t)w) mask[w] |= 1u << (f & 31u);
         ++skip;
     }
-    if (skip != (uint32_t)__popc(mask)) { mask = 0; skip = 0; }
+    uint32_t bits = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) bits += (uint32_t)__popc(mask[w]);
+    if (skip != bits) {
+#pragma unroll
+        for (int w = 0; w < 8; ++w) mask[w] = 0;
+        skip = 0;
+    }
 }
 
-// per tile: longest and shortest list behind the head (max | min << 16), and the 8 head masks
+// per tile: longest and shortest list behind the head (max | min << 16), and the head masks
+// (head / 32 words per document, document-major)
 __global__ void plan_tile_len_kernel(const int32_t *__restrict__ rowptr,
                                      const int32_t *__restrict__ perm,
                                      const uint32_t *__restrict__ doc_off,
@@ -155,16 +167,19 @@ __global__ void plan_tile_len_kernel(const int32_t *__restrict__ rowptr,
 {
     const int64_t tile = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (tile >= n_tiles) return;
+    const uint32_t words = head ? head / 32 : 1;
     uint32_t mx = 0, mn = 0xffffu;
     for (int t = 0; t < 8; ++t) {
         const int64_t p = tile * 8 + t;
-        uint32_t len = 0, mask = 0, skip = 0;
+        uint32_t len = 0, skip = 0, mask[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         if (p < N) {
             const int32_t i = perm[p];
             len = (uint32_t)min(rowptr[i + 1] - rowptr[i], 65535);
             if (head) head_of_doc(ids16 + ((size_t)doc_off[p] + 1) * 8, len, head, mask, skip);
         }
-        tile_head[tile * 8 + t] = mask;
+#pragma unroll
+        for (int w = 0; w < 8; ++w)
+            if ((uint32_t)w < words) tile_head[(tile * 8 + t) * words + w] = mask[w];
         mx = max(mx, len - skip);
         mn = min(mn, len - skip);
     }
@@ -181,8 +196,8 @@ __global__ void __launch_bounds__(256)
 plan_tile_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ perm,
                       const uint32_t *__restrict__ doc_off, const uint16_t *__restrict__ ids16,
                       const uint32_t *__restrict__ tile_len, const uint32_t *__restrict__ tile_off,
-                      const uint32_t *__restrict__ tile_head, int64_t N, int64_t n_tiles,
-                      int interleave, uint4 *__restrict__ tile_ids)
+                      const uint32_t *__restrict__ tile_head, uint32_t head_words, int64_t N,
+                      int64_t n_tiles, int interleave, uint4 *__restrict__ tile_ids)
 {
     const int lane = threadIdx.x & 31;
     const int64_t tile = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -196,7 +211,9 @@ plan_tile_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restr
         src[t] = ids16;
         if (p < N) {
             const int32_t i = perm[p];
-            const uint32_t skip = (uint32_t)__popc(tile_head[tile * 8 + t]);
+            uint32_t skip = 0;
+            for (uint32_t w = 0; w < head_words; ++w)
+                skip += (uint32_t)__popc(tile_head[(tile * 8 + t) * head_words + w]);
             len[t] = (uint32_t)min(rowptr[i + 1] - rowptr[i], 65535) - skip;
             src[t] = ids16 + ((size_t)doc_off[p] + 1) * 8 + skip;
         }
@@ -235,7 +252,7 @@ size_t plan_bytes(int64_t N, int64_t nnz, PlanLayout *l)
     t.tilelen_off = off; off = up(off + (n_tiles + 1) * 4);
     t.tilerows_off = off; off = up(off + (n_tiles + 1) * 4);
     t.tileoff_off = off; off = up(off + (n_tiles + 1) * 4);
-    t.tilehead_off = off; off = up(off + n_tiles * 8 * 4);
+    t.tilehead_off = off; off = up(off + n_tiles * 8 * 4 * (HEAD_ROWS_MAX / 32));
     t.tile_rows_cap = (size_t)nnz / 8 + 65536 + n_tiles;
     t.tileids_off = off; off = up(off + t.tile_rows_cap * 16);
     t.total = off;
@@ -291,8 +308,8 @@ int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head
     BMU_CUDA(cub::DeviceScan::ExclusiveSum(ws + l.scan_off, tmp, tile_rows, tile_off,
                                            (int)(n_tiles + 1), s));
     plan_tile_fill_kernel<<<(unsigned)((n_tiles * 32 + 255) / 256), 256, 0, s>>>(
-        rowptr, perm, doc_off, ids16, tile_len, tile_off, tile_head, N, n_tiles, interleave,
-        tile_ids);
+        rowptr, perm, doc_off, ids16, tile_len, tile_off, tile_head,
+        (uint32_t)(head ? head / 32 : 1), N, n_tiles, interleave, tile_ids);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

@@ -1,0 +1,119 @@
+"""Parity of the tensor-core head + gathered tail sweep (bmu_opts.kernel = 5) against
+the fp64 oracle, through the C ABI.  Same rule as every other kernel
+(tests/parity.py): indices equal except inside a 1e-5 near-tie, distances within
+1e-5 relative.  The head sums come from fp16 (hi, lo) parts of the weights and a
+tensor-core fp32 accumulator, so results are not bit-equal to the gathered
+kernels; they are held to the oracle alone.
+"""
+import numpy as np
+import pytest
+import torch
+
+from inputs import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def bmu():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_05138_b200 as lib
+    lib.load()
+    return lib
+
+
+def opts_of(bmu, **kw):
+    o = bmu.Opts()
+    o.kernel = 5
+    for k, v in kw.items():
+        setattr(o, k, v)
+    return o
+
+
+def run_and_check(bmu, W, rowptr, colidx, opts, cancel_floor=False):
+    Wd, rp, ci = W.cuda(), rowptr.cuda(), colidx.cuda()
+    need = bmu.bmu_search_workspace_bytes(W.shape[0], W.shape[1], rowptr.numel() - 1,
+                                          colidx.numel(), opts)
+    ws = torch.empty(need + 256, dtype=torch.uint8, device="cuda")
+    ob, od = bmu.bmu_search_ws(Wd, rp, ci, opts=opts, workspace=ws)
+    torch.cuda.synchronize()
+    off = (-ws.data_ptr()) % 256
+    assert int(ws[off:off + 4].view(torch.int32)[0]) == 0, "a bounded device-side wait ran out"
+    return parity.compare(ob.cpu().numpy(), od.cpu().numpy(), W.numpy(), rowptr.numpy(),
+                          colidx.numpy(), cancel_floor=cancel_floor)
+
+
+@pytest.mark.parametrize("tile_order", [0, 1])
+@pytest.mark.parametrize("name,n_docs,M,chunk", [("cfg3", 2500, 2048, 1024), ("cfg5", 1203, 1536, 512),
+                                                 ("cfg1", 4001, 1024 + 36, 0), ("cfg2", 777, 512, 0)])
+def test_mma_kernel_matches_oracle(bmu, name, n_docs, M, chunk, tile_order):
+    cfg = synth.CONFIGS[name]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=n_docs)
+    for kind in ("uniform", "scaled"):
+        W = synth.make_codebook(cfg.D, M, 21, kind=kind)
+        res = run_and_check(bmu, W, rowptr, colidx,
+                            opts_of(bmu, tile_order=tile_order, chunk_neurons=chunk))
+        assert res["failed"] == 0 and res["docs"] == n_docs
+
+
+@pytest.mark.parametrize("kind,floor", [("dupes", False), ("const", False), ("sparse", False),
+                                        ("signed", False), ("prototype", True)])
+def test_mma_kernel_codebook_kinds(bmu, kind, floor):
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=1500)
+    W = synth.make_codebook(cfg.D, 1024, 83, kind=kind, docs=(rowptr, colidx))
+    run_and_check(bmu, W, rowptr, colidx, opts_of(bmu), cancel_floor=floor)
+    if kind in ("dupes", "const"):
+        ob, _ = bmu.bmu_search_ws(W.cuda(), rowptr.cuda(), colidx.cuda(), opts=opts_of(bmu))
+        if kind == "dupes":
+            assert int((ob % 2).sum()) == 0        # equal columns: the lower index wins
+        else:
+            assert int(ob.abs().sum()) == 0        # every neuron ties: index 0
+
+
+@pytest.mark.parametrize("scale", [1e-6, 1.0, 3e4, 1e9])
+def test_mma_kernel_weight_magnitudes(bmu, scale):
+    """The power-of-two scaling of the fp16 parts follows the largest head weight."""
+    cfg = synth.CONFIGS["cfg3"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=700)
+    W = synth.make_codebook(cfg.D, 512, 5, kind="signed") * scale
+    run_and_check(bmu, W, rowptr, colidx, opts_of(bmu))
+
+
+def test_mma_kernel_long_empty_unsorted_and_repeated_rows(bmu):
+    D, M = 16384, 1024
+    nnz = torch.tensor([400, 0, 1, 33, 0, 400, 97, 64, 32, 31, 0, 8, 16, 7, 9, 1500, 40] * 19)
+    rowptr, colidx = synth.draw_corpus(nnz.numel(), D, 1.1, nnz, seed=8)
+    ci = colidx.numpy().copy()
+    rp = rowptr.numpy()
+    r = np.random.default_rng(3)
+    for i in range(0, nnz.numel(), 2):
+        r.shuffle(ci[rp[i]:rp[i + 1]])
+    # a row that lists a frequent id twice keeps multiset semantics (added twice, counted twice)
+    ci[rp[3]:rp[3] + 2] = 5
+    # a row made of frequent ids only (no tail at all), one with a single frequent id
+    ci[rp[8]:rp[8 + 1]] = np.arange(32, dtype=np.int32) * 7
+    ci[rp[2]] = 255
+    W = synth.make_codebook(D, M, 11, kind="scaled")
+    run_and_check(bmu, W, rowptr, torch.from_numpy(ci), opts_of(bmu))
+
+
+def test_mma_kernel_unlabelled_vocabulary(bmu):
+    """Feature ids that are not frequency-ordered: still correct, only slower."""
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=900)
+    perm = torch.from_numpy(np.random.default_rng(1).permutation(cfg.D).astype(np.int32))
+    ci = perm[colidx.long()]
+    W = synth.make_codebook(cfg.D, 512, 9, kind="scaled")
+    run_and_check(bmu, W, rowptr, ci, opts_of(bmu))
+
+
+def test_mma_kernel_refuses_what_it_cannot_do(bmu):
+    rp = torch.tensor([0, 1], dtype=torch.int32).cuda()
+    ci = torch.tensor([0], dtype=torch.int32).cuda()
+    for D, M in ((128, 1024), (512, 256)):
+        with pytest.raises(bmu.BmuError) as e:
+            bmu.bmu_search_ws(torch.zeros(D, M, device="cuda"), rp, ci, opts=opts_of(bmu))
+        assert e.value.status == 2
