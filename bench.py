@@ -246,7 +246,9 @@ def run_ours(args, cfg, rank, local_rank, world):
     # launch geometry of the sweep (mirrors the library's defaults; reported, not used by it)
     kernel = opts.kernel
     if kernel == 0:                     # the library's automatic choice
-        kernel = 4 if (float(max_nnz) * cfg.M >= 2e10 and cfg.M >= 128) else 3
+        big = float(max_nnz) * cfg.M >= 2e10
+        kernel = (5 if (big and cfg.M >= 512 and cfg.D >= 256) else 4 if (big and cfg.M >= 128)
+                  else 3)
     vec = opts.vec or (4 if kernel == 1 else 8)
     slab = 32 * vec
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
@@ -255,12 +257,16 @@ def run_ours(args, cfg, rank, local_rank, world):
     n_chunks = (cfg.M + chunk - 1) // chunk
     # documents that share one SM's L1 at a time: resident warps x documents per warp
     kernel_name = {3: "sweep_rows_kernel", 1: "sweep_direct_kernel", 2: "sweep_lanes_kernel",
-                   4: "sweep_tiles_kernel"}[kernel]
+                   4: "sweep_tiles_kernel", 5: "sweep_mma_kernel"}[kernel]
     if kernel == 4:
         vec, slab = 4, 128
         chunk = opts.chunk_neurons or max(slab, (l2_bytes // 2) // (cfg.D * 4) // slab * slab)
         chunk = min((chunk + slab - 1) // slab * slab, (cfg.M + slab - 1) // slab * slab)
         n_chunks = (cfg.M + chunk - 1) // chunk
+    if kernel == 5:
+        vec, slab = 4, 512
+        chunk = min((opts.chunk_neurons or 8192) // slab * slab or slab, cfg.M // slab * slab)
+        n_chunks = (cfg.M // slab * slab + chunk - 1) // chunk
     if kernel == 2:
         docs_per_block, chunk = 992, (opts.chunk_neurons or
                                       max(32, (l2_bytes // 2) // (cfg.D * 4) // 32 * 32))
@@ -269,6 +275,8 @@ def run_ours(args, cfg, rank, local_rank, world):
         docs_per_block = 8 * (opts.warps or 4) * 5
     elif kernel == 1:
         docs_per_block = (opts.warps or 16) * (opts.docs_per_warp or 4) * 2
+    elif kernel == 5:
+        docs_per_block = 128
     else:
         docs_per_block = 48
 
@@ -352,7 +360,7 @@ def run_ours(args, cfg, rank, local_rank, world):
     launch_s = sweep_ms * 1e-3 / (n_chunks * len(batches))
     nnz = total_nnz / len(batches)                              # mean batch
     N = n_docs / len(batches)
-    adds = float(nnz) * chunk                                   # one fp32 add per (nnz, neuron)
+    adds = float(nnz) * chunk                                   # one update per (nnz, neuron)
     union_rows = union_rows_per_block(rowptr, colidx, cfg.D, docs_per_block) * (
         nnz / max(1, colidx.numel()))
     alg = {
@@ -362,6 +370,24 @@ def run_ours(args, cfg, rank, local_rank, world):
         "hbm": ((4.0 * cfg.D * chunk + 4.0 * nnz + 24.0 * N) / launch_s,
                 peaks["hbm_gbs"] * 1e9, "B/s"),
     }
+    extra = {}
+    if kernel == 5:
+        # the frequent features' updates are MMAs, not loads and adds: only the tail's updates
+        # pass through L1 and the fp32 pipe.  The L2 figure stays the algorithmic one (each
+        # block of 128 documents fetches every distinct row it touches once); what the design
+        # really moves is the tail's rows per document plus the head image per block.
+        head = opts.head_rows or 256
+        tail_share = float((colidx >= head).sum().item()) / max(1, colidx.numel())
+        alg["alu"] = (tail_share * adds / launch_s, roofs["fadd2"], "add/s")
+        alg["l1"] = (4.0 * tail_share * adds / launch_s, roofs["smem"], "B/s")
+        moved = 4.0 * chunk * (tail_share * nnz + head * (N / 128.0))
+        mma_flops = 2.0 * 2.0 * head * N * chunk        # hi and lo parts, 2 flops per MAC
+        extra = {"tail_share_of_updates": tail_share,
+                 "l2_bytes_moved_by_design_GBs": moved / launch_s / 1e9,
+                 "l2_moved_frac_of_roof": moved / launch_s / roofs["l2_ldg"],
+                 "head_mma_TFLOPs": mma_flops / launch_s / 1e12,
+                 "head_mma_frac_of_bf16_peak": mma_flops / launch_s / 1e12 /
+                 peaks.get("bf16_tflops_sustained", peaks.get("bf16_tflops", 1590.0))}
     bound = max(alg, key=lambda k: alg[k][0] / alg[k][1])
     ach, peak, unit = alg[bound]
     scale = 1e9
@@ -377,6 +403,7 @@ def run_ours(args, cfg, rank, local_rank, world):
         "launch_ms": launch_s * 1e3, "launches_per_step": n_chunks,
         "units_per_launch": {"adds": adds, "union_rows_x_chunk": float(union_rows) * chunk},
         "fractions": {k: v[0] / v[1] for k, v in alg.items()},
+        **extra,
         "peaks": {"hbm_GBs": peaks["hbm_gbs"], "hbm_source": "MEASURED_PEAKS.json (%s)" % peaks_kind,
                   "l2_GBs": roofs["l2_ldg"] / 1e9, "l1_smem_GBs": roofs["smem"] / 1e9,
                   "fp32_Gadds": roofs["fadd2"] / 1e9,
@@ -398,7 +425,7 @@ def run_ours(args, cfg, rank, local_rank, world):
                         "with the search of the current one)" % len(batches)) +
                        " (codebook resident in HBM; CSR from pinned host memory; results back "
                        "to host)", "matches_device_path": same},
-        "gpu_launches": args.steps * (1 + len(batches) * ({1: 0, 2: 6, 3: 6, 4: 8}[kernel]
+        "gpu_launches": args.steps * (1 + len(batches) * ({1: 0, 2: 6, 3: 6, 4: 8, 5: 10}[kernel]
                                                            + n_chunks + 1)),
         "roofline": roofline,
     }

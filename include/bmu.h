@@ -90,7 +90,9 @@ typedef struct bmu_opts {
                                frequent and the rare half of the lists, 1 ascending ids */
     int32_t tile_head;      /* tiled kernel: 0 sweep the 32 most frequent features (ids < 32)
                                densely, one load per tile, 1 treat them like all other ids */
-    int32_t reserved[6];    /* must be 0 */
+    int32_t head_rows;      /* tensor-core sweep: how many of the most frequent features (ids
+                               below this) are summed by the tensor cores, 256 or 512 */
+    int32_t reserved[5];    /* must be 0 */
 } bmu_opts;
 
 BMU_API const char *bmu_status_string(int status);

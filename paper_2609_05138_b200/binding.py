@@ -33,7 +33,7 @@ class Opts(ctypes.Structure):
                 ("warps", ctypes.c_int32), ("cluster", ctypes.c_int32),
                 ("stage_rows", ctypes.c_int32), ("stages", ctypes.c_int32),
                 ("tile_order", ctypes.c_int32), ("tile_head", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 6)]
+                ("head_rows", ctypes.c_int32), ("reserved", ctypes.c_int32 * 5)]
 
 
 EXPORTS = {

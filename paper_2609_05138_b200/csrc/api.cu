@@ -44,8 +44,16 @@ static bool staged_possible(const float *W, int64_t D, int64_t M)
            (reinterpret_cast<uintptr_t>(W) & 15) == 0;
 }
 
+// Neurons per launch of the tensor-core sweep.  Its blocks all carry the same amount of work
+// and walk the slabs of a launch in the same order, so the rows in use at any moment are those
+// of a few slabs, which L2 holds; a launch therefore spans many slabs (measured flat from
+// 4096 to 65536 neurons at D = 16384, best at 8192) and the blocks' set-up is paid less often.
+static const int64_t MMA_AUTO_CHUNK = 8192;
+
+static int mma_head_rows(const bmu_opts &o) { return o.head_rows ? o.head_rows : MMA_HEAD; }
+
 static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kernel,
-                         bool top2 = false)
+                         bool top2 = false, int head = MMA_HEAD)
 {
     Layout l;
     size_t off = 0;
@@ -56,8 +64,8 @@ static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kerne
     if (top2) off = align_up(off + (size_t)N * sizeof(u64), 256);
     // split image of the frequent rows for the tensor-core sweep (it may be the automatic choice)
     l.head_off = off;
-    if ((kernel == 0 || kernel == 5) && !top2 && D >= MMA_HEAD && D <= LANES_MAX_D && M >= MMA_SLAB)
-        off = align_up(off + head_image_bytes(M), 256);
+    if ((kernel == 0 || kernel == 5) && !top2 && D >= head && D <= LANES_MAX_D && M >= MMA_SLAB)
+        off = align_up(off + head_image_bytes(M, head), 256);
     l.plan_off = off;
     memset(&l.plan, 0, sizeof(l.plan));
     if (kernel != 1 && D <= LANES_MAX_D) off += plan_bytes(N, nnz, &l.plan);
@@ -83,7 +91,8 @@ static int check_opts(const bmu_opts &o)
 {
     if (o.tile_order < 0 || o.tile_order > 1) { set_error("bmu_opts.tile_order must be 0 or 1"); return BMU_ERR_INVALID_ARG; }
     if (o.tile_head < 0 || o.tile_head > 1) { set_error("bmu_opts.tile_head must be 0 or 1"); return BMU_ERR_INVALID_ARG; }
-    for (int i = 0; i < 6; ++i)
+    if (o.head_rows != 0 && o.head_rows != 256 && o.head_rows != 512) { set_error("bmu_opts.head_rows must be 0, 256 or 512"); return BMU_ERR_INVALID_ARG; }
+    for (int i = 0; i < 5; ++i)
         if (o.reserved[i] != 0) { set_error("bmu_opts.reserved must be zero"); return BMU_ERR_INVALID_ARG; }
     if (o.kernel < 0 || o.kernel > 5) { set_error("bmu_opts.kernel must be 0 .. 5"); return BMU_ERR_INVALID_ARG; }
     if (o.cluster < 0 || o.cluster > 2) { set_error("bmu_opts.cluster must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
@@ -131,7 +140,8 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         set_error("empty codebook (D=%lld, M=%lld): no neuron to return", (long long)D, (long long)M);
         return BMU_ERR_INVALID_ARG;
     }
-    const Layout l = layout_for(D, M, N, nnz, o.kernel, top2);
+    const int head = mma_head_rows(o);
+    const Layout l = layout_for(D, M, N, nnz, o.kernel, top2, head);
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < l.total) {
         set_error("workspace missing, not 256-byte aligned, or smaller than %zu bytes", l.total);
         return BMU_ERR_WORKSPACE;
@@ -164,19 +174,19 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
                   LANES_MAX_D);
         return BMU_ERR_UNSUPPORTED;
     }
-    // automatic choice: the tiled kernel once the sweep is large enough to repay its extra
-    // tiling work (a few more small kernels), the planned kernel below that
     const bool tiled_ok = planned_ok && M >= 128 && o.cluster != 2;
     // tensor-core head: additionally whole 512-neuron slabs, at least 256 features, best unit only
-    const bool mma_ok = tiled_ok && !top2 && D >= MMA_HEAD && M >= MMA_SLAB;
+    const bool mma_ok = tiled_ok && !top2 && D >= head && M >= MMA_SLAB;
     if (o.kernel == 5 && !mma_ok) {
         set_error("tensor-core sweep needs what the tiled kernel needs, D >= %d, M >= %d and no "
-                  "second-best unit", MMA_HEAD, MMA_SLAB);
+                  "second-best unit", head, MMA_SLAB);
         return BMU_ERR_UNSUPPORTED;
     }
-    const bool mma = o.kernel == 5;
-    const bool tiled = !mma && (o.kernel == 4 ||
-                       (o.kernel == 0 && tiled_ok && (double)nnz * (double)M >= 2e10));
+    // automatic choice for large sweeps: the tensor-core sweep where it applies, else the tiled
+    // kernel; both repay their extra preparation only when there is enough to sweep
+    const bool big = (double)nnz * (double)M >= 2e10;
+    const bool mma = o.kernel == 5 || (o.kernel == 0 && mma_ok && big);
+    const bool tiled = !mma && (o.kernel == 4 || (o.kernel == 0 && tiled_ok && big));
     if (tiled && !tiled_ok) {
         set_error("tiled kernel needs M %% 4 == 0, M >= 128, D <= %d, W 16-byte aligned and "
                   "length-ordered documents (cluster != 2)", LANES_MAX_D);
@@ -190,8 +200,8 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         const int64_t m_full = M / MMA_SLAB * MMA_SLAB;
         uint32_t *head_max = status + 16;
         unsigned char *img = reinterpret_cast<unsigned char *>(base + l.head_off);
-        if ((rc = launch_head_split(W, M, m_full, head_max, img, s))) return rc;
-        if ((rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, MMA_HEAD, pw, l.plan, s))) return rc;
+        if ((rc = launch_head_split(W, M, m_full, head, head_max, img, s))) return rc;
+        if ((rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, pw, l.plan, s))) return rc;
         MmaArgs a;
         a.W = W; a.M = M; a.N = N; a.n_tiles = (N + 7) / 8; a.norms = norms;
         a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
@@ -199,15 +209,15 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         a.tile_off = reinterpret_cast<const uint32_t *>(pw + l.plan.tileoff_off);
         a.tile_ids = reinterpret_cast<const uint4 *>(pw + l.plan.tileids_off);
         a.tile_head = reinterpret_cast<const uint32_t *>(pw + l.plan.tilehead_off);
-        a.head_max = head_max;
+        a.head_max = head_max; a.head = head;
         a.state = state; a.status = status;
         const int64_t chunk = o.chunk_neurons ? (o.chunk_neurons + MMA_SLAB - 1) / MMA_SLAB * MMA_SLAB
-                                              : auto_chunk(D, M, MMA_SLAB);
+                                              : MMA_AUTO_CHUNK;
         for (int64_t j = 0; j < m_full; j += chunk) {
             a.j_lo = (int32_t)j;
             a.j_hi = (int32_t)(j + chunk < m_full ? j + chunk : m_full);
             a.first = j == 0;
-            a.head_img = img + (size_t)(j / MMA_SLAB) * MMA_STAGES_PER_SLAB * MMA_STAGE_BYTES;
+            a.head_img = img + (size_t)(j / MMA_SLAB) * mma_stages_per_slab(head) * MMA_STAGE_BYTES;
             if ((rc = launch_sweep_mma(a, o, s))) return rc;
         }
         if (m_full < M) {                      // ragged last slab: generic kernel, merged in
@@ -406,7 +416,8 @@ size_t bmu_search_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,
                                   const bmu_opts *opts)
 {
     if (D < 0 || M < 0 || N < 0 || nnz < 0) return 0;
-    return layout_for(D, M, N, nnz, opts ? opts->kernel : 0).total;
+    return layout_for(D, M, N, nnz, opts ? opts->kernel : 0, false,
+                      opts && opts->head_rows == 512 ? 512 : MMA_HEAD).total;
 }
 
 int bmu_search_ws(const float *W, int64_t D, int64_t M, const float *norms,

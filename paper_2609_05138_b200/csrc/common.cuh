@@ -157,7 +157,7 @@ struct PlanLayout {
     size_t tilelen_off, tilerows_off, tileoff_off, tilehead_off, tileids_off, tile_rows_cap;
 };
 static const int TILE_HEAD_ROWS = 32;    // ids below this are swept densely, once per tile
-static const int HEAD_ROWS_MAX = 256;    // widest dense head (the tensor-core sweep's)
+static const int HEAD_ROWS_MAX = 512;    // widest dense head (the tensor-core sweep's)
 int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head, char *ws,
                       const PlanLayout &l, cudaStream_t s);
 
@@ -180,11 +180,13 @@ int launch_sweep_tiles(const TileArgs &a, const bmu_opts &o, cudaStream_t s);
 
 // tensor-core head + gathered tail (sweep_mma.cu): a block carries 128 documents through
 // slabs of 512 neurons
-static const int MMA_HEAD = 256;         // features (ids below this) summed on the tensor cores
+static const int MMA_HEAD = 256;         // features (ids below this) summed on the tensor cores:
+static const int MMA_HEAD_MAX = 512;     // 256 by default, 512 on request (bmu_opts.head_rows)
 static const int MMA_SLAB = 512;         // neurons per slab
 static const int MMA_DOCS = 128;         // documents per block
 static const size_t MMA_STAGE_BYTES = 16384;                  // 128 neurons x 64 features x fp16
-static const int MMA_STAGES_PER_SLAB = 4 * 2 * (MMA_HEAD / 64);   // 4 tiles x (hi, lo) x K blocks
+// stages per slab: 4 tiles x (hi, lo) x blocks of 64 features
+static inline int mma_stages_per_slab(int head) { return 4 * 2 * (head / 64); }
 struct MmaArgs {
     const float *W;
     int64_t M, N, n_tiles;
@@ -193,17 +195,18 @@ struct MmaArgs {
     const uint32_t *tile_len;
     const uint32_t *tile_off;
     const uint4 *tile_ids;
-    const uint32_t *tile_head;  // MMA_HEAD / 32 mask words per planned document
+    int32_t head;               // 256 or 512
+    const uint32_t *tile_head;  // head / 32 mask words per planned document
     const unsigned char *head_img;  // split head of slab j_lo / MMA_SLAB onwards (head_image_bytes)
     const uint32_t *head_max;   // bit pattern of max |W[f][j]| over the head rows
     u64 *state;
     uint32_t *status;           // set non-zero if a bounded wait ran out
     int32_t j_lo, j_hi, first;
 };
-size_t head_image_bytes(int64_t M);
-// writes the fp16 (hi, lo) split of rows [0, MMA_HEAD) of W, scaled by a power of two, as the
+size_t head_image_bytes(int64_t M, int head);
+// writes the fp16 (hi, lo) split of rows [0, head) of W, scaled by a power of two, as the
 // shared-memory images the tensor-core sweep copies; whole slabs of [0, m_full) only
-int launch_head_split(const float *W, int64_t M, int64_t m_full, uint32_t *head_max,
+int launch_head_split(const float *W, int64_t M, int64_t m_full, int head, uint32_t *head_max,
                       unsigned char *head_img, cudaStream_t s);
 int launch_sweep_mma(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
 size_t plan_bytes(int64_t N, int64_t nnz, PlanLayout *l);

@@ -128,30 +128,30 @@ plan_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__
 }
 
 // ---- tiles of 8 documents -------------------------------------------------
-// The ids below `head` (a multiple of 32, at most 256) at the front of a document's
+// The ids below `head` (a multiple of 32, at most HEAD_ROWS_MAX) at the front of a document's
 // ascending list, as a bit mask of head / 32 words, and how many list entries that
 // covers.  A list that repeats one of them keeps multiset semantics by opting out
 // (mask 0, nothing skipped): its ids all stay in the list.
 __device__ __forceinline__ void head_of_doc(const uint16_t *ids, uint32_t len, uint32_t head,
-                                            uint32_t mask[8], uint32_t &skip)
+                                            uint32_t mask[HEAD_ROWS_MAX / 32], uint32_t &skip)
 {
 #pragma unroll
-    for (int w = 0; w < 8; ++w) mask[w] = 0;
+    for (int w = 0; w < HEAD_ROWS_MAX / 32; ++w) mask[w] = 0;
     skip = 0;
     for (uint32_t e = 0; e < len && e <= head; ++e) {
         const uint32_t f = ids[e];
         if (f >= head) break;
 #pragma unroll
-        for (int w = 0; w < 8; ++w)
+        for (int w = 0; w < HEAD_ROWS_MAX / 32; ++w)
             if ((f >> 5) == (uint32_t)w) mask[w] |= 1u << (f & 31u);
         ++skip;
     }
     uint32_t bits = 0;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) bits += (uint32_t)__popc(mask[w]);
+    for (int w = 0; w < HEAD_ROWS_MAX / 32; ++w) bits += (uint32_t)__popc(mask[w]);
     if (skip != bits) {
 #pragma unroll
-        for (int w = 0; w < 8; ++w) mask[w] = 0;
+        for (int w = 0; w < HEAD_ROWS_MAX / 32; ++w) mask[w] = 0;
         skip = 0;
     }
 }
@@ -171,14 +171,14 @@ __global__ void plan_tile_len_kernel(const int32_t *__restrict__ rowptr,
     uint32_t mx = 0, mn = 0xffffu;
     for (int t = 0; t < 8; ++t) {
         const int64_t p = tile * 8 + t;
-        uint32_t len = 0, skip = 0, mask[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        uint32_t len = 0, skip = 0, mask[HEAD_ROWS_MAX / 32] = {};
         if (p < N) {
             const int32_t i = perm[p];
             len = (uint32_t)min(rowptr[i + 1] - rowptr[i], 65535);
             if (head) head_of_doc(ids16 + ((size_t)doc_off[p] + 1) * 8, len, head, mask, skip);
         }
 #pragma unroll
-        for (int w = 0; w < 8; ++w)
+        for (int w = 0; w < HEAD_ROWS_MAX / 32; ++w)
             if ((uint32_t)w < words) tile_head[(tile * 8 + t) * words + w] = mask[w];
         mx = max(mx, len - skip);
         mn = min(mn, len - skip);

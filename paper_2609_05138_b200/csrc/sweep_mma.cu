@@ -6,10 +6,10 @@
 // features is dense enough (about one entry in six) to be a real contraction.
 // So the sum over a document's features is cut in two:
 //
-//   s_ij = sum_{f in x_i, f <  256} W[f][j]      head: binary X_head x W_head on
+//   s_ij = sum_{f in x_i, f <  H} W[f][j]        head: binary X_head x W_head on
 //                                                tcgen05 tensor cores, fp32
 //                                                accumulators in tensor memory
-//        + sum_{f in x_i, f >= 256} W[f][j]      tail: gathered rows, as in the
+//        + sum_{f in x_i, f >= H} W[f][j]        tail: gathered rows, as in the
 //                                                tiled sweep
 //
 // A block carries 128 length-ordered documents through slabs of 512 neurons.
@@ -40,9 +40,11 @@ static const uint32_t MMA_WAIT_LIMIT = 1u << 22;
 static const int MMA_TAIL_WARPS = MMA_DOCS / 8;      // 16
 static const int MMA_THREADS = (MMA_TAIL_WARPS + 2) * 32;
 static const int MMA_TMEM_COLS = 4 * MMA_DOCS;       // 512: four accumulator tiles
-static const size_t MMA_XS_BYTES = (size_t)MMA_DOCS * MMA_HEAD * 2;
-static const size_t MMA_SMEM_BYTES = MMA_XS_BYTES + MMA_NS * MMA_STAGE_BYTES +
-                                     (2 * MMA_NS + 3) * 8 + MMA_DOCS * 8 + 16;
+static inline size_t mma_smem_bytes(int head)
+{
+    return (size_t)MMA_DOCS * head * 2 + MMA_NS * MMA_STAGE_BYTES + (2 * MMA_NS + 3) * 8 +
+           MMA_DOCS * 8 + 16;
+}
 
 // power of two that brings the largest head weight just below 2^15 (fp16 range)
 __host__ __device__ __forceinline__ float head_scale(uint32_t max_bits)
@@ -61,9 +63,9 @@ __host__ __device__ __forceinline__ float head_scale(uint32_t max_bits)
 }
 
 __global__ void head_absmax_kernel(const float *__restrict__ W, int64_t M, int64_t m_full,
-                                   uint32_t *__restrict__ out)
+                                   int head, uint32_t *__restrict__ out)
 {
-    const int64_t n4 = m_full / 4, total = n4 * MMA_HEAD;
+    const int64_t n4 = m_full / 4, total = n4 * head;
     uint32_t mx = 0;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (int64_t)gridDim.x * blockDim.x) {
@@ -84,9 +86,10 @@ __global__ void head_absmax_kernel(const float *__restrict__ W, int64_t M, int64
 // (hi, lo), block of 64 features; inside a stage the core matrix of (8 rows, 8 features)
 // lies at (row / 8) * 1024 + (feature / 8) * 128.
 __global__ void __launch_bounds__(MMA_SLAB)
-head_split_kernel(const float *__restrict__ W, int64_t M, const uint32_t *__restrict__ head_max,
-                  unsigned char *__restrict__ img)
+head_split_kernel(const float *__restrict__ W, int64_t M, int head,
+                  const uint32_t *__restrict__ head_max, unsigned char *__restrict__ img)
 {
+    const int KB = head / 64, SPS = 8 * KB;
     const int sl = blockIdx.x, kcg = blockIdx.y, jin = threadIdx.x;
     const float S = head_scale(*head_max);
     const float *src = W + (int64_t)(kcg * 8) * M + (int64_t)sl * MMA_SLAB + jin;
@@ -101,25 +104,25 @@ head_split_kernel(const float *__restrict__ W, int64_t M, const uint32_t *__rest
     const int c = jin & 3, r = ((jin >> 7) << 5) | ((jin >> 2) & 31);
     const int kb = kcg >> 3, kc = kcg & 7;
     const size_t off = (size_t)(r >> 3) * 1024 + (size_t)kc * 128 + (size_t)(r & 7) * 16;
-    const size_t st_hi = (size_t)sl * MMA_STAGES_PER_SLAB + (size_t)(c * 2 + 0) * (MMA_HEAD / 64) + kb;
-    const size_t st_lo = (size_t)sl * MMA_STAGES_PER_SLAB + (size_t)(c * 2 + 1) * (MMA_HEAD / 64) + kb;
+    const size_t st_hi = (size_t)sl * SPS + (size_t)(c * 2 + 0) * KB + kb;
+    const size_t st_lo = (size_t)sl * SPS + (size_t)(c * 2 + 1) * KB + kb;
     *reinterpret_cast<uint4 *>(img + st_hi * MMA_STAGE_BYTES + off) = *reinterpret_cast<uint4 *>(hi);
     *reinterpret_cast<uint4 *>(img + st_lo * MMA_STAGE_BYTES + off) = *reinterpret_cast<uint4 *>(lo);
 }
 
-size_t head_image_bytes(int64_t M)
+size_t head_image_bytes(int64_t M, int head)
 {
-    return (size_t)(M / MMA_SLAB) * MMA_STAGES_PER_SLAB * MMA_STAGE_BYTES;
+    return (size_t)(M / MMA_SLAB) * mma_stages_per_slab(head) * MMA_STAGE_BYTES;
 }
 
-int launch_head_split(const float *W, int64_t M, int64_t m_full, uint32_t *head_max,
+int launch_head_split(const float *W, int64_t M, int64_t m_full, int head, uint32_t *head_max,
                       unsigned char *head_img, cudaStream_t s)
 {
     if (m_full <= 0) return BMU_OK;
     BMU_CUDA(cudaMemsetAsync(head_max, 0, sizeof(uint32_t), s));
-    head_absmax_kernel<<<592, 256, 0, s>>>(W, M, m_full, head_max);
-    const dim3 grid((unsigned)(m_full / MMA_SLAB), MMA_HEAD / 8);
-    head_split_kernel<<<grid, MMA_SLAB, 0, s>>>(W, M, head_max, head_img);
+    head_absmax_kernel<<<592, 256, 0, s>>>(W, M, m_full, head, head_max);
+    const dim3 grid((unsigned)(m_full / MMA_SLAB), head / 8);
+    head_split_kernel<<<grid, MMA_SLAB, 0, s>>>(W, M, head, head_max, head_img);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
@@ -211,10 +214,10 @@ sweep_mma_kernel(const MmaArgs a)
     constexpr int T = 8;
     constexpr int NS = MMA_NS;
     constexpr int NTW = MMA_TAIL_WARPS;
-    constexpr int SPS = MMA_STAGES_PER_SLAB;
+    const int H = a.head, KB = H / 64, SPS = 8 * KB;           // stages per slab
     extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char *xs = smem;                                   // X_head image, 128 docs x 256
-    unsigned char *ring = smem + MMA_XS_BYTES;                  // NS stages of W_head
+    unsigned char *xs = smem;                                   // X_head image, 128 docs x H
+    unsigned char *ring = smem + (size_t)MMA_DOCS * H * 2;      // NS stages of W_head
     u64 *bars = reinterpret_cast<u64 *>(ring + NS * MMA_STAGE_BYTES);
     u64 *keys = bars + 2 * NS + 3;                              // running minimum per document
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(keys + MMA_DOCS);
@@ -249,20 +252,20 @@ sweep_mma_kernel(const MmaArgs a)
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     // X_head of this block's documents as fp16 zeros and ones: document n, features 8*kc .. +7
-    // at (n / 8) * 4096 + kc * 128 + (n % 8) * 16
-    for (int idx = threadIdx.x; idx < MMA_DOCS * (MMA_HEAD / 8); idx += MMA_THREADS) {
+    // at (n / 8) * (H * 16) + kc * 128 + (n % 8) * 16
+    for (int idx = threadIdx.x; idx < MMA_DOCS * (H / 8); idx += MMA_THREADS) {
         const int n = idx & (MMA_DOCS - 1), kc = idx / MMA_DOCS;
         const int64_t tile = group * (MMA_DOCS / T) + (n >> 3);
         uint32_t bits = 0;
         if (tile < a.n_tiles)
-            bits = (__ldg(a.tile_head + (group * MMA_DOCS + n) * (MMA_HEAD / 32) + (kc >> 2)) >>
+            bits = (__ldg(a.tile_head + (group * MMA_DOCS + n) * (H / 32) + (kc >> 2)) >>
                     ((kc & 3) * 8)) & 0xffu;
         uint4 v;
         v.x = ((bits & 1u) ? 0x3c00u : 0u) | ((bits & 2u) ? 0x3c000000u : 0u);
         v.y = ((bits & 4u) ? 0x3c00u : 0u) | ((bits & 8u) ? 0x3c000000u : 0u);
         v.z = ((bits & 16u) ? 0x3c00u : 0u) | ((bits & 32u) ? 0x3c000000u : 0u);
         v.w = ((bits & 64u) ? 0x3c00u : 0u) | ((bits & 128u) ? 0x3c000000u : 0u);
-        *reinterpret_cast<uint4 *>(xs + (size_t)(n >> 3) * 4096 + (size_t)kc * 128 + (n & 7) * 16) = v;
+        *reinterpret_cast<uint4 *>(xs + (size_t)(n >> 3) * (H * 16) + (size_t)kc * 128 + (n & 7) * 16) = v;
     }
     if (threadIdx.x < MMA_DOCS) keys[threadIdx.x] = KEY_WORST;
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -311,12 +314,12 @@ sweep_mma_kernel(const MmaArgs a)
                         break;
                     }
                     mm_fence_after();
-                    const int tile_c = i >> 3, kb = i & 3;      // i = (tile * 2 + part) * 4 + kb
+                    const int tile_c = i / (2 * KB), kb = i % KB; // i = (tile * 2 + part) * KB + kb
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         const u64 ad = mm_desc(ring_u32 + slot * (uint32_t)MMA_STAGE_BYTES + u * 256, 128, 1024);
-                        const u64 bd = mm_desc(xs_u32 + (kb * 8 + 2 * u) * 128, 128, 4096);
-                        mm_mma(tmem + tile_c * MMA_DOCS, ad, bd, idesc, ((i & 7) | u) != 0);
+                        const u64 bd = mm_desc(xs_u32 + (kb * 8 + 2 * u) * 128, 128, (uint32_t)H * 16);
+                        mm_mma(tmem + tile_c * MMA_DOCS, ad, bd, idesc, ((i % (2 * KB)) | u) != 0);
                     }
                     mm_commit(empty0 + 8 * slot);                // stage free once these MMAs are done
                 }
@@ -458,16 +461,20 @@ int launch_sweep_mma(const MmaArgs &a, const bmu_opts &o, cudaStream_t s)
         set_error("tensor-core sweep handles whole %d-neuron slabs only", MMA_SLAB);
         return BMU_ERR_INVALID_ARG;
     }
+    if (a.head != 256 && a.head != 512) {
+        set_error("tensor-core sweep: head_rows must be 256 or 512");
+        return BMU_ERR_INVALID_ARG;
+    }
     static bool configured[64];
     int dev = 0;
     BMU_CUDA(cudaGetDevice(&dev));
     if (dev >= 0 && dev < 64 && !configured[dev]) {
         BMU_CUDA(cudaFuncSetAttribute(sweep_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)MMA_SMEM_BYTES));
+                                      (int)mma_smem_bytes(MMA_HEAD_MAX)));
         configured[dev] = true;
     }
     const unsigned blocks = (unsigned)((a.N + MMA_DOCS - 1) / MMA_DOCS);
-    sweep_mma_kernel<<<blocks, MMA_THREADS, MMA_SMEM_BYTES, s>>>(a);
+    sweep_mma_kernel<<<blocks, MMA_THREADS, mma_smem_bytes(a.head), s>>>(a);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

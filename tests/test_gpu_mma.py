@@ -45,16 +45,17 @@ def run_and_check(bmu, W, rowptr, colidx, opts, cancel_floor=False):
                           colidx.numpy(), cancel_floor=cancel_floor)
 
 
-@pytest.mark.parametrize("tile_order", [0, 1])
+@pytest.mark.parametrize("tile_order,head_rows", [(0, 0), (1, 256), (0, 512)])
 @pytest.mark.parametrize("name,n_docs,M,chunk", [("cfg3", 2500, 2048, 1024), ("cfg5", 1203, 1536, 512),
                                                  ("cfg1", 4001, 1024 + 36, 0), ("cfg2", 777, 512, 0)])
-def test_mma_kernel_matches_oracle(bmu, name, n_docs, M, chunk, tile_order):
+def test_mma_kernel_matches_oracle(bmu, name, n_docs, M, chunk, tile_order, head_rows):
     cfg = synth.CONFIGS[name]
     rowptr, colidx = synth.make_corpus(cfg, n_docs=n_docs)
     for kind in ("uniform", "scaled"):
         W = synth.make_codebook(cfg.D, M, 21, kind=kind)
         res = run_and_check(bmu, W, rowptr, colidx,
-                            opts_of(bmu, tile_order=tile_order, chunk_neurons=chunk))
+                            opts_of(bmu, tile_order=tile_order, chunk_neurons=chunk,
+                                    head_rows=head_rows))
         assert res["failed"] == 0 and res["docs"] == n_docs
 
 
@@ -98,6 +99,7 @@ def test_mma_kernel_long_empty_unsorted_and_repeated_rows(bmu):
     ci[rp[2]] = 255
     W = synth.make_codebook(D, M, 11, kind="scaled")
     run_and_check(bmu, W, rowptr, torch.from_numpy(ci), opts_of(bmu))
+    run_and_check(bmu, W, rowptr, torch.from_numpy(ci), opts_of(bmu, head_rows=512))
 
 
 def test_mma_kernel_unlabelled_vocabulary(bmu):
