@@ -265,7 +265,8 @@ def run_ours(args, cfg, rank, local_rank, world):
         n_chunks = (cfg.M + chunk - 1) // chunk
     if kernel == 5:
         vec, slab = 4, 512
-        chunk = min((opts.chunk_neurons or 8192) // slab * slab or slab, cfg.M // slab * slab)
+        chunk = opts.chunk_neurons or max(slab, int(l2_bytes * 0.55) // (cfg.D * 4) // slab * slab)
+        chunk = min((chunk + slab - 1) // slab * slab, cfg.M // slab * slab)
         n_chunks = (cfg.M // slab * slab + chunk - 1) // chunk
     if kernel == 2:
         docs_per_block, chunk = 992, (opts.chunk_neurons or

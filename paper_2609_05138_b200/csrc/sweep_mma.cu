@@ -35,7 +35,10 @@
 
 namespace bmu {
 
-static const int MMA_NS = 4;                         // ring stages
+#ifndef BMU_MMA_STAGES
+#define BMU_MMA_STAGES 4
+#endif
+static const int MMA_NS = BMU_MMA_STAGES;            // ring stages
 static const uint32_t MMA_WAIT_LIMIT = 1u << 22;
 static const int MMA_TAIL_WARPS = MMA_DOCS / 8;      // 16
 static const int MMA_THREADS = (MMA_TAIL_WARPS + 2) * 32;
@@ -338,11 +341,51 @@ sweep_mma_kernel(const MmaArgs a)
         const int mydoc = mm_doc_of_lane(lane);
         for (int sl = 0; sl < n_slabs; ++sl) {
             const int j0 = a.j_lo + sl * MMA_SLAB + q * 128;
-            mm_wait(tmem_full, sl & 1, abort_flag, a.status, 8u);
-            mm_fence_after();
             for (int it = 0; it < NTW / 4; ++it) {
                 const int o = g + 4 * it;                        // the block's o-th tile of 8
                 const int64_t tile = group * (MMA_DOCS / T) + o;
+                const bool live = tile < a.n_tiles;
+                u64 acc[T][2];
+#pragma unroll
+                for (int t = 0; t < T; ++t) acc[t][0] = acc[t][1] = 0ull;
+                if (live) {
+                    const uint32_t tl = __ldg(a.tile_len + tile);
+                    const uint32_t rows = tl & 0xffffu, full = tl >> 16;
+                    const uint4 *gp = a.tile_ids + __ldg(a.tile_off + tile);
+                    const char *base = reinterpret_cast<const char *>(a.W + j0 + lane * 4);
+                    uint32_t b = 0;
+                    uint4 qn = __ldg(gp);
+                    for (; b < full; ++b) {
+                        const uint4 qq = qn;
+                        qn = __ldg(gp + b + 1);
+                        const uint32_t f[T] = {qq.x & 0xffffu, qq.x >> 16, qq.y & 0xffffu, qq.y >> 16,
+                                               qq.z & 0xffffu, qq.z >> 16, qq.w & 0xffffu, qq.w >> 16};
+                        ulonglong2 w[T];
+    #pragma unroll
+                        for (int t = 0; t < T; ++t)
+                            w[t] = __ldg(reinterpret_cast<const ulonglong2 *>(base + (u64)f[t] * rowbytes));
+    #pragma unroll
+                        for (int t = 0; t < T; ++t) { add2(acc[t][0], w[t].x); add2(acc[t][1], w[t].y); }
+                    }
+                    for (; b < rows; ++b) {
+                        const uint4 qq = qn;
+                        qn = __ldg(gp + b + 1);
+                        const uint32_t f[T] = {qq.x & 0xffffu, qq.x >> 16, qq.y & 0xffffu, qq.y >> 16,
+                                               qq.z & 0xffffu, qq.z >> 16, qq.w & 0xffffu, qq.w >> 16};
+    #pragma unroll
+                        for (int t = 0; t < T; ++t)
+                            if (f[t] != 0xffffu) {
+                                const ulonglong2 w = __ldg(
+                                    reinterpret_cast<const ulonglong2 *>(base + (u64)f[t] * rowbytes));
+                                add2(acc[t][0], w.x);
+                                add2(acc[t][1], w.y);
+                            }
+                    }
+                }
+                // the head sums of these documents, from tensor memory: the MMAs of this slab ran
+                // while the tail was being gathered
+                if (it == 0) mm_wait(tmem_full, sl & 1, abort_flag, a.status, 8u);
+                mm_fence_after();
                 uint32_t hv[4][8];
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
@@ -353,46 +396,13 @@ sweep_mma_kernel(const MmaArgs a)
                     __syncwarp();
                     if (lane == 0) mm_bar_arrive(tmem_empty);
                 }
-                if (tile >= a.n_tiles) continue;
-                u64 acc[T][2];
+                if (!live) continue;
 #pragma unroll
                 for (int t = 0; t < T; ++t) {
                     const float s0 = __uint_as_float(hv[0][t]) * inv_s, s1 = __uint_as_float(hv[1][t]) * inv_s;
                     const float s2 = __uint_as_float(hv[2][t]) * inv_s, s3 = __uint_as_float(hv[3][t]) * inv_s;
-                    acc[t][0] = ((u64)__float_as_uint(s1) << 32) | __float_as_uint(s0);
-                    acc[t][1] = ((u64)__float_as_uint(s3) << 32) | __float_as_uint(s2);
-                }
-                const uint32_t tl = __ldg(a.tile_len + tile);
-                const uint32_t rows = tl & 0xffffu, full = tl >> 16;
-                const uint4 *gp = a.tile_ids + __ldg(a.tile_off + tile);
-                const char *base = reinterpret_cast<const char *>(a.W + j0 + lane * 4);
-                uint32_t b = 0;
-                uint4 qn = __ldg(gp);
-                for (; b < full; ++b) {
-                    const uint4 qq = qn;
-                    qn = __ldg(gp + b + 1);
-                    const uint32_t f[T] = {qq.x & 0xffffu, qq.x >> 16, qq.y & 0xffffu, qq.y >> 16,
-                                           qq.z & 0xffffu, qq.z >> 16, qq.w & 0xffffu, qq.w >> 16};
-                    ulonglong2 w[T];
-#pragma unroll
-                    for (int t = 0; t < T; ++t)
-                        w[t] = __ldg(reinterpret_cast<const ulonglong2 *>(base + (u64)f[t] * rowbytes));
-#pragma unroll
-                    for (int t = 0; t < T; ++t) { add2(acc[t][0], w[t].x); add2(acc[t][1], w[t].y); }
-                }
-                for (; b < rows; ++b) {
-                    const uint4 qq = qn;
-                    qn = __ldg(gp + b + 1);
-                    const uint32_t f[T] = {qq.x & 0xffffu, qq.x >> 16, qq.y & 0xffffu, qq.y >> 16,
-                                           qq.z & 0xffffu, qq.z >> 16, qq.w & 0xffffu, qq.w >> 16};
-#pragma unroll
-                    for (int t = 0; t < T; ++t)
-                        if (f[t] != 0xffffu) {
-                            const ulonglong2 w = __ldg(
-                                reinterpret_cast<const ulonglong2 *>(base + (u64)f[t] * rowbytes));
-                            add2(acc[t][0], w.x);
-                            add2(acc[t][1], w.y);
-                        }
+                    add2(acc[t][0], ((u64)__float_as_uint(s1) << 32) | __float_as_uint(s0));
+                    add2(acc[t][1], ((u64)__float_as_uint(s3) << 32) | __float_as_uint(s2));
                 }
                 // distances, then the transposing butterfly of the tiled sweep
                 const int col = j0 + lane * 4;
