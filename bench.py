@@ -32,7 +32,7 @@ if ROOT not in sys.path:
 from inputs import synth  # noqa: E402
 
 # DRAM bytes per sweep launch of the default config-4 run, from ncu (profiles/)
-TRAFFIC_CFG4 = {3: 2.0e9, 4: 2.9e9}
+TRAFFIC_CFG4 = {3: 2.0e9, 4: 2.9e9, 5: 4.9e9}
 
 METRIC = "bmu_search_docs_per_s"
 UNIT = "docs/s"
@@ -397,10 +397,11 @@ def run_ours(args, cfg, rank, local_rank, world):
         "achieved": ach / scale, "peak": peak / scale,
         "unit": "GB/s" if unit == "B/s" else "Gadd/s", "frac": ach / peak,
         # DRAM bytes per launch from the ncu capture of this very launch configuration
-        # (profiles/sweep_rows_cfg4_launch_list.md); other workloads were not captured
+        # (profiles/sweep_*_cfg4_launch_list.md); other workloads were not captured
         "traffic": (TRAFFIC_CFG4.get(kernel) if (cfg.name == "cfg4" and n_docs == cfg.N
                                                  and not opts.chunk_neurons and not opts.vec
-                                                 and not opts.warps) else None),
+                                                 and not opts.warps and not opts.head_rows)
+                    else None),
         "launch_ms": launch_s * 1e3, "launches_per_step": n_chunks,
         "units_per_launch": {"adds": adds, "union_rows_x_chunk": float(union_rows) * chunk},
         "fractions": {k: v[0] / v[1] for k, v in alg.items()},

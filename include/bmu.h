@@ -73,9 +73,15 @@ typedef struct bmu_opts {
                                4 tiled (a warp carries 8 documents; frequent rows loaded once
                                per tile; the warps of a block walk the feature axis in step
                                so that L1 serves the rows they share; needs what 3 needs and
-                               length-ordered documents); 2 staged (a lane per document, rows
-                               streamed through shared memory by tensor (TMA) box copies;
-                               needs M % 4 == 0, M >= 32, 256 <= D <= 65024) */
+                               length-ordered documents); 5 tensor-core head (the sum over the
+                               head_rows most frequent features -- ids below head_rows: the
+                               paper keeps its vocabulary frequency-ordered, Table 8 -- is a
+                               dense contraction on tcgen05 tensor cores with fp32
+                               accumulation, the remaining ids are gathered as in 4; needs
+                               what 4 needs, D >= head_rows and M >= 512; best unit only;
+                               the automatic choice for large sweeps); 2 staged (a lane per
+                               document, rows streamed through shared memory by tensor (TMA)
+                               box copies; needs M % 4 == 0, M >= 32, 256 <= D <= 65024) */
     int32_t chunk_neurons;  /* neurons per L2-resident chunk of the codebook (Section 4.2,
                                "neuron-axis chunking"); rounded to the slab width */
     int32_t vec;            /* warp-per-document kernels: floats per lane per row, 4 or 8 */
@@ -110,8 +116,9 @@ BMU_API int bmu_codebook_norms(const float *W, int64_t D, int64_t M, float *norm
 
 /*
  * Scratch bytes bmu_search_ws needs for a problem of this size (norms, the
- * per-document running minimum merged across neuron chunks, and the tiling
- * plan when the staged kernel is selected).  `nnz` is the length of colidx.
+ * per-document running minimum merged across neuron chunks, the tiling plan,
+ * and the split image of the frequent rows for the tensor-core sweep: M KiB at
+ * head_rows = 256).  `nnz` is the length of colidx.
  */
 BMU_API size_t bmu_search_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,
                                   const bmu_opts *opts);
@@ -124,7 +131,8 @@ BMU_API size_t bmu_search_workspace_bytes(int64_t D, int64_t M, int64_t N, int64
  * 256-byte aligned device memory of at least bmu_search_workspace_bytes(...)
  * bytes; its contents are undefined afterwards, except that its first 32-bit
  * word is a status word: 0 after a clean run, non-zero if a bounded device-side
- * wait of the staged kernel ran out (results are then invalid).  Allocates
+ * wait of the staged kernel or of the tensor-core sweep ran out (results are
+ * then invalid).  Allocates
  * nothing.  Calls that share a workspace must not overlap on the GPU.
  */
 BMU_API int bmu_search_ws(const float *W, int64_t D, int64_t M, const float *norms,
