@@ -59,7 +59,10 @@ static int64_t mma_auto_chunk(int64_t D, int64_t M)
     return c;
 }
 
-static int mma_head_rows(const bmu_opts &o) { return o.head_rows ? o.head_rows : MMA_HEAD; }
+static int mma_head_rows(const bmu_opts &o)
+{
+    return o.head_rows ? o.head_rows : (o.kernel == 6 ? 1024 : MMA_HEAD);
+}
 
 static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kernel,
                          bool top2 = false, int head = MMA_HEAD)
@@ -75,9 +78,11 @@ static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kerne
     l.head_off = off;
     if ((kernel == 0 || kernel == 5) && !top2 && D >= head && D <= LANES_MAX_D && M >= MMA_SLAB)
         off = align_up(off + head_image_bytes(M, head), 256);
+    if (kernel == 6 && !top2 && D >= head && D <= LANES_MAX_D && M >= MMA_SLAB)
+        off = align_up(off + head_image2_bytes(M, head), 256);
     l.plan_off = off;
     memset(&l.plan, 0, sizeof(l.plan));
-    if (kernel != 1 && D <= LANES_MAX_D) off += plan_bytes(N, nnz, &l.plan);
+    if (kernel != 1 && D <= LANES_MAX_D) off += plan_bytes(N, nnz, head, &l.plan);
     l.total = off;
     return l;
 }
@@ -100,10 +105,14 @@ static int check_opts(const bmu_opts &o)
 {
     if (o.tile_order < 0 || o.tile_order > 1) { set_error("bmu_opts.tile_order must be 0 or 1"); return BMU_ERR_INVALID_ARG; }
     if (o.tile_head < 0 || o.tile_head > 1) { set_error("bmu_opts.tile_head must be 0 or 1"); return BMU_ERR_INVALID_ARG; }
-    if (o.head_rows != 0 && o.head_rows != 256 && o.head_rows != 512) { set_error("bmu_opts.head_rows must be 0, 256 or 512"); return BMU_ERR_INVALID_ARG; }
+    if (o.head_rows < 0 || o.head_rows > HEAD_ROWS_MAX || o.head_rows % 64 != 0 ||
+        (o.kernel != 6 && o.head_rows != 0 && o.head_rows != 256 && o.head_rows != 512)) {
+        set_error("bmu_opts.head_rows must be 0, 256 or 512 (kernel 6: a multiple of 64 up to %d)", HEAD_ROWS_MAX);
+        return BMU_ERR_INVALID_ARG;
+    }
     for (int i = 0; i < 5; ++i)
         if (o.reserved[i] != 0) { set_error("bmu_opts.reserved must be zero"); return BMU_ERR_INVALID_ARG; }
-    if (o.kernel < 0 || o.kernel > 5) { set_error("bmu_opts.kernel must be 0 .. 5"); return BMU_ERR_INVALID_ARG; }
+    if (o.kernel < 0 || o.kernel > 6) { set_error("bmu_opts.kernel must be 0 .. 6"); return BMU_ERR_INVALID_ARG; }
     if (o.cluster < 0 || o.cluster > 2) { set_error("bmu_opts.cluster must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
     if (o.chunk_neurons < 0) { set_error("bmu_opts.chunk_neurons < 0"); return BMU_ERR_INVALID_ARG; }
     if (o.vec != 0 && o.vec != 4 && o.vec != 8) { set_error("bmu_opts.vec must be 0, 4 or 8"); return BMU_ERR_INVALID_ARG; }
@@ -186,7 +195,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     const bool tiled_ok = planned_ok && M >= 128 && o.cluster != 2;
     // tensor-core head: additionally whole 512-neuron slabs, at least 256 features, best unit only
     const bool mma_ok = tiled_ok && !top2 && D >= head && M >= MMA_SLAB;
-    if (o.kernel == 5 && !mma_ok) {
+    if ((o.kernel == 5 || o.kernel == 6) && !mma_ok) {
         set_error("tensor-core sweep needs what the tiled kernel needs, D >= %d, M >= %d and no "
                   "second-best unit", head, MMA_SLAB);
         return BMU_ERR_UNSUPPORTED;
@@ -194,7 +203,8 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     // automatic choice for large sweeps: the tensor-core sweep where it applies, else the tiled
     // kernel; both repay their extra preparation only when there is enough to sweep
     const bool big = (double)nnz * (double)M >= 2e10;
-    const bool mma = o.kernel == 5 || (o.kernel == 0 && mma_ok && big);
+    const bool mma = o.kernel == 5 || o.kernel == 6 || (o.kernel == 0 && mma_ok && big);
+    const bool wide = o.kernel == 6;
     const bool tiled = !mma && (o.kernel == 4 || (o.kernel == 0 && tiled_ok && big));
     if (tiled && !tiled_ok) {
         set_error("tiled kernel needs M %% 4 == 0, M >= 128, D <= %d, W 16-byte aligned and "
@@ -204,12 +214,14 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     const bool planned = !tiled && !mma && (o.kernel == 3 || (o.kernel == 0 && planned_ok));
     char *pw = base + l.plan_off;
     if (staged || planned || tiled || mma)
-        if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, pw, l.plan, s))) return rc;
+        if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, mma ? head : 0, pw, l.plan, s)))
+            return rc;
     if (mma) {
         const int64_t m_full = M / MMA_SLAB * MMA_SLAB;
         uint32_t *head_max = status + 16;
         unsigned char *img = reinterpret_cast<unsigned char *>(base + l.head_off);
-        if ((rc = launch_head_split(W, M, m_full, head, head_max, img, s))) return rc;
+        if ((rc = wide ? launch_head_split2(W, M, m_full, head, head_max, img, s)
+                       : launch_head_split(W, M, m_full, head, head_max, img, s))) return rc;
         if ((rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, pw, l.plan, s))) return rc;
         MmaArgs a;
         a.W = W; a.M = M; a.N = N; a.n_tiles = (N + 7) / 8; a.norms = norms;
@@ -226,8 +238,9 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
             a.j_lo = (int32_t)j;
             a.j_hi = (int32_t)(j + chunk < m_full ? j + chunk : m_full);
             a.first = j == 0;
-            a.head_img = img + (size_t)(j / MMA_SLAB) * mma_stages_per_slab(head) * MMA_STAGE_BYTES;
-            if ((rc = launch_sweep_mma(a, o, s))) return rc;
+            // both images take 4 * head bytes per neuron, slab after slab
+            a.head_img = img + (size_t)j * head * 4;
+            if ((rc = wide ? launch_sweep_mma2(a, o, s) : launch_sweep_mma(a, o, s))) return rc;
         }
         if (m_full < M) {                      // ragged last slab: generic kernel, merged in
             SweepArgs g;
@@ -425,8 +438,10 @@ size_t bmu_search_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,
                                   const bmu_opts *opts)
 {
     if (D < 0 || M < 0 || N < 0 || nnz < 0) return 0;
-    return layout_for(D, M, N, nnz, opts ? opts->kernel : 0, false,
-                      opts && opts->head_rows == 512 ? 512 : MMA_HEAD).total;
+    bmu_opts o;
+    memset(&o, 0, sizeof(o));
+    if (opts) o = *opts;
+    return layout_for(D, M, N, nnz, o.kernel, false, mma_head_rows(o)).total;
 }
 
 int bmu_search_ws(const float *W, int64_t D, int64_t M, const float *norms,
@@ -512,7 +527,7 @@ int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
     }
     BMU_CUDA(cudaMemsetAsync(base + l.status_off, 0, 256, s));
     char *pw = base + l.plan_off;
-    if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, pw, l.plan, s))) return rc;
+    if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, 0, pw, l.plan, s))) return rc;
     RowsArgs a;
     a.W = static_cast<const float *>(W16); a.M = M; a.N = N; a.norms = norms; a.rowptr = rowptr;
     a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);

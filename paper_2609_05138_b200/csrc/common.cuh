@@ -157,7 +157,7 @@ struct PlanLayout {
     size_t tilelen_off, tilerows_off, tileoff_off, tilehead_off, tileids_off, tile_rows_cap;
 };
 static const int TILE_HEAD_ROWS = 32;    // ids below this are swept densely, once per tile
-static const int HEAD_ROWS_MAX = 512;    // widest dense head (the tensor-core sweep's)
+static const int HEAD_ROWS_MAX = 1024;   // widest dense head (the tensor-core sweep's)
 int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head, char *ws,
                       const PlanLayout &l, cudaStream_t s);
 
@@ -209,9 +209,14 @@ size_t head_image_bytes(int64_t M, int head);
 int launch_head_split(const float *W, int64_t M, int64_t m_full, int head, uint32_t *head_max,
                       unsigned char *head_img, cudaStream_t s);
 int launch_sweep_mma(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
-size_t plan_bytes(int64_t N, int64_t nnz, PlanLayout *l);
+// wide-head variant (sweep_mma2.cu): 256-neuron slabs, head of 64 .. HEAD_ROWS_MAX features
+size_t head_image2_bytes(int64_t M, int head);
+int launch_head_split2(const float *W, int64_t M, int64_t m_full, int head, uint32_t *head_max,
+                       unsigned char *head_img, cudaStream_t s);
+int launch_sweep_mma2(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
+size_t plan_bytes(int64_t N, int64_t nnz, int head, PlanLayout *l);
 int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
-                int order_by_length, char *ws, const PlanLayout &l, cudaStream_t s);
+                int order_by_length, int head, char *ws, const PlanLayout &l, cudaStream_t s);
 
 static const int LANES_MAX_D = 65024;    // 16-bit ids with 0xFFFF as the end marker
 

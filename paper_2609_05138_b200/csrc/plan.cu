@@ -26,12 +26,30 @@ namespace bmu {
 static const int PLAN_BINS = 65536;      // one bin per row length: documents end up exactly
                                          // length-ordered (ids are 16-bit, so rows are shorter)
 
-__global__ void plan_hist_kernel(const int32_t *__restrict__ rowptr, int64_t N,
+// Sorting key of a document: how many of its ids the gather will visit, i.e. the ids at or
+// above `head` (all of them when head == 0).  One warp per document.
+__global__ void __launch_bounds__(256)
+plan_key_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colidx,
+                int64_t N, int32_t head, uint32_t *__restrict__ key)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (i >= N) return;
+    const int beg = rowptr[i], end = rowptr[i + 1];
+    int cnt = 0;
+    for (int e = beg + lane; e < end; e += 32) cnt += colidx[e] >= head;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
+    if (lane == 0) key[i] = (uint32_t)cnt;
+}
+
+__global__ void plan_hist_kernel(const int32_t *__restrict__ rowptr,
+                                 const uint32_t *__restrict__ key, int64_t N,
                                  uint32_t *__restrict__ hist)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
-    const int len = rowptr[i + 1] - rowptr[i];
+    const int len = key ? (int)key[i] : rowptr[i + 1] - rowptr[i];
     const int bin = PLAN_BINS - 1 - min(len, PLAN_BINS - 1);      // longest rows first
     atomicAdd(hist + bin, 1u);
 }
@@ -60,12 +78,13 @@ plan_scan_bins_kernel(const uint32_t *__restrict__ hist, uint32_t *__restrict__ 
     }
 }
 
-__global__ void plan_scatter_kernel(const int32_t *__restrict__ rowptr, int64_t N,
+__global__ void plan_scatter_kernel(const int32_t *__restrict__ rowptr,
+                                    const uint32_t *__restrict__ key, int64_t N,
                                     uint32_t *__restrict__ cursor, int32_t *__restrict__ perm)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
-    const int len = rowptr[i + 1] - rowptr[i];
+    const int len = key ? (int)key[i] : rowptr[i + 1] - rowptr[i];
     const int bin = PLAN_BINS - 1 - min(len, PLAN_BINS - 1);
     perm[atomicAdd(cursor + bin, 1u)] = (int32_t)i;
 }
@@ -129,31 +148,28 @@ plan_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__
 
 // ---- tiles of 8 documents -------------------------------------------------
 // The ids below `head` (a multiple of 32, at most HEAD_ROWS_MAX) at the front of a document's
-// ascending list, as a bit mask of head / 32 words, and how many list entries that
-// covers.  A list that repeats one of them keeps multiset semantics by opting out
-// (mask 0, nothing skipped): its ids all stay in the list.
-__device__ __forceinline__ void head_of_doc(const uint16_t *ids, uint32_t len, uint32_t head,
-                                            uint32_t mask[HEAD_ROWS_MAX / 32], uint32_t &skip)
+// ascending list, as a bit mask of head / 32 words written to `mask`, and how many list
+// entries that covers.  A list that repeats one of them keeps multiset semantics by opting
+// out (mask 0, nothing skipped): its ids all stay in the list.
+__device__ __forceinline__ uint32_t head_of_doc(const uint16_t *ids, uint32_t len, uint32_t head,
+                                                uint32_t *mask)
 {
-#pragma unroll
-    for (int w = 0; w < HEAD_ROWS_MAX / 32; ++w) mask[w] = 0;
-    skip = 0;
+    const uint32_t words = head / 32;
+    for (uint32_t w = 0; w < words; ++w) mask[w] = 0;
+    uint32_t skip = 0, bits = 0;
     for (uint32_t e = 0; e < len && e <= head; ++e) {
         const uint32_t f = ids[e];
         if (f >= head) break;
-#pragma unroll
-        for (int w = 0; w < HEAD_ROWS_MAX / 32; ++w)
-            if ((f >> 5) == (uint32_t)w) mask[w] |= 1u << (f & 31u);
+        const uint32_t old = mask[f >> 5], now = old | (1u << (f & 31u));
+        bits += now != old;
+        mask[f >> 5] = now;
         ++skip;
     }
-    uint32_t bits = 0;
-#pragma unroll
-    for (int w = 0; w < HEAD_ROWS_MAX / 32; ++w) bits += (uint32_t)__popc(mask[w]);
     if (skip != bits) {
-#pragma unroll
-        for (int w = 0; w < HEAD_ROWS_MAX / 32; ++w) mask[w] = 0;
+        for (uint32_t w = 0; w < words; ++w) mask[w] = 0;
         skip = 0;
     }
+    return skip;
 }
 
 // per tile: longest and shortest list behind the head (max | min << 16), and the head masks
@@ -171,15 +187,14 @@ __global__ void plan_tile_len_kernel(const int32_t *__restrict__ rowptr,
     uint32_t mx = 0, mn = 0xffffu;
     for (int t = 0; t < 8; ++t) {
         const int64_t p = tile * 8 + t;
-        uint32_t len = 0, skip = 0, mask[HEAD_ROWS_MAX / 32] = {};
+        uint32_t len = 0, skip = 0;
+        uint32_t *mask = tile_head + (size_t)(tile * 8 + t) * words;
+        for (uint32_t w = 0; w < words; ++w) mask[w] = 0;
         if (p < N) {
             const int32_t i = perm[p];
             len = (uint32_t)min(rowptr[i + 1] - rowptr[i], 65535);
-            if (head) head_of_doc(ids16 + ((size_t)doc_off[p] + 1) * 8, len, head, mask, skip);
+            if (head) skip = head_of_doc(ids16 + ((size_t)doc_off[p] + 1) * 8, len, head, mask);
         }
-#pragma unroll
-        for (int w = 0; w < HEAD_ROWS_MAX / 32; ++w)
-            if ((uint32_t)w < words) tile_head[(tile * 8 + t) * words + w] = mask[w];
         mx = max(mx, len - skip);
         mn = min(mn, len - skip);
     }
@@ -231,7 +246,7 @@ plan_tile_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restr
     }
 }
 
-size_t plan_bytes(int64_t N, int64_t nnz, PlanLayout *l)
+size_t plan_bytes(int64_t N, int64_t nnz, int head, PlanLayout *l)
 {
     auto up = [](size_t x) { return (x + 255) / 256 * 256; };
     size_t off = 0;
@@ -252,7 +267,7 @@ size_t plan_bytes(int64_t N, int64_t nnz, PlanLayout *l)
     t.tilelen_off = off; off = up(off + (n_tiles + 1) * 4);
     t.tilerows_off = off; off = up(off + (n_tiles + 1) * 4);
     t.tileoff_off = off; off = up(off + (n_tiles + 1) * 4);
-    t.tilehead_off = off; off = up(off + n_tiles * 8 * 4 * (HEAD_ROWS_MAX / 32));
+    t.tilehead_off = off; off = up(off + n_tiles * 8 * 4 * (size_t)(head > 32 ? head / 32 : 1));
     t.tile_rows_cap = (size_t)nnz / 8 + 65536 + n_tiles;
     t.tileids_off = off; off = up(off + t.tile_rows_cap * 16);
     t.total = off;
@@ -261,7 +276,7 @@ size_t plan_bytes(int64_t N, int64_t nnz, PlanLayout *l)
 }
 
 int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
-                int order_by_length, char *ws, const PlanLayout &l, cudaStream_t s)
+                int order_by_length, int head, char *ws, const PlanLayout &l, cudaStream_t s)
 {
     (void)nnz;
     int32_t *perm = reinterpret_cast<int32_t *>(ws + l.perm_off);
@@ -272,10 +287,19 @@ int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t
     uint16_t *ids16 = reinterpret_cast<uint16_t *>(ws + l.ids_off);
     const unsigned blocks = (unsigned)((N + 255) / 256);
     if (order_by_length) {
+        // with a dense head the documents are ordered by what is left for the gather, so that
+        // the documents of a tile finish their lists together (the key borrows the ngroups
+        // array, which is written only after the scatter)
+        const uint32_t *key = nullptr;
+        if (head > 0) {
+            plan_key_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(rowptr, colidx, N, head,
+                                                                            ngroups);
+            key = ngroups;
+        }
         BMU_CUDA(cudaMemsetAsync(hist, 0, PLAN_BINS * 4, s));
-        plan_hist_kernel<<<blocks, 256, 0, s>>>(rowptr, N, hist);
+        plan_hist_kernel<<<blocks, 256, 0, s>>>(rowptr, key, N, hist);
         plan_scan_bins_kernel<<<1, 1024, 0, s>>>(hist, cursor);
-        plan_scatter_kernel<<<blocks, 256, 0, s>>>(rowptr, N, cursor, perm);
+        plan_scatter_kernel<<<blocks, 256, 0, s>>>(rowptr, key, N, cursor, perm);
     } else {
         plan_identity_kernel<<<blocks, 256, 0, s>>>(N, perm);
     }

@@ -1,0 +1,412 @@
+// Tensor-core head + gathered tail, second cut: a wide head with double-buffered
+// tensor memory.
+//
+// Same split of the sum as sweep_mma.cu -- the H most frequent features on tcgen05
+// MMAs, the rest gathered -- re-cut so that the head can be much wider (up to 1024
+// features, which takes the features present in about one document in a hundred
+// and more away from the gather):
+//   * a slab is 256 neurons and has two accumulator tiles (tensor-memory lane
+//     32q + t of tile c = neuron 64q + 2t + c), so the head sums of a slab take
+//     half of tensor memory and the MMAs of slab s+1 fill one half while the tail
+//     of slab s is gathered against the other: the MMAs have a whole slab's time,
+//     not the gap between two slabs;
+//   * the K dimension is outermost: for every block of 64 features one warp
+//     expands the documents' mask bits into a 128 x 64 fp16 operand (a 16 KB stage
+//     of a small ring), used by the four W stages of that block (2 tiles x (hi,
+//     lo)); shared memory holds rings and 16 KB of masks instead of the whole
+//     X_head, so L1 keeps its size whatever H is;
+//   * a tail task is 16 documents x 64 neurons: a lane gathers four neurons for
+//     eight of the documents, so a load instruction still moves 512 bytes (two
+//     rows, one per half of the documents) and eight are in flight per warp.
+#include "common.cuh"
+#include "mma_ptx.cuh"
+
+#include <cuda_fp16.h>
+#include <math_constants.h>
+
+namespace bmu {
+
+static const int M2_SLAB = 256;
+static const int M2_NS = 4;                          // W ring stages
+static const int M2_NX = 3;                          // X ring stages
+static const int M2_TAIL_WARPS = 16;
+static const int M2_THREADS = (M2_TAIL_WARPS + 3) * 32;
+static const int M2_TMEM_COLS = 512;                 // 2 buffers x 2 tiles x 128 documents
+
+static inline size_t m2_smem_bytes(int head)
+{
+    return (size_t)MMA_DOCS * (head / 8) + (M2_NS + M2_NX) * MMA_STAGE_BYTES +
+           (2 * M2_NS + 2 * M2_NX + 5) * 8 + MMA_DOCS * 8 + 16;
+}
+
+// One thread per (slab, group of 8 features, neuron).  Stage order inside a slab: block of
+// 64 features, tile c (neuron % 2), part (hi, lo).
+__global__ void __launch_bounds__(M2_SLAB)
+head_split2_kernel(const float *__restrict__ W, int64_t M, const uint32_t *__restrict__ head_max,
+                   int head, unsigned char *__restrict__ img)
+{
+    const int sl = blockIdx.x, kcg = blockIdx.y, jin = threadIdx.x;
+    const int SPS = 4 * (head / 64);
+    const float S = head_scale(*head_max);
+    const float *src = W + (int64_t)(kcg * 8) * M + (int64_t)sl * M2_SLAB + jin;
+    __align__(16) __half hi[8];
+    __align__(16) __half lo[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const float w = __ldg(src + (int64_t)e * M) * S;
+        hi[e] = __float2half_rn(w);
+        lo[e] = __float2half_rn(w - __half2float(hi[e]));
+    }
+    const int c = jin & 1, r = ((jin >> 6) << 5) | ((jin >> 1) & 31);
+    const int kb = kcg >> 3, kc = kcg & 7;
+    const size_t off = (size_t)(r >> 3) * 1024 + (size_t)kc * 128 + (size_t)(r & 7) * 16;
+    const size_t st = (size_t)sl * SPS + (size_t)(kb * 2 + c) * 2;
+    *reinterpret_cast<uint4 *>(img + st * MMA_STAGE_BYTES + off) = *reinterpret_cast<uint4 *>(hi);
+    *reinterpret_cast<uint4 *>(img + (st + 1) * MMA_STAGE_BYTES + off) = *reinterpret_cast<uint4 *>(lo);
+}
+
+__global__ void head_absmax2_kernel(const float *__restrict__ W, int64_t M, int64_t m_full,
+                                    int head, uint32_t *__restrict__ out)
+{
+    const int64_t n4 = m_full / 4, total = n4 * head;
+    uint32_t mx = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t f = i / n4, c = i - f * n4;
+        const float4 v = __ldg(reinterpret_cast<const float4 *>(W + f * M) + c);
+        mx = max(mx, __float_as_uint(fabsf(v.x)));
+        mx = max(mx, __float_as_uint(fabsf(v.y)));
+        mx = max(mx, __float_as_uint(fabsf(v.z)));
+        mx = max(mx, __float_as_uint(fabsf(v.w)));
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    if ((threadIdx.x & 31) == 0 && mx) atomicMax(out, mx);
+}
+
+size_t head_image2_bytes(int64_t M, int head)
+{
+    return (size_t)(M / M2_SLAB) * 4 * (head / 64) * MMA_STAGE_BYTES;
+}
+
+int launch_head_split2(const float *W, int64_t M, int64_t m_full, int head, uint32_t *head_max,
+                       unsigned char *head_img, cudaStream_t s)
+{
+    if (m_full <= 0) return BMU_OK;
+    BMU_CUDA(cudaMemsetAsync(head_max, 0, sizeof(uint32_t), s));
+    head_absmax2_kernel<<<592, 256, 0, s>>>(W, M, m_full, head, head_max);
+    const dim3 grid((unsigned)(m_full / M2_SLAB), head / 8);
+    head_split2_kernel<<<grid, M2_SLAB, 0, s>>>(W, M, head_max, head, head_img);
+    BMU_CUDA(cudaGetLastError());
+    return BMU_OK;
+}
+
+__device__ __forceinline__ void m2_unpack(const uint4 q, uint32_t f[8])
+{
+    f[0] = q.x & 0xffffu; f[1] = q.x >> 16; f[2] = q.y & 0xffffu; f[3] = q.y >> 16;
+    f[4] = q.z & 0xffffu; f[5] = q.z >> 16; f[6] = q.w & 0xffffu; f[7] = q.w >> 16;
+}
+
+__global__ void __launch_bounds__(M2_THREADS, 1)
+sweep_mma2_kernel(const MmaArgs a)
+{
+    constexpr int NS = M2_NS, NX = M2_NX, NTW = M2_TAIL_WARPS;
+    const int H = a.head, KB = H / 64;
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char *masks = smem;                                 // 128 documents x H bits
+    unsigned char *xring = smem + (size_t)MMA_DOCS * (H / 8);    // NX stages of X_head
+    unsigned char *wring = xring + NX * MMA_STAGE_BYTES;         // NS stages of W_head
+    u64 *bars = reinterpret_cast<u64 *>(wring + NS * MMA_STAGE_BYTES);
+    u64 *keys = bars + 2 * NS + 2 * NX + 5;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(keys + MMA_DOCS);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+    uint32_t *skip_flag = tmem_slot + 2;
+    const uint32_t wfull0 = mm_smem(bars), wempty0 = mm_smem(bars + NS);
+    const uint32_t xfull0 = mm_smem(bars + 2 * NS), xempty0 = mm_smem(bars + 2 * NS + NX);
+    const uint32_t tfull0 = mm_smem(bars + 2 * NS + 2 * NX), tempty0 = tfull0 + 16;
+    const uint32_t drain = tfull0 + 32;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t group = blockIdx.x;
+    const int n_slabs = (a.j_hi - a.j_lo) / M2_SLAB;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < NS; ++i) { mm_bar_init(wfull0 + 8 * i, 1); mm_bar_init(wempty0 + 8 * i, 1); }
+        for (int i = 0; i < NX; ++i) { mm_bar_init(xfull0 + 8 * i, 1); mm_bar_init(xempty0 + 8 * i, 1); }
+        for (int i = 0; i < 2; ++i) { mm_bar_init(tfull0 + 8 * i, 1); mm_bar_init(tempty0 + 8 * i, NTW); }
+        mm_bar_init(drain, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        *abort_flag = 0u;
+        *skip_flag = *reinterpret_cast<volatile uint32_t *>(a.status);
+    }
+    __syncthreads();
+    if (*skip_flag) return;          // a block before this one gave up: let the grid drain
+
+    if (warp == NTW) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(mm_smem(tmem_slot)), "r"((uint32_t)M2_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    {   // the block's head masks into shared memory (document-major, H / 8 bytes each)
+        const int words = H / 32;
+        uint32_t *mw = reinterpret_cast<uint32_t *>(masks);
+        for (int idx = threadIdx.x; idx < MMA_DOCS * words; idx += M2_THREADS) {
+            const int n = idx / words;
+            const int64_t tile = group * (MMA_DOCS / 8) + (n >> 3);
+            mw[idx] = tile < a.n_tiles ? __ldg(a.tile_head + (size_t)group * MMA_DOCS * words + idx) : 0u;
+        }
+    }
+    if (threadIdx.x < MMA_DOCS) keys[threadIdx.x] = KEY_WORST;
+    mm_fence_before();
+    __syncthreads();
+    mm_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == NTW) {
+        // ---------------- producer: W stages of every slab, in order
+        if (lane == 0) {
+            const unsigned char *src = a.head_img;
+            const int total = n_slabs * 4 * KB;
+            int issued = 0;
+            for (int c = 0; c < total; ++c) {
+                const int slot = c % NS;
+                if (c >= NS && !mm_wait(wempty0 + 8 * slot, ((c / NS) - 1) & 1, abort_flag, a.status, 1u))
+                    break;
+                mm_bar_expect_tx(wfull0 + 8 * slot, (uint32_t)MMA_STAGE_BYTES);
+                mm_bulk_load(mm_smem(wring + (size_t)slot * MMA_STAGE_BYTES),
+                             src + (size_t)c * MMA_STAGE_BYTES, (uint32_t)MMA_STAGE_BYTES,
+                             wfull0 + 8 * slot);
+                issued = c + 1;
+            }
+            if (*abort_flag)         // gave up: let the copies in flight land before leaving
+                for (int c = issued > NS ? issued - NS : 0; c < issued; ++c)
+                    for (uint32_t spin = 0; spin < MMA_WAIT_LIMIT; ++spin)
+                        if (mm_bar_try(wfull0 + 8 * (c % NS), (c / NS) & 1)) break;
+        }
+        __syncwarp();
+    } else if (warp == NTW + 1) {
+        // ---------------- expander: X_head, one block of 64 features per stage
+        const int total = n_slabs * KB;
+        for (int x = 0; x < total; ++x) {
+            const int slot = x % NX, kb = x % KB;
+            if (x >= NX && !mm_wait(xempty0 + 8 * slot, ((x / NX) - 1) & 1, abort_flag, a.status, 16u))
+                break;
+            unsigned char *dst = xring + (size_t)slot * MMA_STAGE_BYTES;
+#ifndef M2_DEBUG_NOEXPAND
+            for (int idx = lane; idx < MMA_DOCS * 8; idx += 32) {
+                const int n = idx & (MMA_DOCS - 1), kc = idx >> 7;
+                const uint32_t bits = masks[(size_t)n * (H / 8) + kb * 8 + kc];
+                uint4 v;
+                v.x = ((bits & 1u) ? 0x3c00u : 0u) | ((bits & 2u) ? 0x3c000000u : 0u);
+                v.y = ((bits & 4u) ? 0x3c00u : 0u) | ((bits & 8u) ? 0x3c000000u : 0u);
+                v.z = ((bits & 16u) ? 0x3c00u : 0u) | ((bits & 32u) ? 0x3c000000u : 0u);
+                v.w = ((bits & 64u) ? 0x3c00u : 0u) | ((bits & 128u) ? 0x3c000000u : 0u);
+                *reinterpret_cast<uint4 *>(dst + (size_t)(n >> 3) * 1024 + kc * 128 + (n & 7) * 16) = v;
+            }
+#endif
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mm_bar_arrive(xfull0 + 8 * slot);
+        }
+        __syncwarp();
+    } else if (warp == NTW + 2) {
+        // ---------------- one thread issues every MMA
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | ((uint32_t)(MMA_DOCS >> 3) << 17) | (8u << 24);
+            const uint32_t wring_u32 = mm_smem(wring), xring_u32 = mm_smem(xring);
+            bool ok = true;
+            int wc = 0, xc = 0;
+            for (int sl = 0; sl < n_slabs && ok; ++sl) {
+                const int buf = sl & 1;
+                if (sl >= 2) ok = mm_wait(tempty0 + 8 * buf, ((sl >> 1) - 1) & 1, abort_flag, a.status, 2u);
+                if (!ok) break;
+                mm_fence_after();
+                for (int kb = 0; kb < KB && ok; ++kb, ++xc) {
+                    const int xslot = xc % NX;
+                    if (!mm_wait(xfull0 + 8 * xslot, (xc / NX) & 1, abort_flag, a.status, 32u)) { ok = false; break; }
+                    for (int cp = 0; cp < 4; ++cp, ++wc) {       // cp = tile * 2 + part
+                        const int slot = wc % NS;
+                        if (!mm_wait(wfull0 + 8 * slot, (wc / NS) & 1, abort_flag, a.status, 4u)) { ok = false; break; }
+                        mm_fence_after();
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const u64 ad = mm_desc(wring_u32 + slot * (uint32_t)MMA_STAGE_BYTES + u * 256, 128, 1024);
+                            const u64 bd = mm_desc(xring_u32 + xslot * (uint32_t)MMA_STAGE_BYTES + u * 256, 128, 1024);
+                            mm_mma(tmem + buf * 256 + (cp >> 1) * MMA_DOCS, ad, bd, idesc,
+                                   (kb | (cp & 1) | u) != 0);
+                        }
+                        mm_commit(wempty0 + 8 * slot);
+                    }
+                    if (ok) mm_commit(xempty0 + 8 * xslot);
+                }
+                if (ok) mm_commit(tfull0 + 8 * buf);
+            }
+            mm_commit(drain);
+            for (uint32_t spin = 0; spin < MMA_WAIT_LIMIT; ++spin)
+                if (mm_bar_try(drain, 0)) break;
+        }
+        __syncwarp();
+    } else {
+        // ---------------- tail: 16 documents x 64 neurons per task.  Lane (i, h) = (lane / 2,
+        // lane % 2) gathers neurons 4i .. 4i+3 for the documents 8h .. 8h+7 of the task: one
+        // 128-bit load per lane and row, two rows (one per half of the documents) per instruction.
+        const int q = warp & 3, g = warp >> 2;
+        const int li = lane >> 1, lh = lane & 1;
+        const float inv_s = 1.f / head_scale(__ldg(a.head_max));
+        const uint32_t rowbytes = (uint32_t)(a.M * 4);
+        const int mydoc = 8 * lh + (((lane >> 1) & 1) << 2 | ((lane >> 2) & 1) << 1 | ((lane >> 3) & 1));
+        for (int sl = 0; sl < n_slabs; ++sl) {
+            const int buf = sl & 1;
+            const int j0 = a.j_lo + sl * M2_SLAB + q * 64;
+            for (int it = 0; it < 2; ++it) {
+                const int dg = g + 4 * it;                       // the block's dg-th set of 16
+                const int64_t tile_a = group * (MMA_DOCS / 8) + 2 * dg, tile_b = tile_a + 1;
+                const bool live = tile_a < a.n_tiles;
+                u64 acc[8][2];
+#pragma unroll
+                for (int t = 0; t < 8; ++t) acc[t][0] = acc[t][1] = 0ull;
+                if (live) {
+                    const bool has_b = tile_b < a.n_tiles;
+                    const uint32_t tla = __ldg(a.tile_len + tile_a);
+                    const uint32_t tlb = has_b ? __ldg(a.tile_len + tile_b) : 0u;
+                    const uint32_t full = min(tla >> 16, tlb >> 16);
+                    const uint32_t rows = max(tla & 0xffffu, tlb & 0xffffu);
+                    const uint32_t my_rows = (lh ? tlb : tla) & 0xffffu;
+                    const uint4 *gp = (lh && has_b) ? a.tile_ids + __ldg(a.tile_off + tile_b)
+                                                    : a.tile_ids + __ldg(a.tile_off + tile_a);
+                    const char *base = reinterpret_cast<const char *>(a.W + j0 + li * 4);
+                    uint32_t b = 0;
+                    uint4 qn = __ldg(gp);
+                    for (; b < full; ++b) {
+                        uint32_t f[8];
+                        m2_unpack(qn, f);
+                        qn = __ldg(gp + b + 1);
+                        ulonglong2 w[8];
+#pragma unroll
+                        for (int t = 0; t < 8; ++t)
+                            w[t] = __ldg(reinterpret_cast<const ulonglong2 *>(base + (u64)f[t] * rowbytes));
+#pragma unroll
+                        for (int t = 0; t < 8; ++t) { add2(acc[t][0], w[t].x); add2(acc[t][1], w[t].y); }
+                    }
+                    for (; b < rows; ++b) {                      // some documents have run out
+                        uint32_t f[8];
+                        m2_unpack(qn, f);
+                        qn = __ldg(gp + b + 1);
+                        const bool in = b < my_rows;
+                        ulonglong2 w[8];
+#pragma unroll
+                        for (int t = 0; t < 8; ++t)
+                            w[t] = (in && f[t] != 0xffffu)
+                                       ? __ldg(reinterpret_cast<const ulonglong2 *>(base + (u64)f[t] * rowbytes))
+                                       : make_ulonglong2(0ull, 0ull);
+#pragma unroll
+                        for (int t = 0; t < 8; ++t) { add2(acc[t][0], w[t].x); add2(acc[t][1], w[t].y); }
+                    }
+                }
+                // head sums of these documents: the MMAs of this slab ran during the gather.
+                // Tensor-memory lane 32q + lane holds neurons 4i + 2h, 4i + 2h + 1 for all 16
+                // documents; the two lanes of a pair swap halves so that each ends up with four
+                // neurons of its own eight documents.
+#ifndef M2_DEBUG_NOWAIT
+                if (it == 0) mm_wait(tfull0 + 8 * buf, (sl >> 1) & 1, abort_flag, a.status, 8u);
+#endif
+                mm_fence_after();
+                uint32_t h0[16], h1[16];
+                const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 256 + dg * 16);
+                mm_tmem_ld16(taddr, h0);
+                mm_tmem_ld16(taddr + MMA_DOCS, h1);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (it == 1) {                                   // this half of tensor memory is free
+                    mm_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mm_bar_arrive(tempty0 + 8 * buf);
+                }
+                if (!live) continue;
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    const uint32_t mine0 = lh ? h0[8 + t] : h0[t], mine1 = lh ? h1[8 + t] : h1[t];
+                    const uint32_t send0 = lh ? h0[t] : h0[8 + t], send1 = lh ? h1[t] : h1[8 + t];
+                    const uint32_t got0 = __shfl_xor_sync(0xffffffffu, send0, 1);
+                    const uint32_t got1 = __shfl_xor_sync(0xffffffffu, send1, 1);
+                    const float s0 = __uint_as_float(lh ? got0 : mine0) * inv_s;
+                    const float s1 = __uint_as_float(lh ? got1 : mine1) * inv_s;
+                    const float s2 = __uint_as_float(lh ? mine0 : got0) * inv_s;
+                    const float s3 = __uint_as_float(lh ? mine1 : got1) * inv_s;
+                    add2(acc[t][0], ((u64)__float_as_uint(s1) << 32) | __float_as_uint(s0));
+                    add2(acc[t][1], ((u64)__float_as_uint(s3) << 32) | __float_as_uint(s2));
+                }
+                const int col = j0 + li * 4;
+                const float4 n = __ldg(reinterpret_cast<const float4 *>(a.norms + col));
+                const float n4[4] = {n.x, n.y, n.z, n.w};
+                u64 k[8];
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    const float s4[4] = {lo_f(acc[t][0]), hi_f(acc[t][0]), lo_f(acc[t][1]), hi_f(acc[t][1])};
+                    Best<false> bst;
+                    bst.init();
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) bst.push(fmaf(-2.f, s4[c], n4[c]), col + c);
+                    k[t] = make_key(bst.d1, bst.j1);
+                }
+                // transposing butterfly among the 16 lanes that hold the same documents
+#pragma unroll
+                for (int st = 0; st < 3; ++st) {
+                    const int m = 2 << st, cnt = 4 >> st;
+#pragma unroll
+                    for (int i = 0; i < cnt; ++i) {
+                        const u64 send = (lane & m) ? k[i] : k[i + cnt];
+                        const u64 keep = (lane & m) ? k[i + cnt] : k[i];
+                        const u64 got = __shfl_xor_sync(0xffffffffu, send, m);
+                        k[i] = got < keep ? got : keep;
+                    }
+                }
+                const u64 got = __shfl_xor_sync(0xffffffffu, k[0], 16);
+                k[0] = got < k[0] ? got : k[0];
+                if (lane < 16) atomicMin(reinterpret_cast<unsigned long long *>(keys + dg * 16 + mydoc), k[0]);
+            }
+        }
+        __syncwarp();
+    }
+
+    mm_fence_before();
+    __syncthreads();
+    mm_fence_after();
+    if (threadIdx.x < MMA_DOCS) {
+        const int64_t p = group * MMA_DOCS + threadIdx.x;
+        if (p < a.N) {
+            const int32_t orig = __ldg(a.perm + p);
+            Best<false>::commit(keys[threadIdx.x], KEY_WORST, a.state, nullptr, orig, a.first);
+        }
+    }
+    if (warp == NTW)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                     ::"r"(tmem), "r"((uint32_t)M2_TMEM_COLS) : "memory");
+}
+
+int launch_sweep_mma2(const MmaArgs &a, const bmu_opts &o, cudaStream_t s)
+{
+    (void)o;
+    if (a.N == 0 || a.j_lo >= a.j_hi) return BMU_OK;
+    if ((a.j_hi - a.j_lo) % M2_SLAB != 0 || a.j_lo % M2_SLAB != 0) {
+        set_error("wide-head sweep handles whole %d-neuron slabs only", M2_SLAB);
+        return BMU_ERR_INVALID_ARG;
+    }
+    if (a.head < 64 || a.head > HEAD_ROWS_MAX || a.head % 64 != 0) {
+        set_error("wide-head sweep: head_rows must be a multiple of 64 up to %d", HEAD_ROWS_MAX);
+        return BMU_ERR_INVALID_ARG;
+    }
+    static bool configured[64];
+    int dev = 0;
+    BMU_CUDA(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        BMU_CUDA(cudaFuncSetAttribute(sweep_mma2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)m2_smem_bytes(HEAD_ROWS_MAX)));
+        configured[dev] = true;
+    }
+    const unsigned blocks = (unsigned)((a.N + MMA_DOCS - 1) / MMA_DOCS);
+    sweep_mma2_kernel<<<blocks, M2_THREADS, m2_smem_bytes(a.head), s>>>(a);
+    BMU_CUDA(cudaGetLastError());
+    return BMU_OK;
+}
+
+}  // namespace bmu
