@@ -247,7 +247,7 @@ def run_ours(args, cfg, rank, local_rank, world):
     kernel = opts.kernel
     if kernel == 0:                     # the library's automatic choice
         big = float(max_nnz) * cfg.M >= 2e10
-        kernel = (5 if (big and cfg.M >= 512 and cfg.D >= 256) else 4 if (big and cfg.M >= 128)
+        kernel = (6 if (big and cfg.M >= 512 and cfg.D >= 64) else 4 if (big and cfg.M >= 128)
                   else 3)
     vec = opts.vec or (4 if kernel == 1 else 8)
     slab = 32 * vec
@@ -257,13 +257,13 @@ def run_ours(args, cfg, rank, local_rank, world):
     n_chunks = (cfg.M + chunk - 1) // chunk
     # documents that share one SM's L1 at a time: resident warps x documents per warp
     kernel_name = {3: "sweep_rows_kernel", 1: "sweep_direct_kernel", 2: "sweep_lanes_kernel",
-                   4: "sweep_tiles_kernel", 5: "sweep_mma_kernel"}[kernel]
+                   4: "sweep_tiles_kernel", 5: "sweep_mma_kernel", 6: "sweep_mma2_kernel"}[kernel]
     if kernel == 4:
         vec, slab = 4, 128
         chunk = opts.chunk_neurons or max(slab, (l2_bytes // 2) // (cfg.D * 4) // slab * slab)
         chunk = min((chunk + slab - 1) // slab * slab, (cfg.M + slab - 1) // slab * slab)
         n_chunks = (cfg.M + chunk - 1) // chunk
-    if kernel == 5:
+    if kernel in (5, 6):
         vec, slab = 4, 512
         chunk = opts.chunk_neurons or max(slab, int(l2_bytes * 0.55) // (cfg.D * 4) // slab * slab)
         chunk = min((chunk + slab - 1) // slab * slab, cfg.M // slab * slab)
@@ -276,7 +276,7 @@ def run_ours(args, cfg, rank, local_rank, world):
         docs_per_block = 8 * (opts.warps or 4) * 5
     elif kernel == 1:
         docs_per_block = (opts.warps or 16) * (opts.docs_per_warp or 4) * 2
-    elif kernel == 5:
+    elif kernel in (5, 6):
         docs_per_block = 128
     else:
         docs_per_block = 48
@@ -372,12 +372,12 @@ def run_ours(args, cfg, rank, local_rank, world):
                 peaks["hbm_gbs"] * 1e9, "B/s"),
     }
     extra = {}
-    if kernel == 5:
+    if kernel in (5, 6):
         # the frequent features' updates are MMAs, not loads and adds: only the tail's updates
         # pass through L1 and the fp32 pipe.  The L2 figure stays the algorithmic one (each
         # block of 128 documents fetches every distinct row it touches once); what the design
         # really moves is the tail's rows per document plus the head image per block.
-        head = opts.head_rows or 256
+        head = opts.head_rows or (256 if kernel == 5 else min(768, cfg.D // 64 * 64))
         tail_share = float((colidx >= head).sum().item()) / max(1, colidx.numel())
         alg["alu"] = (tail_share * adds / launch_s, roofs["fadd2"], "add/s")
         alg["l1"] = (4.0 * tail_share * adds / launch_s, roofs["smem"], "B/s")
@@ -427,8 +427,11 @@ def run_ours(args, cfg, rank, local_rank, world):
                         "with the search of the current one)" % len(batches)) +
                        " (codebook resident in HBM; CSR from pinned host memory; results back "
                        "to host)", "matches_device_path": same},
-        "gpu_launches": args.steps * (1 + len(batches) * ({1: 0, 2: 6, 3: 6, 4: 8, 5: 10}[kernel]
-                                                           + n_chunks + 1)),
+        "gpu_launches": args.steps * (1 + len(batches) * ({1: 0, 2: 6, 3: 6, 4: 8, 5: 11, 6: 11}[kernel]
+                                                           + n_chunks * (2 if kernel in (5, 6) and
+                                                                         opts.repack != 2 and
+                                                                         n_chunks > 1 else 1)
+                                                           + 1)),
         "roofline": roofline,
     }
     if world == 1 and not args.no_cpu_baseline:

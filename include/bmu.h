@@ -98,7 +98,10 @@ typedef struct bmu_opts {
                                densely, one load per tile, 1 treat them like all other ids */
     int32_t head_rows;      /* tensor-core sweep: how many of the most frequent features (ids
                                below this) are summed by the tensor cores, 256 or 512 */
-    int32_t reserved[5];    /* must be 0 */
+    int32_t repack;         /* tensor-core sweeps: 0/1 gather from a compact [D][chunk] copy
+                               of the chunk's columns, made before each launch, 2 gather
+                               from the codebook itself */
+    int32_t reserved[4];    /* must be 0 */
 } bmu_opts;
 
 BMU_API const char *bmu_status_string(int status);

@@ -33,7 +33,8 @@ class Opts(ctypes.Structure):
                 ("warps", ctypes.c_int32), ("cluster", ctypes.c_int32),
                 ("stage_rows", ctypes.c_int32), ("stages", ctypes.c_int32),
                 ("tile_order", ctypes.c_int32), ("tile_head", ctypes.c_int32),
-                ("head_rows", ctypes.c_int32), ("reserved", ctypes.c_int32 * 5)]
+                ("head_rows", ctypes.c_int32), ("repack", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 4)]
 
 
 EXPORTS = {

@@ -164,7 +164,7 @@ sweep_mma_kernel(const MmaArgs a)
         const int64_t tile = group * (MMA_DOCS / T) + (n >> 3);
         uint32_t bits = 0;
         if (tile < a.n_tiles)
-            bits = (__ldg(a.tile_head + (group * MMA_DOCS + n) * (H / 32) + (kc >> 2)) >>
+            bits = (__ldcs(a.tile_head + (group * MMA_DOCS + n) * (H / 32) + (kc >> 2)) >>
                     ((kc & 3) * 8)) & 0xffu;
         uint4 v;
         v.x = ((bits & 1u) ? 0x3c00u : 0u) | ((bits & 2u) ? 0x3c000000u : 0u);
@@ -257,10 +257,10 @@ sweep_mma_kernel(const MmaArgs a)
                     const uint4 *gp = a.tile_ids + __ldg(a.tile_off + tile);
                     const char *base = reinterpret_cast<const char *>(a.W + j0 + lane * 4);
                     uint32_t b = 0;
-                    uint4 qn = __ldg(gp);
+                    uint4 qn = __ldcs(gp);
                     for (; b < full; ++b) {
                         const uint4 qq = qn;
-                        qn = __ldg(gp + b + 1);
+                        qn = __ldcs(gp + b + 1);
                         const uint32_t f[T] = {qq.x & 0xffffu, qq.x >> 16, qq.y & 0xffffu, qq.y >> 16,
                                                qq.z & 0xffffu, qq.z >> 16, qq.w & 0xffffu, qq.w >> 16};
                         ulonglong2 w[T];
@@ -272,7 +272,7 @@ sweep_mma_kernel(const MmaArgs a)
                     }
                     for (; b < rows; ++b) {                          // some documents have run out
                         const uint4 qq = qn;
-                        qn = __ldg(gp + b + 1);
+                        qn = __ldcs(gp + b + 1);
                         const uint32_t f[T] = {qq.x & 0xffffu, qq.x >> 16, qq.y & 0xffffu, qq.y >> 16,
                                                qq.z & 0xffffu, qq.z >> 16, qq.w & 0xffffu, qq.w >> 16};
                         ulonglong2 w[T];

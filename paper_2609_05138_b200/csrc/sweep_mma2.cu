@@ -6,7 +6,7 @@
 // features, which takes the features present in about one document in a hundred
 // and more away from the gather):
 //   * a slab is 256 neurons and has two accumulator tiles (tensor-memory lane
-//     32q + t of tile c = neuron 64q + 2t + c), so the head sums of a slab take
+//     32q + 16h + i of tile c = neuron 64q + 4i + 2h + c), so the head sums of a slab take
 //     half of tensor memory and the MMAs of slab s+1 fill one half while the tail
 //     of slab s is gathered against the other: the MMAs have a whole slab's time,
 //     not the gap between two slabs;
@@ -35,7 +35,7 @@ static const int M2_TMEM_COLS = 512;                 // 2 buffers x 2 tiles x 12
 
 static inline size_t m2_smem_bytes(int head)
 {
-    return (size_t)MMA_DOCS * (head / 8) + (M2_NS + M2_NX) * MMA_STAGE_BYTES +
+    return (size_t)MMA_DOCS * (head / 8) + 4096 + (M2_NS + M2_NX) * MMA_STAGE_BYTES +
            (2 * M2_NS + 2 * M2_NX + 5) * 8 + MMA_DOCS * 8 + 16;
 }
 
@@ -57,7 +57,8 @@ head_split2_kernel(const float *__restrict__ W, int64_t M, const uint32_t *__res
         hi[e] = __float2half_rn(w);
         lo[e] = __float2half_rn(w - __half2float(hi[e]));
     }
-    const int c = jin & 1, r = ((jin >> 6) << 5) | ((jin >> 1) & 31);
+    // neuron 64q + 4i + 2h + c sits in row 32q + 16h + i of tile c
+    const int c = jin & 1, r = ((jin >> 6) << 5) | (((jin >> 1) & 1) << 4) | ((jin >> 2) & 15);
     const int kb = kcg >> 3, kc = kcg & 7;
     const size_t off = (size_t)(r >> 3) * 1024 + (size_t)kc * 128 + (size_t)(r & 7) * 16;
     const size_t st = (size_t)sl * SPS + (size_t)(kb * 2 + c) * 2;
@@ -114,7 +115,8 @@ sweep_mma2_kernel(const MmaArgs a)
     const int H = a.head, KB = H / 64;
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char *masks = smem;                                 // 128 documents x H bits
-    unsigned char *xring = smem + (size_t)MMA_DOCS * (H / 8);    // NX stages of X_head
+    uint4 *lut = reinterpret_cast<uint4 *>(smem + (size_t)MMA_DOCS * (H / 8));   // byte -> 8 fp16
+    unsigned char *xring = smem + (size_t)MMA_DOCS * (H / 8) + 4096;   // NX stages of X_head
     unsigned char *wring = xring + NX * MMA_STAGE_BYTES;         // NS stages of W_head
     u64 *bars = reinterpret_cast<u64 *>(wring + NS * MMA_STAGE_BYTES);
     u64 *keys = bars + 2 * NS + 2 * NX + 5;
@@ -153,10 +155,19 @@ sweep_mma2_kernel(const MmaArgs a)
         for (int idx = threadIdx.x; idx < MMA_DOCS * words; idx += M2_THREADS) {
             const int n = idx / words;
             const int64_t tile = group * (MMA_DOCS / 8) + (n >> 3);
-            mw[idx] = tile < a.n_tiles ? __ldg(a.tile_head + (size_t)group * MMA_DOCS * words + idx) : 0u;
+            mw[idx] = tile < a.n_tiles ? __ldcs(a.tile_head + (size_t)group * MMA_DOCS * words + idx) : 0u;
         }
     }
     if (threadIdx.x < MMA_DOCS) keys[threadIdx.x] = KEY_WORST;
+    if (threadIdx.x < 256) {         // the eight mask bits of a byte as eight fp16 zeros and ones
+        const uint32_t bits = threadIdx.x;
+        uint4 v;
+        v.x = ((bits & 1u) ? 0x3c00u : 0u) | ((bits & 2u) ? 0x3c000000u : 0u);
+        v.y = ((bits & 4u) ? 0x3c00u : 0u) | ((bits & 8u) ? 0x3c000000u : 0u);
+        v.z = ((bits & 16u) ? 0x3c00u : 0u) | ((bits & 32u) ? 0x3c000000u : 0u);
+        v.w = ((bits & 64u) ? 0x3c00u : 0u) | ((bits & 128u) ? 0x3c000000u : 0u);
+        lut[bits] = v;
+    }
     mm_fence_before();
     __syncthreads();
     mm_fence_after();
@@ -192,18 +203,19 @@ sweep_mma2_kernel(const MmaArgs a)
             if (x >= NX && !mm_wait(xempty0 + 8 * slot, ((x / NX) - 1) & 1, abort_flag, a.status, 16u))
                 break;
             unsigned char *dst = xring + (size_t)slot * MMA_STAGE_BYTES;
-#ifndef M2_DEBUG_NOEXPAND
-            for (int idx = lane; idx < MMA_DOCS * 8; idx += 32) {
-                const int n = idx & (MMA_DOCS - 1), kc = idx >> 7;
-                const uint32_t bits = masks[(size_t)n * (H / 8) + kb * 8 + kc];
-                uint4 v;
-                v.x = ((bits & 1u) ? 0x3c00u : 0u) | ((bits & 2u) ? 0x3c000000u : 0u);
-                v.y = ((bits & 4u) ? 0x3c00u : 0u) | ((bits & 8u) ? 0x3c000000u : 0u);
-                v.z = ((bits & 16u) ? 0x3c00u : 0u) | ((bits & 32u) ? 0x3c000000u : 0u);
-                v.w = ((bits & 64u) ? 0x3c00u : 0u) | ((bits & 128u) ? 0x3c000000u : 0u);
-                *reinterpret_cast<uint4 *>(dst + (size_t)(n >> 3) * 1024 + kc * 128 + (n & 7) * 16) = v;
+            // a lane takes documents lane, lane + 32, ..: its 8 mask bytes of this block of 64
+            // features in one load, then one table look-up and one 16-byte store per byte
+#pragma unroll
+            for (int j = 0; j < MMA_DOCS / 32; ++j) {
+                const int n = lane + 32 * j;
+                const uint2 mb = *reinterpret_cast<const uint2 *>(masks + (size_t)n * (H / 8) + kb * 8);
+                unsigned char *row = dst + (size_t)(n >> 3) * 1024 + (n & 7) * 16;
+#pragma unroll
+                for (int kc = 0; kc < 8; ++kc) {
+                    const uint32_t byte = ((kc < 4 ? mb.x : mb.y) >> ((kc & 3) * 8)) & 0xffu;
+                    *reinterpret_cast<uint4 *>(row + kc * 128) = lut[byte];
+                }
             }
-#endif
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) mm_bar_arrive(xfull0 + 8 * slot);
@@ -247,14 +259,14 @@ sweep_mma2_kernel(const MmaArgs a)
         }
         __syncwarp();
     } else {
-        // ---------------- tail: 16 documents x 64 neurons per task.  Lane (i, h) = (lane / 2,
-        // lane % 2) gathers neurons 4i .. 4i+3 for the documents 8h .. 8h+7 of the task: one
-        // 128-bit load per lane and row, two rows (one per half of the documents) per instruction.
+        // ---------------- tail: 16 documents x 64 neurons per task.  Lane (h, i) = (lane / 16,
+        // lane % 16) gathers neurons 4i .. 4i+3 for the documents 8h .. 8h+7 of the task: one
+        // 128-bit load per lane and row, two rows (one per half-warp) per instruction.
         const int q = warp & 3, g = warp >> 2;
-        const int li = lane >> 1, lh = lane & 1;
+        const int li = lane & 15, lh = lane >> 4;
         const float inv_s = 1.f / head_scale(__ldg(a.head_max));
         const uint32_t rowbytes = (uint32_t)(a.M * 4);
-        const int mydoc = 8 * lh + (((lane >> 1) & 1) << 2 | ((lane >> 2) & 1) << 1 | ((lane >> 3) & 1));
+        const int mydoc = 8 * lh + ((lane & 1) << 2 | (lane & 2) | ((lane >> 2) & 1));
         for (int sl = 0; sl < n_slabs; ++sl) {
             const int buf = sl & 1;
             const int j0 = a.j_lo + sl * M2_SLAB + q * 64;
@@ -276,11 +288,11 @@ sweep_mma2_kernel(const MmaArgs a)
                                                     : a.tile_ids + __ldg(a.tile_off + tile_a);
                     const char *base = reinterpret_cast<const char *>(a.W + j0 + li * 4);
                     uint32_t b = 0;
-                    uint4 qn = __ldg(gp);
+                    uint4 qn = __ldcs(gp);
                     for (; b < full; ++b) {
                         uint32_t f[8];
                         m2_unpack(qn, f);
-                        qn = __ldg(gp + b + 1);
+                        qn = __ldcs(gp + b + 1);
                         ulonglong2 w[8];
 #pragma unroll
                         for (int t = 0; t < 8; ++t)
@@ -291,7 +303,7 @@ sweep_mma2_kernel(const MmaArgs a)
                     for (; b < rows; ++b) {                      // some documents have run out
                         uint32_t f[8];
                         m2_unpack(qn, f);
-                        qn = __ldg(gp + b + 1);
+                        qn = __ldcs(gp + b + 1);
                         const bool in = b < my_rows;
                         ulonglong2 w[8];
 #pragma unroll
@@ -305,7 +317,7 @@ sweep_mma2_kernel(const MmaArgs a)
                 }
                 // head sums of these documents: the MMAs of this slab ran during the gather.
                 // Tensor-memory lane 32q + lane holds neurons 4i + 2h, 4i + 2h + 1 for all 16
-                // documents; the two lanes of a pair swap halves so that each ends up with four
+                // documents; lanes l and l ^ 16 swap halves so that each ends up with four
                 // neurons of its own eight documents.
 #ifndef M2_DEBUG_NOWAIT
                 if (it == 0) mm_wait(tfull0 + 8 * buf, (sl >> 1) & 1, abort_flag, a.status, 8u);
@@ -326,8 +338,8 @@ sweep_mma2_kernel(const MmaArgs a)
                 for (int t = 0; t < 8; ++t) {
                     const uint32_t mine0 = lh ? h0[8 + t] : h0[t], mine1 = lh ? h1[8 + t] : h1[t];
                     const uint32_t send0 = lh ? h0[t] : h0[8 + t], send1 = lh ? h1[t] : h1[8 + t];
-                    const uint32_t got0 = __shfl_xor_sync(0xffffffffu, send0, 1);
-                    const uint32_t got1 = __shfl_xor_sync(0xffffffffu, send1, 1);
+                    const uint32_t got0 = __shfl_xor_sync(0xffffffffu, send0, 16);
+                    const uint32_t got1 = __shfl_xor_sync(0xffffffffu, send1, 16);
                     const float s0 = __uint_as_float(lh ? got0 : mine0) * inv_s;
                     const float s1 = __uint_as_float(lh ? got1 : mine1) * inv_s;
                     const float s2 = __uint_as_float(lh ? mine0 : got0) * inv_s;
@@ -351,7 +363,7 @@ sweep_mma2_kernel(const MmaArgs a)
                 // transposing butterfly among the 16 lanes that hold the same documents
 #pragma unroll
                 for (int st = 0; st < 3; ++st) {
-                    const int m = 2 << st, cnt = 4 >> st;
+                    const int m = 1 << st, cnt = 4 >> st;
 #pragma unroll
                     for (int i = 0; i < cnt; ++i) {
                         const u64 send = (lane & m) ? k[i] : k[i + cnt];
@@ -360,9 +372,9 @@ sweep_mma2_kernel(const MmaArgs a)
                         k[i] = got < keep ? got : keep;
                     }
                 }
-                const u64 got = __shfl_xor_sync(0xffffffffu, k[0], 16);
+                const u64 got = __shfl_xor_sync(0xffffffffu, k[0], 8);
                 k[0] = got < k[0] ? got : k[0];
-                if (lane < 16) atomicMin(reinterpret_cast<unsigned long long *>(keys + dg * 16 + mydoc), k[0]);
+                if ((lane & 8) == 0) atomicMin(reinterpret_cast<unsigned long long *>(keys + dg * 16 + mydoc), k[0]);
             }
         }
         __syncwarp();

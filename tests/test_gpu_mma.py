@@ -1,5 +1,6 @@
-"""Parity of the tensor-core head + gathered tail sweep (bmu_opts.kernel = 5) against
-the fp64 oracle, through the C ABI.  Same rule as every other kernel
+"""Parity of the tensor-core head + gathered tail sweeps (bmu_opts.kernel = 5: 512-neuron
+slabs, head of 256 or 512 features; 6: 256-neuron slabs, double-buffered tensor memory,
+head of 64 .. 1024 features) against the fp64 oracle, through the C ABI.  Same rule as every other kernel
 (tests/parity.py): indices equal except inside a 1e-5 near-tie, distances within
 1e-5 relative.  The head sums come from fp16 (hi, lo) parts of the weights and a
 tensor-core fp32 accumulator, so results are not bit-equal to the gathered
@@ -24,9 +25,9 @@ def bmu():
     return lib
 
 
-def opts_of(bmu, **kw):
+def opts_of(bmu, kernel=5, **kw):
     o = bmu.Opts()
-    o.kernel = 5
+    o.kernel = kernel
     for k, v in kw.items():
         setattr(o, k, v)
     return o
@@ -45,42 +46,46 @@ def run_and_check(bmu, W, rowptr, colidx, opts, cancel_floor=False):
                           colidx.numpy(), cancel_floor=cancel_floor)
 
 
-@pytest.mark.parametrize("tile_order,head_rows", [(0, 0), (1, 256), (0, 512)])
+@pytest.mark.parametrize("kernel,tile_order,head_rows", [(5, 0, 0), (5, 1, 256), (5, 0, 512),
+                                                         (6, 0, 0), (6, 1, 64), (6, 0, 512),
+                                                         (6, 0, 1024), (6, 1, 320)])
 @pytest.mark.parametrize("name,n_docs,M,chunk", [("cfg3", 2500, 2048, 1024), ("cfg5", 1203, 1536, 512),
                                                  ("cfg1", 4001, 1024 + 36, 0), ("cfg2", 777, 512, 0)])
-def test_mma_kernel_matches_oracle(bmu, name, n_docs, M, chunk, tile_order, head_rows):
+def test_mma_kernel_matches_oracle(bmu, name, n_docs, M, chunk, kernel, tile_order, head_rows):
     cfg = synth.CONFIGS[name]
     rowptr, colidx = synth.make_corpus(cfg, n_docs=n_docs)
     for kind in ("uniform", "scaled"):
         W = synth.make_codebook(cfg.D, M, 21, kind=kind)
         res = run_and_check(bmu, W, rowptr, colidx,
-                            opts_of(bmu, tile_order=tile_order, chunk_neurons=chunk,
+                            opts_of(bmu, kernel, tile_order=tile_order, chunk_neurons=chunk,
                                     head_rows=head_rows))
         assert res["failed"] == 0 and res["docs"] == n_docs
 
 
+@pytest.mark.parametrize("kernel", [5, 6])
 @pytest.mark.parametrize("kind,floor", [("dupes", False), ("const", False), ("sparse", False),
                                         ("signed", False), ("prototype", True)])
-def test_mma_kernel_codebook_kinds(bmu, kind, floor):
+def test_mma_kernel_codebook_kinds(bmu, kind, floor, kernel):
     cfg = synth.CONFIGS["cfg1"]
     rowptr, colidx = synth.make_corpus(cfg, n_docs=1500)
     W = synth.make_codebook(cfg.D, 1024, 83, kind=kind, docs=(rowptr, colidx))
-    run_and_check(bmu, W, rowptr, colidx, opts_of(bmu), cancel_floor=floor)
+    run_and_check(bmu, W, rowptr, colidx, opts_of(bmu, kernel), cancel_floor=floor)
     if kind in ("dupes", "const"):
-        ob, _ = bmu.bmu_search_ws(W.cuda(), rowptr.cuda(), colidx.cuda(), opts=opts_of(bmu))
+        ob, _ = bmu.bmu_search_ws(W.cuda(), rowptr.cuda(), colidx.cuda(), opts=opts_of(bmu, kernel))
         if kind == "dupes":
             assert int((ob % 2).sum()) == 0        # equal columns: the lower index wins
         else:
             assert int(ob.abs().sum()) == 0        # every neuron ties: index 0
 
 
+@pytest.mark.parametrize("kernel", [5, 6])
 @pytest.mark.parametrize("scale", [1e-6, 1.0, 3e4, 1e9])
-def test_mma_kernel_weight_magnitudes(bmu, scale):
+def test_mma_kernel_weight_magnitudes(bmu, scale, kernel):
     """The power-of-two scaling of the fp16 parts follows the largest head weight."""
     cfg = synth.CONFIGS["cfg3"]
     rowptr, colidx = synth.make_corpus(cfg, n_docs=700)
     W = synth.make_codebook(cfg.D, 512, 5, kind="signed") * scale
-    run_and_check(bmu, W, rowptr, colidx, opts_of(bmu))
+    run_and_check(bmu, W, rowptr, colidx, opts_of(bmu, kernel))
 
 
 def test_mma_kernel_long_empty_unsorted_and_repeated_rows(bmu):
@@ -100,6 +105,8 @@ def test_mma_kernel_long_empty_unsorted_and_repeated_rows(bmu):
     W = synth.make_codebook(D, M, 11, kind="scaled")
     run_and_check(bmu, W, rowptr, torch.from_numpy(ci), opts_of(bmu))
     run_and_check(bmu, W, rowptr, torch.from_numpy(ci), opts_of(bmu, head_rows=512))
+    run_and_check(bmu, W, rowptr, torch.from_numpy(ci), opts_of(bmu, 6))
+    run_and_check(bmu, W, rowptr, torch.from_numpy(ci), opts_of(bmu, 6, head_rows=256, tile_order=1))
 
 
 def test_mma_kernel_unlabelled_vocabulary(bmu):
@@ -110,12 +117,13 @@ def test_mma_kernel_unlabelled_vocabulary(bmu):
     ci = perm[colidx.long()]
     W = synth.make_codebook(cfg.D, 512, 9, kind="scaled")
     run_and_check(bmu, W, rowptr, ci, opts_of(bmu))
+    run_and_check(bmu, W, rowptr, ci, opts_of(bmu, 6))
 
 
 def test_mma_kernel_refuses_what_it_cannot_do(bmu):
     rp = torch.tensor([0, 1], dtype=torch.int32).cuda()
     ci = torch.tensor([0], dtype=torch.int32).cuda()
-    for D, M in ((128, 1024), (512, 256)):
+    for kernel, D, M in ((5, 128, 1024), (5, 512, 256), (6, 32, 1024), (6, 2048, 256)):
         with pytest.raises(bmu.BmuError) as e:
-            bmu.bmu_search_ws(torch.zeros(D, M, device="cuda"), rp, ci, opts=opts_of(bmu))
+            bmu.bmu_search_ws(torch.zeros(D, M, device="cuda"), rp, ci, opts=opts_of(bmu, kernel))
         assert e.value.status == 2
