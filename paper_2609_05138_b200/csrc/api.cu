@@ -124,6 +124,13 @@ static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kerne
     return l;
 }
 
+// the layout search_impl uses for these options (the workspace-size queries must agree with it)
+static Layout layout_of(const bmu_opts &o, int64_t D, int64_t M, int64_t N, int64_t nnz, bool top2)
+{
+    return layout_for(D, M, N, nnz, o.kernel, top2, mma_head_rows(o, D),
+                      mma_repack_bytes(o, D, M, N, nnz, top2));
+}
+
 static int check_sizes(int64_t D, int64_t M, int64_t N, int64_t nnz)
 {
     if (D < 0 || M < 0 || N < 0 || nnz < 0) {
@@ -198,7 +205,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     }
     const int head = mma_head_rows(o, D);
     const size_t repack_bytes = mma_repack_bytes(o, D, M, N, nnz, top2);
-    const Layout l = layout_for(D, M, N, nnz, o.kernel, top2, head, repack_bytes);
+    const Layout l = layout_of(o, D, M, N, nnz, top2);
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < l.total) {
         set_error("workspace missing, not 256-byte aligned, or smaller than %zu bytes", l.total);
         return BMU_ERR_WORKSPACE;
@@ -487,8 +494,7 @@ size_t bmu_search_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,
     bmu_opts o;
     memset(&o, 0, sizeof(o));
     if (opts) o = *opts;
-    return layout_for(D, M, N, nnz, o.kernel, false, mma_head_rows(o, D),
-                      mma_repack_bytes(o, D, M, N, nnz, false)).total;
+    return layout_of(o, D, M, N, nnz, false).total;
 }
 
 int bmu_search_ws(const float *W, int64_t D, int64_t M, const float *norms,
@@ -504,7 +510,10 @@ size_t bmu_search_top2_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t 
                                        const bmu_opts *opts)
 {
     if (D < 0 || M < 0 || N < 0 || nnz < 0) return 0;
-    return layout_for(D, M, N, nnz, opts ? opts->kernel : 0, true).total;
+    bmu_opts o;
+    memset(&o, 0, sizeof(o));
+    if (opts) o = *opts;
+    return layout_of(o, D, M, N, nnz, true).total;
 }
 
 int bmu_search_top2_ws(const float *W, int64_t D, int64_t M, const float *norms,
