@@ -27,15 +27,21 @@
 namespace bmu {
 
 static const int M2_SLAB = 256;
-static const int M2_NS = 4;                          // W ring stages
-static const int M2_NX = 3;                          // X ring stages
+#ifndef BMU_M2_WSTAGES
+#define BMU_M2_WSTAGES 4
+#endif
+#ifndef BMU_M2_XSTAGES
+#define BMU_M2_XSTAGES 3
+#endif
+static const int M2_NS = BMU_M2_WSTAGES;             // W ring stages
+static const int M2_NX = BMU_M2_XSTAGES;             // X ring stages
 static const int M2_TAIL_WARPS = 16;
 static const int M2_THREADS = (M2_TAIL_WARPS + 3) * 32;
 static const int M2_TMEM_COLS = 512;                 // 2 buffers x 2 tiles x 128 documents
 
 static inline size_t m2_smem_bytes(int head)
 {
-    return (size_t)MMA_DOCS * (head / 8) + 4096 + (M2_NS + M2_NX) * MMA_STAGE_BYTES +
+    return (size_t)MMA_DOCS * (head / 8) + (M2_NS + M2_NX) * MMA_STAGE_BYTES +
            (2 * M2_NS + 2 * M2_NX + 5) * 8 + MMA_DOCS * 8 + 16;
 }
 
@@ -115,8 +121,7 @@ sweep_mma2_kernel(const MmaArgs a)
     const int H = a.head, KB = H / 64;
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char *masks = smem;                                 // 128 documents x H bits
-    uint4 *lut = reinterpret_cast<uint4 *>(smem + (size_t)MMA_DOCS * (H / 8));   // byte -> 8 fp16
-    unsigned char *xring = smem + (size_t)MMA_DOCS * (H / 8) + 4096;   // NX stages of X_head
+    unsigned char *xring = smem + (size_t)MMA_DOCS * (H / 8);    // NX stages of X_head
     unsigned char *wring = xring + NX * MMA_STAGE_BYTES;         // NS stages of W_head
     u64 *bars = reinterpret_cast<u64 *>(wring + NS * MMA_STAGE_BYTES);
     u64 *keys = bars + 2 * NS + 2 * NX + 5;
@@ -159,15 +164,6 @@ sweep_mma2_kernel(const MmaArgs a)
         }
     }
     if (threadIdx.x < MMA_DOCS) keys[threadIdx.x] = KEY_WORST;
-    if (threadIdx.x < 256) {         // the eight mask bits of a byte as eight fp16 zeros and ones
-        const uint32_t bits = threadIdx.x;
-        uint4 v;
-        v.x = ((bits & 1u) ? 0x3c00u : 0u) | ((bits & 2u) ? 0x3c000000u : 0u);
-        v.y = ((bits & 4u) ? 0x3c00u : 0u) | ((bits & 8u) ? 0x3c000000u : 0u);
-        v.z = ((bits & 16u) ? 0x3c00u : 0u) | ((bits & 32u) ? 0x3c000000u : 0u);
-        v.w = ((bits & 64u) ? 0x3c00u : 0u) | ((bits & 128u) ? 0x3c000000u : 0u);
-        lut[bits] = v;
-    }
     mm_fence_before();
     __syncthreads();
     mm_fence_after();
@@ -204,7 +200,8 @@ sweep_mma2_kernel(const MmaArgs a)
                 break;
             unsigned char *dst = xring + (size_t)slot * MMA_STAGE_BYTES;
             // a lane takes documents lane, lane + 32, ..: its 8 mask bytes of this block of 64
-            // features in one load, then one table look-up and one 16-byte store per byte
+            // features in one load, then eight 16-byte stores of fp16 zeros and ones (bit e of
+            // a byte -> half e; 0x3c00 is 1.0)
 #pragma unroll
             for (int j = 0; j < MMA_DOCS / 32; ++j) {
                 const int n = lane + 32 * j;
@@ -212,8 +209,13 @@ sweep_mma2_kernel(const MmaArgs a)
                 unsigned char *row = dst + (size_t)(n >> 3) * 1024 + (n & 7) * 16;
 #pragma unroll
                 for (int kc = 0; kc < 8; ++kc) {
-                    const uint32_t byte = ((kc < 4 ? mb.x : mb.y) >> ((kc & 3) * 8)) & 0xffu;
-                    *reinterpret_cast<uint4 *>(row + kc * 128) = lut[byte];
+                    const uint32_t b = (kc < 4 ? mb.x : mb.y) >> ((kc & 3) * 8);
+                    uint4 v;
+                    v.x = (b & 1u) * 0x3c00u + (b & 2u) * 0x1e000000u;
+                    v.y = ((b >> 2) & 1u) * 0x3c00u + ((b >> 2) & 2u) * 0x1e000000u;
+                    v.z = ((b >> 4) & 1u) * 0x3c00u + ((b >> 4) & 2u) * 0x1e000000u;
+                    v.w = ((b >> 6) & 1u) * 0x3c00u + ((b >> 6) & 2u) * 0x1e000000u;
+                    *reinterpret_cast<uint4 *>(row + kc * 128) = v;
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
