@@ -32,7 +32,7 @@ if ROOT not in sys.path:
 from inputs import synth  # noqa: E402
 
 # DRAM bytes per sweep launch of the default config-4 run, from ncu (profiles/)
-TRAFFIC_CFG4 = {3: 2.0e9, 4: 2.9e9, 5: 4.9e9}
+TRAFFIC_CFG4 = {3: 2.0e9, 4: 2.9e9, 5: 4.9e9, 6: 3.6e9}
 
 METRIC = "bmu_search_docs_per_s"
 UNIT = "docs/s"
@@ -400,7 +400,8 @@ def run_ours(args, cfg, rank, local_rank, world):
         # (profiles/sweep_*_cfg4_launch_list.md); other workloads were not captured
         "traffic": (TRAFFIC_CFG4.get(kernel) if (cfg.name == "cfg4" and n_docs == cfg.N
                                                  and not opts.chunk_neurons and not opts.vec
-                                                 and not opts.warps and not opts.head_rows)
+                                                 and not opts.warps and not opts.head_rows
+                                                 and not opts.repack)
                     else None),
         "launch_ms": launch_s * 1e3, "launches_per_step": n_chunks,
         "units_per_launch": {"adds": adds, "union_rows_x_chunk": float(union_rows) * chunk},

@@ -42,7 +42,7 @@ static const int M2_TMEM_COLS = 512;                 // 2 buffers x 2 tiles x 12
 static inline size_t m2_smem_bytes(int head)
 {
     return (size_t)MMA_DOCS * (head / 8) + (M2_NS + M2_NX) * MMA_STAGE_BYTES +
-           (2 * M2_NS + 2 * M2_NX + 5) * 8 + MMA_DOCS * 8 + 16;
+           (2 * M2_NS + 2 * M2_NX + 6) * 8 + MMA_DOCS * 8 + 16 + 16 * 16 + 2 * 16 * 4;
 }
 
 // One thread per (slab, group of 8 features, neuron).  Stage order inside a slab: block of
@@ -124,10 +124,14 @@ sweep_mma2_kernel(const MmaArgs a)
     unsigned char *xring = smem + (size_t)MMA_DOCS * (H / 8);    // NX stages of X_head
     unsigned char *wring = xring + NX * MMA_STAGE_BYTES;         // NS stages of W_head
     u64 *bars = reinterpret_cast<u64 *>(wring + NS * MMA_STAGE_BYTES);
-    u64 *keys = bars + 2 * NS + 2 * NX + 5;
+    u64 *keys = bars + 2 * NS + 2 * NX + 6;                      // (16-byte aligned)
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(keys + MMA_DOCS);
     volatile uint32_t *abort_flag = tmem_slot + 1;
     uint32_t *skip_flag = tmem_slot + 2;
+    // the block's 16 tiles: first row of each id matrix, its length word and its offset
+    uint4 *s_first = reinterpret_cast<uint4 *>(tmem_slot + 4);
+    uint32_t *s_len = reinterpret_cast<uint32_t *>(s_first + 16);
+    uint32_t *s_off = s_len + 16;
     const uint32_t wfull0 = mm_smem(bars), wempty0 = mm_smem(bars + NS);
     const uint32_t xfull0 = mm_smem(bars + 2 * NS), xempty0 = mm_smem(bars + 2 * NS + NX);
     const uint32_t tfull0 = mm_smem(bars + 2 * NS + 2 * NX), tempty0 = tfull0 + 16;
@@ -164,6 +168,15 @@ sweep_mma2_kernel(const MmaArgs a)
         }
     }
     if (threadIdx.x < MMA_DOCS) keys[threadIdx.x] = KEY_WORST;
+    if (threadIdx.x >= M2_THREADS - 16) {            // 16 threads of the last control warp
+        const int t = threadIdx.x - (M2_THREADS - 16);
+        const int64_t tile = group * (MMA_DOCS / 8) + t;
+        const bool there = tile < a.n_tiles;
+        const uint32_t off = there ? __ldg(a.tile_off + tile) : 0u;
+        s_len[t] = there ? __ldg(a.tile_len + tile) : 0u;
+        s_off[t] = off;
+        s_first[t] = __ldcs(a.tile_ids + off);
+    }
     mm_fence_before();
     __syncthreads();
     mm_fence_after();
@@ -281,16 +294,15 @@ sweep_mma2_kernel(const MmaArgs a)
                 for (int t = 0; t < 8; ++t) acc[t][0] = acc[t][1] = 0ull;
                 if (live) {
                     const bool has_b = tile_b < a.n_tiles;
-                    const uint32_t tla = __ldg(a.tile_len + tile_a);
-                    const uint32_t tlb = has_b ? __ldg(a.tile_len + tile_b) : 0u;
+                    const uint32_t tla = s_len[2 * dg], tlb = s_len[2 * dg + 1];
                     const uint32_t full = min(tla >> 16, tlb >> 16);
                     const uint32_t rows = max(tla & 0xffffu, tlb & 0xffffu);
                     const uint32_t my_rows = (lh ? tlb : tla) & 0xffffu;
-                    const uint4 *gp = (lh && has_b) ? a.tile_ids + __ldg(a.tile_off + tile_b)
-                                                    : a.tile_ids + __ldg(a.tile_off + tile_a);
+                    const int mine = 2 * dg + ((lh && has_b) ? 1 : 0);
+                    const uint4 *gp = a.tile_ids + s_off[mine];
                     const char *base = reinterpret_cast<const char *>(a.W + j0 + li * 4);
                     uint32_t b = 0;
-                    uint4 qn = __ldcs(gp);
+                    uint4 qn = s_first[mine];
                     for (; b < full; ++b) {
                         uint32_t f[8];
                         m2_unpack(qn, f);
