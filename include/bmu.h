@@ -73,13 +73,15 @@ typedef struct bmu_opts {
                                4 tiled (a warp carries 8 documents; frequent rows loaded once
                                per tile; the warps of a block walk the feature axis in step
                                so that L1 serves the rows they share; needs what 3 needs and
-                               length-ordered documents); 5 tensor-core head (the sum over the
-                               head_rows most frequent features -- ids below head_rows: the
-                               paper keeps its vocabulary frequency-ordered, Table 8 -- is a
-                               dense contraction on tcgen05 tensor cores with fp32
-                               accumulation, the remaining ids are gathered as in 4; needs
-                               what 4 needs, D >= head_rows and M >= 512; best unit only;
-                               the automatic choice for large sweeps); 2 staged (a lane per
+                               length-ordered documents); 6 wide tensor-core head (the sum over
+                               the head_rows most frequent features -- ids below head_rows:
+                               the paper keeps its vocabulary frequency-ordered, Table 8 --
+                               is a dense contraction on tcgen05 tensor cores with fp32
+                               accumulation into double-buffered tensor memory, the
+                               remaining ids are gathered as in 4; needs what 4 needs,
+                               D >= head_rows and M >= 512; best unit only; the automatic
+                               choice for large sweeps); 5 first tensor-core sweep (same
+                               split, 512-neuron slabs, head of 256 or 512); 2 staged (a lane per
                                document, rows streamed through shared memory by tensor (TMA)
                                box copies; needs M % 4 == 0, M >= 32, 256 <= D <= 65024) */
     int32_t chunk_neurons;  /* neurons per L2-resident chunk of the codebook (Section 4.2,
@@ -96,8 +98,9 @@ typedef struct bmu_opts {
                                frequent and the rare half of the lists, 1 ascending ids */
     int32_t tile_head;      /* tiled kernel: 0 sweep the 32 most frequent features (ids < 32)
                                densely, one load per tile, 1 treat them like all other ids */
-    int32_t head_rows;      /* tensor-core sweep: how many of the most frequent features (ids
-                               below this) are summed by the tensor cores, 256 or 512 */
+    int32_t head_rows;      /* tensor-core sweeps: how many of the most frequent features (ids
+                               below this) are summed by the tensor cores: a multiple of 64
+                               up to 1024 (kernel 5: 256 or 512); 0 = 768 (kernel 5: 256) */
     int32_t repack;         /* tensor-core sweeps: 0/1 gather from a compact [D][chunk] copy
                                of the chunk's columns, made before each launch, 2 gather
                                from the codebook itself */
@@ -120,8 +123,8 @@ BMU_API int bmu_codebook_norms(const float *W, int64_t D, int64_t M, float *norm
 /*
  * Scratch bytes bmu_search_ws needs for a problem of this size (norms, the
  * per-document running minimum merged across neuron chunks, the tiling plan,
- * and the split image of the frequent rows for the tensor-core sweep: M KiB at
- * head_rows = 256).  `nnz` is the length of colidx.
+ * the split image of the frequent rows (4 * head_rows bytes per neuron) and the
+ * compact chunk copy of the tensor-core sweeps).  `nnz` is the length of colidx.
  */
 BMU_API size_t bmu_search_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,
                                   const bmu_opts *opts);
