@@ -44,6 +44,12 @@ def _load():
         lib.oracle_bmu.restype = ci
         lib.oracle_bmu2.argtypes = [vp, i64, i64, vp, vp, vp, i64, vp, vp, vp, vp, ci]
         lib.oracle_bmu2.restype = ci
+        lib.oracle_scatter.argtypes = [vp, vp, i64, vp, i64, vp, vp]
+        lib.oracle_scatter.restype = None
+        lib.oracle_blur_plane.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_double, vp]
+        lib.oracle_blur_plane.restype = None
+        lib.oracle_writeback.argtypes = [vp, vp, i64, i64, vp]
+        lib.oracle_writeback.restype = None
         lib.oracle_max_threads.argtypes = []
         lib.oracle_max_threads.restype = ci
         _lib = lib
@@ -118,3 +124,34 @@ def eval_pair(W, rowptr, colidx, norms_, i: int, j: int) -> float:
     n = np.ascontiguousarray(norms_, dtype=np.float64)
     return float(_load().oracle_eval(_p(W), D, M, _p(n), _p(rowptr), _p(colidx),
                                      int(i), int(j)))
+
+
+# ---- the rest of a batch epoch: scatter, blur, write-back (Table 4) ----------
+def scatter(rowptr, colidx, bmu_, D: int, M: int):
+    """(num uint64 [D, M], cnt uint64 [M]): how many documents of each unit have each feature."""
+    rowptr, colidx, b = _i32(rowptr), _i32(colidx), _i32(bmu_)
+    N = rowptr.shape[0] - 1
+    num = np.zeros((D, M), dtype=np.uint64)
+    cnt = np.zeros(M, dtype=np.uint64)
+    _load().oracle_scatter(_p(rowptr), _p(colidx), N, _p(b), M, _p(num), _p(cnt))
+    return num, cnt
+
+
+def blur(planes, edge_x: int, edge_y: int, sigma: float) -> np.ndarray:
+    """Truncated Gaussian neighbourhood sum of every plane ([..., edge_y * edge_x]) in float64."""
+    a = np.ascontiguousarray(planes, dtype=np.float64)
+    flat = a.reshape(-1, edge_x * edge_y)
+    out = np.empty_like(flat)
+    for r in range(flat.shape[0]):
+        _load().oracle_blur_plane(_p(flat[r]), edge_x, edge_y, float(sigma), _p(out[r]))
+    return out.reshape(a.shape)
+
+
+def writeback(B, c, W) -> np.ndarray:
+    """New codebook (float32 copy of W with W[f][j] = B[f][j] / c[j] where c[j] > 0)."""
+    B = np.ascontiguousarray(B, dtype=np.float64)
+    c = np.ascontiguousarray(c, dtype=np.float64)
+    out = _f32(W).copy()
+    D, M = out.shape
+    _load().oracle_writeback(_p(B), _p(c), D, M, _p(out))
+    return out

@@ -146,3 +146,63 @@ int oracle_max_threads(void)
     return 1;
 #endif
 }
+
+/* ------------------------------------------------------------------------
+ * The rest of a batch epoch (Table 4: "scatter", "blur", "write-back"; Section 6:
+ * "the scatter into accumulators is O(N.nnz) ... the blur is the O(M) term").
+ * The paper times these steps but does not print their formulas; what follows is
+ * the textbook batch self-organizing-map update written out, on a rectangular,
+ * non-periodic map of edge_y rows by edge_x columns (neuron j = y * edge_x + x):
+ *
+ *   scatter     num[f][j] = #{ i : bmu_i = j and f in x_i }   (a repeated id counts
+ *               twice), cnt[j] = #{ i : bmu_i = j }           -- exact integers
+ *   blur        B[f][j] = sum_k h(j, k) num[f][k],  c[j] = sum_k h(j, k) cnt[k],
+ *               h(j, k) = exp(-((xj-xk)^2 + (yj-yk)^2) / (2 sigma^2)) when both
+ *               |xj-xk| and |yj-yk| are at most R = ceil(3 sigma), else 0;
+ *               sigma == 0 means h = identity
+ *   write-back  W[f][j] = B[f][j] / c[j] where c[j] > 0, otherwise W[f][j] stays
+ *
+ * Parity status: pinned by mathematics only (dense brute force with the explicit
+ * h matrix, closed forms, invariants; tests/test_oracle_pins_update.py) -- the
+ * paper prints no formula or value for these steps, so against the paper they
+ * are "parity unpinned".
+ */
+void oracle_scatter(const int32_t *rowptr, const int32_t *colidx, int64_t N, const int32_t *bmu,
+                    int64_t M, uint64_t *num, uint64_t *cnt)
+{
+    for (int64_t i = 0; i < N; ++i) {
+        const int64_t j = bmu[i];
+        cnt[j] += 1;
+        for (int32_t e = rowptr[i]; e < rowptr[i + 1]; ++e)
+            num[(int64_t)colidx[e] * M + j] += 1;
+    }
+}
+
+/* One plane (edge_y x edge_x doubles in, doubles out), by the definition: a
+ * double loop over the neighbours inside the square of half-width R. */
+void oracle_blur_plane(const double *in, int32_t edge_x, int32_t edge_y, double sigma, double *out)
+{
+    const int R = sigma > 0.0 ? (int)ceil(3.0 * sigma) : 0;
+    for (int y = 0; y < edge_y; ++y)
+        for (int x = 0; x < edge_x; ++x) {
+            double s = 0.0;
+            for (int dy = -R; dy <= R; ++dy)
+                for (int dx = -R; dx <= R; ++dx) {
+                    const int yy = y + dy, xx = x + dx;
+                    if (yy < 0 || yy >= edge_y || xx < 0 || xx >= edge_x)
+                        continue;
+                    const double h = sigma > 0.0
+                        ? exp(-((double)(dx * dx + dy * dy)) / (2.0 * sigma * sigma)) : 1.0;
+                    s += h * in[(int64_t)yy * edge_x + xx];
+                }
+            out[(int64_t)y * edge_x + x] = s;
+        }
+}
+
+void oracle_writeback(const double *B, const double *c, int64_t D, int64_t M, float *W)
+{
+    for (int64_t f = 0; f < D; ++f)
+        for (int64_t j = 0; j < M; ++j)
+            if (c[j] > 0.0)
+                W[f * M + j] = (float)(B[f * M + j] / c[j]);
+}
