@@ -274,6 +274,38 @@ BMU_API int bmu_search_static(const float *W, int64_t D, int64_t M, const int32_
                               float *out_dist, void *stream);
 
 /*
+ * The rest of a batch epoch after the search (Table 4 columns "scatter", "blur",
+ * "write-back"; Section 6: "the scatter into accumulators is O(N.nnz) ... the
+ * blur is the O(M) term").  The paper times these steps and prints no formula;
+ * they are the textbook batch update of a self-organizing map on a rectangular,
+ * non-periodic map of edge_y rows by edge_x columns, neuron j = y * edge_x + x.
+ * All arrays are device memory, feature-major like W; every call is
+ * asynchronous on `stream` and uses no scratch.
+ *
+ * bmu_update_scatter: for every document i, cnt[bmu[i]] += 1 and, for every
+ *   listed feature f, num[f*M + bmu[i]] += 1 (a repeated id counts twice).
+ *   num uint32 [D][M] and cnt uint32 [M] are accumulated into: zero them at the
+ *   start of an epoch, call once per corpus batch.  Exact integer counters.
+ *   bmu[i] must lie in [0, M) (unchecked, like colidx).
+ * bmu_update_blur: num_blur[f][j] = sum_k h(j, k) * num[f][k] and cnt_blur[j] =
+ *   sum_k h(j, k) * cnt[k] in fp32, h(j, k) = exp(-(dx^2 + dy^2) / (2 sigma^2))
+ *   for |dx|, |dy| <= ceil(3 sigma) and 0 beyond (no wrap-around, no
+ *   normalisation: the write-back divides it out); sigma == 0 copies.  Limits:
+ *   sigma <= 8, D <= 65024.  Outputs must not alias inputs.
+ * bmu_update_writeback: W[f*M + j] = num_blur[f*M + j] / cnt_blur[j] where
+ *   cnt_blur[j] > 0; other neurons keep their weights.  D <= 65535.
+ * The norms of the new codebook are bmu_codebook_norms.
+ */
+BMU_API int bmu_update_scatter(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
+                               const int32_t *bmu, int64_t D, int64_t M, uint32_t *num,
+                               uint32_t *cnt, void *stream);
+BMU_API int bmu_update_blur(const uint32_t *num, const uint32_t *cnt, int64_t D, int32_t edge_x,
+                            int32_t edge_y, float sigma, float *num_blur, float *cnt_blur,
+                            void *stream);
+BMU_API int bmu_update_writeback(const float *num_blur, const float *cnt_blur, int64_t D, int64_t M,
+                                 float *W, void *stream);
+
+/*
  * Measures one on-chip ceiling of the current device with a microbenchmark, so
  * that achieved throughput can be quoted against the roof that binds (the paper
  * quotes its kernel against the L2 roof of its card, Section 6 / Table 3).

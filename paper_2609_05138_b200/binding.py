@@ -87,6 +87,15 @@ EXPORTS = {
     "bmu_release_scratch": (ctypes.c_int, []),
     "bmu_validate_csr": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                         ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
+    "bmu_update_scatter": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                                          ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64,
+                                          ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
+                                          ctypes.c_void_p]),
+    "bmu_update_blur": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                                       ctypes.c_int32, ctypes.c_int32, ctypes.c_float,
+                                       ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "bmu_update_writeback": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                                            ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]),
     "bmu_measure_roof": (ctypes.c_int, [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t,
                                         ctypes.c_int, ctypes.POINTER(ctypes.c_double),
                                         ctypes.c_void_p]),
@@ -331,6 +340,45 @@ def bmu_validate_csr(rowptr, colidx, D: int):
             _dev(rowptr, torch.int32, "rowptr"),
             _dev(colidx, torch.int32, "colidx") if colidx.numel() else None, N, colidx.numel(),
             D, _stream(rowptr)))
+
+
+# ---- the rest of a batch epoch: scatter, blur, write-back (Table 4) ----------
+def bmu_update_scatter(rowptr, colidx, bmu, num, cnt):
+    """Adds this batch to the integer accumulators num uint32 [D, M] and cnt uint32 [M]."""
+    D, M = num.shape
+    N = rowptr.numel() - 1
+    nnz = colidx.numel()
+    for t, name in ((num, "num"), (cnt, "cnt")):
+        if t.dtype not in (torch.uint32, torch.int32) or not t.is_cuda or not t.is_contiguous():
+            raise ValueError("%s must be a contiguous CUDA uint32 (or int32) tensor" % name)
+    with torch.cuda.device(num.device):
+        _check(load().bmu_update_scatter(
+            _dev(rowptr, torch.int32, "rowptr"),
+            _dev(colidx, torch.int32, "colidx") if nnz else None, N, nnz,
+            _dev(bmu, torch.int32, "bmu"), D, M, num.data_ptr(), cnt.data_ptr(), _stream(num)))
+
+
+def bmu_update_blur(num, cnt, edge_x: int, edge_y: int, sigma: float):
+    """Neighbourhood-weighted sums of the accumulators: (num_blur float32 [D, M], cnt_blur [M])."""
+    D, M = num.shape
+    if edge_x * edge_y != M:
+        raise ValueError("edge_x * edge_y must equal M")
+    nb = torch.empty((D, M), dtype=torch.float32, device=num.device)
+    cb = torch.empty(M, dtype=torch.float32, device=num.device)
+    with torch.cuda.device(num.device):
+        _check(load().bmu_update_blur(num.data_ptr(), cnt.data_ptr(), D, edge_x, edge_y,
+                                      float(sigma), nb.data_ptr(), cb.data_ptr(), _stream(num)))
+    return nb, cb
+
+
+def bmu_update_writeback(num_blur, cnt_blur, W):
+    """W[f, j] = num_blur[f, j] / cnt_blur[j] where cnt_blur[j] > 0 (in place)."""
+    wp, D, M = _codebook(W)
+    with torch.cuda.device(W.device):
+        _check(load().bmu_update_writeback(_dev(num_blur, torch.float32, "num_blur"),
+                                           _dev(cnt_blur, torch.float32, "cnt_blur"), D, M, wp,
+                                           _stream(W)))
+    return W
 
 
 ROOFS = {"l2_ldg": 0, "l2_bulk": 1, "smem": 2, "l1": 3, "fadd": 4, "fadd2": 5}

@@ -817,6 +817,51 @@ int bmu_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, in
     return BMU_OK;
 }
 
+// ---- the rest of a batch epoch (Table 4: scatter, blur, write-back) -----------
+int bmu_update_scatter(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
+                       const int32_t *bmu, int64_t D, int64_t M, uint32_t *num, uint32_t *cnt,
+                       void *stream)
+{
+    int rc = check_sizes(D, M, N, nnz);
+    if (rc) return rc;
+    if (N == 0) return BMU_OK;
+    if (!rowptr || !bmu || !num || !cnt || (nnz > 0 && !colidx)) {
+        set_error("null pointer argument");
+        return BMU_ERR_INVALID_ARG;
+    }
+    return launch_update_scatter(rowptr, colidx, N, bmu, M, num, cnt, static_cast<cudaStream_t>(stream));
+}
+
+int bmu_update_blur(const uint32_t *num, const uint32_t *cnt, int64_t D, int32_t edge_x,
+                    int32_t edge_y, float sigma, float *num_blur, float *cnt_blur, void *stream)
+{
+    if (D < 0 || edge_x < 0 || edge_y < 0 || !(sigma >= 0.f)) {
+        set_error("negative size or sigma");
+        return BMU_ERR_INVALID_ARG;
+    }
+    int rc = check_sizes(D, (int64_t)edge_x * edge_y, 0, 0);
+    if (rc) return rc;
+    if (D > LANES_MAX_D) { set_error("blur: D beyond %d", LANES_MAX_D); return BMU_ERR_UNSUPPORTED; }
+    if ((int64_t)edge_x * edge_y == 0) return BMU_OK;
+    if (!cnt || !cnt_blur || (D > 0 && (!num || !num_blur))) {
+        set_error("null pointer argument");
+        return BMU_ERR_INVALID_ARG;
+    }
+    return launch_update_blur(num, cnt, D, edge_x, edge_y, sigma, num_blur, cnt_blur,
+                              static_cast<cudaStream_t>(stream));
+}
+
+int bmu_update_writeback(const float *num_blur, const float *cnt_blur, int64_t D, int64_t M,
+                         float *W, void *stream)
+{
+    int rc = check_sizes(D, M, 0, 0);
+    if (rc) return rc;
+    if (D * M == 0) return BMU_OK;
+    if (D > 65535) { set_error("write-back: D beyond 65535"); return BMU_ERR_UNSUPPORTED; }
+    if (!num_blur || !cnt_blur || !W) { set_error("null pointer argument"); return BMU_ERR_INVALID_ARG; }
+    return launch_update_writeback(num_blur, cnt_blur, D, M, W, static_cast<cudaStream_t>(stream));
+}
+
 }  // extern "C"
 
 // ---- search with library-resident scratch (no allocation anywhere) ---------

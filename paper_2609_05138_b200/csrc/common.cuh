@@ -256,6 +256,16 @@ int launch_sweep_rows(const RowsArgs &a, const bmu_opts &o, cudaStream_t s);
 // same with W pointing at an fp16 codebook (row pitch 2*M bytes), 256-neuron slabs
 int launch_sweep_rows_f16(const RowsArgs &a, const bmu_opts &o, cudaStream_t s);
 
+// update step (update.cu): scatter, neighbourhood blur, write-back
+int launch_update_scatter(const int32_t *rowptr, const int32_t *colidx, int64_t N,
+                          const int32_t *bmu, int64_t M, uint32_t *num, uint32_t *cnt,
+                          cudaStream_t s);
+int launch_update_blur(const uint32_t *num, const uint32_t *cnt, int64_t D, int32_t edge_x,
+                       int32_t edge_y, float sigma, float *num_blur, float *cnt_blur,
+                       cudaStream_t s);
+int launch_update_writeback(const float *num_blur, const float *cnt_blur, int64_t D, int64_t M,
+                            float *W, cudaStream_t s);
+
 int launch_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                         int64_t D, int32_t *flags, cudaStream_t s);
 

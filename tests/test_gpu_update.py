@@ -1,0 +1,127 @@
+"""Parity of the update step (scatter, neighbourhood blur, write-back; Table 4) against
+the oracle, through the C ABI.  The scatter's integer counters must be bit-exact; the
+blur (fp32 sums of at most 49 + 49 terms against fp64) within 2e-6 of the plane's largest
+value; the write-back within one fp32 rounding."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from inputs import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def bmu():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_05138_b200 as lib
+    lib.load()
+    return lib
+
+
+def gpu_scatter(bmu, rowptr, colidx, units, D, M, num=None, cnt=None):
+    if num is None:
+        num = torch.zeros((D, M), dtype=torch.int32, device="cuda")
+        cnt = torch.zeros(M, dtype=torch.int32, device="cuda")
+    bmu.bmu_update_scatter(rowptr.cuda(), colidx.cuda(), units.cuda(), num, cnt)
+    torch.cuda.synchronize()
+    return num, cnt
+
+
+@pytest.mark.parametrize("mode", ["random", "one_unit", "few_units"])
+def test_scatter_is_bit_exact(bmu, mode):
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=3001)
+    D, M = cfg.D, 400
+    g = torch.Generator().manual_seed(5)
+    N = rowptr.numel() - 1
+    units = {"random": torch.randint(0, M, (N,), generator=g),
+             "one_unit": torch.full((N,), 37),
+             "few_units": torch.randint(0, 3, (N,), generator=g) * 199}[mode].to(torch.int32)
+    num, cnt = gpu_scatter(bmu, rowptr, colidx, units, D, M)
+    onum, ocnt = oracle.scatter(rowptr.numpy(), colidx.numpy(), units.numpy(), D, M)
+    assert np.array_equal(num.cpu().numpy().astype(np.uint64), onum)
+    assert np.array_equal(cnt.cpu().numpy().astype(np.uint64), ocnt)
+
+
+def test_scatter_accumulates_batches_and_takes_odd_rows(bmu):
+    D, M = 300, 37
+    nnz = torch.tensor([0, 5, 1, 40, 0, 33, 2] * 30)
+    rowptr, colidx = synth.draw_corpus(nnz.numel(), D, 1.0, nnz, seed=2)
+    ci = colidx.numpy().copy()
+    ci[rowptr[3]:rowptr[3] + 2] = 7                       # a repeated id counts twice
+    colidx = torch.from_numpy(ci)
+    units = (torch.arange(nnz.numel()) % M).to(torch.int32)
+    num, cnt = gpu_scatter(bmu, rowptr, colidx, units, D, M)
+    num, cnt = gpu_scatter(bmu, rowptr, colidx, units, D, M, num, cnt)     # second batch: same docs
+    onum, ocnt = oracle.scatter(rowptr.numpy(), ci, units.numpy(), D, M)
+    assert np.array_equal(num.cpu().numpy().astype(np.uint64), 2 * onum)
+    assert np.array_equal(cnt.cpu().numpy().astype(np.uint64), 2 * ocnt)
+
+
+@pytest.mark.parametrize("ex,ey,sigma,D", [(32, 32, 1.0, 5), (64, 64, 2.5, 3), (45, 70, 0.4, 4),
+                                          (33, 31, 8.0, 2), (7, 5, 1.5, 6), (128, 16, 0.0, 3),
+                                          (100, 100, 3.3, 2)])
+def test_blur_matches_oracle(bmu, ex, ey, sigma, D):
+    M = ex * ey
+    g = torch.Generator().manual_seed(ex + ey)
+    num = torch.randint(0, 2_000_000, (D, M), generator=g, dtype=torch.int32)
+    num[0] = 0
+    num[0, (ey // 2) * ex + ex // 2] = 1000               # an impulse plane
+    cnt = torch.randint(0, 50, (M,), generator=g, dtype=torch.int32)
+    nb, cb = bmu.bmu_update_blur(num.cuda(), cnt.cuda(), ex, ey, sigma)
+    torch.cuda.synchronize()
+    ref_n = oracle.blur(num.numpy(), ex, ey, sigma)
+    ref_c = oracle.blur(cnt.numpy(), ex, ey, sigma)
+    for got, ref in ((nb.cpu().numpy(), ref_n), (cb.cpu().numpy()[None], ref_c[None])):
+        tol = 2e-6 * np.abs(ref).max(axis=-1, keepdims=True)
+        assert np.all(np.abs(got - ref) <= tol), float(np.abs(got - ref).max())
+    if sigma == 0.0:
+        assert np.array_equal(nb.cpu().numpy(), num.numpy().astype(np.float32))
+
+
+def test_blur_refuses_a_neighbourhood_it_cannot_hold(bmu):
+    num = torch.zeros((1, 64), dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(64, dtype=torch.int32, device="cuda")
+    with pytest.raises(bmu.BmuError) as e:
+        bmu.bmu_update_blur(num, cnt, 8, 8, 8.5)
+    assert e.value.status == 2
+
+
+@pytest.mark.parametrize("D,M", [(40, 256), (33, 101)])
+def test_writeback_matches_oracle(bmu, D, M):
+    r = np.random.default_rng(D)
+    B = r.random((D, M)).astype(np.float32) * 1000
+    c = (r.random(M).astype(np.float32) * 50) * (r.random(M) > 0.2)
+    W0 = r.random((D, M)).astype(np.float32)
+    W = torch.from_numpy(W0.copy()).cuda()
+    bmu.bmu_update_writeback(torch.from_numpy(B).cuda(), torch.from_numpy(c.astype(np.float32)).cuda(), W)
+    torch.cuda.synchronize()
+    ref = oracle.writeback(B, c, W0)
+    got = W.cpu().numpy()
+    np.testing.assert_allclose(got, ref, rtol=1.2e-7, atol=0)
+    assert np.array_equal(got[:, c == 0], W0[:, c == 0])   # units without weight keep theirs
+
+
+def test_whole_epoch_against_oracle_chain(bmu):
+    """search -> scatter -> blur -> write-back -> norms, the oracle fed the same assignments."""
+    cfg = synth.CONFIGS["cfg1"]
+    ex, ey, sigma = 32, 20, 1.3
+    M = ex * ey
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=4000)
+    W0 = synth.make_codebook(cfg.D, M, 17, kind="scaled")
+    W = W0.clone().cuda()
+    units, _ = bmu.bmu_search_ws(W, rowptr.cuda(), colidx.cuda())
+    num, cnt = gpu_scatter(bmu, rowptr, colidx, units.cpu(), cfg.D, M)
+    nb, cb = bmu.bmu_update_blur(num, cnt, ex, ey, sigma)
+    bmu.bmu_update_writeback(nb, cb, W)
+    nrm = bmu.bmu_codebook_norms(W)
+    torch.cuda.synchronize()
+    onum, ocnt = oracle.scatter(rowptr.numpy(), colidx.numpy(), units.cpu().numpy(), cfg.D, M)
+    ref = oracle.writeback(oracle.blur(onum, ex, ey, sigma), oracle.blur(ocnt, ex, ey, sigma), W0.numpy())
+    got = W.cpu().numpy()
+    assert np.all(np.abs(got - ref) <= 4e-6 * np.maximum(np.abs(ref), 1e-3))
+    assert got.min() >= 0.0 and got.max() <= 1.0 + 1e-6     # weighted means of binary vectors
+    np.testing.assert_allclose(nrm.cpu().numpy(), oracle.norms(got), rtol=1e-6)
