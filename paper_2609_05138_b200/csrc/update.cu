@@ -34,51 +34,83 @@ update_scatter_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restr
         atomicAdd(num + (int64_t)__ldg(colidx + e) * M + j, 1u);
 }
 
-static const int BLUR_TILE = 32;
-static const int BLUR_RMAX = 24;           // sigma <= 8
+static const int BLUR_TX = 64, BLUR_TY = 32;   // outputs per block
+static const int BLUR_RMAX = 24;               // sigma <= 8
 
-struct BlurTaps { int32_t R; float g[2 * BLUR_RMAX + 1]; };
+// taps g[-R..R] at gp[3 .. 3 + 2R], three zeros on either side so that a window value can be
+// offered to four neighbouring outputs without a range test
+struct BlurTaps { int32_t R; float gp[2 * BLUR_RMAX + 1 + 6]; };
 
-// One block per 32 x 32 tile of one plane: the tile and its halo (zero outside the map) into
-// shared memory, the row pass there, the column pass into the output.  Planes 0 .. D-1 are the
-// feature planes of `num`, plane D is `cnt`.
+// One block per 32 x 64 tile of one plane: the tile and its halo (zero outside the map) into
+// shared memory; the row pass there, four neighbouring outputs per thread from 128-bit
+// shared-memory loads; the column pass into the output, four outputs down a column per thread.
+// Planes 0 .. D-1 are the feature planes of `num`, plane D is `cnt`.
 __global__ void __launch_bounds__(256)
 update_blur_kernel(const uint32_t *__restrict__ num, const uint32_t *__restrict__ cnt, int64_t D,
                    int32_t edge_x, int32_t edge_y, const BlurTaps taps, float *__restrict__ num_blur,
                    float *__restrict__ cnt_blur)
 {
-    extern __shared__ float sm[];
-    const int R = taps.R, span = BLUR_TILE + 2 * R;
-    float *in = sm;                          // span x span
-    float *mid = sm + span * span;           // span rows x BLUR_TILE columns
+    extern __shared__ __align__(16) float sm[];
+    const int R = taps.R, span_y = BLUR_TY + 2 * R;
+    const int pitch = (BLUR_TX + 2 * R + 3) / 4 * 4 + 4;     // floats per staged row (16-byte rows)
+    float *in = sm;                          // span_y x pitch
+    float *mid = sm + span_y * pitch;        // span_y x BLUR_TX
     const int64_t plane = blockIdx.z, M = (int64_t)edge_x * edge_y;
     const uint32_t *src = plane < D ? num + plane * M : cnt;
     float *dst = plane < D ? num_blur + plane * M : cnt_blur;
-    const int x0 = blockIdx.x * BLUR_TILE, y0 = blockIdx.y * BLUR_TILE;
+    const int x0 = blockIdx.x * BLUR_TX, y0 = blockIdx.y * BLUR_TY;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
 
-    for (int idx = threadIdx.x; idx < span * span; idx += blockDim.x) {
-        const int r = idx / span, c = idx - r * span;
-        const int y = y0 - R + r, x = x0 - R + c;
-        in[idx] = (y >= 0 && y < edge_y && x >= 0 && x < edge_x)
-                      ? (float)__ldg(src + (int64_t)y * edge_x + x) : 0.f;
+    for (int r = ty; r < span_y; r += 8) {
+        const int y = y0 - R + r;
+        const bool row_in = y >= 0 && y < edge_y;
+        for (int c = tx; c < pitch; c += 32) {
+            const int x = x0 - R + c;
+            in[r * pitch + c] = (row_in && x >= 0 && x < edge_x)
+                                    ? (float)__ldg(src + (int64_t)y * edge_x + x) : 0.f;
+        }
     }
     __syncthreads();
-    for (int idx = threadIdx.x; idx < span * BLUR_TILE; idx += blockDim.x) {
-        const int r = idx / BLUR_TILE, c = idx - r * BLUR_TILE;
-        const float *row = in + r * span + c;
-        float s = 0.f;
-        for (int d = 0; d <= 2 * R; ++d) s = fmaf(taps.g[d], row[d], s);
-        mid[idx] = s;
+    // row pass: item = (row r, group of four outputs c4); output x = 4 c4 + o reads in[r][x + d]
+    const int groups = BLUR_TX / 4;
+    for (int item = threadIdx.x; item < span_y * groups; item += 256) {
+        const int r = item / groups, c4 = item - r * groups;
+        const float4 *win = reinterpret_cast<const float4 *>(in + r * pitch + 4 * c4);
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        const int pieces = (4 + 2 * R + 3) / 4;
+        for (int k = 0; k < pieces; ++k) {
+            const float4 v = win[k];
+            const float *g = taps.gp + 4 * k;                // value e = 4k + i serves output o with
+            a0 = fmaf(g[3], v.x, a0); a1 = fmaf(g[2], v.x, a1);   // tap d = e - o: gp[e - o + 3]
+            a2 = fmaf(g[1], v.x, a2); a3 = fmaf(g[0], v.x, a3);
+            a0 = fmaf(g[4], v.y, a0); a1 = fmaf(g[3], v.y, a1);
+            a2 = fmaf(g[2], v.y, a2); a3 = fmaf(g[1], v.y, a3);
+            a0 = fmaf(g[5], v.z, a0); a1 = fmaf(g[4], v.z, a1);
+            a2 = fmaf(g[3], v.z, a2); a3 = fmaf(g[2], v.z, a3);
+            a0 = fmaf(g[6], v.w, a0); a1 = fmaf(g[5], v.w, a1);
+            a2 = fmaf(g[4], v.w, a2); a3 = fmaf(g[3], v.w, a3);
+        }
+        *reinterpret_cast<float4 *>(mid + r * BLUR_TX + 4 * c4) = make_float4(a0, a1, a2, a3);
     }
     __syncthreads();
-    for (int idx = threadIdx.x; idx < BLUR_TILE * BLUR_TILE; idx += blockDim.x) {
-        const int r = idx / BLUR_TILE, c = idx - r * BLUR_TILE;
-        const int y = y0 + r, x = x0 + c;
-        if (y >= edge_y || x >= edge_x) continue;
-        const float *col = mid + r * BLUR_TILE + c;
-        float s = 0.f;
-        for (int d = 0; d <= 2 * R; ++d) s = fmaf(taps.g[d], col[d * BLUR_TILE], s);
-        dst[(int64_t)y * edge_x + x] = s;
+    // column pass: item = (group of four rows r4, column c)
+    for (int item = threadIdx.x; item < (BLUR_TY / 4) * BLUR_TX; item += 256) {
+        const int r4 = item / BLUR_TX, c = item - r4 * BLUR_TX;
+        const float *col = mid + (4 * r4) * BLUR_TX + c;
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        for (int e = 0; e < 4 + 2 * R; ++e) {
+            const float v = col[e * BLUR_TX];
+            const float *g = taps.gp + e;
+            a0 = fmaf(g[3], v, a0); a1 = fmaf(g[2], v, a1);
+            a2 = fmaf(g[1], v, a2); a3 = fmaf(g[0], v, a3);
+        }
+        const int x = x0 + c, y = y0 + 4 * r4;
+        if (x < edge_x) {
+            if (y < edge_y) dst[(int64_t)y * edge_x + x] = a0;
+            if (y + 1 < edge_y) dst[(int64_t)(y + 1) * edge_x + x] = a1;
+            if (y + 2 < edge_y) dst[(int64_t)(y + 2) * edge_x + x] = a2;
+            if (y + 3 < edge_y) dst[(int64_t)(y + 3) * edge_x + x] = a3;
+        }
     }
 }
 
@@ -133,13 +165,23 @@ int launch_update_blur(const uint32_t *num, const uint32_t *cnt, int64_t D, int3
                   (double)sigma, t.R, BLUR_RMAX);
         return BMU_ERR_UNSUPPORTED;
     }
+    for (int i = 0; i < 2 * BLUR_RMAX + 1 + 6; ++i) t.gp[i] = 0.f;
     for (int d = -t.R; d <= t.R; ++d)
-        t.g[d + t.R] = sigma > 0.f
+        t.gp[d + t.R + 3] = sigma > 0.f
             ? (float)exp(-(double)(d * d) / (2.0 * (double)sigma * (double)sigma)) : 1.f;
-    const int span = BLUR_TILE + 2 * t.R;
-    const size_t smem = (size_t)(span * span + span * BLUR_TILE) * sizeof(float);
-    const dim3 grid((unsigned)((edge_x + BLUR_TILE - 1) / BLUR_TILE),
-                    (unsigned)((edge_y + BLUR_TILE - 1) / BLUR_TILE), (unsigned)(D + 1));
+    const int span_y = BLUR_TY + 2 * t.R;
+    const int pitch = (BLUR_TX + 2 * t.R + 3) / 4 * 4 + 4;
+    const size_t smem = (size_t)(span_y * pitch + span_y * BLUR_TX) * sizeof(float);
+    static bool configured[64];
+    int dev = 0;
+    BMU_CUDA(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        BMU_CUDA(cudaFuncSetAttribute(update_blur_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      64 * 1024));
+        configured[dev] = true;
+    }
+    const dim3 grid((unsigned)((edge_x + BLUR_TX - 1) / BLUR_TX),
+                    (unsigned)((edge_y + BLUR_TY - 1) / BLUR_TY), (unsigned)(D + 1));
     update_blur_kernel<<<grid, 256, smem, s>>>(num, cnt, D, edge_x, edge_y, t, num_blur, cnt_blur);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
