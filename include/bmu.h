@@ -147,6 +147,34 @@ BMU_API int bmu_search_ws(const float *W, int64_t D, int64_t M, const float *nor
                   void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Reusable tiling plan.  The paper's epochs run over a frozen, pre-ordered corpus
+ * (Section 5: the corpus is clustered once, offline; Section 4.2, tile
+ * membership), so the document-tiling pass -- ordering, id re-packing, tile
+ * matrices, head masks -- can be done once and reused by every epoch's search.
+ *   bmu_plan_workspace_bytes  bytes of 256-byte aligned device memory a plan needs
+ *       (the plan itself plus the scratch of the searches that use it).
+ *   bmu_plan_create  runs the tiling pass into `workspace` (asynchronous on
+ *       `stream`) and returns a host handle in *plan.  rowptr, colidx and the
+ *       workspace stay owned by the caller and must stay alive and unchanged
+ *       until bmu_plan_destroy; `nnz` is the length of colidx.
+ *   bmu_search_planned  the search of bmu_search_ws without its tiling pass:
+ *       norms (NULL = computed), sweep, outputs.  W must be 16-byte aligned.
+ *       Allocates nothing, asynchronous on `stream`; searches that share a plan
+ *       must not overlap on the GPU.  Results equal bmu_search_ws with the same
+ *       options bit for bit.
+ *   bmu_plan_destroy  frees the host handle (not the workspace).
+ */
+typedef struct bmu_plan bmu_plan;
+BMU_API size_t bmu_plan_workspace_bytes(int64_t N, int64_t nnz, int64_t D, int64_t M,
+                                        const bmu_opts *opts);
+BMU_API int bmu_plan_create(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
+                            int64_t D, int64_t M, const bmu_opts *opts, void *workspace,
+                            size_t workspace_bytes, bmu_plan **plan, void *stream);
+BMU_API int bmu_search_planned(const bmu_plan *plan, const float *W, const float *norms,
+                               int32_t *out_bmu, float *out_dist, void *stream);
+BMU_API void bmu_plan_destroy(bmu_plan *plan);
+
+/*
  * The same search that also returns the second-best unit, which the paper's
  * kernel tracks because topographic error -- gated on by its stopping rules --
  * needs it (Table 5, "bmu1-only").  out_bmu2[i] is the lowest index j !=

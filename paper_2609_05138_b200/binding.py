@@ -87,6 +87,15 @@ EXPORTS = {
     "bmu_release_scratch": (ctypes.c_int, []),
     "bmu_validate_csr": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                         ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
+    "bmu_plan_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
+                                                   ctypes.c_int64, ctypes.c_void_p]),
+    "bmu_plan_create": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                                       ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
+                                       ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
+                                       ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p]),
+    "bmu_search_planned": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "bmu_plan_destroy": (None, [ctypes.c_void_p]),
     "bmu_update_scatter": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                           ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64,
                                           ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
@@ -340,6 +349,53 @@ def bmu_validate_csr(rowptr, colidx, D: int):
             _dev(rowptr, torch.int32, "rowptr"),
             _dev(colidx, torch.int32, "colidx") if colidx.numel() else None, N, colidx.numel(),
             D, _stream(rowptr)))
+
+
+class Plan:
+    """A tiling plan of one corpus batch for a codebook shape (bmu_plan_create); keeps the
+    tensors it refers to alive."""
+
+    def __init__(self, rowptr, colidx, D: int, M: int, opts: Opts | None = None):
+        self.rowptr, self.colidx, self.D, self.M, self.opts = rowptr, colidx, D, M, opts
+        self.N = rowptr.numel() - 1
+        nnz = colidx.numel()
+        op = ctypes.byref(opts) if opts else None
+        need = int(load().bmu_plan_workspace_bytes(self.N, nnz, D, M, op))
+        self.workspace = torch.empty(need + 256, dtype=torch.uint8, device=rowptr.device)
+        ws_ptr = (self.workspace.data_ptr() + 255) // 256 * 256
+        handle = ctypes.c_void_p()
+        with torch.cuda.device(rowptr.device):
+            _check(load().bmu_plan_create(
+                _dev(rowptr, torch.int32, "rowptr"),
+                _dev(colidx, torch.int32, "colidx") if nnz else None, self.N, nnz, D, M, op,
+                ws_ptr, need, ctypes.byref(handle), _stream(rowptr)))
+        self.handle = handle
+
+    def search(self, W, norms=None, out_bmu=None, out_dist=None):
+        wp, D, M = _codebook(W)
+        if (D, M) != (self.D, self.M):
+            raise ValueError("codebook shape differs from the plan's")
+        if out_bmu is None:
+            out_bmu = torch.empty(self.N, dtype=torch.int32, device=W.device)
+        if out_dist is None:
+            out_dist = torch.empty(self.N, dtype=torch.float32, device=W.device)
+        with torch.cuda.device(W.device):
+            _check(load().bmu_search_planned(
+                self.handle, wp, _dev(norms, torch.float32, "norms") if norms is not None else None,
+                _dev(out_bmu, torch.int32, "out_bmu"), _dev(out_dist, torch.float32, "out_dist"),
+                _stream(W)))
+        return out_bmu, out_dist
+
+    def close(self):
+        if self.handle:
+            load().bmu_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 # ---- the rest of a batch epoch: scatter, blur, write-back (Table 4) ----------

@@ -6,6 +6,7 @@
 #include <string.h>
 
 #include <mutex>
+#include <new>
 
 namespace bmu {
 
@@ -184,8 +185,10 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
                        const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                        int32_t *out_bmu, float *out_dist, const bmu_opts *opts_in, void *ws,
                        size_t ws_bytes, cudaStream_t s, int32_t *out_bmu2 = nullptr,
-                       float *out_dist2 = nullptr)
+                       float *out_dist2 = nullptr, int phase = 0)
 {
+    // phase 0: the whole search; 1: only the tiling pass (bmu_plan_create); 2: everything but
+    // the tiling pass, whose results are still in the workspace (bmu_search_planned)
     const bool top2 = out_bmu2 != nullptr || out_dist2 != nullptr;
     int rc = check_sizes(D, M, N, nnz);
     if (rc) return rc;
@@ -194,10 +197,17 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     if (opts_in) o = *opts_in;
     if ((rc = check_opts(o))) return rc;
     if (N == 0) return BMU_OK;
-    if (!W || !rowptr || !out_bmu || !out_dist || (nnz > 0 && !colidx) ||
-        (top2 && (!out_bmu2 || !out_dist2))) {
+    if (!rowptr || (nnz > 0 && !colidx) ||
+        (phase != 1 && (!W || !out_bmu || !out_dist || (top2 && (!out_bmu2 || !out_dist2))))) {
         set_error("null pointer argument");
         return BMU_ERR_INVALID_ARG;
+    }
+    // a plan is made before the codebook is known: it assumes the aligned fast path, and the
+    // search that uses it insists on it
+    const uintptr_t w_addr = phase == 1 ? 0 : reinterpret_cast<uintptr_t>(W);
+    if (phase == 2 && (w_addr & 15) != 0) {
+        set_error("a planned search needs W 16-byte aligned");
+        return BMU_ERR_UNSUPPORTED;
     }
     if (M == 0 || D == 0) {
         set_error("empty codebook (D=%lld, M=%lld): no neuron to return", (long long)D, (long long)M);
@@ -213,7 +223,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     char *base = static_cast<char *>(ws);
     u64 *state = reinterpret_cast<u64 *>(base + l.state_off);
     u64 *state2 = top2 ? reinterpret_cast<u64 *>(base + l.state2_off) : nullptr;
-    if (!norms) {
+    if (!norms && phase != 1) {
         float *n = reinterpret_cast<float *>(base + l.norms_off);
         if ((rc = launch_norms(W, D, M, n, s))) return rc;
         norms = n;
@@ -225,14 +235,14 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         set_error("the staged kernel does not track the second-best unit");
         return BMU_ERR_UNSUPPORTED;
     }
-    if (staged && !staged_possible(W, D, M)) {
+    if (staged && !staged_possible(reinterpret_cast<const float *>(w_addr), D, M)) {
         set_error("staged kernel needs M %% 4 == 0, M >= 32, 256 <= D <= %d and W 16-byte aligned",
                   LANES_MAX_D);
         return BMU_ERR_UNSUPPORTED;
     }
     // the planned warp-per-document kernel needs 16-bit ids and whole 16-byte row pieces
     const bool planned_ok = D <= LANES_MAX_D && M % 4 == 0 && M >= rows_slab_width(o) &&
-                            (reinterpret_cast<uintptr_t>(W) & 15) == 0;
+                            (w_addr & 15) == 0;
     if (o.kernel == 3 && !planned_ok) {
         set_error("planned kernel needs M %% 4 == 0, M >= 128, D <= %d and W 16-byte aligned",
                   LANES_MAX_D);
@@ -259,16 +269,18 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     }
     const bool planned = !tiled && !mma && (o.kernel == 3 || (o.kernel == 0 && planned_ok));
     char *pw = base + l.plan_off;
-    if (staged || planned || tiled || mma)
+    if ((staged || planned || tiled || mma) && phase != 2)
         if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, mma ? head : 0, pw, l.plan, s)))
             return rc;
     if (mma) {
+        if (phase != 2 &&
+            (rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, pw, l.plan, s))) return rc;
+        if (phase == 1) return BMU_OK;
         const int64_t m_full = M / MMA_SLAB * MMA_SLAB;
         uint32_t *head_max = status + 16;
         unsigned char *img = reinterpret_cast<unsigned char *>(base + l.head_off);
         if ((rc = wide ? launch_head_split2(W, M, m_full, head, head_max, img, s)
                        : launch_head_split(W, M, m_full, head, head_max, img, s))) return rc;
-        if ((rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, pw, l.plan, s))) return rc;
         MmaArgs a;
         a.W = W; a.M = M; a.N = N; a.n_tiles = (N + 7) / 8; a.norms = norms;
         a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
@@ -308,7 +320,9 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     }
     if (tiled) {
         const int head = (o.tile_head == 1 || D < TILE_HEAD_ROWS) ? 0 : TILE_HEAD_ROWS;
-        if ((rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, pw, l.plan, s))) return rc;
+        if (phase != 2 &&
+            (rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, pw, l.plan, s))) return rc;
+        if (phase == 1) return BMU_OK;
         TileArgs a;
         a.W = W; a.M = M; a.N = N; a.n_tiles = (N + 7) / 8; a.norms = norms;
         a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
@@ -338,6 +352,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         }
         return launch_finalize(state, state2, rowptr, N, out_bmu, out_dist, out_bmu2, out_dist2, s);
     }
+    if (phase == 1) return BMU_OK;           // nothing more to prepare for the other kernels
     if (planned) {
         const int slab = rows_slab_width(o);
         RowsArgs a;
@@ -816,6 +831,52 @@ int bmu_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, in
     }
     return BMU_OK;
 }
+
+// ---- reusable tiling plan: a frozen corpus searched once per epoch ------------
+struct bmu_plan {
+    int64_t D, M, N, nnz;
+    bmu_opts opts;
+    const int32_t *rowptr, *colidx;
+    void *ws;
+    size_t ws_bytes;
+};
+
+size_t bmu_plan_workspace_bytes(int64_t N, int64_t nnz, int64_t D, int64_t M, const bmu_opts *opts)
+{
+    return bmu_search_workspace_bytes(D, M, N, nnz, opts);
+}
+
+int bmu_plan_create(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz, int64_t D,
+                    int64_t M, const bmu_opts *opts, void *workspace, size_t workspace_bytes,
+                    bmu_plan **plan, void *stream)
+{
+    if (!plan) { set_error("null pointer argument"); return BMU_ERR_INVALID_ARG; }
+    *plan = nullptr;
+    if (N <= 0) { set_error("a plan needs at least one document"); return BMU_ERR_INVALID_ARG; }
+    int rc = search_impl(nullptr, D, M, nullptr, rowptr, colidx, N, nnz, nullptr, nullptr, opts,
+                         workspace, workspace_bytes, static_cast<cudaStream_t>(stream), nullptr,
+                         nullptr, 1);
+    if (rc) return rc;
+    bmu_plan *p = new (std::nothrow) bmu_plan;
+    if (!p) { set_error("out of host memory"); return BMU_ERR_INVALID_ARG; }
+    p->D = D; p->M = M; p->N = N; p->nnz = nnz;
+    memset(&p->opts, 0, sizeof(p->opts));
+    if (opts) p->opts = *opts;
+    p->rowptr = rowptr; p->colidx = colidx; p->ws = workspace; p->ws_bytes = workspace_bytes;
+    *plan = p;
+    return BMU_OK;
+}
+
+int bmu_search_planned(const bmu_plan *plan, const float *W, const float *norms, int32_t *out_bmu,
+                       float *out_dist, void *stream)
+{
+    if (!plan) { set_error("null plan"); return BMU_ERR_INVALID_ARG; }
+    return search_impl(W, plan->D, plan->M, norms, plan->rowptr, plan->colidx, plan->N, plan->nnz,
+                       out_bmu, out_dist, &plan->opts, plan->ws, plan->ws_bytes,
+                       static_cast<cudaStream_t>(stream), nullptr, nullptr, 2);
+}
+
+void bmu_plan_destroy(bmu_plan *plan) { delete plan; }
 
 // ---- the rest of a batch epoch (Table 4: scatter, blur, write-back) -----------
 int bmu_update_scatter(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,

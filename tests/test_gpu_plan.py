@@ -1,0 +1,50 @@
+"""The reusable tiling plan (bmu_plan_create / bmu_search_planned): the plan is made once for
+a frozen corpus and every search that uses it returns exactly what bmu_search_ws returns."""
+import pytest
+import torch
+
+from inputs import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def bmu():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_05138_b200 as lib
+    lib.load()
+    return lib
+
+
+@pytest.mark.parametrize("kernel", [0, 1, 3, 4, 5, 6])
+def test_planned_search_equals_one_shot_search_and_is_reusable(bmu, kernel):
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=2300)
+    rp, ci = rowptr.cuda(), colidx.cuda()
+    o = bmu.Opts()
+    o.kernel = kernel
+    plan = bmu.Plan(rp, ci, cfg.D, 1024 + 40, o)
+    for seed in (3, 4):                                   # two "epochs": two codebooks, one plan
+        W = synth.make_codebook(cfg.D, 1024 + 40, seed, kind="scaled").cuda()
+        a = plan.search(W)
+        b = bmu.bmu_search_ws(W, rp, ci, opts=o)
+        torch.cuda.synchronize()
+        assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    nrm = bmu.bmu_codebook_norms(W)
+    c = plan.search(W, norms=nrm)
+    assert torch.equal(c[0], b[0]) and torch.equal(c[1], b[1])
+    plan.close()
+
+
+def test_planned_search_argument_checks(bmu):
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=50)
+    plan = bmu.Plan(rowptr.cuda(), colidx.cuda(), cfg.D, 256)
+    with pytest.raises(ValueError):
+        plan.search(torch.zeros(cfg.D, 128, device="cuda"))
+    W = torch.zeros(cfg.D * 256 + 1, device="cuda")[1:].view(cfg.D, 256)      # 4-byte aligned only
+    with pytest.raises(bmu.BmuError) as e:
+        plan.search(W)
+    assert e.value.status == 2
+    assert bmu.load().bmu_search_planned(None, None, None, None, None, None) == 1
