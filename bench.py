@@ -437,18 +437,19 @@ def run_ours(args, cfg, rank, local_rank, world):
     }
     # ---- the same step with the tiling pass done beforehand (a frozen corpus, reused per epoch)
     if len(batches) == 1:
+        n0 = rowptr.numel() - 1
         plan = bmu.Plan(rowptr, colidx, cfg.D, cfg.M, opts)
-        plan.search(W, norms=norms, out_bmu=out_bmu[:N], out_dist=out_dist[:N])
+        plan.search(W, norms=norms, out_bmu=out_bmu[:n0], out_dist=out_dist[:n0])
         torch.cuda.synchronize(dev)
         p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         p0.record()
         for _ in range(args.steps):
             bmu.bmu_codebook_norms(W, norms)
-            plan.search(W, norms=norms, out_bmu=out_bmu[:N], out_dist=out_dist[:N])
+            plan.search(W, norms=norms, out_bmu=out_bmu[:n0], out_dist=out_dist[:n0])
         p1.record()
         torch.cuda.synchronize(dev)
         planned_ms = p0.elapsed_time(p1) / args.steps
-        line["planned"] = {"ms_per_step": planned_ms, "value": N / (planned_ms * 1e-3), "unit": UNIT,
+        line["planned"] = {"ms_per_step": planned_ms, "value": n0 / (planned_ms * 1e-3), "unit": UNIT,
                            "api": "bmu_plan_create once, then bmu_codebook_norms + "
                                   "bmu_search_planned per step (rank 0's figure)"}
         plan.close()
