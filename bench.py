@@ -454,12 +454,54 @@ def run_ours(args, cfg, rank, local_rank, world):
                                   "bmu_search_planned per step (rank 0's figure)"}
         plan.close()
         del plan
+    if args.comparator:
+        line["comparator"] = comparator_spmm(cfg, W, norms, rowptr, colidx)
     if args.epoch:
         line["epoch"] = epoch_phases(bmu, cfg, W, batches, opts, ws, norms, out_bmu, out_dist,
                                      peaks, args.sigma)
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(cfg, W, rowptr, colidx, rowptr.numel() - 1)
     return line
+
+
+def comparator_spmm(cfg, W, norms, rowptr, colidx, budget_docs=200_000):
+    """The other side of the paper's comparison (Section 3: a library sparse-dense product that
+    materialises the score block, then a separate arg-min), on this GPU and these arrays:
+    torch.sparse CSR x dense fp32 (cuSPARSE SpMM) per document batch, then n_j - 2 s_ij and
+    torch.argmin.  A comparator only: nothing of it is part of the library.  Timed on a bounded
+    prefix of the workload (documents are independent, so docs/s extrapolates)."""
+    dev = W.device
+    n_docs = min(rowptr.numel() - 1, budget_docs)
+    batch = int(max(1024, min(n_docs, (2 << 30) // (cfg.M * 4))))      # score block <= 2 GiB
+    rp64 = rowptr[: n_docs + 1].to(torch.int64)
+    ci64 = colidx[: int(rp64[-1])].to(torch.int64)
+    ones = torch.ones(ci64.numel(), device=dev)
+
+    def one_pass():
+        out = torch.empty(n_docs, dtype=torch.int64, device=dev)
+        for lo in range(0, n_docs, batch):
+            hi = min(n_docs, lo + batch)
+            a, b = int(rp64[lo]), int(rp64[hi])
+            X = torch.sparse_csr_tensor(rp64[lo:hi + 1] - a, ci64[a:b], ones[a:b],
+                                        size=(hi - lo, cfg.D))
+            S = X @ W
+            out[lo:hi] = torch.argmin(torch.addcmul(norms[None, :], S, S.new_full((), -2.0)), dim=1)
+        return out
+
+    import warnings
+    with warnings.catch_warnings():
+        warnings.simplefilter("ignore")
+        one_pass()
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        one_pass()
+        e1.record()
+        torch.cuda.synchronize(dev)
+    ms = e0.elapsed_time(e1)
+    return {"kind": "materialised score block: torch.sparse CSR x dense fp32 (cuSPARSE SpMM) + "
+                    "torch.argmin, batches of %d documents" % batch,
+            "value": n_docs / (ms * 1e-3), "unit": UNIT, "sample_docs": n_docs, "ms": ms}
 
 
 def epoch_phases(bmu, cfg, W, batches, opts, ws, norms, out_bmu, out_dist, peaks, sigma):
@@ -522,6 +564,8 @@ def main():
     ap.add_argument("--opt", action="append", default=[], help="bmu_opts field=value")
     ap.add_argument("--ref-sample", type=int, default=4000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--comparator", action="store_true",
+                    help="also time the materialised-score route (library SpMM + argmin)")
     ap.add_argument("--epoch", action="store_true",
                     help="also time one whole epoch (search + scatter + blur + write-back)")
     ap.add_argument("--sigma", type=float, default=2.0, help="neighbourhood width of --epoch")
