@@ -79,9 +79,9 @@ typedef struct bmu_opts {
                                is a dense contraction on tcgen05 tensor cores with fp32
                                accumulation into double-buffered tensor memory, the
                                remaining ids are gathered as in 4; needs what 4 needs,
-                               D >= head_rows and M >= 512; best unit only; the automatic
-                               choice for large sweeps); 5 first tensor-core sweep (same
-                               split, 512-neuron slabs, head of 256 or 512); 2 staged (a lane per
+                               D >= head_rows and M >= 512; the automatic choice for large
+                               sweeps); 5 first tensor-core sweep (same split, 512-neuron
+                               slabs, head of 256 or 512, best unit only); 2 staged (a lane per
                                document, rows streamed through shared memory by tensor (TMA)
                                box copies; needs M % 4 == 0, M >= 32, 256 <= D <= 65024) */
     int32_t chunk_neurons;  /* neurons per L2-resident chunk of the codebook (Section 4.2,

@@ -73,7 +73,8 @@ static int64_t mma_chunk(const bmu_opts &o, int64_t D, int64_t M)
 static size_t mma_repack_bytes(const bmu_opts &o, int64_t D, int64_t M, int64_t N, int64_t nnz,
                                bool top2)
 {
-    if (o.repack == 2 || top2 || (o.kernel != 0 && o.kernel != 5 && o.kernel != 6)) return 0;
+    if (o.repack == 2 || (top2 && o.kernel == 5) ||
+        (o.kernel != 0 && o.kernel != 5 && o.kernel != 6)) return 0;
     if (D > LANES_MAX_D || M < MMA_SLAB) return 0;
     const int64_t chunk = mma_chunk(o, D, M);
     if (M <= chunk) return 0;                      // one launch: the codebook is the chunk
@@ -114,7 +115,7 @@ static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kerne
     l.head_off = off;
     if (kernel == 5 && !top2 && D >= head && D <= LANES_MAX_D && M >= MMA_SLAB)
         off = align_up(off + head_image_bytes(M, head), 256);
-    if ((kernel == 0 || kernel == 6) && !top2 && D >= head && D <= LANES_MAX_D && M >= MMA_SLAB)
+    if ((kernel == 0 || kernel == 6) && D >= head && D <= LANES_MAX_D && M >= MMA_SLAB)
         off = align_up(off + head_image2_bytes(M, head), 256);
     l.repack_off = off;                  // compact copy of the codebook chunk being swept
     off = align_up(off + repack_bytes, 256);
@@ -250,10 +251,10 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     }
     const bool tiled_ok = planned_ok && M >= 128 && o.cluster != 2;
     // tensor-core head: additionally whole 512-neuron slabs, at least 256 features, best unit only
-    const bool mma_ok = tiled_ok && !top2 && D >= head && M >= MMA_SLAB;
+    const bool mma_ok = tiled_ok && !(top2 && o.kernel == 5) && D >= head && M >= MMA_SLAB;
     if ((o.kernel == 5 || o.kernel == 6) && !mma_ok) {
-        set_error("tensor-core sweep needs what the tiled kernel needs, D >= %d, M >= %d and no "
-                  "second-best unit", head, MMA_SLAB);
+        set_error("tensor-core sweep needs what the tiled kernel needs, D >= %d and M >= %d "
+                  "(kernel 5: no second-best unit)", head, MMA_SLAB);
         return BMU_ERR_UNSUPPORTED;
     }
     // automatic choice for large sweeps: the tensor-core sweep where it applies, else the tiled
@@ -289,7 +290,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         a.tile_ids = reinterpret_cast<const uint4 *>(pw + l.plan.tileids_off);
         a.tile_head = reinterpret_cast<const uint32_t *>(pw + l.plan.tilehead_off);
         a.head_max = head_max; a.head = head;
-        a.state = state; a.status = status;
+        a.state = state; a.state2 = state2; a.status = status;
         const int64_t chunk = mma_chunk(o, D, M);
         float *compact = repack_bytes ? reinterpret_cast<float *>(base + l.repack_off) : nullptr;
         for (int64_t j = 0; j < m_full; j += chunk) {
@@ -310,13 +311,13 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         if (m_full < M) {                      // ragged last slab: generic kernel, merged in
             SweepArgs g;
             g.W = W; g.D = D; g.M = M; g.norms = norms; g.rowptr = rowptr; g.colidx = colidx;
-            g.N = N; g.state = state; g.state2 = nullptr; g.j_lo = (int32_t)m_full;
+            g.N = N; g.state = state; g.state2 = state2; g.j_lo = (int32_t)m_full;
             g.j_hi = (int32_t)M; g.first = 0;
             bmu_opts go;
             memset(&go, 0, sizeof(go));
             if ((rc = launch_sweep_direct(g, go, s))) return rc;
         }
-        return launch_finalize(state, nullptr, rowptr, N, out_bmu, out_dist, nullptr, nullptr, s);
+        return launch_finalize(state, state2, rowptr, N, out_bmu, out_dist, out_bmu2, out_dist2, s);
     }
     if (tiled) {
         const int head = (o.tile_head == 1 || D < TILE_HEAD_ROWS) ? 0 : TILE_HEAD_ROWS;

@@ -200,6 +200,7 @@ struct MmaArgs {
     const unsigned char *head_img;  // split head of slab j_lo / MMA_SLAB onwards (head_image_bytes)
     const uint32_t *head_max;   // bit pattern of max |W[f][j]| over the head rows
     u64 *state;
+    u64 *state2;                // wide-head sweep only: second-best unit (NULL unless wanted)
     uint32_t *status;           // set non-zero if a bounded wait ran out
     int32_t j_lo, j_hi, first;
 };

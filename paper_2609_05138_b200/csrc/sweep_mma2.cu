@@ -39,10 +39,11 @@ static const int M2_TAIL_WARPS = 16;
 static const int M2_THREADS = (M2_TAIL_WARPS + 3) * 32;
 static const int M2_TMEM_COLS = 512;                 // 2 buffers x 2 tiles x 128 documents
 
-static inline size_t m2_smem_bytes(int head)
+static inline size_t m2_smem_bytes(int head, bool top2)
 {
     return (size_t)MMA_DOCS * (head / 8) + (M2_NS + M2_NX) * MMA_STAGE_BYTES +
-           (2 * M2_NS + 2 * M2_NX + 6) * 8 + MMA_DOCS * 8 + 16 + 16 * 16 + 2 * 16 * 4;
+           (2 * M2_NS + 2 * M2_NX + 6) * 8 + MMA_DOCS * 8 + 16 + 16 * 16 + 2 * 16 * 4 +
+           (top2 ? 4 * MMA_DOCS * 16 : 0);
 }
 
 // One thread per (slab, group of 8 features, neuron).  Stage order inside a slab: block of
@@ -114,6 +115,8 @@ __device__ __forceinline__ void m2_unpack(const uint4 q, uint32_t f[8])
     f[4] = q.z & 0xffffu; f[5] = q.z >> 16; f[6] = q.w & 0xffffu; f[7] = q.w >> 16;
 }
 
+// TOP2: also the second-best unit (Table 5: the paper's kernel tracks it for topographic error)
+template <bool TOP2>
 __global__ void __launch_bounds__(M2_THREADS, 1)
 sweep_mma2_kernel(const MmaArgs a)
 {
@@ -132,6 +135,9 @@ sweep_mma2_kernel(const MmaArgs a)
     uint4 *s_first = reinterpret_cast<uint4 *>(tmem_slot + 4);
     uint32_t *s_len = reinterpret_cast<uint32_t *>(s_first + 16);
     uint32_t *s_off = s_len + 16;
+    // TOP2: (best, second) per neuron quarter and document; the warp that owns a quarter of a
+    // document is the same in every slab, so it merges without atomics
+    u64 *kq = reinterpret_cast<u64 *>(s_off + 16);
     const uint32_t wfull0 = mm_smem(bars), wempty0 = mm_smem(bars + NS);
     const uint32_t xfull0 = mm_smem(bars + 2 * NS), xempty0 = mm_smem(bars + 2 * NS + NX);
     const uint32_t tfull0 = mm_smem(bars + 2 * NS + 2 * NX), tempty0 = tfull0 + 16;
@@ -168,6 +174,8 @@ sweep_mma2_kernel(const MmaArgs a)
         }
     }
     if (threadIdx.x < MMA_DOCS) keys[threadIdx.x] = KEY_WORST;
+    if (TOP2)
+        for (int idx = threadIdx.x; idx < 4 * MMA_DOCS * 2; idx += M2_THREADS) kq[idx] = KEY_WORST;
     if (threadIdx.x >= M2_THREADS - 16) {            // 16 threads of the last control warp
         const int t = threadIdx.x - (M2_THREADS - 16);
         const int64_t tile = group * (MMA_DOCS / 8) + t;
@@ -364,15 +372,16 @@ sweep_mma2_kernel(const MmaArgs a)
                 const int col = j0 + li * 4;
                 const float4 n = __ldg(reinterpret_cast<const float4 *>(a.norms + col));
                 const float n4[4] = {n.x, n.y, n.z, n.w};
-                u64 k[8];
+                u64 k[8], k2[8];
 #pragma unroll
                 for (int t = 0; t < 8; ++t) {
                     const float s4[4] = {lo_f(acc[t][0]), hi_f(acc[t][0]), lo_f(acc[t][1]), hi_f(acc[t][1])};
-                    Best<false> bst;
+                    Best<TOP2> bst;
                     bst.init();
 #pragma unroll
                     for (int c = 0; c < 4; ++c) bst.push(fmaf(-2.f, s4[c], n4[c]), col + c);
                     k[t] = make_key(bst.d1, bst.j1);
+                    k2[t] = TOP2 ? make_key(bst.d2, bst.j2) : KEY_WORST;
                 }
                 // transposing butterfly among the 16 lanes that hold the same documents
 #pragma unroll
@@ -383,12 +392,34 @@ sweep_mma2_kernel(const MmaArgs a)
                         const u64 send = (lane & m) ? k[i] : k[i + cnt];
                         const u64 keep = (lane & m) ? k[i + cnt] : k[i];
                         const u64 got = __shfl_xor_sync(0xffffffffu, send, m);
-                        k[i] = got < keep ? got : keep;
+                        if (TOP2) {
+                            const u64 send2 = (lane & m) ? k2[i] : k2[i + cnt];
+                            u64 keep2 = (lane & m) ? k2[i + cnt] : k2[i];
+                            const u64 got2 = __shfl_xor_sync(0xffffffffu, send2, m);
+                            u64 b1 = keep;
+                            Best<true>::merge(b1, keep2, got, got2);
+                            k[i] = b1;
+                            k2[i] = keep2;
+                        } else {
+                            k[i] = got < keep ? got : keep;
+                        }
                     }
                 }
                 const u64 got = __shfl_xor_sync(0xffffffffu, k[0], 8);
-                k[0] = got < k[0] ? got : k[0];
-                if ((lane & 8) == 0) atomicMin(reinterpret_cast<unsigned long long *>(keys + dg * 16 + mydoc), k[0]);
+                if (TOP2) {
+                    const u64 got2 = __shfl_xor_sync(0xffffffffu, k2[0], 8);
+                    Best<true>::merge(k[0], k2[0], got, got2);
+                    if ((lane & 8) == 0) {
+                        u64 *slot = kq + ((size_t)q * MMA_DOCS + dg * 16 + mydoc) * 2;
+                        Best<true>::merge(k[0], k2[0], slot[0], slot[1]);
+                        slot[0] = k[0];
+                        slot[1] = k2[0];
+                    }
+                } else {
+                    k[0] = got < k[0] ? got : k[0];
+                    if ((lane & 8) == 0)
+                        atomicMin(reinterpret_cast<unsigned long long *>(keys + dg * 16 + mydoc), k[0]);
+                }
             }
         }
         __syncwarp();
@@ -401,7 +432,17 @@ sweep_mma2_kernel(const MmaArgs a)
         const int64_t p = group * MMA_DOCS + threadIdx.x;
         if (p < a.N) {
             const int32_t orig = __ldg(a.perm + p);
-            Best<false>::commit(keys[threadIdx.x], KEY_WORST, a.state, nullptr, orig, a.first);
+            if (TOP2) {
+                u64 b1 = KEY_WORST, b2 = KEY_WORST;
+#pragma unroll
+                for (int qq = 0; qq < 4; ++qq) {
+                    const u64 *slot = kq + ((size_t)qq * MMA_DOCS + threadIdx.x) * 2;
+                    Best<true>::merge(b1, b2, slot[0], slot[1]);
+                }
+                Best<true>::commit(b1, b2, a.state, a.state2, orig, a.first);
+            } else {
+                Best<false>::commit(keys[threadIdx.x], KEY_WORST, a.state, nullptr, orig, a.first);
+            }
         }
     }
     if (warp == NTW)
@@ -425,12 +466,15 @@ int launch_sweep_mma2(const MmaArgs &a, const bmu_opts &o, cudaStream_t s)
     int dev = 0;
     BMU_CUDA(cudaGetDevice(&dev));
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        BMU_CUDA(cudaFuncSetAttribute(sweep_mma2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)m2_smem_bytes(HEAD_ROWS_MAX)));
+        BMU_CUDA(cudaFuncSetAttribute(sweep_mma2_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)m2_smem_bytes(HEAD_ROWS_MAX, false)));
+        BMU_CUDA(cudaFuncSetAttribute(sweep_mma2_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)m2_smem_bytes(HEAD_ROWS_MAX, true)));
         configured[dev] = true;
     }
     const unsigned blocks = (unsigned)((a.N + MMA_DOCS - 1) / MMA_DOCS);
-    sweep_mma2_kernel<<<blocks, M2_THREADS, m2_smem_bytes(a.head), s>>>(a);
+    if (a.state2) sweep_mma2_kernel<true><<<blocks, M2_THREADS, m2_smem_bytes(a.head, true), s>>>(a);
+    else sweep_mma2_kernel<false><<<blocks, M2_THREADS, m2_smem_bytes(a.head, false), s>>>(a);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

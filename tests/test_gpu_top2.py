@@ -48,7 +48,7 @@ def check(bmu, W, rowptr, colidx, **kw):
     return b1, b2
 
 
-@pytest.mark.parametrize("kernel", [1, 3])
+@pytest.mark.parametrize("kernel", [1, 3, 6])
 @pytest.mark.parametrize("kind", ["uniform", "scaled", "signed"])
 def test_top2_against_oracle(bmu, kernel, kind):
     cfg = synth.CONFIGS["cfg1"]
@@ -57,7 +57,7 @@ def test_top2_against_oracle(bmu, kernel, kind):
     check(bmu, W, rowptr, colidx, kernel=kernel, chunk_neurons=256)
 
 
-@pytest.mark.parametrize("kernel", [1, 3])
+@pytest.mark.parametrize("kernel", [1, 3, 6])
 def test_top2_ties_take_lower_indices(bmu, kernel):
     cfg = synth.CONFIGS["cfg1"]
     rowptr, colidx = synth.make_corpus(cfg, n_docs=600)
