@@ -104,7 +104,14 @@ typedef struct bmu_opts {
     int32_t repack;         /* tensor-core sweeps: 0/1 gather from a compact [D][chunk] copy
                                of the chunk's columns, made before each launch, 2 gather
                                from the codebook itself */
-    int32_t reserved[4];    /* must be 0 */
+    int32_t relabel;        /* tensor-core sweeps: which features form the dense head.
+                               1 the head_rows features listed by the most documents of
+                               this corpus (ranked inside the tiling pass; the caller's ids
+                               stay as they are); 2 the ids below head_rows (a vocabulary
+                               already labelled by frequency, as the paper's is, Table 8);
+                               0 decide: keep the ids if they cover at least 98 % of what
+                               the most frequent features would */
+    int32_t reserved[3];    /* must be 0 */
 } bmu_opts;
 
 BMU_API const char *bmu_status_string(int status);

@@ -34,7 +34,7 @@ class Opts(ctypes.Structure):
                 ("stage_rows", ctypes.c_int32), ("stages", ctypes.c_int32),
                 ("tile_order", ctypes.c_int32), ("tile_head", ctypes.c_int32),
                 ("head_rows", ctypes.c_int32), ("repack", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 4)]
+                ("relabel", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3)]
 
 
 EXPORTS = {

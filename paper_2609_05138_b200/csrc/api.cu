@@ -121,7 +121,7 @@ static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kerne
     off = align_up(off + repack_bytes, 256);
     l.plan_off = off;
     memset(&l.plan, 0, sizeof(l.plan));
-    if (kernel != 1 && D <= LANES_MAX_D) off += plan_bytes(N, nnz, head, &l.plan);
+    if (kernel != 1 && D <= LANES_MAX_D) off += plan_bytes(N, nnz, head, D, &l.plan);
     l.total = off;
     return l;
 }
@@ -157,7 +157,8 @@ static int check_opts(const bmu_opts &o)
         return BMU_ERR_INVALID_ARG;
     }
     if (o.repack < 0 || o.repack > 2) { set_error("bmu_opts.repack must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
-    for (int i = 0; i < 4; ++i)
+    if (o.relabel < 0 || o.relabel > 2) { set_error("bmu_opts.relabel must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
+    for (int i = 0; i < 3; ++i)
         if (o.reserved[i] != 0) { set_error("bmu_opts.reserved must be zero"); return BMU_ERR_INVALID_ARG; }
     if (o.kernel < 0 || o.kernel > 6) { set_error("bmu_opts.kernel must be 0 .. 6"); return BMU_ERR_INVALID_ARG; }
     if (o.cluster < 0 || o.cluster > 2) { set_error("bmu_opts.cluster must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
@@ -270,18 +271,24 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     }
     const bool planned = !tiled && !mma && (o.kernel == 3 || (o.kernel == 0 && planned_ok));
     char *pw = base + l.plan_off;
+    // dense head = the most frequent features by the corpus's own counts (bmu_opts.relabel)
+    const int relabel = mma ? o.relabel : 2;        // 0 decide from the counts, 1 always, 2 never
     if ((staged || planned || tiled || mma) && phase != 2)
-        if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, mma ? head : 0, pw, l.plan, s)))
+        if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, mma ? head : 0, relabel, D, pw,
+                              l.plan, s)))
             return rc;
     if (mma) {
         if (phase != 2 &&
-            (rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, pw, l.plan, s))) return rc;
+            (rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, relabel, pw, l.plan, s)))
+            return rc;
         if (phase == 1) return BMU_OK;
         const int64_t m_full = M / MMA_SLAB * MMA_SLAB;
         uint32_t *head_max = status + 16;
         unsigned char *img = reinterpret_cast<unsigned char *>(base + l.head_off);
-        if ((rc = wide ? launch_head_split2(W, M, m_full, head, head_max, img, s)
-                       : launch_head_split(W, M, m_full, head, head_max, img, s))) return rc;
+        const uint16_t *feat = (relabel != 2 && l.plan.fsort_tmp_bytes > 0)
+                                   ? reinterpret_cast<const uint16_t *>(pw + l.plan.feat_off) : nullptr;
+        if ((rc = wide ? launch_head_split2(W, M, m_full, head, feat, head_max, img, s)
+                       : launch_head_split(W, M, m_full, head, feat, head_max, img, s))) return rc;
         MmaArgs a;
         a.W = W; a.M = M; a.N = N; a.n_tiles = (N + 7) / 8; a.norms = norms;
         a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
@@ -322,7 +329,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     if (tiled) {
         const int head = (o.tile_head == 1 || D < TILE_HEAD_ROWS) ? 0 : TILE_HEAD_ROWS;
         if (phase != 2 &&
-            (rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, pw, l.plan, s))) return rc;
+            (rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, 2, pw, l.plan, s))) return rc;
         if (phase == 1) return BMU_OK;
         TileArgs a;
         a.W = W; a.M = M; a.N = N; a.n_tiles = (N + 7) / 8; a.norms = norms;
@@ -599,7 +606,7 @@ int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
     }
     BMU_CUDA(cudaMemsetAsync(base + l.status_off, 0, 256, s));
     char *pw = base + l.plan_off;
-    if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, 0, pw, l.plan, s))) return rc;
+    if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, 0, 2, D, pw, l.plan, s))) return rc;
     RowsArgs a;
     a.W = static_cast<const float *>(W16); a.M = M; a.N = N; a.norms = norms; a.rowptr = rowptr;
     a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);

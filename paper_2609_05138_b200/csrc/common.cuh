@@ -155,11 +155,12 @@ int launch_finalize(const u64 *state, const u64 *state2, const int32_t *rowptr, 
 struct PlanLayout {
     size_t perm_off, docoff_off, ngroups_off, bins_off, ids_off, scan_off, scan_bytes, total;
     size_t tilelen_off, tilerows_off, tileoff_off, tilehead_off, tileids_off, tile_rows_cap;
+    size_t rank_off, feat_off, fsort_off, fsort_tmp_off, fsort_tmp_bytes;   // feature ranks
 };
 static const int TILE_HEAD_ROWS = 32;    // ids below this are swept densely, once per tile
 static const int HEAD_ROWS_MAX = 1024;   // widest dense head (the tensor-core sweep's)
-int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head, char *ws,
-                      const PlanLayout &l, cudaStream_t s);
+int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head, int relabel,
+                      char *ws, const PlanLayout &l, cudaStream_t s);
 
 // tiled sweep (sweep_tiles.cu): a warp carries 8 documents, 128-neuron slabs
 struct TileArgs {
@@ -207,17 +208,19 @@ struct MmaArgs {
 size_t head_image_bytes(int64_t M, int head);
 // writes the fp16 (hi, lo) split of rows [0, head) of W, scaled by a power of two, as the
 // shared-memory images the tensor-core sweep copies; whole slabs of [0, m_full) only
-int launch_head_split(const float *W, int64_t M, int64_t m_full, int head, uint32_t *head_max,
-                      unsigned char *head_img, cudaStream_t s);
+// `feat` (may be NULL = identity): the feature whose row of W is head row r
+int launch_head_split(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
+                      uint32_t *head_max, unsigned char *head_img, cudaStream_t s);
 int launch_sweep_mma(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
 // wide-head variant (sweep_mma2.cu): 256-neuron slabs, head of 64 .. HEAD_ROWS_MAX features
 size_t head_image2_bytes(int64_t M, int head);
-int launch_head_split2(const float *W, int64_t M, int64_t m_full, int head, uint32_t *head_max,
-                       unsigned char *head_img, cudaStream_t s);
+int launch_head_split2(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
+                       uint32_t *head_max, unsigned char *head_img, cudaStream_t s);
 int launch_sweep_mma2(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
-size_t plan_bytes(int64_t N, int64_t nnz, int head, PlanLayout *l);
+size_t plan_bytes(int64_t N, int64_t nnz, int head, int64_t D, PlanLayout *l);
 int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
-                int order_by_length, int head, char *ws, const PlanLayout &l, cudaStream_t s);
+                int order_by_length, int head, int relabel, int64_t D, char *ws, const PlanLayout &l,
+                cudaStream_t s);
 
 static const int LANES_MAX_D = 65024;    // 16-bit ids with 0xFFFF as the end marker
 

@@ -19,6 +19,7 @@
 // every document is reduced on its own.
 #include "common.cuh"
 
+#include <cub/device/device_radix_sort.cuh>
 #include <cub/device/device_scan.cuh>
 
 namespace bmu {
@@ -26,18 +27,77 @@ namespace bmu {
 static const int PLAN_BINS = 65536;      // one bin per row length: documents end up exactly
                                          // length-ordered (ids are 16-bit, so rows are shorter)
 
+// ---- frequency ranks of the features (Table 8: the paper relabels its vocabulary by
+// frequency and keeps that as substrate; here the relabelling is internal to the plan, so the
+// dense head is the `head` most frequent features whatever ids the caller uses) -------------
+__global__ void plan_feat_hist_kernel(const int32_t *__restrict__ colidx, int64_t nnz,
+                                      uint32_t *__restrict__ count)
+{
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < nnz;
+         e += (int64_t)gridDim.x * blockDim.x)
+        atomicAdd(count + colidx[e], 1u);
+}
+
+__global__ void plan_iota_kernel(int32_t D, uint32_t *__restrict__ v)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < D) v[i] = (uint32_t)i;
+}
+
+// Is the vocabulary labelled by frequency already?  If the ids below `head` cover at least 98 %
+// of the listings that the `head` most frequent features cover, the ids are kept as ranks (rows
+// then stay ascending and need no re-sorting).  One block.
+__global__ void __launch_bounds__(1024)
+plan_rank_decide_kernel(const uint32_t *__restrict__ count, const uint32_t *__restrict__ count_sorted,
+                        int32_t D, int32_t head, int force, uint32_t *__restrict__ keep_ids)
+{
+    __shared__ unsigned long long s_id[32], s_rk[32];
+    unsigned long long by_id = 0, by_rank = 0;
+    for (int i = threadIdx.x; i < head && i < D; i += 1024) {
+        by_id += count[i];
+        by_rank += count_sorted[i];
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        by_id += __shfl_xor_sync(0xffffffffu, by_id, off);
+        by_rank += __shfl_xor_sync(0xffffffffu, by_rank, off);
+    }
+    if ((threadIdx.x & 31) == 0) { s_id[threadIdx.x >> 5] = by_id; s_rk[threadIdx.x >> 5] = by_rank; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        by_id = by_rank = 0;
+        for (int w = 0; w < 32; ++w) { by_id += s_id[w]; by_rank += s_rk[w]; }
+        *keep_ids = (!force && by_id * 100ull >= by_rank * 98ull) ? 1u : 0u;
+    }
+}
+
+// sorted[r] = the feature of rank r (most frequent first, ties by ascending id)
+__global__ void plan_rank_tables_kernel(const uint32_t *__restrict__ sorted, int32_t D,
+                                        const uint32_t *__restrict__ keep_ids,
+                                        uint16_t *__restrict__ rank_of_feat,
+                                        uint16_t *__restrict__ feat_of_rank)
+{
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= D) return;
+    const uint32_t f = *keep_ids ? (uint32_t)r : sorted[r];
+    feat_of_rank[r] = (uint16_t)f;
+    rank_of_feat[f] = (uint16_t)r;
+}
+
 // Sorting key of a document: how many of its ids the gather will visit, i.e. the ids at or
 // above `head` (all of them when head == 0).  One warp per document.
 __global__ void __launch_bounds__(256)
 plan_key_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colidx,
-                int64_t N, int32_t head, uint32_t *__restrict__ key)
+                const uint16_t *__restrict__ rank, int64_t N, int32_t head,
+                uint32_t *__restrict__ key)
 {
     const int lane = threadIdx.x & 31;
     const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (i >= N) return;
     const int beg = rowptr[i], end = rowptr[i + 1];
     int cnt = 0;
-    for (int e = beg + lane; e < end; e += 32) cnt += colidx[e] >= head;
+    for (int e = beg + lane; e < end; e += 32)
+        cnt += (rank ? (int32_t)rank[colidx[e]] : colidx[e]) >= head;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
     if (lane == 0) key[i] = (uint32_t)cnt;
@@ -112,9 +172,11 @@ __global__ void plan_groups_kernel(const int32_t *__restrict__ rowptr,
 // must precede it (quadratic in the row length, rows are short).
 __global__ void __launch_bounds__(256)
 plan_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colidx,
-                 const int32_t *__restrict__ perm, const uint32_t *__restrict__ doc_off,
-                 int64_t N, uint16_t *__restrict__ ids16)
+                 const uint16_t *__restrict__ rank, const int32_t *__restrict__ perm,
+                 const uint32_t *__restrict__ doc_off, int64_t N, uint16_t *__restrict__ ids16)
 {
+    // with a rank table the list holds ranks (ascending: most frequent first), not ids
+#define BMU_PLAN_ID(e) (rank ? (int32_t)rank[row[e]] : row[e])
     const int lane = threadIdx.x & 31;
     const int64_t p = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (p >= N) return;
@@ -125,23 +187,24 @@ plan_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__
     const int padded = ((len + 7) / 8 + 1) * 8;
 
     bool sorted = true;
-    for (int e = lane; e + 1 < len; e += 32) sorted &= row[e] < row[e + 1];
+    for (int e = lane; e + 1 < len; e += 32) sorted &= BMU_PLAN_ID(e) < BMU_PLAN_ID(e + 1);
     sorted = __all_sync(0xffffffffu, sorted);
     if (sorted) {
-        for (int e = lane; e < padded; e += 32) dst[e] = e < len ? (uint16_t)row[e] : 0xFFFFu;
+        for (int e = lane; e < padded; e += 32) dst[e] = e < len ? (uint16_t)BMU_PLAN_ID(e) : 0xFFFFu;
     } else {
         for (int e = lane; e < padded; e += 32)
             if (e >= len) dst[e] = 0xFFFFu;
         for (int e = lane; e < len; e += 32) {
-            const int32_t f = row[e];
-            int rank = 0;
+            const int32_t f = BMU_PLAN_ID(e);
+            int pos = 0;
             for (int k = 0; k < len; ++k) {
-                const int32_t g = row[k];
-                rank += (g < f) || (g == f && k < e);
+                const int32_t g = BMU_PLAN_ID(k);
+                pos += (g < f) || (g == f && k < e);
             }
-            dst[rank] = (uint16_t)f;
+            dst[pos] = (uint16_t)f;
         }
     }
+#undef BMU_PLAN_ID
     if (p == 0 && lane < 8) ids16[lane] = 0xFFFFu;                  // global sentinel group
     if (p == N - 1 && lane < 16) dst[padded + lane] = 0xFFFFu;      // two groups of slack at the end
 }
@@ -211,8 +274,9 @@ __global__ void __launch_bounds__(256)
 plan_tile_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ perm,
                       const uint32_t *__restrict__ doc_off, const uint16_t *__restrict__ ids16,
                       const uint32_t *__restrict__ tile_len, const uint32_t *__restrict__ tile_off,
-                      const uint32_t *__restrict__ tile_head, uint32_t head_words, int64_t N,
-                      int64_t n_tiles, int interleave, uint4 *__restrict__ tile_ids)
+                      const uint32_t *__restrict__ tile_head, uint32_t head_words,
+                      const uint16_t *__restrict__ feat_of_rank, int64_t N, int64_t n_tiles,
+                      int interleave, uint4 *__restrict__ tile_ids)
 {
     const int lane = threadIdx.x & 31;
     const int64_t tile = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -240,13 +304,14 @@ plan_tile_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restr
             uint32_t e = r;
             if (interleave) e = (r & 1u) ? (len[t] + 1) / 2 + r / 2 : r / 2;
             f[t] = r < len[t] ? src[t][e] : 0xffffu;
+            if (feat_of_rank && f[t] != 0xffffu) f[t] = feat_of_rank[f[t]];   // rank -> row of W
         }
         dst[r] = make_uint4(f[0] | (f[1] << 16), f[2] | (f[3] << 16), f[4] | (f[5] << 16),
                             f[6] | (f[7] << 16));
     }
 }
 
-size_t plan_bytes(int64_t N, int64_t nnz, int head, PlanLayout *l)
+size_t plan_bytes(int64_t N, int64_t nnz, int head, int64_t D, PlanLayout *l)
 {
     auto up = [](size_t x) { return (x + 255) / 256 * 256; };
     size_t off = 0;
@@ -270,15 +335,54 @@ size_t plan_bytes(int64_t N, int64_t nnz, int head, PlanLayout *l)
     t.tilehead_off = off; off = up(off + n_tiles * 8 * 4 * (size_t)(head > 32 ? head / 32 : 1));
     t.tile_rows_cap = (size_t)nnz / 8 + 65536 + n_tiles;
     t.tileids_off = off; off = up(off + t.tile_rows_cap * 16);
+    // frequency ranks of the features (dense head only): counts, sort buffers, the two tables
+    t.rank_off = t.feat_off = t.fsort_off = t.fsort_tmp_off = off;
+    t.fsort_tmp_bytes = 0;
+    if (head > 0 && D > 0 && D <= 65535) {
+        const size_t d4 = up((size_t)D * 4), d2 = up((size_t)D * 2);
+        t.rank_off = off; off += d2;
+        t.feat_off = off; off += d2;
+        t.fsort_off = off; off += 4 * d4;            // counts, sorted counts, ids, sorted ids
+        size_t tmp = 0;
+        cub::DeviceRadixSort::SortPairsDescending(nullptr, tmp, (uint32_t *)nullptr, (uint32_t *)nullptr,
+                                                  (uint32_t *)nullptr, (uint32_t *)nullptr, (int)D);
+        t.fsort_tmp_off = off; t.fsort_tmp_bytes = tmp; off = up(off + tmp);
+    }
     t.total = off;
     if (l) *l = t;
     return off;
 }
 
 int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
-                int order_by_length, int head, char *ws, const PlanLayout &l, cudaStream_t s)
+                int order_by_length, int head, int relabel, int64_t D, char *ws, const PlanLayout &l,
+                cudaStream_t s)
 {
-    (void)nnz;
+    // dense head: rank the features by how many documents list them, so that the head is the
+    // `head` most frequent features whatever their ids
+    const uint16_t *rank = nullptr;
+    if (head > 0 && relabel != 2 && l.fsort_tmp_bytes > 0) {
+        const size_t d4 = ((size_t)D * 4 + 255) / 256 * 256;
+        uint32_t *count = reinterpret_cast<uint32_t *>(ws + l.fsort_off);
+        uint32_t *count_sorted = reinterpret_cast<uint32_t *>(ws + l.fsort_off + d4);
+        uint32_t *ids = reinterpret_cast<uint32_t *>(ws + l.fsort_off + 2 * d4);
+        uint32_t *ids_sorted = reinterpret_cast<uint32_t *>(ws + l.fsort_off + 3 * d4);
+        uint16_t *rank_of_feat = reinterpret_cast<uint16_t *>(ws + l.rank_off);
+        uint16_t *feat_of_rank = reinterpret_cast<uint16_t *>(ws + l.feat_off);
+        BMU_CUDA(cudaMemsetAsync(count, 0, (size_t)D * 4, s));
+        if (nnz > 0) plan_feat_hist_kernel<<<1184, 256, 0, s>>>(colidx, nnz, count);
+        plan_iota_kernel<<<(unsigned)((D + 255) / 256), 256, 0, s>>>((int32_t)D, ids);
+        size_t tmp = l.fsort_tmp_bytes;
+        BMU_CUDA(cub::DeviceRadixSort::SortPairsDescending(ws + l.fsort_tmp_off, tmp, count, count_sorted,
+                                                           ids, ids_sorted, (int)D, 0, 32, s));
+        // the decision word borrows the first counter of the length histogram (cleared below)
+        uint32_t *keep_ids = reinterpret_cast<uint32_t *>(ws + l.bins_off);
+        plan_rank_decide_kernel<<<1, 1024, 0, s>>>(count, count_sorted, (int32_t)D, head, relabel == 1,
+                                                   keep_ids);
+        plan_rank_tables_kernel<<<(unsigned)((D + 255) / 256), 256, 0, s>>>(ids_sorted, (int32_t)D,
+                                                                            keep_ids, rank_of_feat,
+                                                                            feat_of_rank);
+        rank = rank_of_feat;
+    }
     int32_t *perm = reinterpret_cast<int32_t *>(ws + l.perm_off);
     uint32_t *doc_off = reinterpret_cast<uint32_t *>(ws + l.docoff_off);
     uint32_t *ngroups = reinterpret_cast<uint32_t *>(ws + l.ngroups_off);
@@ -292,8 +396,8 @@ int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t
         // array, which is written only after the scatter)
         const uint32_t *key = nullptr;
         if (head > 0) {
-            plan_key_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(rowptr, colidx, N, head,
-                                                                            ngroups);
+            plan_key_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(rowptr, colidx, rank, N,
+                                                                            head, ngroups);
             key = ngroups;
         }
         BMU_CUDA(cudaMemsetAsync(hist, 0, PLAN_BINS * 4, s));
@@ -307,15 +411,17 @@ int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t
     BMU_CUDA(cudaMemsetAsync(ngroups + N, 0, 4, s));
     size_t tmp = l.scan_bytes;
     BMU_CUDA(cub::DeviceScan::ExclusiveSum(ws + l.scan_off, tmp, ngroups, doc_off, (int)(N + 1), s));
-    plan_fill_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(rowptr, colidx, perm,
+    plan_fill_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(rowptr, colidx, rank, perm,
                                                                        doc_off, N, ids16);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
 
-int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head, char *ws,
-                      const PlanLayout &l, cudaStream_t s)
+int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head, int relabel,
+                      char *ws, const PlanLayout &l, cudaStream_t s)
 {
+    const uint16_t *feat_of_rank = (head > 0 && relabel != 2 && l.fsort_tmp_bytes > 0)
+                                       ? reinterpret_cast<const uint16_t *>(ws + l.feat_off) : nullptr;
     const int64_t n_tiles = (N + 7) / 8;
     const int32_t *perm = reinterpret_cast<const int32_t *>(ws + l.perm_off);
     const uint32_t *doc_off = reinterpret_cast<const uint32_t *>(ws + l.docoff_off);
@@ -333,7 +439,7 @@ int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head
                                            (int)(n_tiles + 1), s));
     plan_tile_fill_kernel<<<(unsigned)((n_tiles * 32 + 255) / 256), 256, 0, s>>>(
         rowptr, perm, doc_off, ids16, tile_len, tile_off, tile_head,
-        (uint32_t)(head ? head / 32 : 1), N, n_tiles, interleave, tile_ids);
+        (uint32_t)(head ? head / 32 : 1), feat_of_rank, N, n_tiles, interleave, tile_ids);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

@@ -50,14 +50,16 @@ static inline size_t mma_smem_bytes(int head)
 }
 
 __global__ void head_absmax_kernel(const float *__restrict__ W, int64_t M, int64_t m_full,
-                                   int head, uint32_t *__restrict__ out)
+                                   int head, const uint16_t *__restrict__ feat,
+                                   uint32_t *__restrict__ out)
 {
     const int64_t n4 = m_full / 4, total = n4 * head;
     uint32_t mx = 0;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (int64_t)gridDim.x * blockDim.x) {
         const int64_t f = i / n4, c = i - f * n4;
-        const float4 v = __ldg(reinterpret_cast<const float4 *>(W + f * M) + c);
+        const int64_t row = feat ? (int64_t)feat[f] : f;
+        const float4 v = __ldg(reinterpret_cast<const float4 *>(W + row * M) + c);
         mx = max(mx, __float_as_uint(fabsf(v.x)));
         mx = max(mx, __float_as_uint(fabsf(v.y)));
         mx = max(mx, __float_as_uint(fabsf(v.z)));
@@ -73,18 +75,19 @@ __global__ void head_absmax_kernel(const float *__restrict__ W, int64_t M, int64
 // (hi, lo), block of 64 features; inside a stage the core matrix of (8 rows, 8 features)
 // lies at (row / 8) * 1024 + (feature / 8) * 128.
 __global__ void __launch_bounds__(MMA_SLAB)
-head_split_kernel(const float *__restrict__ W, int64_t M, int head,
+head_split_kernel(const float *__restrict__ W, int64_t M, int head, const uint16_t *__restrict__ feat,
                   const uint32_t *__restrict__ head_max, unsigned char *__restrict__ img)
 {
     const int KB = head / 64, SPS = 8 * KB;
     const int sl = blockIdx.x, kcg = blockIdx.y, jin = threadIdx.x;
     const float S = head_scale(*head_max);
-    const float *src = W + (int64_t)(kcg * 8) * M + (int64_t)sl * MMA_SLAB + jin;
+    const float *col = W + (int64_t)sl * MMA_SLAB + jin;
     __align__(16) __half hi[8];
     __align__(16) __half lo[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-        const float w = __ldg(src + (int64_t)e * M) * S;
+        const int64_t row = feat ? (int64_t)feat[kcg * 8 + e] : (int64_t)(kcg * 8 + e);
+        const float w = __ldg(col + row * M) * S;
         hi[e] = __float2half_rn(w);
         lo[e] = __float2half_rn(w - __half2float(hi[e]));
     }
@@ -102,14 +105,14 @@ size_t head_image_bytes(int64_t M, int head)
     return (size_t)(M / MMA_SLAB) * mma_stages_per_slab(head) * MMA_STAGE_BYTES;
 }
 
-int launch_head_split(const float *W, int64_t M, int64_t m_full, int head, uint32_t *head_max,
-                      unsigned char *head_img, cudaStream_t s)
+int launch_head_split(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
+                      uint32_t *head_max, unsigned char *head_img, cudaStream_t s)
 {
     if (m_full <= 0) return BMU_OK;
     BMU_CUDA(cudaMemsetAsync(head_max, 0, sizeof(uint32_t), s));
-    head_absmax_kernel<<<592, 256, 0, s>>>(W, M, m_full, head, head_max);
+    head_absmax_kernel<<<592, 256, 0, s>>>(W, M, m_full, head, feat, head_max);
     const dim3 grid((unsigned)(m_full / MMA_SLAB), head / 8);
-    head_split_kernel<<<grid, MMA_SLAB, 0, s>>>(W, M, head, head_max, head_img);
+    head_split_kernel<<<grid, MMA_SLAB, 0, s>>>(W, M, head, feat, head_max, head_img);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

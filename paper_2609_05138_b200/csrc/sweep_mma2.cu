@@ -50,17 +50,18 @@ static inline size_t m2_smem_bytes(int head, bool top2)
 // 64 features, tile c (neuron % 2), part (hi, lo).
 __global__ void __launch_bounds__(M2_SLAB)
 head_split2_kernel(const float *__restrict__ W, int64_t M, const uint32_t *__restrict__ head_max,
-                   int head, unsigned char *__restrict__ img)
+                   int head, const uint16_t *__restrict__ feat, unsigned char *__restrict__ img)
 {
     const int sl = blockIdx.x, kcg = blockIdx.y, jin = threadIdx.x;
     const int SPS = 4 * (head / 64);
     const float S = head_scale(*head_max);
-    const float *src = W + (int64_t)(kcg * 8) * M + (int64_t)sl * M2_SLAB + jin;
+    const float *col = W + (int64_t)sl * M2_SLAB + jin;
     __align__(16) __half hi[8];
     __align__(16) __half lo[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-        const float w = __ldg(src + (int64_t)e * M) * S;
+        const int64_t row = feat ? (int64_t)feat[kcg * 8 + e] : (int64_t)(kcg * 8 + e);
+        const float w = __ldg(col + row * M) * S;
         hi[e] = __float2half_rn(w);
         lo[e] = __float2half_rn(w - __half2float(hi[e]));
     }
@@ -74,14 +75,16 @@ head_split2_kernel(const float *__restrict__ W, int64_t M, const uint32_t *__res
 }
 
 __global__ void head_absmax2_kernel(const float *__restrict__ W, int64_t M, int64_t m_full,
-                                    int head, uint32_t *__restrict__ out)
+                                    int head, const uint16_t *__restrict__ feat,
+                                    uint32_t *__restrict__ out)
 {
     const int64_t n4 = m_full / 4, total = n4 * head;
     uint32_t mx = 0;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (int64_t)gridDim.x * blockDim.x) {
         const int64_t f = i / n4, c = i - f * n4;
-        const float4 v = __ldg(reinterpret_cast<const float4 *>(W + f * M) + c);
+        const int64_t row = feat ? (int64_t)feat[f] : f;
+        const float4 v = __ldg(reinterpret_cast<const float4 *>(W + row * M) + c);
         mx = max(mx, __float_as_uint(fabsf(v.x)));
         mx = max(mx, __float_as_uint(fabsf(v.y)));
         mx = max(mx, __float_as_uint(fabsf(v.z)));
@@ -97,14 +100,14 @@ size_t head_image2_bytes(int64_t M, int head)
     return (size_t)(M / M2_SLAB) * 4 * (head / 64) * MMA_STAGE_BYTES;
 }
 
-int launch_head_split2(const float *W, int64_t M, int64_t m_full, int head, uint32_t *head_max,
-                       unsigned char *head_img, cudaStream_t s)
+int launch_head_split2(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
+                       uint32_t *head_max, unsigned char *head_img, cudaStream_t s)
 {
     if (m_full <= 0) return BMU_OK;
     BMU_CUDA(cudaMemsetAsync(head_max, 0, sizeof(uint32_t), s));
-    head_absmax2_kernel<<<592, 256, 0, s>>>(W, M, m_full, head, head_max);
+    head_absmax2_kernel<<<592, 256, 0, s>>>(W, M, m_full, head, feat, head_max);
     const dim3 grid((unsigned)(m_full / M2_SLAB), head / 8);
-    head_split2_kernel<<<grid, M2_SLAB, 0, s>>>(W, M, head_max, head, head_img);
+    head_split2_kernel<<<grid, M2_SLAB, 0, s>>>(W, M, head_max, head, feat, head_img);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

@@ -109,15 +109,27 @@ def test_mma_kernel_long_empty_unsorted_and_repeated_rows(bmu):
     run_and_check(bmu, W, rowptr, torch.from_numpy(ci), opts_of(bmu, 6, head_rows=256, tile_order=1))
 
 
-def test_mma_kernel_unlabelled_vocabulary(bmu):
-    """Feature ids that are not frequency-ordered: still correct, only slower."""
+@pytest.mark.parametrize("kernel", [5, 6])
+@pytest.mark.parametrize("relabel", [0, 2])
+def test_mma_kernel_unlabelled_vocabulary(bmu, kernel, relabel):
+    """Feature ids that are not frequency-ordered: the tiling pass ranks the features itself
+    (relabel = 0); with relabel = 2 the head is the ids below head_rows -- exact either way."""
     cfg = synth.CONFIGS["cfg1"]
     rowptr, colidx = synth.make_corpus(cfg, n_docs=900)
     perm = torch.from_numpy(np.random.default_rng(1).permutation(cfg.D).astype(np.int32))
-    ci = perm[colidx.long()]
+    ci = perm[colidx.long()]                              # rows are no longer ascending either
     W = synth.make_codebook(cfg.D, 512, 9, kind="scaled")
-    run_and_check(bmu, W, rowptr, ci, opts_of(bmu))
-    run_and_check(bmu, W, rowptr, ci, opts_of(bmu, 6))
+    run_and_check(bmu, W, rowptr, ci, opts_of(bmu, kernel, relabel=relabel))
+
+
+def test_mma_kernel_relabel_off_matches_on_for_ordered_ids(bmu):
+    """On a vocabulary already labelled by frequency both choices of head pass the oracle rule
+    (they differ only in which of the near-equally frequent features fall inside the head)."""
+    cfg = synth.CONFIGS["cfg3"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=1500)
+    W = synth.make_codebook(cfg.D, 1024, 4, kind="scaled")
+    for relabel in (0, 2):
+        run_and_check(bmu, W, rowptr, colidx, opts_of(bmu, 6, relabel=relabel))
 
 
 def test_mma_kernel_refuses_what_it_cannot_do(bmu):
