@@ -428,7 +428,7 @@ def run_ours(args, cfg, rank, local_rank, world):
                         "with the search of the current one)" % len(batches)) +
                        " (codebook resident in HBM; CSR from pinned host memory; results back "
                        "to host)", "matches_device_path": same},
-        "gpu_launches": args.steps * (1 + len(batches) * ({1: 0, 2: 6, 3: 6, 4: 8, 5: 11, 6: 11}[kernel]
+        "gpu_launches": args.steps * (1 + len(batches) * ({1: 0, 2: 7, 3: 7, 4: 11, 5: 24, 6: 24}[kernel]
                                                            + n_chunks * (2 if kernel in (5, 6) and
                                                                          opts.repack != 2 and
                                                                          n_chunks > 1 else 1)

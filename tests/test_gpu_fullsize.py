@@ -104,3 +104,35 @@ def test_cfg2_full_size_against_library_product(bmu):
         d_at = d.gather(1, got_j[:, None])[:, 0]
         bad_j += int(((got_j != jmin) & (d_at > dmin + tol)).sum())
     assert bad_d == 0 and bad_j == 0
+
+
+def test_cfg2_full_size_update_step_properties(bmu):
+    """Scatter, blur and write-back at full size: what must hold at any size (integer totals,
+    a weighted mean of binary vectors stays in [0, 1], untouched units keep their weights),
+    plus sampled planes against the oracle."""
+    import oracle
+    cfg = synth.CONFIGS["cfg2"]
+    dev = torch.device("cuda")
+    W = synth.make_codebook(cfg.D, cfg.M, synth.codebook_seed(cfg), device=dev)
+    rowptr, colidx = synth.make_corpus(cfg, device=dev)
+    units, _ = bmu.bmu_search(W, rowptr, colidx)
+    num = torch.zeros((cfg.D, cfg.M), dtype=torch.int32, device=dev)
+    cnt = torch.zeros(cfg.M, dtype=torch.int32, device=dev)
+    bmu.bmu_update_scatter(rowptr, colidx, units, num, cnt)
+    torch.cuda.synchronize()
+    assert int(cnt.sum()) == cfg.N
+    assert int(num.sum(dtype=torch.int64)) == colidx.numel()
+    assert torch.equal(num.sum(1, dtype=torch.int64), torch.bincount(colidx.long(), minlength=cfg.D))
+    assert torch.equal(cnt.long(), torch.bincount(units.long(), minlength=cfg.M))
+    sigma = 1.5
+    nb, cb = bmu.bmu_update_blur(num, cnt, cfg.edge, cfg.edge, sigma)
+    for f in (0, 17, 4095, cfg.D - 1):                               # sampled planes
+        ref = oracle.blur(num[f].cpu().numpy(), cfg.edge, cfg.edge, sigma)
+        got = nb[f].cpu().numpy()
+        assert np.all(np.abs(got - ref) <= 2e-6 * max(1.0, np.abs(ref).max()))
+    W1 = W.clone()
+    bmu.bmu_update_writeback(nb, cb, W1)
+    torch.cuda.synchronize()
+    live = cb > 0
+    assert float(W1[:, live].min()) >= 0.0 and float(W1[:, live].max()) <= 1.0 + 1e-6
+    assert torch.equal(W1[:, ~live], W[:, ~live])
