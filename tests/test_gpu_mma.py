@@ -139,3 +139,16 @@ def test_mma_kernel_refuses_what_it_cannot_do(bmu):
         with pytest.raises(bmu.BmuError) as e:
             bmu.bmu_search_ws(torch.zeros(D, M, device="cuda"), rp, ci, opts=opts_of(bmu, kernel))
         assert e.value.status == 2
+
+
+@pytest.mark.parametrize("kernel", [5, 6])
+@pytest.mark.parametrize("N", [1, 7, 9, 129])
+def test_mma_kernel_few_documents_and_empty_corpus_rows(bmu, kernel, N):
+    """Blocks and tiles that are mostly padding; a corpus whose rows are all empty."""
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=N)
+    W = synth.make_codebook(cfg.D, 512, 5 + N, kind="scaled")
+    run_and_check(bmu, W, rowptr, colidx, opts_of(bmu, kernel))
+    empty_rp = torch.zeros(N + 1, dtype=torch.int32)
+    res = run_and_check(bmu, W, empty_rp, torch.zeros(0, dtype=torch.int32), opts_of(bmu, kernel))
+    assert res["docs"] == N
