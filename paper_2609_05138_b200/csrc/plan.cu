@@ -30,12 +30,25 @@ static const int PLAN_BINS = 65536;      // one bin per row length: documents en
 // ---- frequency ranks of the features (Table 8: the paper relabels its vocabulary by
 // frequency and keeps that as substrate; here the relabelling is internal to the plan, so the
 // dense head is the `head` most frequent features whatever ids the caller uses) -------------
-__global__ void plan_feat_hist_kernel(const int32_t *__restrict__ colidx, int64_t nnz,
-                                      uint32_t *__restrict__ count)
+// Listings per feature for the ids in [lo, hi): counted in shared memory first (a frequent
+// feature is listed by most documents, and that many atomics on one global counter crawl),
+// then flushed.
+__global__ void __launch_bounds__(1024)
+plan_feat_hist_kernel(const int32_t *__restrict__ colidx, int64_t nnz, int32_t lo, int32_t hi,
+                      uint32_t *__restrict__ count)
 {
+    extern __shared__ uint32_t bins[];
+    const int n_bins = hi - lo;
+    for (int b = threadIdx.x; b < n_bins; b += blockDim.x) bins[b] = 0u;
+    __syncthreads();
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < nnz;
-         e += (int64_t)gridDim.x * blockDim.x)
-        atomicAdd(count + colidx[e], 1u);
+         e += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t f = __ldg(colidx + e);
+        if (f >= lo && f < hi) atomicAdd(bins + (f - lo), 1u);
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < n_bins; b += blockDim.x)
+        if (bins[b]) atomicAdd(count + lo + b, bins[b]);
 }
 
 __global__ void plan_iota_kernel(int32_t D, uint32_t *__restrict__ v)
@@ -236,33 +249,38 @@ __device__ __forceinline__ uint32_t head_of_doc(const uint16_t *ids, uint32_t le
 }
 
 // per tile: longest and shortest list behind the head (max | min << 16), and the head masks
-// (head / 32 words per document, document-major)
-__global__ void plan_tile_len_kernel(const int32_t *__restrict__ rowptr,
-                                     const int32_t *__restrict__ perm,
-                                     const uint32_t *__restrict__ doc_off,
-                                     const uint16_t *__restrict__ ids16, int64_t N, int64_t n_tiles,
-                                     uint32_t head, uint32_t *__restrict__ tile_rows,
-                                     uint32_t *__restrict__ tile_len, uint32_t *__restrict__ tile_head)
+// (head / 32 words per document, document-major).  One thread per planned document; the eight
+// threads of a tile combine their lengths with shuffles.
+__global__ void __launch_bounds__(256)
+plan_tile_len_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ perm,
+                     const uint32_t *__restrict__ doc_off, const uint16_t *__restrict__ ids16,
+                     int64_t N, int64_t n_tiles, uint32_t head, uint32_t *__restrict__ tile_rows,
+                     uint32_t *__restrict__ tile_len, uint32_t *__restrict__ tile_head)
 {
-    const int64_t tile = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (tile >= n_tiles) return;
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;     // planned position
+    const int64_t tile = p >> 3;
+    const bool there = tile < n_tiles;
     const uint32_t words = head ? head / 32 : 1;
-    uint32_t mx = 0, mn = 0xffffu;
-    for (int t = 0; t < 8; ++t) {
-        const int64_t p = tile * 8 + t;
-        uint32_t len = 0, skip = 0;
-        uint32_t *mask = tile_head + (size_t)(tile * 8 + t) * words;
+    uint32_t len = 0, skip = 0;
+    if (there) {
+        uint32_t *mask = tile_head + (size_t)p * words;
         for (uint32_t w = 0; w < words; ++w) mask[w] = 0;
         if (p < N) {
             const int32_t i = perm[p];
             len = (uint32_t)min(rowptr[i + 1] - rowptr[i], 65535);
             if (head) skip = head_of_doc(ids16 + ((size_t)doc_off[p] + 1) * 8, len, head, mask);
         }
-        mx = max(mx, len - skip);
-        mn = min(mn, len - skip);
     }
-    tile_rows[tile] = mx;
-    tile_len[tile] = mx | (mn << 16);
+    uint32_t mx = len - skip, mn = len - skip;
+#pragma unroll
+    for (int off = 1; off < 8; off <<= 1) {
+        mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+        mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, off));
+    }
+    if (there && (threadIdx.x & 7) == 0) {
+        tile_rows[tile] = mx;
+        tile_len[tile] = mx | (mn << 16);
+    }
 }
 
 // One warp per tile: row r of the matrix = the r-th id, in visiting order, of each of its
@@ -369,7 +387,21 @@ int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t
         uint16_t *rank_of_feat = reinterpret_cast<uint16_t *>(ws + l.rank_off);
         uint16_t *feat_of_rank = reinterpret_cast<uint16_t *>(ws + l.feat_off);
         BMU_CUDA(cudaMemsetAsync(count, 0, (size_t)D * 4, s));
-        if (nnz > 0) plan_feat_hist_kernel<<<1184, 256, 0, s>>>(colidx, nnz, count);
+        if (nnz > 0) {
+            const int32_t span = 32768;                   // 128 KB of shared-memory counters
+            static bool configured[64];
+            int dev = 0;
+            BMU_CUDA(cudaGetDevice(&dev));
+            if (dev >= 0 && dev < 64 && !configured[dev]) {
+                BMU_CUDA(cudaFuncSetAttribute(plan_feat_hist_kernel,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, span * 4));
+                configured[dev] = true;
+            }
+            for (int32_t lo = 0; lo < (int32_t)D; lo += span) {
+                const int32_t hi = lo + span < (int32_t)D ? lo + span : (int32_t)D;
+                plan_feat_hist_kernel<<<148, 1024, (size_t)(hi - lo) * 4, s>>>(colidx, nnz, lo, hi, count);
+            }
+        }
         plan_iota_kernel<<<(unsigned)((D + 255) / 256), 256, 0, s>>>((int32_t)D, ids);
         size_t tmp = l.fsort_tmp_bytes;
         BMU_CUDA(cub::DeviceRadixSort::SortPairsDescending(ws + l.fsort_tmp_off, tmp, count, count_sorted,
@@ -431,7 +463,7 @@ int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head
     uint32_t *tile_off = reinterpret_cast<uint32_t *>(ws + l.tileoff_off);
     uint4 *tile_ids = reinterpret_cast<uint4 *>(ws + l.tileids_off);
     uint32_t *tile_head = reinterpret_cast<uint32_t *>(ws + l.tilehead_off);
-    plan_tile_len_kernel<<<(unsigned)((n_tiles + 255) / 256), 256, 0, s>>>(
+    plan_tile_len_kernel<<<(unsigned)((n_tiles * 8 + 255) / 256), 256, 0, s>>>(
         rowptr, perm, doc_off, ids16, N, n_tiles, (uint32_t)head, tile_rows, tile_len, tile_head);
     BMU_CUDA(cudaMemsetAsync(tile_rows + n_tiles, 0, 4, s));
     size_t tmp = l.scan_bytes;
