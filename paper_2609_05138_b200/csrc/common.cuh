@@ -209,6 +209,8 @@ size_t head_image_bytes(int64_t M, int head);
 // writes the fp16 (hi, lo) split of rows [0, head) of W, scaled by a power of two, as the
 // shared-memory images the tensor-core sweep copies; whole slabs of [0, m_full) only
 // `feat` (may be NULL = identity): the feature whose row of W is head row r
+int launch_head_absmax(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
+                       uint32_t *head_max, cudaStream_t s);
 int launch_head_split(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
                       uint32_t *head_max, unsigned char *head_img, cudaStream_t s);
 int launch_sweep_mma(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);

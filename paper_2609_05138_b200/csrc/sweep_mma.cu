@@ -105,12 +105,22 @@ size_t head_image_bytes(int64_t M, int head)
     return (size_t)(M / MMA_SLAB) * mma_stages_per_slab(head) * MMA_STAGE_BYTES;
 }
 
+// bit pattern of the largest |weight| among the head rows (both tensor-core sweeps)
+int launch_head_absmax(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
+                       uint32_t *head_max, cudaStream_t s)
+{
+    BMU_CUDA(cudaMemsetAsync(head_max, 0, sizeof(uint32_t), s));
+    head_absmax_kernel<<<592, 256, 0, s>>>(W, M, m_full, head, feat, head_max);
+    BMU_CUDA(cudaGetLastError());
+    return BMU_OK;
+}
+
 int launch_head_split(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
                       uint32_t *head_max, unsigned char *head_img, cudaStream_t s)
 {
     if (m_full <= 0) return BMU_OK;
-    BMU_CUDA(cudaMemsetAsync(head_max, 0, sizeof(uint32_t), s));
-    head_absmax_kernel<<<592, 256, 0, s>>>(W, M, m_full, head, feat, head_max);
+    int rc = launch_head_absmax(W, M, m_full, head, feat, head_max, s);
+    if (rc) return rc;
     const dim3 grid((unsigned)(m_full / MMA_SLAB), head / 8);
     head_split_kernel<<<grid, MMA_SLAB, 0, s>>>(W, M, head, feat, head_max, head_img);
     BMU_CUDA(cudaGetLastError());

@@ -74,27 +74,6 @@ head_split2_kernel(const float *__restrict__ W, int64_t M, const uint32_t *__res
     *reinterpret_cast<uint4 *>(img + (st + 1) * MMA_STAGE_BYTES + off) = *reinterpret_cast<uint4 *>(lo);
 }
 
-__global__ void head_absmax2_kernel(const float *__restrict__ W, int64_t M, int64_t m_full,
-                                    int head, const uint16_t *__restrict__ feat,
-                                    uint32_t *__restrict__ out)
-{
-    const int64_t n4 = m_full / 4, total = n4 * head;
-    uint32_t mx = 0;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-         i += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t f = i / n4, c = i - f * n4;
-        const int64_t row = feat ? (int64_t)feat[f] : f;
-        const float4 v = __ldg(reinterpret_cast<const float4 *>(W + row * M) + c);
-        mx = max(mx, __float_as_uint(fabsf(v.x)));
-        mx = max(mx, __float_as_uint(fabsf(v.y)));
-        mx = max(mx, __float_as_uint(fabsf(v.z)));
-        mx = max(mx, __float_as_uint(fabsf(v.w)));
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-    if ((threadIdx.x & 31) == 0 && mx) atomicMax(out, mx);
-}
-
 size_t head_image2_bytes(int64_t M, int head)
 {
     return (size_t)(M / M2_SLAB) * 4 * (head / 64) * MMA_STAGE_BYTES;
@@ -104,8 +83,8 @@ int launch_head_split2(const float *W, int64_t M, int64_t m_full, int head, cons
                        uint32_t *head_max, unsigned char *head_img, cudaStream_t s)
 {
     if (m_full <= 0) return BMU_OK;
-    BMU_CUDA(cudaMemsetAsync(head_max, 0, sizeof(uint32_t), s));
-    head_absmax2_kernel<<<592, 256, 0, s>>>(W, M, m_full, head, feat, head_max);
+    int rc = launch_head_absmax(W, M, m_full, head, feat, head_max, s);
+    if (rc) return rc;
     const dim3 grid((unsigned)(m_full / M2_SLAB), head / 8);
     head_split2_kernel<<<grid, M2_SLAB, 0, s>>>(W, M, head_max, head, feat, head_img);
     BMU_CUDA(cudaGetLastError());
