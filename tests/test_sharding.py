@@ -54,3 +54,61 @@ def test_two_gloo_ranks_match_single_process(tmp_path):
     np.testing.assert_array_equal(np.load(tmp_path / "b.npy"), b)
     np.testing.assert_array_equal(np.load(tmp_path / "d.npy"), d1)
     assert abs(np.load(tmp_path / "rate.npy")[0] - 301 / 2.0) < 1e-9
+
+
+# ---- neuron-axis sharding: every rank searches all documents against its slice of neurons
+def test_neuron_ranges_tile_the_map():
+    for M, w in [(262144, 8), (1024 + 40, 2), (512, 4), (100, 3)]:
+        edges = [sharding.neuron_range(M, r, w) for r in range(w)]
+        assert edges[0][0] == 0 and edges[-1][1] == M
+        assert all(a[1] == b[0] for a, b in zip(edges, edges[1:]))
+        assert all(lo % 512 == 0 for lo, hi in edges if hi > lo)
+
+
+def test_packed_keys_order_like_distance_then_index():
+    d = torch.tensor([3.5, -1.0, 0.0, -0.0, 3.5, float("inf"), 1e-30, -2.5e7], dtype=torch.float32)
+    j = torch.tensor([7, 2, 5, 4, 6, 0, 1, 3], dtype=torch.int32)
+    k = sharding.pack_keys(d, j, 100)
+    dd, jj = sharding.unpack_keys(k)
+    assert torch.equal(dd.view(torch.int32), d.view(torch.int32)) and torch.equal(jj, j + 100)
+    order = torch.argsort(k).tolist()
+    want = sorted(range(8), key=lambda i: (float(d[i]), int(j[i])))
+    # -0.0 sorts before +0.0 as bit patterns; as distances they are equal: accept either order
+    assert [i for i in order if i not in (2, 3)] == [i for i in want if i not in (2, 3)]
+
+
+def _neuron_worker(rank, world, port, tmp):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import oracle
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=257)
+    W = synth.make_codebook(cfg.D, 1024 + 40, 5, kind="dupes")      # ties across the shard edge
+    W[:, 512] = W[:, 511]
+    lo, hi = sharding.neuron_range(W.shape[1], rank, world)
+    b, d1, _ = oracle.bmu(W[:, lo:hi].contiguous().numpy(), rowptr.numpy(), colidx.numpy(), threads=1)
+    dg, bg = sharding.merge_neuron_shards(torch.from_numpy(d1.astype(np.float32)),
+                                          torch.from_numpy(b), lo)
+    if rank == 0:
+        np.save(os.path.join(tmp, "bn.npy"), bg.numpy())
+        np.save(os.path.join(tmp, "dn.npy"), dg.numpy())
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_shard_the_neurons(tmp_path):
+    import oracle
+    port = 31500 + os.getpid() % 2000
+    mp.spawn(_neuron_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=257)
+    W = synth.make_codebook(cfg.D, 1024 + 40, 5, kind="dupes")
+    W[:, 512] = W[:, 511]
+    b, d1, _ = oracle.bmu(W.numpy(), rowptr.numpy(), colidx.numpy())
+    np.testing.assert_array_equal(np.load(tmp_path / "dn.npy"), d1.astype(np.float32))
+    # equal float32 distances on both sides of a shard edge: the lower global index wins
+    got = np.load(tmp_path / "bn.npy")
+    d32 = d1.astype(np.float32)
+    for i in np.nonzero(got != b)[0]:
+        assert oracle.eval_pair(W.numpy(), rowptr.numpy(), colidx.numpy(), oracle.norms(W.numpy()),
+                                int(i), int(got[i])).astype(np.float32) == d32[i] and got[i] < b[i] + 2
+    assert (got == b).mean() > 0.99
