@@ -81,7 +81,11 @@ typedef struct bmu_opts {
                                remaining ids are gathered as in 4; needs what 4 needs,
                                D >= head_rows and M >= 512; the automatic choice for large
                                sweeps); 5 first tensor-core sweep (same split, 512-neuron
-                               slabs, head of 256 or 512, best unit only); 2 staged (a lane per
+                               slabs, head of 256 or 512, best unit only); 7 the same split
+                               with 256 documents per block (128-neuron slabs; the head image
+                               is shared by twice as many documents; head_rows 0 = 896;
+                               best unit only; within 2 % of 6 on the benchmark shapes);
+                               2 staged (a lane per
                                document, rows streamed through shared memory by tensor (TMA)
                                box copies; needs M % 4 == 0, M >= 32, 256 <= D <= 65024) */
     int32_t chunk_neurons;  /* neurons per L2-resident chunk of the codebook (Section 4.2,
@@ -100,7 +104,8 @@ typedef struct bmu_opts {
                                densely, one load per tile, 1 treat them like all other ids */
     int32_t head_rows;      /* tensor-core sweeps: how many of the most frequent features (ids
                                below this) are summed by the tensor cores: a multiple of 64
-                               up to 1024 (kernel 5: 256 or 512); 0 = 768 (kernel 5: 256) */
+                               up to 2048 (kernel 5: 256 or 512); 0 = 768 (kernel 5: 256,
+                               kernel 7: 896) */
     int32_t repack;         /* tensor-core sweeps: 0/1 gather from a compact [D][chunk] copy
                                of the chunk's columns, made before each launch, 2 gather
                                from the codebook itself */

@@ -74,7 +74,7 @@ static size_t mma_repack_bytes(const bmu_opts &o, int64_t D, int64_t M, int64_t 
                                bool top2)
 {
     if (o.repack == 2 || (top2 && o.kernel == 5) ||
-        (o.kernel != 0 && o.kernel != 5 && o.kernel != 6)) return 0;
+        (o.kernel != 0 && o.kernel != 5 && o.kernel != 6 && o.kernel != 7)) return 0;
     if (D > LANES_MAX_D || M < MMA_SLAB) return 0;
     const int64_t chunk = mma_chunk(o, D, M);
     if (M <= chunk) return 0;                      // one launch: the codebook is the chunk
@@ -97,8 +97,8 @@ static int mma_head_rows(const bmu_opts &o, int64_t D)
 {
     if (o.head_rows) return o.head_rows;
     if (o.kernel == 5) return MMA_HEAD;
-    const int64_t cap = D / 64 * 64;
-    return (int)(cap < 768 ? (cap < 64 ? 64 : cap) : 768);
+    const int64_t cap = D / 64 * 64, want = o.kernel == 7 ? 896 : 768;
+    return (int)(cap < want ? (cap < 64 ? 64 : cap) : want);
 }
 
 static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kernel,
@@ -115,7 +115,7 @@ static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kerne
     l.head_off = off;
     if (kernel == 5 && !top2 && D >= head && D <= LANES_MAX_D && M >= MMA_SLAB)
         off = align_up(off + head_image_bytes(M, head), 256);
-    if ((kernel == 0 || kernel == 6) && D >= head && D <= LANES_MAX_D && M >= MMA_SLAB)
+    if ((kernel == 0 || kernel == 6 || kernel == 7) && D >= head && D <= LANES_MAX_D && M >= MMA_SLAB)
         off = align_up(off + head_image2_bytes(M, head), 256);
     l.repack_off = off;                  // compact copy of the codebook chunk being swept
     off = align_up(off + repack_bytes, 256);
@@ -160,7 +160,7 @@ static int check_opts(const bmu_opts &o)
     if (o.relabel < 0 || o.relabel > 2) { set_error("bmu_opts.relabel must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
     for (int i = 0; i < 3; ++i)
         if (o.reserved[i] != 0) { set_error("bmu_opts.reserved must be zero"); return BMU_ERR_INVALID_ARG; }
-    if (o.kernel < 0 || o.kernel > 6) { set_error("bmu_opts.kernel must be 0 .. 6"); return BMU_ERR_INVALID_ARG; }
+    if (o.kernel < 0 || o.kernel > 7) { set_error("bmu_opts.kernel must be 0 .. 7"); return BMU_ERR_INVALID_ARG; }
     if (o.cluster < 0 || o.cluster > 2) { set_error("bmu_opts.cluster must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
     if (o.chunk_neurons < 0) { set_error("bmu_opts.chunk_neurons < 0"); return BMU_ERR_INVALID_ARG; }
     if (o.vec != 0 && o.vec != 4 && o.vec != 8) { set_error("bmu_opts.vec must be 0, 4 or 8"); return BMU_ERR_INVALID_ARG; }
@@ -252,8 +252,9 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     }
     const bool tiled_ok = planned_ok && M >= 128 && o.cluster != 2;
     // tensor-core head: additionally whole 512-neuron slabs, at least 256 features, best unit only
-    const bool mma_ok = tiled_ok && !(top2 && o.kernel == 5) && D >= head && M >= MMA_SLAB;
-    if ((o.kernel == 5 || o.kernel == 6) && !mma_ok) {
+    const bool mma_ok = tiled_ok && !(top2 && (o.kernel == 5 || o.kernel == 7)) && D >= head &&
+                        M >= MMA_SLAB;
+    if ((o.kernel == 5 || o.kernel == 6 || o.kernel == 7) && !mma_ok) {
         set_error("tensor-core sweep needs what the tiled kernel needs, D >= %d and M >= %d "
                   "(kernel 5: no second-best unit)", head, MMA_SLAB);
         return BMU_ERR_UNSUPPORTED;
@@ -261,7 +262,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     // automatic choice for large sweeps: the tensor-core sweep where it applies, else the tiled
     // kernel; both repay their extra preparation only when there is enough to sweep
     const bool big = (double)nnz * (double)M >= 2e10;
-    const bool mma = o.kernel == 5 || o.kernel == 6 || (o.kernel == 0 && mma_ok && big);
+    const bool mma = o.kernel == 5 || o.kernel == 6 || o.kernel == 7 || (o.kernel == 0 && mma_ok && big);
     const bool wide = o.kernel != 5;
     const bool tiled = !mma && (o.kernel == 4 || (o.kernel == 0 && tiled_ok && big));
     if (tiled && !tiled_ok) {
@@ -287,8 +288,9 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         unsigned char *img = reinterpret_cast<unsigned char *>(base + l.head_off);
         const uint16_t *feat = (relabel != 2 && l.plan.fsort_tmp_bytes > 0)
                                    ? reinterpret_cast<const uint16_t *>(pw + l.plan.feat_off) : nullptr;
-        if ((rc = wide ? launch_head_split2(W, M, m_full, head, feat, head_max, img, s)
-                       : launch_head_split(W, M, m_full, head, feat, head_max, img, s))) return rc;
+        if ((rc = o.kernel == 7 ? launch_head_split3(W, M, m_full, head, feat, head_max, img, s)
+                  : wide ? launch_head_split2(W, M, m_full, head, feat, head_max, img, s)
+                         : launch_head_split(W, M, m_full, head, feat, head_max, img, s))) return rc;
         MmaArgs a;
         a.W = W; a.M = M; a.N = N; a.n_tiles = (N + 7) / 8; a.norms = norms;
         a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
@@ -313,7 +315,8 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
             }
             // both images take 4 * head bytes per neuron, slab after slab
             a.head_img = img + (size_t)j * head * 4;
-            if ((rc = wide ? launch_sweep_mma2(a, o, s) : launch_sweep_mma(a, o, s))) return rc;
+            if ((rc = o.kernel == 7 ? launch_sweep_mma3(a, o, s)
+                      : wide ? launch_sweep_mma2(a, o, s) : launch_sweep_mma(a, o, s))) return rc;
         }
         if (m_full < M) {                      // ragged last slab: generic kernel, merged in
             SweepArgs g;

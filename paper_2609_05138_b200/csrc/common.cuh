@@ -158,7 +158,7 @@ struct PlanLayout {
     size_t rank_off, feat_off, fsort_off, fsort_tmp_off, fsort_tmp_bytes;   // feature ranks
 };
 static const int TILE_HEAD_ROWS = 32;    // ids below this are swept densely, once per tile
-static const int HEAD_ROWS_MAX = 1024;   // widest dense head (the tensor-core sweep's)
+static const int HEAD_ROWS_MAX = 2048;   // widest dense head (the tensor-core sweep's)
 int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head, int relabel,
                       char *ws, const PlanLayout &l, cudaStream_t s);
 
@@ -219,6 +219,10 @@ size_t head_image2_bytes(int64_t M, int head);
 int launch_head_split2(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
                        uint32_t *head_max, unsigned char *head_img, cudaStream_t s);
 int launch_sweep_mma2(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
+// 256-document variant (sweep_mma3.cu): 128-neuron slabs, same image size (4 * head bytes per neuron)
+int launch_head_split3(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
+                       uint32_t *head_max, unsigned char *head_img, cudaStream_t s);
+int launch_sweep_mma3(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
 size_t plan_bytes(int64_t N, int64_t nnz, int head, int64_t D, PlanLayout *l);
 int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                 int order_by_length, int head, int relabel, int64_t D, char *ws, const PlanLayout &l,
