@@ -43,7 +43,7 @@ static inline size_t m2_smem_bytes(int head, bool top2)
 {
     return (size_t)MMA_DOCS * (head / 8) + (M2_NS + M2_NX) * MMA_STAGE_BYTES +
            (2 * M2_NS + 2 * M2_NX + 6) * 8 + MMA_DOCS * 8 + 16 + 16 * 16 + 2 * 16 * 4 +
-           (top2 ? 4 * MMA_DOCS * 16 : 0);
+           16 * 8 + (top2 ? 4 * MMA_DOCS * 16 : 0);
 }
 
 // One thread per (slab, group of 8 features, neuron).  Stage order inside a slab: block of
@@ -119,7 +119,8 @@ sweep_mma2_kernel(const MmaArgs a)
     uint32_t *s_off = s_len + 16;
     // TOP2: (best, second) per neuron quarter and document; the warp that owns a quarter of a
     // document is the same in every slab, so it merges without atomics
-    u64 *kq = reinterpret_cast<u64 *>(s_off + 16);
+    uint2 *lut = reinterpret_cast<uint2 *>(s_off + 16);          // 4 mask bits -> 4 fp16 zeros and ones
+    u64 *kq = reinterpret_cast<u64 *>(lut + 16);
     const uint32_t wfull0 = mm_smem(bars), wempty0 = mm_smem(bars + NS);
     const uint32_t xfull0 = mm_smem(bars + 2 * NS), xempty0 = mm_smem(bars + 2 * NS + NX);
     const uint32_t tfull0 = mm_smem(bars + 2 * NS + 2 * NX), tempty0 = tfull0 + 16;
@@ -156,6 +157,11 @@ sweep_mma2_kernel(const MmaArgs a)
         }
     }
     if (threadIdx.x < MMA_DOCS) keys[threadIdx.x] = KEY_WORST;
+    if (threadIdx.x < 16) {
+        const uint32_t b = threadIdx.x;
+        lut[b] = make_uint2((b & 1u) * 0x3c00u + (b & 2u) * 0x1e000000u,
+                            ((b >> 2) & 1u) * 0x3c00u + ((b >> 2) & 2u) * 0x1e000000u);
+    }
     if (TOP2)
         for (int idx = threadIdx.x; idx < 4 * MMA_DOCS * 2; idx += M2_THREADS) kq[idx] = KEY_WORST;
     if (threadIdx.x >= M2_THREADS - 16) {            // 16 threads of the last control warp
@@ -204,7 +210,7 @@ sweep_mma2_kernel(const MmaArgs a)
             unsigned char *dst = xring + (size_t)slot * MMA_STAGE_BYTES;
             // a lane takes documents lane, lane + 32, ..: its 8 mask bytes of this block of 64
             // features in one load, then eight 16-byte stores of fp16 zeros and ones (bit e of
-            // a byte -> half e; 0x3c00 is 1.0)
+            // a byte -> half e; 0x3c00 is 1.0), four bits at a time through a 16-entry table
 #pragma unroll
             for (int j = 0; j < MMA_DOCS / 32; ++j) {
                 const int n = lane + 32 * j;
@@ -213,12 +219,8 @@ sweep_mma2_kernel(const MmaArgs a)
 #pragma unroll
                 for (int kc = 0; kc < 8; ++kc) {
                     const uint32_t b = (kc < 4 ? mb.x : mb.y) >> ((kc & 3) * 8);
-                    uint4 v;
-                    v.x = (b & 1u) * 0x3c00u + (b & 2u) * 0x1e000000u;
-                    v.y = ((b >> 2) & 1u) * 0x3c00u + ((b >> 2) & 2u) * 0x1e000000u;
-                    v.z = ((b >> 4) & 1u) * 0x3c00u + ((b >> 4) & 2u) * 0x1e000000u;
-                    v.w = ((b >> 6) & 1u) * 0x3c00u + ((b >> 6) & 2u) * 0x1e000000u;
-                    *reinterpret_cast<uint4 *>(row + kc * 128) = v;
+                    const uint2 lo4 = lut[b & 15u], hi4 = lut[(b >> 4) & 15u];
+                    *reinterpret_cast<uint4 *>(row + kc * 128) = make_uint4(lo4.x, lo4.y, hi4.x, hi4.y);
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
