@@ -208,8 +208,11 @@ BMU_API int bmu_search_top2_ws(const float *W, int64_t D, int64_t M, const float
  * [D][M], feature-major, 16-byte aligned; sums and distances are still fp32
  * (norms: fp64 accumulate).  Needs M % 256 == 0 (M % 8 == 0 for the norms
  * alone) and D <= 65024.  out_bmu2 / out_dist2 may both be NULL, or both given
- * to get the second-best unit as in bmu_search_top2_ws.  Workspace:
- * bmu_search_top2_workspace_bytes(...) covers either case.
+ * to get the second-best unit as in bmu_search_top2_ws.  bmu_opts.kernel: 3 the
+ * planned kernel, 6 the wide tensor-core sweep (needs M % 512 == 0 and D >=
+ * head_rows; the weights being fp16 already, its head image has one part), 0
+ * the tensor-core sweep for large sweeps, else the planned kernel.  Workspace:
+ * bmu_search_top2_workspace_bytes(...) with the same options covers either case.
  */
 BMU_API int bmu_codebook_norms_f16(const void *W16, int64_t D, int64_t M, float *norms,
                                    void *stream);

@@ -82,13 +82,14 @@ static size_t mma_repack_bytes(const bmu_opts &o, int64_t D, int64_t M, int64_t 
     return (size_t)D * (size_t)(chunk < M ? chunk : M) * sizeof(float);
 }
 
+// one block per codebook row: `width_bytes` (a multiple of 16) from byte `off_bytes` of the row
 __global__ void __launch_bounds__(256)
-repack_chunk_kernel(const float *__restrict__ W, int64_t M, int64_t j_lo, int32_t width,
-                    float *__restrict__ out)
+repack_chunk_kernel(const char *__restrict__ W, int64_t pitch_bytes, int64_t off_bytes,
+                    int32_t width_bytes, char *__restrict__ out)
 {
-    const float4 *src = reinterpret_cast<const float4 *>(W + (int64_t)blockIdx.x * M + j_lo);
-    float4 *dst = reinterpret_cast<float4 *>(out + (int64_t)blockIdx.x * width);
-    for (int i = threadIdx.x; i < width / 4; i += 256) dst[i] = __ldcs(src + i);
+    const uint4 *src = reinterpret_cast<const uint4 *>(W + (int64_t)blockIdx.x * pitch_bytes + off_bytes);
+    uint4 *dst = reinterpret_cast<uint4 *>(out + (int64_t)blockIdx.x * width_bytes);
+    for (int i = threadIdx.x; i < width_bytes / 16; i += 256) dst[i] = __ldcs(src + i);
 }
 
 // Features summed on the tensor cores: 256 for the first tensor-core sweep; 768 for the wide
@@ -298,7 +299,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         a.tile_off = reinterpret_cast<const uint32_t *>(pw + l.plan.tileoff_off);
         a.tile_ids = reinterpret_cast<const uint4 *>(pw + l.plan.tileids_off);
         a.tile_head = reinterpret_cast<const uint32_t *>(pw + l.plan.tilehead_off);
-        a.head_max = head_max; a.head = head;
+        a.head_max = head_max; a.head = head; a.f16 = 0;
         a.state = state; a.state2 = state2; a.status = status;
         const int64_t chunk = mma_chunk(o, D, M);
         float *compact = repack_bytes ? reinterpret_cast<float *>(base + l.repack_off) : nullptr;
@@ -308,7 +309,9 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
             a.first = j == 0;
             if (compact) {                 // gather from a compact copy of this chunk's columns
                 const int32_t width = a.j_hi - a.j_lo;
-                repack_chunk_kernel<<<(unsigned)D, 256, 0, s>>>(W, M, j, width, compact);
+                repack_chunk_kernel<<<(unsigned)D, 256, 0, s>>>(
+                    reinterpret_cast<const char *>(W), M * 4, j * 4, width * 4,
+                    reinterpret_cast<char *>(compact));
                 a.W = reinterpret_cast<const float *>(reinterpret_cast<uintptr_t>(compact) -
                                                       (uintptr_t)j * sizeof(float));
                 a.M = width;
@@ -589,12 +592,23 @@ int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
         return BMU_ERR_INVALID_ARG;
     }
     if (M % 256 != 0 || D < 1 || D > LANES_MAX_D || (reinterpret_cast<uintptr_t>(W16) & 15) != 0 ||
-        (o.kernel != 0 && o.kernel != 3)) {
+        (o.kernel != 0 && o.kernel != 3 && o.kernel != 6)) {
         set_error("half-precision search needs M %% 256 == 0, 1 <= D <= %d, 16-byte alignment and "
-                  "the planned kernel", LANES_MAX_D);
+                  "the planned (3) or the wide tensor-core (6) kernel", LANES_MAX_D);
         return BMU_ERR_UNSUPPORTED;
     }
-    const Layout l = layout_for(D, M, N, nnz, 3, top2);
+    // large sweeps take the wide tensor-core sweep (whole 512-neuron slabs only)
+    bmu_opts ow = o;
+    ow.kernel = 6;
+    const int head = mma_head_rows(ow, D);
+    const bool wide_ok = M % MMA_SLAB == 0 && D >= head && o.cluster != 2;
+    if (o.kernel == 6 && !wide_ok) {
+        set_error("half-precision tensor-core sweep needs M %% %d == 0, D >= %d and length-ordered "
+                  "documents", MMA_SLAB, head);
+        return BMU_ERR_UNSUPPORTED;
+    }
+    const bool wide = o.kernel == 6 || (o.kernel == 0 && wide_ok && (double)nnz * (double)M >= 2e10);
+    const Layout l = wide ? layout_of(ow, D, M, N, nnz, top2) : layout_for(D, M, N, nnz, 3, top2);
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < l.total) {
         set_error("workspace missing, not 256-byte aligned, or smaller than %zu bytes", l.total);
         return BMU_ERR_WORKSPACE;
@@ -606,6 +620,48 @@ int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
         float *n = reinterpret_cast<float *>(base + l.norms_off);
         if ((rc = launch_norms_f16(W16, D, M, n, s))) return rc;
         norms = n;
+    }
+    if (wide) {
+        uint32_t *status = reinterpret_cast<uint32_t *>(base + l.status_off);
+        BMU_CUDA(cudaMemsetAsync(status, 0, 256, s));
+        char *pw = base + l.plan_off;
+        const int relabel = o.relabel;
+        if ((rc = launch_plan(rowptr, colidx, N, nnz, 1, head, relabel, D, pw, l.plan, s))) return rc;
+        if ((rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, relabel, pw, l.plan, s))) return rc;
+        unsigned char *img = reinterpret_cast<unsigned char *>(base + l.head_off);
+        const uint16_t *feat = (relabel != 2 && l.plan.fsort_tmp_bytes > 0)
+                                   ? reinterpret_cast<const uint16_t *>(pw + l.plan.feat_off) : nullptr;
+        if ((rc = launch_head_split2_f16(W16, M, M, head, feat, img, s))) return rc;
+        MmaArgs a;
+        a.W = static_cast<const float *>(W16); a.M = M; a.N = N; a.n_tiles = (N + 7) / 8; a.norms = norms;
+        a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
+        a.tile_len = reinterpret_cast<const uint32_t *>(pw + l.plan.tilelen_off);
+        a.tile_off = reinterpret_cast<const uint32_t *>(pw + l.plan.tileoff_off);
+        a.tile_ids = reinterpret_cast<const uint4 *>(pw + l.plan.tileids_off);
+        a.tile_head = reinterpret_cast<const uint32_t *>(pw + l.plan.tilehead_off);
+        a.head_max = status + 16; a.head = head; a.f16 = 1;
+        a.state = state; a.state2 = state2; a.status = status;
+        // twice the neurons per L2-resident chunk: the rows are half as wide
+        const int64_t chunk = o.chunk_neurons ? mma_chunk(o, D, M) : 2 * mma_auto_chunk(D, M);
+        const size_t repack_bytes = mma_repack_bytes(ow, D, M, N, nnz, top2);
+        char *compact = (repack_bytes && M > chunk) ? base + l.repack_off : nullptr;
+        for (int64_t j = 0; j < M; j += chunk) {
+            a.j_lo = (int32_t)j;
+            a.j_hi = (int32_t)(j + chunk < M ? j + chunk : M);
+            a.first = j == 0;
+            a.W = static_cast<const float *>(W16); a.M = M;
+            if (compact) {                 // a compact copy of this chunk's columns (2 bytes each)
+                const int32_t width = a.j_hi - a.j_lo;
+                repack_chunk_kernel<<<(unsigned)D, 256, 0, s>>>(static_cast<const char *>(W16), M * 2,
+                                                              j * 2, width * 2, compact);
+                a.W = reinterpret_cast<const float *>(reinterpret_cast<uintptr_t>(compact) -
+                                                      (uintptr_t)j * 2);
+                a.M = width;
+            }
+            a.head_img = img + (size_t)j * head * 2;     // one part: 2 * head bytes per neuron
+            if ((rc = launch_sweep_mma2(a, o, s))) return rc;
+        }
+        return launch_finalize(state, state2, rowptr, N, out_bmu, out_dist, out_bmu2, out_dist2, s);
     }
     BMU_CUDA(cudaMemsetAsync(base + l.status_off, 0, 256, s));
     char *pw = base + l.plan_off;

@@ -204,6 +204,7 @@ struct MmaArgs {
     u64 *state2;                // wide-head sweep only: second-best unit (NULL unless wanted)
     uint32_t *status;           // set non-zero if a bounded wait ran out
     int32_t j_lo, j_hi, first;
+    int32_t f16;                // wide-head sweep only: W is an fp16 codebook (row pitch 2 * M bytes)
 };
 size_t head_image_bytes(int64_t M, int head);
 // writes the fp16 (hi, lo) split of rows [0, head) of W, scaled by a power of two, as the
@@ -219,6 +220,8 @@ size_t head_image2_bytes(int64_t M, int head);
 int launch_head_split2(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
                        uint32_t *head_max, unsigned char *head_img, cudaStream_t s);
 int launch_sweep_mma2(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
+int launch_head_split2_f16(const void *W16, int64_t M, int64_t m_full, int head, const uint16_t *feat,
+                           unsigned char *head_img, cudaStream_t s);
 // 256-document variant (sweep_mma3.cu): 128-neuron slabs, same image size (4 * head bytes per neuron)
 int launch_head_split3(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
                        uint32_t *head_max, unsigned char *head_img, cudaStream_t s);

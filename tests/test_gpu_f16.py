@@ -60,3 +60,26 @@ def test_f16_top2_and_limits(bmu):
     with pytest.raises(bmu.BmuError) as e:
         bmu.bmu_search_f16_ws(W16[:, :100].contiguous().cuda(), rowptr.cuda(), colidx.cuda())
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("name,n_docs,M,kind,head", [("cfg1", 4000, 1024, "uniform", 0),
+                                                     ("cfg3", 1500, 2048, "scaled", 0),
+                                                     ("cfg5", 700, 512, "signed", 256),
+                                                     ("cfg1", 900, 512, "dupes", 1024)])
+def test_f16_tensor_core_sweep_matches_oracle(bmu, name, n_docs, M, kind, head):
+    """The wide tensor-core sweep on a half-precision codebook: the weights are fp16 already, so
+    the head image has one part and the tail gathers 8-byte pieces."""
+    cfg = synth.CONFIGS[name]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=n_docs)
+    W16 = synth.make_codebook(cfg.D, M, 52, kind=kind).half()
+    W32 = W16.float()
+    o = bmu.Opts()
+    o.kernel = 6
+    o.head_rows = head
+    ob, od = bmu.bmu_search_f16_ws(W16.cuda(), rowptr.cuda(), colidx.cuda(), opts=o)
+    torch.cuda.synchronize()
+    parity.compare(ob.cpu().numpy(), od.cpu().numpy(), W32.numpy(), rowptr.numpy(), colidx.numpy())
+    if kind == "dupes":
+        assert int((ob % 2).sum()) == 0
+    b1, d1, b2, d2 = bmu.bmu_search_f16_ws(W16.cuda(), rowptr.cuda(), colidx.cuda(), opts=o, top2=True)
+    assert torch.equal(b1, ob) and torch.equal(d1, od) and bool((b2 != b1).all())
