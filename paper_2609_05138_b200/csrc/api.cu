@@ -659,7 +659,7 @@ int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
                 a.M = width;
             }
             a.head_img = img + (size_t)j * head * 2;     // one part: 2 * head bytes per neuron
-            if ((rc = launch_sweep_mma2(a, o, s))) return rc;
+            if ((rc = launch_sweep_mma2_f16(a, o, s))) return rc;
         }
         return launch_finalize(state, state2, rowptr, N, out_bmu, out_dist, out_bmu2, out_dist2, s);
     }

@@ -220,6 +220,7 @@ size_t head_image2_bytes(int64_t M, int head);
 int launch_head_split2(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
                        uint32_t *head_max, unsigned char *head_img, cudaStream_t s);
 int launch_sweep_mma2(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
+int launch_sweep_mma2_f16(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
 int launch_head_split2_f16(const void *W16, int64_t M, int64_t m_full, int head, const uint16_t *feat,
                            unsigned char *head_img, cudaStream_t s);
 // 256-document variant (sweep_mma3.cu): 128-neuron slabs, same image size (4 * head bytes per neuron)

@@ -91,63 +91,18 @@ int launch_head_split2(const float *W, int64_t M, int64_t m_full, int head, cons
     return BMU_OK;
 }
 
-// Half-precision codebook: the weights are fp16 already, so the image is a re-layout (one part,
-// no scale): stage order inside a slab: block of 64 features, tile c.
-__global__ void __launch_bounds__(M2_SLAB)
-head_split2_f16_kernel(const __half *__restrict__ W16, int64_t M, int head,
-                       const uint16_t *__restrict__ feat, unsigned char *__restrict__ img)
-{
-    const int sl = blockIdx.x, kcg = blockIdx.y, jin = threadIdx.x;
-    const int SPS = 2 * (head / 64);
-    const __half *col = W16 + (int64_t)sl * M2_SLAB + jin;
-    __align__(16) __half h[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        const int64_t row = feat ? (int64_t)feat[kcg * 8 + e] : (int64_t)(kcg * 8 + e);
-        h[e] = col[row * M];
-    }
-    const int c = jin & 1, r = ((jin >> 6) << 5) | (((jin >> 1) & 1) << 4) | ((jin >> 2) & 15);
-    const int kb = kcg >> 3, kc = kcg & 7;
-    const size_t off = (size_t)(r >> 3) * 1024 + (size_t)kc * 128 + (size_t)(r & 7) * 16;
-    const size_t st = (size_t)sl * SPS + (size_t)(kb * 2 + c);
-    *reinterpret_cast<uint4 *>(img + st * MMA_STAGE_BYTES + off) = *reinterpret_cast<uint4 *>(h);
-}
-
-int launch_head_split2_f16(const void *W16, int64_t M, int64_t m_full, int head, const uint16_t *feat,
-                           unsigned char *head_img, cudaStream_t s)
-{
-    if (m_full <= 0) return BMU_OK;
-    const dim3 grid((unsigned)(m_full / M2_SLAB), head / 8);
-    head_split2_f16_kernel<<<grid, M2_SLAB, 0, s>>>(static_cast<const __half *>(W16), M, head, feat,
-                                                    head_img);
-    BMU_CUDA(cudaGetLastError());
-    return BMU_OK;
-}
-
-// two fp16 pairs (8 bytes of a half-precision row) widened and added to four fp32 sums
-__device__ __forceinline__ void m2_add_h4(u64 &a0, u64 &a1, u64 raw)
-{
-    const uint32_t lo = (uint32_t)raw, hi = (uint32_t)(raw >> 32);
-    const float2 f0 = __half22float2(*reinterpret_cast<const __half2 *>(&lo));
-    const float2 f1 = __half22float2(*reinterpret_cast<const __half2 *>(&hi));
-    add2(a0, ((u64)__float_as_uint(f0.y) << 32) | __float_as_uint(f0.x));
-    add2(a1, ((u64)__float_as_uint(f1.y) << 32) | __float_as_uint(f1.x));
-}
-
 __device__ __forceinline__ void m2_unpack(const uint4 q, uint32_t f[8])
 {
     f[0] = q.x & 0xffffu; f[1] = q.x >> 16; f[2] = q.y & 0xffffu; f[3] = q.y >> 16;
     f[4] = q.z & 0xffffu; f[5] = q.z >> 16; f[6] = q.w & 0xffffu; f[7] = q.w >> 16;
 }
 
-// TOP2: also the second-best unit (Table 5: the paper's kernel tracks it for topographic error).
-// F16: the codebook is half precision (the paper's storage): one image part, 8-byte row pieces.
-template <bool TOP2, bool F16>
+// TOP2: also the second-best unit (Table 5: the paper's kernel tracks it for topographic error)
+template <bool TOP2>
 __global__ void __launch_bounds__(M2_THREADS, 1)
 sweep_mma2_kernel(const MmaArgs a)
 {
     constexpr int NS = M2_NS, NX = M2_NX, NTW = M2_TAIL_WARPS;
-    constexpr int PARTS = F16 ? 1 : 2;                           // (hi, lo) unless the weights are fp16
     const int H = a.head, KB = H / 64;
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char *masks = smem;                                 // 128 documents x H bits
@@ -227,7 +182,7 @@ sweep_mma2_kernel(const MmaArgs a)
         // ---------------- producer: W stages of every slab, in order
         if (lane == 0) {
             const unsigned char *src = a.head_img;
-            const int total = n_slabs * 2 * PARTS * KB;
+            const int total = n_slabs * 4 * KB;
             int issued = 0;
             for (int c = 0; c < total; ++c) {
                 const int slot = c % NS;
@@ -288,7 +243,7 @@ sweep_mma2_kernel(const MmaArgs a)
                 for (int kb = 0; kb < KB && ok; ++kb, ++xc) {
                     const int xslot = xc % NX;
                     if (!mm_wait(xfull0 + 8 * xslot, (xc / NX) & 1, abort_flag, a.status, 32u)) { ok = false; break; }
-                    for (int cp = 0; cp < 2 * PARTS; ++cp, ++wc) {   // cp = tile * PARTS + part
+                    for (int cp = 0; cp < 4; ++cp, ++wc) {       // cp = tile * 2 + part
                         const int slot = wc % NS;
                         if (!mm_wait(wfull0 + 8 * slot, (wc / NS) & 1, abort_flag, a.status, 4u)) { ok = false; break; }
                         mm_fence_after();
@@ -296,8 +251,8 @@ sweep_mma2_kernel(const MmaArgs a)
                         for (int u = 0; u < 4; ++u) {
                             const u64 ad = mm_desc(wring_u32 + slot * (uint32_t)MMA_STAGE_BYTES + u * 256, 128, 1024);
                             const u64 bd = mm_desc(xring_u32 + xslot * (uint32_t)MMA_STAGE_BYTES + u * 256, 128, 1024);
-                            mm_mma(tmem + buf * 256 + (cp / PARTS) * MMA_DOCS, ad, bd, idesc,
-                                   (kb | (cp % PARTS) | u) != 0);
+                            mm_mma(tmem + buf * 256 + (cp >> 1) * MMA_DOCS, ad, bd, idesc,
+                                   (kb | (cp & 1) | u) != 0);
                         }
                         mm_commit(wempty0 + 8 * slot);
                     }
@@ -316,8 +271,8 @@ sweep_mma2_kernel(const MmaArgs a)
         // 128-bit load per lane and row, two rows (one per half-warp) per instruction.
         const int q = warp & 3, g = warp >> 2;
         const int li = lane & 15, lh = lane >> 4;
-        const float inv_s = F16 ? 1.f : 1.f / head_scale(__ldg(a.head_max));
-        const uint32_t rowbytes = (uint32_t)(a.M * (F16 ? 2 : 4));
+        const float inv_s = 1.f / head_scale(__ldg(a.head_max));
+        const uint32_t rowbytes = (uint32_t)(a.M * 4);
         const int mydoc = 8 * lh + ((lane & 1) << 2 | (lane & 2) | ((lane >> 2) & 1));
         for (int sl = 0; sl < n_slabs; ++sl) {
             const int buf = sl & 1;
@@ -337,38 +292,9 @@ sweep_mma2_kernel(const MmaArgs a)
                     const uint32_t my_rows = (lh ? tlb : tla) & 0xffffu;
                     const int mine = 2 * dg + ((lh && has_b) ? 1 : 0);
                     const uint4 *gp = a.tile_ids + s_off[mine];
-                    const char *base = reinterpret_cast<const char *>(a.W) +
-                                       (size_t)(j0 + li * 4) * (F16 ? 2 : 4);
+                    const char *base = reinterpret_cast<const char *>(a.W + j0 + li * 4);
                     uint32_t b = 0;
                     uint4 qn = s_first[mine];
-                    if (F16) {
-                        // 8-byte pieces: two rows of ids per turn keep sixteen loads in flight
-                        for (; b + 1 < full; b += 2) {
-                            uint32_t f[16];
-                            m2_unpack(qn, f);
-                            m2_unpack(__ldcs(gp + b + 1), f + 8);
-                            qn = __ldcs(gp + b + 2);
-                            u64 w[16];
-#pragma unroll
-                            for (int t = 0; t < 16; ++t)
-                                w[t] = __ldg(reinterpret_cast<const u64 *>(base + (u64)f[t] * rowbytes));
-#pragma unroll
-                            for (int t = 0; t < 16; ++t) m2_add_h4(acc[t & 7][0], acc[t & 7][1], w[t]);
-                        }
-                        for (; b < rows; ++b) {
-                            uint32_t f[8];
-                            m2_unpack(qn, f);
-                            qn = __ldcs(gp + b + 1);
-                            const bool in = b < my_rows;
-                            u64 w[8];
-#pragma unroll
-                            for (int t = 0; t < 8; ++t)
-                                w[t] = (in && f[t] != 0xffffu)
-                                           ? __ldg(reinterpret_cast<const u64 *>(base + (u64)f[t] * rowbytes)) : 0ull;
-#pragma unroll
-                            for (int t = 0; t < 8; ++t) m2_add_h4(acc[t][0], acc[t][1], w[t]);
-                        }
-                    } else {
                     for (; b < full; ++b) {
                         uint32_t f[8];
                         m2_unpack(qn, f);
@@ -393,7 +319,6 @@ sweep_mma2_kernel(const MmaArgs a)
                                        : make_ulonglong2(0ull, 0ull);
 #pragma unroll
                         for (int t = 0; t < 8; ++t) { add2(acc[t][0], w[t].x); add2(acc[t][1], w[t].y); }
-                    }
                     }
                 }
                 // head sums of these documents: the MMAs of this slab ran during the gather.
@@ -525,22 +450,15 @@ int launch_sweep_mma2(const MmaArgs &a, const bmu_opts &o, cudaStream_t s)
     int dev = 0;
     BMU_CUDA(cudaGetDevice(&dev));
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        const int plain = (int)m2_smem_bytes(HEAD_ROWS_MAX, false), two = (int)m2_smem_bytes(HEAD_ROWS_MAX, true);
-        BMU_CUDA(cudaFuncSetAttribute(sweep_mma2_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, plain));
-        BMU_CUDA(cudaFuncSetAttribute(sweep_mma2_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, two));
-        BMU_CUDA(cudaFuncSetAttribute(sweep_mma2_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, plain));
-        BMU_CUDA(cudaFuncSetAttribute(sweep_mma2_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, two));
+        BMU_CUDA(cudaFuncSetAttribute(sweep_mma2_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)m2_smem_bytes(HEAD_ROWS_MAX, false)));
+        BMU_CUDA(cudaFuncSetAttribute(sweep_mma2_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)m2_smem_bytes(HEAD_ROWS_MAX, true)));
         configured[dev] = true;
     }
     const unsigned blocks = (unsigned)((a.N + MMA_DOCS - 1) / MMA_DOCS);
-    const size_t smem = m2_smem_bytes(a.head, a.state2 != nullptr);
-    if (a.f16) {
-        if (a.state2) sweep_mma2_kernel<true, true><<<blocks, M2_THREADS, smem, s>>>(a);
-        else sweep_mma2_kernel<false, true><<<blocks, M2_THREADS, smem, s>>>(a);
-    } else {
-        if (a.state2) sweep_mma2_kernel<true, false><<<blocks, M2_THREADS, smem, s>>>(a);
-        else sweep_mma2_kernel<false, false><<<blocks, M2_THREADS, smem, s>>>(a);
-    }
+    if (a.state2) sweep_mma2_kernel<true><<<blocks, M2_THREADS, m2_smem_bytes(a.head, true), s>>>(a);
+    else sweep_mma2_kernel<false><<<blocks, M2_THREADS, m2_smem_bytes(a.head, false), s>>>(a);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
