@@ -68,14 +68,30 @@ int launch_head_split2_f16(const void *W16, int64_t M, int64_t m_full, int head,
     return BMU_OK;
 }
 
-// two fp16 pairs (8 bytes of a half-precision row) widened and added to four fp32 sums
+// fp32 sum + fp16 term in one instruction (mixed-precision add of sm_100: the widening is exact,
+// so the result is the one a convert followed by an fp32 add gives)
+__device__ __forceinline__ uint32_t m2_addh(uint32_t c, uint16_t h)
+{
+    float d;
+    asm("add.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(__uint_as_float(c)));
+    return __float_as_uint(d);
+}
+
+// two fp16 pairs (8 bytes of a half-precision row) added to four fp32 sums
 __device__ __forceinline__ void m2_add_h4(u64 &a0, u64 &a1, u64 raw)
 {
+#ifdef BMU_F16_CONVERT_ADD
     const uint32_t lo = (uint32_t)raw, hi = (uint32_t)(raw >> 32);
     const float2 f0 = __half22float2(*reinterpret_cast<const __half2 *>(&lo));
     const float2 f1 = __half22float2(*reinterpret_cast<const __half2 *>(&hi));
     add2(a0, ((u64)__float_as_uint(f0.y) << 32) | __float_as_uint(f0.x));
     add2(a1, ((u64)__float_as_uint(f1.y) << 32) | __float_as_uint(f1.x));
+#else
+    uint16_t h0, h1, h2, h3;
+    asm("mov.b64 {%0, %1, %2, %3}, %4;" : "=h"(h0), "=h"(h1), "=h"(h2), "=h"(h3) : "l"(raw));
+    a0 = ((u64)m2_addh((uint32_t)(a0 >> 32), h1) << 32) | m2_addh((uint32_t)a0, h0);
+    a1 = ((u64)m2_addh((uint32_t)(a1 >> 32), h3) << 32) | m2_addh((uint32_t)a1, h2);
+#endif
 }
 
 __device__ __forceinline__ void m2_unpack(const uint4 q, uint32_t f[8])
@@ -85,13 +101,11 @@ __device__ __forceinline__ void m2_unpack(const uint4 q, uint32_t f[8])
 }
 
 // TOP2: also the second-best unit (Table 5: the paper's kernel tracks it for topographic error).
-// F16: the codebook is half precision (the paper's storage): one image part, 8-byte row pieces.
 template <bool TOP2>
 __global__ void __launch_bounds__(M2_THREADS, 1)
 sweep_mma2_f16_kernel(const MmaArgs a)
 {
     constexpr int NS = M2_NS, NX = M2_NX, NTW = M2_TAIL_WARPS;
-    constexpr bool F16 = true;
     constexpr int PARTS = 1;                                     // the weights are fp16: no lo part
     const int H = a.head, KB = H / 64;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -261,8 +275,8 @@ sweep_mma2_f16_kernel(const MmaArgs a)
         // 128-bit load per lane and row, two rows (one per half-warp) per instruction.
         const int q = warp & 3, g = warp >> 2;
         const int li = lane & 15, lh = lane >> 4;
-        const float inv_s = F16 ? 1.f : 1.f / head_scale(__ldg(a.head_max));
-        const uint32_t rowbytes = (uint32_t)(a.M * (F16 ? 2 : 4));
+        const float inv_s = 1.f;                                 // the image is unscaled
+        const uint32_t rowbytes = (uint32_t)(a.M * 2);
         const int mydoc = 8 * lh + ((lane & 1) << 2 | (lane & 2) | ((lane >> 2) & 1));
         for (int sl = 0; sl < n_slabs; ++sl) {
             const int buf = sl & 1;
@@ -283,62 +297,34 @@ sweep_mma2_f16_kernel(const MmaArgs a)
                     const int mine = 2 * dg + ((lh && has_b) ? 1 : 0);
                     const uint4 *gp = a.tile_ids + s_off[mine];
                     const char *base = reinterpret_cast<const char *>(a.W) +
-                                       (size_t)(j0 + li * 4) * (F16 ? 2 : 4);
+                                       (size_t)(j0 + li * 4) * 2;
                     uint32_t b = 0;
                     uint4 qn = s_first[mine];
-                    if (F16) {
-                        // 8-byte pieces: two rows of ids per turn keep sixteen loads in flight
-                        for (; b + 1 < full; b += 2) {
-                            uint32_t f[16];
-                            m2_unpack(qn, f);
-                            m2_unpack(__ldcs(gp + b + 1), f + 8);
-                            qn = __ldcs(gp + b + 2);
-                            u64 w[16];
-#pragma unroll
-                            for (int t = 0; t < 16; ++t)
-                                w[t] = __ldg(reinterpret_cast<const u64 *>(base + (u64)f[t] * rowbytes));
-#pragma unroll
-                            for (int t = 0; t < 16; ++t) m2_add_h4(acc[t & 7][0], acc[t & 7][1], w[t]);
-                        }
-                        for (; b < rows; ++b) {
-                            uint32_t f[8];
-                            m2_unpack(qn, f);
-                            qn = __ldcs(gp + b + 1);
-                            const bool in = b < my_rows;
-                            u64 w[8];
-#pragma unroll
-                            for (int t = 0; t < 8; ++t)
-                                w[t] = (in && f[t] != 0xffffu)
-                                           ? __ldg(reinterpret_cast<const u64 *>(base + (u64)f[t] * rowbytes)) : 0ull;
-#pragma unroll
-                            for (int t = 0; t < 8; ++t) m2_add_h4(acc[t][0], acc[t][1], w[t]);
-                        }
-                    } else {
-                    for (; b < full; ++b) {
-                        uint32_t f[8];
+                    // 8-byte pieces: two rows of ids per turn keep sixteen loads in flight
+                    for (; b + 1 < full; b += 2) {
+                        uint32_t f[16];
                         m2_unpack(qn, f);
-                        qn = __ldcs(gp + b + 1);
-                        ulonglong2 w[8];
+                        m2_unpack(__ldcs(gp + b + 1), f + 8);
+                        qn = __ldcs(gp + b + 2);
+                        u64 w[16];
 #pragma unroll
-                        for (int t = 0; t < 8; ++t)
-                            w[t] = __ldg(reinterpret_cast<const ulonglong2 *>(base + (u64)f[t] * rowbytes));
+                        for (int t = 0; t < 16; ++t)
+                            w[t] = __ldg(reinterpret_cast<const u64 *>(base + (u64)f[t] * rowbytes));
 #pragma unroll
-                        for (int t = 0; t < 8; ++t) { add2(acc[t][0], w[t].x); add2(acc[t][1], w[t].y); }
+                        for (int t = 0; t < 16; ++t) m2_add_h4(acc[t & 7][0], acc[t & 7][1], w[t]);
                     }
-                    for (; b < rows; ++b) {                      // some documents have run out
+                    for (; b < rows; ++b) {
                         uint32_t f[8];
                         m2_unpack(qn, f);
                         qn = __ldcs(gp + b + 1);
                         const bool in = b < my_rows;
-                        ulonglong2 w[8];
+                        u64 w[8];
 #pragma unroll
                         for (int t = 0; t < 8; ++t)
                             w[t] = (in && f[t] != 0xffffu)
-                                       ? __ldg(reinterpret_cast<const ulonglong2 *>(base + (u64)f[t] * rowbytes))
-                                       : make_ulonglong2(0ull, 0ull);
+                                       ? __ldg(reinterpret_cast<const u64 *>(base + (u64)f[t] * rowbytes)) : 0ull;
 #pragma unroll
-                        for (int t = 0; t < 8; ++t) { add2(acc[t][0], w[t].x); add2(acc[t][1], w[t].y); }
-                    }
+                        for (int t = 0; t < 8; ++t) m2_add_h4(acc[t][0], acc[t][1], w[t]);
                     }
                 }
                 // head sums of these documents: the MMAs of this slab ran during the gather.
