@@ -255,14 +255,17 @@ sweep_rows_f16_kernel(const RowsArgs a)
 
     for (int j0 = a.j_lo; j0 < a.j_hi; j0 += 256) {
         const char *base = reinterpret_cast<const char *>(W16 + j0 + lane * 8);
-        u64 acc[4] = {0ull, 0ull, 0ull, 0ull};
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        // fp32 sum + fp16 weight in one instruction (the mixed-precision add of sm_100; the
+        // widening is exact, so this equals convert-then-add bit for bit)
         auto add_row = [&](const uint4 h) {
             const uint32_t w[4] = {h.x, h.y, h.z, h.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const float2 f2 = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
-                const u64 pk = ((u64)__float_as_uint(f2.y) << 32) | __float_as_uint(f2.x);
-                add2(acc[i], pk);
+                uint16_t h0, h1;
+                asm("mov.b32 {%0, %1}, %2;" : "=h"(h0), "=h"(h1) : "r"(w[i]));
+                asm("add.rn.f32.f16 %0, %1, %0;" : "+f"(acc[2 * i]) : "h"(h0));
+                asm("add.rn.f32.f16 %0, %1, %0;" : "+f"(acc[2 * i + 1]) : "h"(h1));
             }
         };
         for (int g = 0; g < full; ++g) {
@@ -289,8 +292,8 @@ sweep_rows_f16_kernel(const RowsArgs a)
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const float2 n = __ldg(reinterpret_cast<const float2 *>(a.norms + col + 2 * i));
-            best.push(fmaf(-2.f, lo_f(acc[i]), n.x), col + 2 * i);
-            best.push(fmaf(-2.f, hi_f(acc[i]), n.y), col + 2 * i + 1);
+            best.push(fmaf(-2.f, acc[2 * i], n.x), col + 2 * i);
+            best.push(fmaf(-2.f, acc[2 * i + 1], n.y), col + 2 * i + 1);
         }
     }
     u64 k1, k2;
