@@ -211,9 +211,12 @@ BMU_API int bmu_search_top2_ws(const float *W, int64_t D, int64_t M, const float
  * to get the second-best unit as in bmu_search_top2_ws.  bmu_opts.kernel: 3 the
  * planned kernel, 6 the wide tensor-core sweep (needs M % 512 == 0 and D >=
  * head_rows; the weights being fp16 already, its head image has one part), 0
- * the tensor-core sweep for large sweeps, else the planned kernel.  Workspace:
- * bmu_search_top2_workspace_bytes(...) with the same options covers either case.
+ * the tensor-core sweep for large sweeps, else the planned kernel; head_rows
+ * defaults to 512 here.  Workspace: bmu_search_f16_workspace_bytes(...) with the
+ * same sizes and options (enough with or without the second-best outputs).
  */
+BMU_API size_t bmu_search_f16_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,
+                                              const bmu_opts *opts);
 BMU_API int bmu_codebook_norms_f16(const void *W16, int64_t D, int64_t M, float *norms,
                                    void *stream);
 BMU_API int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,

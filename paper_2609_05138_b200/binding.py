@@ -55,6 +55,9 @@ EXPORTS = {
     "bmu_search_top2_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int64, ctypes.c_int64,
                                                           ctypes.c_int64, ctypes.c_int64,
                                                           ctypes.c_void_p]),
+    "bmu_search_f16_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int64, ctypes.c_int64,
+                                                         ctypes.c_int64, ctypes.c_int64,
+                                                         ctypes.c_void_p]),
     "bmu_search_top2_ws": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                           ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
@@ -245,8 +248,8 @@ def bmu_search_f16_ws(W16, rowptr, colidx, norms=None, opts: Opts | None = None,
     od = torch.empty(N, dtype=torch.float32, device=dev)
     ob2 = torch.empty(N, dtype=torch.int32, device=dev) if top2 else None
     od2 = torch.empty(N, dtype=torch.float32, device=dev) if top2 else None
-    need = int(load().bmu_search_top2_workspace_bytes(D, M, N, nnz,
-                                                      ctypes.byref(opts) if opts else None))
+    need = int(load().bmu_search_f16_workspace_bytes(D, M, N, nnz,
+                                                     ctypes.byref(opts) if opts else None))
     ws = workspace if workspace is not None else torch.empty(need + 256, dtype=torch.uint8,
                                                              device=dev)
     ws_ptr = (ws.data_ptr() + 255) // 256 * 256

@@ -572,6 +572,35 @@ int bmu_codebook_norms_f16(const void *W16, int64_t D, int64_t M, float *norms, 
     return launch_norms_f16(W16, D, M, norms, static_cast<cudaStream_t>(stream));
 }
 
+// Which kernel a half-precision search takes: large sweeps the wide tensor-core sweep (whole
+// 512-neuron slabs only), the rest the planned kernel.  `ow` = the options of the wide sweep, its
+// head resolved (512 by default: with 2-byte rows the gathered tail is cheap, so the balance
+// point sits lower than the fp32 sweep's 768).
+static bool f16_route(const bmu_opts &o, int64_t D, int64_t M, int64_t nnz, bmu_opts &ow, bool &wide)
+{
+    ow = o;
+    ow.kernel = 6;
+    if (!ow.head_rows) {
+        const int64_t cap = D / 64 * 64;
+        ow.head_rows = (int32_t)(cap < 512 ? (cap < 64 ? 64 : cap) : 512);
+    }
+    const bool wide_ok = M % MMA_SLAB == 0 && D >= ow.head_rows && o.cluster != 2;
+    wide = wide_ok && (o.kernel == 6 || (o.kernel == 0 && (double)nnz * (double)M >= 2e10));
+    return wide_ok;
+}
+
+size_t bmu_search_f16_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,
+                                      const bmu_opts *opts)
+{
+    if (D < 0 || M < 0 || N < 0 || nnz < 0) return 0;
+    bmu_opts o, ow;
+    memset(&o, 0, sizeof(o));
+    if (opts) o = *opts;
+    bool wide = false;
+    f16_route(o, D, M, nnz, ow, wide);
+    return (wide ? layout_of(ow, D, M, N, nnz, true) : layout_for(D, M, N, nnz, 3, true)).total;
+}
+
 int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
                       const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                       int32_t *out_bmu, float *out_dist, int32_t *out_bmu2, float *out_dist2,
@@ -597,17 +626,15 @@ int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
                   "the planned (3) or the wide tensor-core (6) kernel", LANES_MAX_D);
         return BMU_ERR_UNSUPPORTED;
     }
-    // large sweeps take the wide tensor-core sweep (whole 512-neuron slabs only)
-    bmu_opts ow = o;
-    ow.kernel = 6;
-    const int head = mma_head_rows(ow, D);
-    const bool wide_ok = M % MMA_SLAB == 0 && D >= head && o.cluster != 2;
+    bmu_opts ow;
+    bool wide = false;
+    const bool wide_ok = f16_route(o, D, M, nnz, ow, wide);
+    const int head = ow.head_rows;
     if (o.kernel == 6 && !wide_ok) {
         set_error("half-precision tensor-core sweep needs M %% %d == 0, D >= %d and length-ordered "
                   "documents", MMA_SLAB, head);
         return BMU_ERR_UNSUPPORTED;
     }
-    const bool wide = o.kernel == 6 || (o.kernel == 0 && wide_ok && (double)nnz * (double)M >= 2e10);
     const Layout l = wide ? layout_of(ow, D, M, N, nnz, top2) : layout_for(D, M, N, nnz, 3, top2);
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < l.total) {
         set_error("workspace missing, not 256-byte aligned, or smaller than %zu bytes", l.total);

@@ -2,11 +2,14 @@
 // storage (Section 4.2: "two bytes per half-precision weight"; Section 4.3: __half2 loads).
 // Same structure -- 256-neuron slabs, two accumulator tiles, double-buffered tensor memory,
 // K-outermost with X expanded per block of 64 features, tail tasks of 16 documents x 64
-// neurons -- with two differences: the weights are fp16 already, so the head image is a plain
-// re-layout with ONE part (half the MMAs, 2 bytes per weight, no scale), and the tail gathers
-// 8-byte pieces (four fp16 neurons per lane), two id rows per turn so that sixteen loads are in
-// flight per warp, widened to fp32 in registers.  Kept as its own kernel so that the fp32
-// sweep's code generation is not disturbed.
+// neurons -- with these differences: the weights are fp16 already, so the head image is a plain
+// re-layout with ONE part (half the MMAs, 2 bytes per weight, no scale); the tail gathers
+// 16-byte pieces (eight fp16 neurons per lane, a quarter-warp per 128-byte row piece, four rows
+// per load instruction, three id rows = twelve loads in flight per lane) and adds each weight to
+// its fp32 sum with the mixed-precision add of sm_100; the head sums leave tensor memory through
+// a per-warp transposing buffer in shared memory; and the control warpgroup hands registers to
+// the tail warpgroups.  Kept as its own kernel so that the fp32 sweep's code generation is not
+// disturbed.
 #include "common.cuh"
 #include "mma_ptx.cuh"
 
@@ -16,23 +19,27 @@
 namespace bmu {
 
 static const int M2_SLAB = 256;
-#ifndef BMU_M2_WSTAGES
-#define BMU_M2_WSTAGES 4
+#ifndef BMU_M2F_WSTAGES
+#define BMU_M2F_WSTAGES 4
 #endif
-#ifndef BMU_M2_XSTAGES
-#define BMU_M2_XSTAGES 3
+#ifndef BMU_M2F_XSTAGES
+#define BMU_M2F_XSTAGES 3
 #endif
-static const int M2_NS = BMU_M2_WSTAGES;             // W ring stages
-static const int M2_NX = BMU_M2_XSTAGES;             // X ring stages
+static const int M2_NS = BMU_M2F_WSTAGES;             // W ring stages
+static const int M2_NX = BMU_M2F_XSTAGES;             // X ring stages
 static const int M2_TAIL_WARPS = 16;
-static const int M2_THREADS = (M2_TAIL_WARPS + 3) * 32;
+static const int M2_THREADS = (M2_TAIL_WARPS + 4) * 32;      // 4 tail warpgroups + 1 control warpgroup
+#ifndef BMU_M2F_ROWS
+#define BMU_M2F_ROWS 3                               // id rows per turn: 4 x ROWS loads in flight per lane
+#endif
 static const int M2_TMEM_COLS = 512;                 // 2 buffers x 2 tiles x 128 documents
+static const int M2_XCH_BYTES = 16 * 64 * 4;         // a tail warp's 16 documents x 64 head sums
 
 static inline size_t m2_smem_bytes(int head, bool top2)
 {
     return (size_t)MMA_DOCS * (head / 8) + (M2_NS + M2_NX) * MMA_STAGE_BYTES +
            (2 * M2_NS + 2 * M2_NX + 6) * 8 + MMA_DOCS * 8 + 16 + 16 * 16 + 2 * 16 * 4 +
-           16 * 8 + (top2 ? 4 * MMA_DOCS * 16 : 0);
+           16 * 8 + (top2 ? 4 * MMA_DOCS * 16 : 0) + (size_t)M2_TAIL_WARPS * M2_XCH_BYTES;
 }
 
 // Half-precision codebook: the weights are fp16 already, so the image is a re-layout (one part,
@@ -50,7 +57,9 @@ head_split2_f16_kernel(const __half *__restrict__ W16, int64_t M, int head,
         const int64_t row = feat ? (int64_t)feat[kcg * 8 + e] : (int64_t)(kcg * 8 + e);
         h[e] = col[row * M];
     }
-    const int c = jin & 1, r = ((jin >> 6) << 5) | (((jin >> 1) & 1) << 4) | ((jin >> 2) & 15);
+    // accumulator row 32q + 8s + i of tile c holds neuron 64q + 32 (s / 2) + 4i + 2 (s % 2) + c of
+    // the slab, so that the 16 lanes of a half-warp hold 32 consecutive neurons
+    const int c = jin & 1, r = ((jin >> 6) << 5) | (((jin >> 5) & 1) << 4) | (((jin >> 1) & 1) << 3) | ((jin >> 2) & 7);
     const int kb = kcg >> 3, kc = kcg & 7;
     const size_t off = (size_t)(r >> 3) * 1024 + (size_t)kc * 128 + (size_t)(r & 7) * 16;
     const size_t st = (size_t)sl * SPS + (size_t)(kb * 2 + c);
@@ -70,34 +79,31 @@ int launch_head_split2_f16(const void *W16, int64_t M, int64_t m_full, int head,
 
 // fp32 sum + fp16 term in one instruction (mixed-precision add of sm_100: the widening is exact,
 // so the result is the one a convert followed by an fp32 add gives)
-__device__ __forceinline__ uint32_t m2_addh(uint32_t c, uint16_t h)
+__device__ __forceinline__ float m2_addh(float c, uint16_t h)
 {
     float d;
-    asm("add.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(__uint_as_float(c)));
-    return __float_as_uint(d);
+    asm("add.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(c));
+    return d;
 }
 
-// two fp16 pairs (8 bytes of a half-precision row) added to four fp32 sums
-__device__ __forceinline__ void m2_add_h4(u64 &a0, u64 &a1, u64 raw)
+// eight fp16 weights (16 bytes of a half-precision row) added to eight fp32 sums
+__device__ __forceinline__ void m2_add_h8(float (&s)[8], const uint4 w)
 {
-#ifdef BMU_F16_CONVERT_ADD
-    const uint32_t lo = (uint32_t)raw, hi = (uint32_t)(raw >> 32);
-    const float2 f0 = __half22float2(*reinterpret_cast<const __half2 *>(&lo));
-    const float2 f1 = __half22float2(*reinterpret_cast<const __half2 *>(&hi));
-    add2(a0, ((u64)__float_as_uint(f0.y) << 32) | __float_as_uint(f0.x));
-    add2(a1, ((u64)__float_as_uint(f1.y) << 32) | __float_as_uint(f1.x));
-#else
-    uint16_t h0, h1, h2, h3;
-    asm("mov.b64 {%0, %1, %2, %3}, %4;" : "=h"(h0), "=h"(h1), "=h"(h2), "=h"(h3) : "l"(raw));
-    a0 = ((u64)m2_addh((uint32_t)(a0 >> 32), h1) << 32) | m2_addh((uint32_t)a0, h0);
-    a1 = ((u64)m2_addh((uint32_t)(a1 >> 32), h3) << 32) | m2_addh((uint32_t)a1, h2);
-#endif
+    const uint32_t p[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint16_t h0, h1;
+        asm("mov.b32 {%0, %1}, %2;" : "=h"(h0), "=h"(h1) : "r"(p[i]));
+        s[2 * i] = m2_addh(s[2 * i], h0);
+        s[2 * i + 1] = m2_addh(s[2 * i + 1], h1);
+    }
 }
 
-__device__ __forceinline__ void m2_unpack(const uint4 q, uint32_t f[8])
+// the four ids of a lane's documents: the low or the high half of a row of eight
+__device__ __forceinline__ void m2_ids4(const uint4 q, bool upper, uint32_t f[4])
 {
-    f[0] = q.x & 0xffffu; f[1] = q.x >> 16; f[2] = q.y & 0xffffu; f[3] = q.y >> 16;
-    f[4] = q.z & 0xffffu; f[5] = q.z >> 16; f[6] = q.w & 0xffffu; f[7] = q.w >> 16;
+    const uint32_t a = upper ? q.z : q.x, b = upper ? q.w : q.y;
+    f[0] = a & 0xffffu; f[1] = a >> 16; f[2] = b & 0xffffu; f[3] = b >> 16;
 }
 
 // TOP2: also the second-best unit (Table 5: the paper's kernel tracks it for topographic error).
@@ -125,6 +131,7 @@ sweep_mma2_f16_kernel(const MmaArgs a)
     // document is the same in every slab, so it merges without atomics
     uint2 *lut = reinterpret_cast<uint2 *>(s_off + 16);          // 4 mask bits -> 4 fp16 zeros and ones
     u64 *kq = reinterpret_cast<u64 *>(lut + 16);
+    float *xch0 = reinterpret_cast<float *>(kq + (TOP2 ? 4 * MMA_DOCS * 2 : 0));   // per tail warp
     const uint32_t wfull0 = mm_smem(bars), wempty0 = mm_smem(bars + NS);
     const uint32_t xfull0 = mm_smem(bars + 2 * NS), xempty0 = mm_smem(bars + 2 * NS + NX);
     const uint32_t tfull0 = mm_smem(bars + 2 * NS + 2 * NX), tempty0 = tfull0 + 16;
@@ -182,6 +189,12 @@ sweep_mma2_f16_kernel(const MmaArgs a)
     mm_fence_after();
     const uint32_t tmem = *tmem_slot;
 
+    // The control warpgroup (producer, expander, MMA issuer and one idle warp) hands registers
+    // to the four tail warpgroups, whose loads in flight are bounded by their registers.  The
+    // block is launched with 96 per thread (640 x 96 = 61440); 128 x 56 + 512 x 104 = 60416 fits,
+    // so the increase below never waits for registers that nobody releases.
+    if (warp >= NTW) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (warp == NTW) {
         // ---------------- producer: W stages of every slab, in order
         if (lane == 0) {
@@ -269,15 +282,17 @@ sweep_mma2_f16_kernel(const MmaArgs a)
                 if (mm_bar_try(drain, 0)) break;
         }
         __syncwarp();
+    }   // (the fourth warp only completes the control warpgroup)
     } else {
-        // ---------------- tail: 16 documents x 64 neurons per task.  Lane (h, i) = (lane / 16,
-        // lane % 16) gathers neurons 4i .. 4i+3 for the documents 8h .. 8h+7 of the task: one
-        // 128-bit load per lane and row, two rows (one per half-warp) per instruction.
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 104;");
+        // ---------------- tail: 16 documents x 64 neurons per task.  Lane (s, i) = (lane / 8,
+        // lane % 8) gathers neurons 8i .. 8i+7 for the documents 4s .. 4s+3 of the task: one
+        // 128-bit load per lane and row, four rows (one per quarter-warp) per instruction.
         const int q = warp & 3, g = warp >> 2;
-        const int li = lane & 15, lh = lane >> 4;
-        const float inv_s = 1.f;                                 // the image is unscaled
+        const int li = lane & 7, ls = lane >> 3;
         const uint32_t rowbytes = (uint32_t)(a.M * 2);
-        const int mydoc = 8 * lh + ((lane & 1) << 2 | (lane & 2) | ((lane >> 2) & 1));
+        const int mydoc = 4 * ls + (((lane & 1) << 1) | ((lane >> 1) & 1));
+        float *xch = xch0 + (size_t)warp * (M2_XCH_BYTES / 4);
         for (int sl = 0; sl < n_slabs; ++sl) {
             const int buf = sl & 1;
             const int j0 = a.j_lo + sl * M2_SLAB + q * 64;
@@ -285,52 +300,57 @@ sweep_mma2_f16_kernel(const MmaArgs a)
                 const int dg = g + 4 * it;                       // the block's dg-th set of 16
                 const int64_t tile_a = group * (MMA_DOCS / 8) + 2 * dg, tile_b = tile_a + 1;
                 const bool live = tile_a < a.n_tiles;
-                u64 acc[8][2];
+                float acc[4][8];
 #pragma unroll
-                for (int t = 0; t < 8; ++t) acc[t][0] = acc[t][1] = 0ull;
+                for (int t = 0; t < 4; ++t)
+#pragma unroll
+                    for (int n = 0; n < 8; ++n) acc[t][n] = 0.f;
                 if (live) {
                     const bool has_b = tile_b < a.n_tiles;
                     const uint32_t tla = s_len[2 * dg], tlb = s_len[2 * dg + 1];
                     const uint32_t full = min(tla >> 16, tlb >> 16);
                     const uint32_t rows = max(tla & 0xffffu, tlb & 0xffffu);
-                    const uint32_t my_rows = (lh ? tlb : tla) & 0xffffu;
-                    const int mine = 2 * dg + ((lh && has_b) ? 1 : 0);
+                    const uint32_t my_rows = ((ls >> 1) ? tlb : tla) & 0xffffu;
+                    const int mine = 2 * dg + (((ls >> 1) && has_b) ? 1 : 0);
+                    const bool upper = ls & 1;
                     const uint4 *gp = a.tile_ids + s_off[mine];
-                    const char *base = reinterpret_cast<const char *>(a.W) +
-                                       (size_t)(j0 + li * 4) * 2;
+                    const char *base = reinterpret_cast<const char *>(a.W) + (size_t)(j0 + li * 8) * 2;
                     uint32_t b = 0;
                     uint4 qn = s_first[mine];
-                    // 8-byte pieces: two rows of ids per turn keep sixteen loads in flight
-                    for (; b + 1 < full; b += 2) {
-                        uint32_t f[16];
-                        m2_unpack(qn, f);
-                        m2_unpack(__ldcs(gp + b + 1), f + 8);
-                        qn = __ldcs(gp + b + 2);
-                        u64 w[16];
+                    // ROWS rows of ids per turn keep 4 x ROWS 16-byte loads in flight per lane
+                    constexpr int ROWS = BMU_M2F_ROWS;
+                    for (; b + ROWS - 1 < full; b += ROWS) {
+                        uint32_t f[4 * ROWS];
+                        m2_ids4(qn, upper, f);
 #pragma unroll
-                        for (int t = 0; t < 16; ++t)
-                            w[t] = __ldg(reinterpret_cast<const u64 *>(base + (u64)f[t] * rowbytes));
+                        for (int r = 1; r < ROWS; ++r) m2_ids4(__ldcs(gp + b + r), upper, f + 4 * r);
+                        qn = __ldcs(gp + b + ROWS);
+                        uint4 w[4 * ROWS];
 #pragma unroll
-                        for (int t = 0; t < 16; ++t) m2_add_h4(acc[t & 7][0], acc[t & 7][1], w[t]);
+                        for (int t = 0; t < 4 * ROWS; ++t)
+                            w[t] = __ldg(reinterpret_cast<const uint4 *>(base + (u64)f[t] * rowbytes));
+#pragma unroll
+                        for (int t = 0; t < 4 * ROWS; ++t) m2_add_h8(acc[t & 3], w[t]);
                     }
-                    for (; b < rows; ++b) {
-                        uint32_t f[8];
-                        m2_unpack(qn, f);
+                    for (; b < rows; ++b) {                      // left-over rows, then documents that ran out
+                        uint32_t f[4];
+                        m2_ids4(qn, upper, f);
                         qn = __ldcs(gp + b + 1);
                         const bool in = b < my_rows;
-                        u64 w[8];
+                        uint4 w[4];
 #pragma unroll
-                        for (int t = 0; t < 8; ++t)
+                        for (int t = 0; t < 4; ++t)
                             w[t] = (in && f[t] != 0xffffu)
-                                       ? __ldg(reinterpret_cast<const u64 *>(base + (u64)f[t] * rowbytes)) : 0ull;
+                                       ? __ldg(reinterpret_cast<const uint4 *>(base + (u64)f[t] * rowbytes))
+                                       : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-                        for (int t = 0; t < 8; ++t) m2_add_h4(acc[t][0], acc[t][1], w[t]);
+                        for (int t = 0; t < 4; ++t) m2_add_h8(acc[t], w[t]);
                     }
                 }
                 // head sums of these documents: the MMAs of this slab ran during the gather.
-                // Tensor-memory lane 32q + lane holds neurons 4i + 2h, 4i + 2h + 1 for all 16
-                // documents; lanes l and l ^ 16 swap halves so that each ends up with four
-                // neurons of its own eight documents.
+                // Tensor-memory lane 32q + lane holds neurons 32 (s / 2) + 4i + 2 (s % 2) + {0, 1}
+                // for all 16 documents; the warp's buffer turns that into eight neurons of
+                // four documents per lane.
 #ifndef M2_DEBUG_NOWAIT
                 if (it == 0) mm_wait(tfull0 + 8 * buf, (sl >> 1) & 1, abort_flag, a.status, 8u);
 #endif
@@ -346,37 +366,39 @@ sweep_mma2_f16_kernel(const MmaArgs a)
                     if (lane == 0) mm_bar_arrive(tempty0 + 8 * buf);
                 }
                 if (!live) continue;
+                __syncwarp();                                    // the buffer's last readers are done
 #pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    const uint32_t mine0 = lh ? h0[8 + t] : h0[t], mine1 = lh ? h1[8 + t] : h1[t];
-                    const uint32_t send0 = lh ? h0[t] : h0[8 + t], send1 = lh ? h1[t] : h1[8 + t];
-                    const uint32_t got0 = __shfl_xor_sync(0xffffffffu, send0, 16);
-                    const uint32_t got1 = __shfl_xor_sync(0xffffffffu, send1, 16);
-                    const float s0 = __uint_as_float(lh ? got0 : mine0) * inv_s;
-                    const float s1 = __uint_as_float(lh ? got1 : mine1) * inv_s;
-                    const float s2 = __uint_as_float(lh ? mine0 : got0) * inv_s;
-                    const float s3 = __uint_as_float(lh ? mine1 : got1) * inv_s;
-                    add2(acc[t][0], ((u64)__float_as_uint(s1) << 32) | __float_as_uint(s0));
-                    add2(acc[t][1], ((u64)__float_as_uint(s3) << 32) | __float_as_uint(s2));
+                for (int d = 0; d < 16; ++d)                     // 128 contiguous bytes per half-warp
+                    *reinterpret_cast<uint2 *>(xch + d * 64 + 32 * (ls >> 1) + 4 * li + 2 * (ls & 1)) =
+                        make_uint2(h0[d], h1[d]);
+                __syncwarp();
+                const int sw = li >> 2;                          // lanes 4..7 of a quarter read the
+#pragma unroll                                                   // upper half first: no bank conflict
+                for (int t = 0; t < 4; ++t) {
+                    const float4 *r = reinterpret_cast<const float4 *>(xch + (4 * ls + t) * 64 + 8 * li);
+                    const float4 u = r[sw], v = r[sw ^ 1];
+                    const float4 lo = sw ? v : u, hi = sw ? u : v;
+                    acc[t][0] += lo.x; acc[t][1] += lo.y; acc[t][2] += lo.z; acc[t][3] += lo.w;
+                    acc[t][4] += hi.x; acc[t][5] += hi.y; acc[t][6] += hi.z; acc[t][7] += hi.w;
                 }
-                const int col = j0 + li * 4;
-                const float4 n = __ldg(reinterpret_cast<const float4 *>(a.norms + col));
-                const float n4[4] = {n.x, n.y, n.z, n.w};
-                u64 k[8], k2[8];
+                const int col = j0 + li * 8;
+                const float4 na = __ldg(reinterpret_cast<const float4 *>(a.norms + col));
+                const float4 nb = __ldg(reinterpret_cast<const float4 *>(a.norms + col + 4));
+                const float n8[8] = {na.x, na.y, na.z, na.w, nb.x, nb.y, nb.z, nb.w};
+                u64 k[4], k2[4];
 #pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    const float s4[4] = {lo_f(acc[t][0]), hi_f(acc[t][0]), lo_f(acc[t][1]), hi_f(acc[t][1])};
+                for (int t = 0; t < 4; ++t) {
                     Best<TOP2> bst;
                     bst.init();
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) bst.push(fmaf(-2.f, s4[c], n4[c]), col + c);
+                    for (int c = 0; c < 8; ++c) bst.push(fmaf(-2.f, acc[t][c], n8[c]), col + c);
                     k[t] = make_key(bst.d1, bst.j1);
                     k2[t] = TOP2 ? make_key(bst.d2, bst.j2) : KEY_WORST;
                 }
-                // transposing butterfly among the 16 lanes that hold the same documents
+                // transposing butterfly among the 8 lanes that hold the same documents
 #pragma unroll
-                for (int st = 0; st < 3; ++st) {
-                    const int m = 1 << st, cnt = 4 >> st;
+                for (int st = 0; st < 2; ++st) {
+                    const int m = 1 << st, cnt = 2 >> st;
 #pragma unroll
                     for (int i = 0; i < cnt; ++i) {
                         const u64 send = (lane & m) ? k[i] : k[i + cnt];
@@ -395,11 +417,11 @@ sweep_mma2_f16_kernel(const MmaArgs a)
                         }
                     }
                 }
-                const u64 got = __shfl_xor_sync(0xffffffffu, k[0], 8);
+                const u64 got = __shfl_xor_sync(0xffffffffu, k[0], 4);
                 if (TOP2) {
-                    const u64 got2 = __shfl_xor_sync(0xffffffffu, k2[0], 8);
+                    const u64 got2 = __shfl_xor_sync(0xffffffffu, k2[0], 4);
                     Best<true>::merge(k[0], k2[0], got, got2);
-                    if ((lane & 8) == 0) {
+                    if ((lane & 4) == 0) {
                         u64 *slot = kq + ((size_t)q * MMA_DOCS + dg * 16 + mydoc) * 2;
                         Best<true>::merge(k[0], k2[0], slot[0], slot[1]);
                         slot[0] = k[0];
@@ -407,7 +429,7 @@ sweep_mma2_f16_kernel(const MmaArgs a)
                     }
                 } else {
                     k[0] = got < k[0] ? got : k[0];
-                    if ((lane & 8) == 0)
+                    if ((lane & 4) == 0)
                         atomicMin(reinterpret_cast<unsigned long long *>(keys + dg * 16 + mydoc), k[0]);
                 }
             }
