@@ -456,12 +456,40 @@ def run_ours(args, cfg, rank, local_rank, world):
         del plan
     if args.comparator:
         line["comparator"] = comparator_spmm(cfg, W, norms, rowptr, colidx)
+    if args.f16 and len(batches) == 1:
+        line["f16_codebook"] = f16_codebook(bmu, cfg, W, rowptr, colidx, args)
     if args.epoch:
         line["epoch"] = epoch_phases(bmu, cfg, W, batches, opts, ws, norms, out_bmu, out_dist,
                                      peaks, args.sigma)
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(cfg, W, rowptr, colidx, rowptr.numel() - 1)
     return line
+
+
+def f16_codebook(bmu, cfg, W, rowptr, colidx, args):
+    """The same sweep with the paper's own storage (Section 4.2: two bytes per half-precision
+    weight): the codebook rounded to fp16 once, sums and distances still fp32.  Context beside
+    the fp32 headline, not a substitute for it: the rounding changes the weights."""
+    W16 = W.half()
+    n16 = bmu.bmu_codebook_norms_f16(W16)
+    n0, nnz = rowptr.numel() - 1, colidx.numel()
+    D, M = W16.shape
+    need = int(bmu.load().bmu_search_f16_workspace_bytes(D, M, n0, nnz, None))
+    ws = torch.empty(need + 256, dtype=torch.uint8, device=W.device)
+    for _ in range(max(1, args.warmup)):
+        bmu.bmu_search_f16_ws(W16, rowptr, colidx, norms=n16, workspace=ws)
+    torch.cuda.synchronize(W.device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        bmu.bmu_codebook_norms_f16(W16)
+        bmu.bmu_search_f16_ws(W16, rowptr, colidx, norms=n16, workspace=ws)
+    e1.record()
+    torch.cuda.synchronize(W.device)
+    ms = e0.elapsed_time(e1) / args.steps
+    return {"ms_per_step": ms, "value": n0 / (ms * 1e-3), "unit": UNIT,
+            "updates_per_s": nnz * float(M) / (ms * 1e-3), "dtype": "f16 storage, f32 sums",
+            "api": "bmu_codebook_norms_f16 + bmu_search_f16_ws per step (rank 0's figure)"}
 
 
 def comparator_spmm(cfg, W, norms, rowptr, colidx, budget_docs=200_000):
@@ -566,6 +594,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--comparator", action="store_true",
                     help="also time the materialised-score route (library SpMM + argmin)")
+    ap.add_argument("--f16", action="store_true",
+                    help="also time the same sweep on the codebook rounded to fp16 (the paper's storage)")
     ap.add_argument("--epoch", action="store_true",
                     help="also time one whole epoch (search + scatter + blur + write-back)")
     ap.add_argument("--sigma", type=float, default=2.0, help="neighbourhood width of --epoch")
