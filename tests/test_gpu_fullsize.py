@@ -62,6 +62,34 @@ def test_cfg4_full_size_sampled(bmu):
     check_sample(W, rowptr, colidx, ob, od, 256, seed=4)
 
 
+def test_cfg3_full_size_sampled(bmu):
+    cfg = synth.CONFIGS["cfg3"]
+    dev = torch.device("cuda")
+    W = synth.make_codebook(cfg.D, cfg.M, synth.codebook_seed(cfg), device=dev)
+    rowptr, colidx = synth.make_corpus(cfg, device=dev)
+    assert rowptr.numel() - 1 == cfg.N
+    norms = bmu.bmu_codebook_norms(W)
+    ob, od = bmu.bmu_search_ws(W, rowptr, colidx, norms=norms)
+    torch.cuda.synchronize()
+    check_properties(W, norms, rowptr, colidx, ob, od, cfg.M)
+    check_sample(W, rowptr, colidx, ob, od, 2000, seed=3)
+
+
+def test_cfg3_full_size_half_precision_codebook_sampled(bmu):
+    """The paper's storage at full size: the codebook rounded to fp16 once; the oracle reads the
+    same rounded weights widened to fp32, so the rule and its tolerance are unchanged."""
+    cfg = synth.CONFIGS["cfg3"]
+    dev = torch.device("cuda")
+    W16 = synth.make_codebook(cfg.D, cfg.M, synth.codebook_seed(cfg), device=dev).half()
+    Ww = W16.float()
+    rowptr, colidx = synth.make_corpus(cfg, device=dev)
+    n16 = bmu.bmu_codebook_norms_f16(W16)
+    ob, od = bmu.bmu_search_f16_ws(W16, rowptr, colidx, norms=n16)   # the wide tensor-core sweep
+    torch.cuda.synchronize()
+    check_properties(Ww, n16, rowptr, colidx, ob, od, cfg.M)
+    check_sample(Ww, rowptr, colidx, ob, od, 2000, seed=33)
+
+
 def test_cfg5_one_streamed_batch_sampled(bmu):
     cfg = synth.CONFIGS["cfg5"]
     dev = torch.device("cuda")
