@@ -50,6 +50,9 @@ def _load():
         lib.oracle_blur_plane.restype = None
         lib.oracle_writeback.argtypes = [vp, vp, i64, i64, vp]
         lib.oracle_writeback.restype = None
+        lib.oracle_map_errors.argtypes = [vp, vp, vp, i64, ctypes.c_int32, ctypes.c_int32,
+                                          ctypes.c_int32, vp]
+        lib.oracle_map_errors.restype = None
         lib.oracle_max_threads.argtypes = []
         lib.oracle_max_threads.restype = ci
         _lib = lib
@@ -154,4 +157,17 @@ def writeback(B, c, W) -> np.ndarray:
     out = _f32(W).copy()
     D, M = out.shape
     _load().oracle_writeback(_p(B), _p(c), D, M, _p(out))
+    return out
+
+
+def map_errors(bmu, bmu2, dist, edge_x: int, edge_y: int, adjacency: int = 4) -> np.ndarray:
+    """(mean squared quantisation error, mean quantisation error, topographic error) of a
+    search with second-best units on an edge_y x edge_x map."""
+    b1 = np.ascontiguousarray(bmu, dtype=np.int32)
+    b2 = np.ascontiguousarray(bmu2, dtype=np.int32)
+    d = _f32(dist)
+    if adjacency not in (4, 8):
+        raise ValueError("adjacency must be 4 or 8")
+    out = np.zeros(3, dtype=np.float64)
+    _load().oracle_map_errors(_p(b1), _p(b2), _p(d), b1.size, edge_x, edge_y, adjacency, _p(out))
     return out

@@ -206,3 +206,47 @@ void oracle_writeback(const double *B, const double *c, int64_t D, int64_t M, fl
             if (c[j] > 0.0)
                 W[f * M + j] = (float)(B[f * M + j] / c[j]);
 }
+
+/* ------------------------------------------------------------------------
+ * Stopping metrics of an epoch (Table 4 column "stopping metric"; Section 5: the
+ * second-best unit "feeds topographic error", which the stopping rules gate on
+ * together with the quantisation error).  The paper names the two measures and
+ * prints no formula; these are their textbook definitions over the outputs of a
+ * search with second-best units, on the map of edge_y rows by edge_x columns
+ * (neuron j = y * edge_x + x):
+ *
+ *   out[0]  mean of d_i                  (mean squared quantisation error: d is the
+ *                                         squared distance to the best unit)
+ *   out[1]  mean of sqrt(max(d_i, 0))    (quantisation error; a d_i rounded below
+ *                                         zero counts as zero)
+ *   out[2]  fraction of documents whose best and second-best units are not
+ *           neighbours on the map (topographic error): neighbours share an edge
+ *           (adjacency == 4: |dx| + |dy| == 1) or an edge or a corner (adjacency
+ *           == 8: max(|dx|, |dy|) == 1); a document without a second unit
+ *           (bmu2 < 0, a one-neuron map) is not an error.
+ *
+ * N == 0 gives zeros.  Parity status: pinned by hand-computed cases and
+ * invariants (tests/test_oracle_pins_update.py); against the paper "parity
+ * unpinned" (no formula, no value printed).
+ */
+void oracle_map_errors(const int32_t *bmu, const int32_t *bmu2, const float *dist, int64_t N,
+                       int32_t edge_x, int32_t edge_y, int32_t adjacency, double *out)
+{
+    double sum_d = 0.0, sum_r = 0.0;
+    int64_t errors = 0;
+    (void)edge_y;
+    for (int64_t i = 0; i < N; ++i) {
+        const double d = (double)dist[i];
+        sum_d += d;
+        sum_r += d > 0.0 ? sqrt(d) : 0.0;
+        if (bmu2[i] < 0) continue;
+        const int32_t x1 = bmu[i] % edge_x, y1 = bmu[i] / edge_x;
+        const int32_t x2 = bmu2[i] % edge_x, y2 = bmu2[i] / edge_x;
+        const int32_t dx = x1 > x2 ? x1 - x2 : x2 - x1, dy = y1 > y2 ? y1 - y2 : y2 - y1;
+        const int near = adjacency == 8 ? ((dx > dy ? dx : dy) == 1) : (dx + dy == 1);
+        if (!near) ++errors;
+    }
+    out[0] = N ? sum_d / (double)N : 0.0;
+    out[1] = N ? sum_r / (double)N : 0.0;
+    out[2] = N ? (double)errors / (double)N : 0.0;
+}

@@ -173,3 +173,55 @@ def test_identical_documents_pull_their_unit_onto_the_document():
     want = np.zeros(8, np.float32)
     want[[1, 4, 6]] = 1.0
     assert np.array_equal(W1[:, 2], want) and np.all(W1[:, [0, 1, 3]] == 0.5)
+
+
+# ------------------------------------------------------------------ stopping metrics
+def test_map_errors_hand_computed_case():
+    # a 4-column, 3-row map: unit j sits at (x, y) = (j % 4, j // 4)
+    #   0  1  2  3
+    #   4  5  6  7
+    #   8  9 10 11
+    bmu = np.array([5, 5, 5, 0, 11, 3], np.int32)
+    bmu2 = np.array([6, 10, 7, 4, 7, 4], np.int32)
+    #  5-6 share an edge; 5-10 share a corner; 5-7 are two apart; 0-4 share an edge (a row
+    #  apart, not neighbours by index); 11-7 share an edge; 3-4 are index neighbours but sit at
+    #  opposite ends of two rows
+    dist = np.array([4.0, 9.0, 0.25, 16.0, 1.0, 0.0], np.float32)
+    e4 = oracle.map_errors(bmu, bmu2, dist, 4, 3, adjacency=4)
+    e8 = oracle.map_errors(bmu, bmu2, dist, 4, 3, adjacency=8)
+    assert e4[0] == pytest.approx(30.25 / 6, rel=1e-15)            # mean of d
+    assert e4[1] == pytest.approx((2 + 3 + 0.5 + 4 + 1 + 0) / 6, rel=1e-15)   # mean of sqrt(d)
+    assert e4[2] == pytest.approx(3 / 6, rel=1e-15)                # 5-10, 5-7, 3-4
+    assert e8[2] == pytest.approx(2 / 6, rel=1e-15)                # 5-7, 3-4
+    assert np.array_equal(e4[:2], e8[:2])
+
+
+def test_map_errors_edge_cases_and_invariants():
+    assert np.array_equal(oracle.map_errors([], [], [], 5, 5), np.zeros(3))
+    # a distance rounded below zero counts as zero in the root, as itself in the mean
+    e = oracle.map_errors([0, 1], [1, 0], np.array([-1e-6, 4.0], np.float32), 2, 1)
+    assert e[0] == pytest.approx((float(np.float32(-1e-6)) + 4.0) / 2, rel=1e-12) and e[1] == 1.0 and e[2] == 0.0
+    # no second unit (one-neuron map): not an error
+    assert oracle.map_errors([0, 0], [-1, -1], [1.0, 1.0], 1, 1)[2] == 0.0
+    # a non-square map: x runs along a row of edge_x units
+    assert oracle.map_errors([0], [7], [0.0], 7, 2)[2] == 0.0      # (0,0)-(0,1): an edge
+    assert oracle.map_errors([0], [7], [0.0], 2, 7)[2] == 1.0      # (0,0)-(1,3)
+    r = np.random.default_rng(17)
+    ex, ey, N = 9, 6, 4000
+    b1 = r.integers(0, ex * ey, N).astype(np.int32)
+    b2 = r.integers(0, ex * ey, N).astype(np.int32)
+    d = (r.random(N) * 50).astype(np.float32)
+    e4, e8 = oracle.map_errors(b1, b2, d, ex, ey, 4), oracle.map_errors(b1, b2, d, ex, ey, 8)
+    assert e8[2] <= e4[2]                                          # corners only ever help
+    # the definition written with array operations
+    dx, dy = np.abs(b1 % ex - b2 % ex), np.abs(b1 // ex - b2 // ex)
+    assert e4[2] == pytest.approx(np.mean(dx + dy != 1), rel=1e-15)
+    assert e8[2] == pytest.approx(np.mean(np.maximum(dx, dy) != 1), rel=1e-15)
+    assert e4[0] == pytest.approx(d.astype(np.float64).mean(), rel=1e-12)
+    assert e4[1] == pytest.approx(np.sqrt(d.astype(np.float64)).mean(), rel=1e-12)
+    # swapping best and second-best changes no adjacency; permuting documents changes nothing
+    assert oracle.map_errors(b2, b1, d, ex, ey, 4)[2] == e4[2]
+    p = r.permutation(N)
+    np.testing.assert_allclose(oracle.map_errors(b1[p], b2[p], d[p], ex, ey, 4), e4, rtol=1e-12)
+    # by Jensen the mean root is at most the root of the mean
+    assert e4[1] <= np.sqrt(e4[0])
