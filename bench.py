@@ -533,7 +533,8 @@ def comparator_spmm(cfg, W, norms, rowptr, colidx, budget_docs=200_000):
 
 
 def epoch_phases(bmu, cfg, W, batches, opts, ws, norms, out_bmu, out_dist, peaks, sigma):
-    """One whole batch epoch (Table 4 of the paper: norms, search, scatter, blur, write-back),
+    """One whole batch epoch (Table 4 of the paper: norms, search, stopping metric on held-out
+    documents, scatter, blur, write-back),
     timed phase by phase with CUDA events; HBM-bound phases against the measured copy roof.
     The codebook is overwritten by the update (random data either way)."""
     dev = W.device
@@ -542,8 +543,14 @@ def epoch_phases(bmu, cfg, W, batches, opts, ws, norms, out_bmu, out_dist, peaks
     cnt = torch.zeros(M, dtype=torch.int32, device=dev)
     nnz = sum(ci.numel() for _, ci in batches)
     n_docs = sum(rp.numel() - 1 for rp, _ in batches)
-    names = ["norms", "search", "scatter", "blur", "writeback"]
+    names = ["norms", "search", "stopping_metric", "scatter", "blur", "writeback"]
     acc = {k: 0.0 for k in names}
+    # held-out documents for the stopping metrics: a tenth of the corpus (the paper trains on
+    # 90 % and holds 10 % out, Section 5), drawn as a batch of its own
+    n_held = max(1, n_docs // 9)
+    held_rp, held_ci = synth.make_corpus(cfg, n_docs=min(n_held, synth.batch_size(cfg)),
+                                         seed=synth.corpus_seed(cfg, 40), device=dev)
+    quality = None
 
     def timed(name, fn):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -560,6 +567,11 @@ def epoch_phases(bmu, cfg, W, batches, opts, ws, norms, out_bmu, out_dist, peaks
         num.zero_()
         cnt.zero_()
         timed("norms", lambda: bmu.bmu_codebook_norms(W, norms))
+
+        def stopping_metric():
+            b1, d1, b2, _ = bmu.bmu_search_top2_ws(W, held_rp, held_ci, norms=norms, opts=opts)
+            return bmu.bmu_map_errors(b1, b2, d1, cfg.edge, cfg.edge, 4)
+        quality = timed("stopping_metric", stopping_metric)
         for rp_b, ci_b in batches:
             nb = rp_b.numel() - 1
             timed("search", lambda: bmu.bmu_search_ws(W, rp_b, ci_b, norms=norms, opts=opts,
@@ -574,8 +586,12 @@ def epoch_phases(bmu, cfg, W, batches, opts, ws, norms, out_bmu, out_dist, peaks
     plane = 4.0 * D * M
     alg = {"scatter": 12.0 * nnz + 12.0 * n_docs,      # id + counter read-modify-write per listing
            "blur": 2.0 * plane, "writeback": 3.0 * plane, "norms": plane}
+    q = quality.cpu().tolist()
     return {"sigma": sigma, "phases_ms": dict(acc), "total_ms": total,
             "search_share": acc["search"] / total,
+            "held_out_docs": held_rp.numel() - 1,
+            "held_out_quality": {"mean_sq_quantisation_error": q[0], "quantisation_error": q[1],
+                                 "topographic_error_4": q[2]},
             "hbm_frac": {k: alg[k] / (acc[k] * 1e-3) / hbm for k in alg if acc[k] > 0},
             "note": "paper (RTX 4090, Table 4): search 73.7-94.0 % of the epoch"}
 

@@ -352,6 +352,29 @@ BMU_API int bmu_update_writeback(const float *num_blur, const float *cnt_blur, i
                                  float *W, void *stream);
 
 /*
+ * Stopping metrics of an epoch (Table 4 column "stopping metric"; Section 5: the
+ * second-best unit feeds the topographic error, which the stopping rules gate on
+ * together with the quantisation error).  The paper names the measures and
+ * prints no formula; these are the textbook definitions over the outputs of
+ * bmu_search_top2_ws for a batch of (held-out) documents, on the map of edge_y
+ * rows by edge_x columns (neuron j = y * edge_x + x):
+ *   out[0] = mean of dist[i]               (mean squared quantisation error)
+ *   out[1] = mean of sqrt(max(dist[i], 0)) (quantisation error)
+ *   out[2] = fraction of documents whose bmu[i] and bmu2[i] are not neighbours
+ *            (topographic error): adjacency 4 = the units share an edge, 8 = an
+ *            edge or a corner; bmu2[i] < 0 (one-neuron map) is not an error.
+ * bmu, bmu2 int32[N], dist fp32[N], out double[3]: device memory.  Sums are
+ * fp64 in a fixed order (same bits on every call).  N == 0 gives zeros.
+ * workspace: bmu_map_errors_workspace_bytes() bytes of device memory, 256-byte
+ * aligned, contents irrelevant.  Asynchronous on `stream`; BMU_ERR_INVALID_ARG for
+ * an adjacency other than 4 or 8, edges < 1 or null pointers.
+ */
+BMU_API size_t bmu_map_errors_workspace_bytes(void);
+BMU_API int bmu_map_errors(const int32_t *bmu, const int32_t *bmu2, const float *dist, int64_t N,
+                           int32_t edge_x, int32_t edge_y, int32_t adjacency, double *out,
+                           void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Measures one on-chip ceiling of the current device with a microbenchmark, so
  * that achieved throughput can be quoted against the roof that binds (the paper
  * quotes its kernel against the L2 roof of its card, Section 6 / Table 3).

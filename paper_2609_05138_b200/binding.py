@@ -108,6 +108,11 @@ EXPORTS = {
                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "bmu_update_writeback": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                             ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]),
+    "bmu_map_errors_workspace_bytes": (ctypes.c_size_t, []),
+    "bmu_map_errors": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                      ctypes.c_int64, ctypes.c_int32, ctypes.c_int32,
+                                      ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                      ctypes.c_size_t, ctypes.c_void_p]),
     "bmu_measure_roof": (ctypes.c_int, [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t,
                                         ctypes.c_int, ctypes.POINTER(ctypes.c_double),
                                         ctypes.c_void_p]),
@@ -439,6 +444,24 @@ def bmu_update_writeback(num_blur, cnt_blur, W):
                                            _dev(cnt_blur, torch.float32, "cnt_blur"), D, M, wp,
                                            _stream(W)))
     return W
+
+
+def bmu_map_errors(bmu, bmu2, dist, edge_x: int, edge_y: int, adjacency: int = 4) -> torch.Tensor:
+    """Device tensor of three float64: mean squared quantisation error, mean quantisation
+    error, topographic error of a search with second-best units."""
+    N = bmu.numel()
+    dev = dist.device
+    out = torch.empty(3, dtype=torch.float64, device=dev)
+    need = int(load().bmu_map_errors_workspace_bytes())
+    ws = torch.empty(need + 256, dtype=torch.uint8, device=dev)
+    ws_ptr = (ws.data_ptr() + 255) // 256 * 256
+    with torch.cuda.device(dev):
+        _check(load().bmu_map_errors(_dev(bmu, torch.int32, "bmu") if N else None,
+                                     _dev(bmu2, torch.int32, "bmu2") if N else None,
+                                     _dev(dist, torch.float32, "dist") if N else None, N,
+                                     int(edge_x), int(edge_y), int(adjacency), out.data_ptr(),
+                                     ws_ptr, need, _stream(dist)))
+    return out
 
 
 ROOFS = {"l2_ldg": 0, "l2_bulk": 1, "smem": 2, "l1": 3, "fadd": 4, "fadd2": 5}

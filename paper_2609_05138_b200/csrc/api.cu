@@ -1017,6 +1017,30 @@ int bmu_update_writeback(const float *num_blur, const float *cnt_blur, int64_t D
     return launch_update_writeback(num_blur, cnt_blur, D, M, W, static_cast<cudaStream_t>(stream));
 }
 
+size_t bmu_map_errors_workspace_bytes(void) { return map_errors_workspace_bytes(); }
+
+int bmu_map_errors(const int32_t *bmu, const int32_t *bmu2, const float *dist, int64_t N,
+                   int32_t edge_x, int32_t edge_y, int32_t adjacency, double *out, void *workspace,
+                   size_t workspace_bytes, void *stream)
+{
+    if (N < 0 || N > MAX_I32 || edge_x < 1 || edge_y < 1 || (adjacency != 4 && adjacency != 8)) {
+        set_error("map errors: need 0 <= N < 2^31, edges >= 1 and adjacency 4 or 8");
+        return BMU_ERR_INVALID_ARG;
+    }
+    if (!out || (N > 0 && (!bmu || !bmu2 || !dist))) {
+        set_error("null pointer argument");
+        return BMU_ERR_INVALID_ARG;
+    }
+    if (N > 0 && (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0 ||
+                  workspace_bytes < map_errors_workspace_bytes())) {
+        set_error("workspace missing, not 256-byte aligned, or smaller than %zu bytes",
+                  map_errors_workspace_bytes());
+        return BMU_ERR_WORKSPACE;
+    }
+    return launch_map_errors(bmu, bmu2, dist, N, edge_x, adjacency, out, workspace,
+                             static_cast<cudaStream_t>(stream));
+}
+
 }  // extern "C"
 
 // ---- search with library-resident scratch (no allocation anywhere) ---------

@@ -277,6 +277,9 @@ int launch_update_scatter(const int32_t *rowptr, const int32_t *colidx, int64_t 
 int launch_update_blur(const uint32_t *num, const uint32_t *cnt, int64_t D, int32_t edge_x,
                        int32_t edge_y, float sigma, float *num_blur, float *cnt_blur,
                        cudaStream_t s);
+size_t map_errors_workspace_bytes();
+int launch_map_errors(const int32_t *bmu, const int32_t *bmu2, const float *dist, int64_t N,
+                      int32_t edge_x, int32_t adjacency, double *out, void *ws, cudaStream_t s);
 int launch_update_writeback(const float *num_blur, const float *cnt_blur, int64_t D, int64_t M,
                             float *W, cudaStream_t s);
 

@@ -143,6 +143,64 @@ update_writeback_kernel(const float *__restrict__ num_blur, const float *__restr
     }
 }
 
+
+// Stopping metrics of an epoch (Table 4 "stopping metric"; Section 5: the second-best unit feeds
+// the topographic error): mean d, mean sqrt(max(d, 0)) and the fraction of documents whose best
+// and second-best units are not neighbours on the map.  fp64 sums in a fixed order (grid-stride
+// partition, shuffle tree, warps in order, blocks in order by the last block to finish), so a
+// call gives the same bits every time.
+static const int ME_BLOCKS = 592, ME_THREADS = 256;
+
+__global__ void __launch_bounds__(ME_THREADS)
+map_errors_kernel(const int32_t *__restrict__ bmu, const int32_t *__restrict__ bmu2,
+                  const float *__restrict__ dist, int64_t N, int32_t edge_x, int32_t adjacency,
+                  double *__restrict__ part, unsigned int *__restrict__ ticket,
+                  double *__restrict__ out)
+{
+    double sd = 0.0, sr = 0.0, er = 0.0;
+    for (int64_t i = (int64_t)blockIdx.x * ME_THREADS + threadIdx.x; i < N;
+         i += (int64_t)ME_BLOCKS * ME_THREADS) {
+        const double d = (double)__ldg(dist + i);
+        sd += d;
+        sr += d > 0.0 ? sqrt(d) : 0.0;
+        const int32_t b2 = __ldg(bmu2 + i);
+        if (b2 >= 0) {
+            const int32_t b1 = __ldg(bmu + i);
+            const int32_t dx = abs(b1 % edge_x - b2 % edge_x), dy = abs(b1 / edge_x - b2 / edge_x);
+            const bool near = adjacency == 8 ? max(dx, dy) == 1 : dx + dy == 1;
+            er += near ? 0.0 : 1.0;
+        }
+    }
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) {
+        sd += __shfl_xor_sync(0xffffffffu, sd, m);
+        sr += __shfl_xor_sync(0xffffffffu, sr, m);
+        er += __shfl_xor_sync(0xffffffffu, er, m);
+    }
+    __shared__ double wsum[3][ME_THREADS / 32];
+    __shared__ bool last;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) { wsum[0][warp] = sd; wsum[1][warp] = sr; wsum[2][warp] = er; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double a = 0.0, b = 0.0, e = 0.0;
+        for (int w = 0; w < ME_THREADS / 32; ++w) { a += wsum[0][w]; b += wsum[1][w]; e += wsum[2][w]; }
+        part[blockIdx.x] = a;
+        part[ME_BLOCKS + blockIdx.x] = b;
+        part[2 * ME_BLOCKS + blockIdx.x] = e;
+        __threadfence();
+        last = atomicAdd(ticket, 1u) == ME_BLOCKS - 1;
+    }
+    __syncthreads();
+    if (last && threadIdx.x < 3) {
+        __threadfence();
+        const volatile double *p = part + threadIdx.x * ME_BLOCKS;
+        double s = 0.0;
+        for (int b = 0; b < ME_BLOCKS; ++b) s += p[b];
+        out[threadIdx.x] = s / (double)N;
+    }
+}
+
 int launch_update_scatter(const int32_t *rowptr, const int32_t *colidx, int64_t N,
                           const int32_t *bmu, int64_t M, uint32_t *num, uint32_t *cnt,
                           cudaStream_t s)
@@ -197,6 +255,24 @@ int launch_update_writeback(const float *num_blur, const float *cnt_blur, int64_
     const dim3 grid((unsigned)((per_row + 255) / 256 < 64 ? (per_row + 255) / 256 : 64), (unsigned)D);
     if (vec) update_writeback_kernel<true><<<grid, 256, 0, s>>>(num_blur, cnt_blur, M, W);
     else update_writeback_kernel<false><<<grid, 256, 0, s>>>(num_blur, cnt_blur, M, W);
+    BMU_CUDA(cudaGetLastError());
+    return BMU_OK;
+}
+
+size_t map_errors_workspace_bytes() { return 256 + (size_t)3 * ME_BLOCKS * sizeof(double); }
+
+int launch_map_errors(const int32_t *bmu, const int32_t *bmu2, const float *dist, int64_t N,
+                      int32_t edge_x, int32_t adjacency, double *out, void *ws, cudaStream_t s)
+{
+    if (N == 0) {
+        BMU_CUDA(cudaMemsetAsync(out, 0, 3 * sizeof(double), s));
+        return BMU_OK;
+    }
+    unsigned int *ticket = static_cast<unsigned int *>(ws);
+    double *part = reinterpret_cast<double *>(static_cast<char *>(ws) + 256);
+    BMU_CUDA(cudaMemsetAsync(ticket, 0, sizeof(unsigned int), s));
+    map_errors_kernel<<<ME_BLOCKS, ME_THREADS, 0, s>>>(bmu, bmu2, dist, N, edge_x, adjacency, part,
+                                                      ticket, out);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

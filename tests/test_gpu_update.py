@@ -125,3 +125,49 @@ def test_whole_epoch_against_oracle_chain(bmu):
     assert np.all(np.abs(got - ref) <= 4e-6 * np.maximum(np.abs(ref), 1e-3))
     assert got.min() >= 0.0 and got.max() <= 1.0 + 1e-6     # weighted means of binary vectors
     np.testing.assert_allclose(nrm.cpu().numpy(), oracle.norms(got), rtol=1e-6)
+
+
+@pytest.mark.parametrize("ex,ey,N", [(16, 16, 100_000), (23, 7, 777), (1, 1, 50), (40, 3, 1)])
+@pytest.mark.parametrize("adjacency", [4, 8])
+def test_map_errors_match_oracle(bmu, ex, ey, N, adjacency):
+    g = torch.Generator().manual_seed(ex * 1000 + N)
+    M = ex * ey
+    b1 = torch.randint(0, M, (N,), generator=g, dtype=torch.int32)
+    # second-best units: neighbours for half of the documents, anything for the rest
+    step = torch.tensor([1, -1, ex, -ex, ex + 1, -ex - 1, 2, 3 * ex])[torch.randint(0, 8, (N,), generator=g)]
+    b2 = torch.where(torch.rand(N, generator=g) < 0.5, (b1 + step) % M,
+                     torch.randint(0, M, (N,), generator=g)).to(torch.int32)
+    if M == 1:
+        b2 = torch.full((N,), -1, dtype=torch.int32)
+    d = (torch.rand(N, generator=g) * 300 - 0.001).float()           # a few just below zero
+    got = bmu.bmu_map_errors(b1.cuda(), b2.cuda(), d.cuda(), ex, ey, adjacency).cpu().numpy()
+    ref = oracle.map_errors(b1.numpy(), b2.numpy(), d.numpy(), ex, ey, adjacency)
+    assert got[2] == ref[2]                                           # a count over N: exact
+    np.testing.assert_allclose(got[:2], ref[:2], rtol=1e-12)          # fp64 sums, another order
+    again = bmu.bmu_map_errors(b1.cuda(), b2.cuda(), d.cuda(), ex, ey, adjacency).cpu().numpy()
+    assert np.array_equal(got, again)                                 # fixed summation order
+
+
+def test_map_errors_empty_and_bad_arguments(bmu):
+    e = torch.empty(0, dtype=torch.int32, device="cuda")
+    out = bmu.bmu_map_errors(e, e, torch.empty(0, device="cuda"), 4, 4)
+    assert out.cpu().tolist() == [0.0, 0.0, 0.0]
+    one = torch.zeros(1, dtype=torch.int32, device="cuda")
+    with pytest.raises(bmu.BmuError):
+        bmu.bmu_map_errors(one, one, torch.zeros(1, device="cuda"), 4, 4, adjacency=6)
+    with pytest.raises(bmu.BmuError):
+        bmu.bmu_map_errors(one, one, torch.zeros(1, device="cuda"), 0, 4)
+
+
+def test_stopping_metrics_of_a_search(bmu):
+    """Search with second-best units on a small map, then the metrics, against the oracle chain."""
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=3000)
+    W = synth.make_codebook(cfg.D, cfg.M, 5) * 0.02                    # the gathered sum decides
+    b1, d1, b2, _ = bmu.bmu_search_top2_ws(W.cuda(), rowptr.cuda(), colidx.cuda())
+    got = bmu.bmu_map_errors(b1, b2, d1, cfg.edge, cfg.edge, 8).cpu().numpy()
+    ob1, od1, ob2, _ = oracle.bmu2(W.numpy(), rowptr.numpy(), colidx.numpy())
+    ref = oracle.map_errors(ob1, ob2, od1.astype(np.float32), cfg.edge, cfg.edge, 8)
+    np.testing.assert_allclose(got[:2], ref[:2], rtol=2e-6)            # fp32 distances vs fp64
+    # the units agree except inside near-ties, so the error fractions differ by a few documents
+    assert abs(got[2] - ref[2]) <= 5 / 3000
