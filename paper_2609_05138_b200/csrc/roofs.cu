@@ -1,5 +1,5 @@
 // Microbenchmarks that measure, on the GPU the library runs on, the on-chip
-// ceilings the gather-accumulate sweep is judged against: L2->SM read
+// ceilings the gather-accumulate sweep is measured against: L2->SM read
 // bandwidth (128-bit loads and bulk copies into shared memory), the
 // L1 / shared-memory -> register bandwidth, and the fp32 add issue rate.
 // The paper reports its kernel against the L2 roof of its own card
