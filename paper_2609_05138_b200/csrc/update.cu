@@ -114,6 +114,146 @@ update_blur_kernel(const uint32_t *__restrict__ num, const uint32_t *__restrict_
     }
 }
 
+
+// ---- the same blur for radii 1 .. 8 on maps whose rows are whole 16-byte pieces ----------
+// One block per 64 x 64 tile of one plane, radius a template parameter so that every loop
+// unrolls and the taps sit in registers.  Packed fp32 arithmetic throughout (fma.rn.f32x2):
+// the row pass works on two map rows at once (the tile is staged as (row 2p, row 2p+1) pairs),
+// the column pass on two neighbouring columns at once, and the outputs leave as 8-byte stores:
+// 47 warp instructions per 32 outputs against 84 for the general kernel above.
+__device__ __forceinline__ void fma2(u64 &acc, u64 a, u64 b)
+{
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
+}
+__device__ __forceinline__ u64 pack2(float lo, float hi)
+{
+    return ((u64)__float_as_uint(hi) << 32) | __float_as_uint(lo);
+}
+
+template <int R> struct BlurFast {
+    static constexpr int TX = 64, TY = 64;
+    static constexpr int RP = (R + 3) / 4 * 4;          // halo in x, whole 16-byte pieces
+    static constexpr int SPAN = TY + 2 * R;             // staged rows (even)
+    static constexpr int NRP = SPAN / 2;                // staged row pairs
+    static constexpr int NC = (TX + 2 * RP) / 4;        // 16-byte pieces per staged row
+    static constexpr int PX = TX + 2 * RP + 1;          // pairs per staged row pair (odd pitch:
+                                                        // lanes over row pairs hit distinct banks)
+    static constexpr int PM = TX + 4;                   // floats per row of the row-pass result
+    static constexpr size_t SMEM = (size_t)SPAN * PM * 4 + (size_t)NRP * PX * 8;
+};
+
+template <int R>
+__global__ void __launch_bounds__(256)
+update_blur_fast_kernel(const uint32_t *__restrict__ num, const uint32_t *__restrict__ cnt, int64_t D,
+                        int32_t edge_x, int32_t edge_y, const BlurTaps taps,
+                        float *__restrict__ num_blur, float *__restrict__ cnt_blur)
+{
+    using F = BlurFast<R>;
+    extern __shared__ __align__(16) unsigned char smraw[];
+    float *mid = reinterpret_cast<float *>(smraw);                          // SPAN x PM
+    float2 *in2 = reinterpret_cast<float2 *>(smraw + (size_t)F::SPAN * F::PM * 4);   // NRP x PX
+    const int64_t plane = blockIdx.z, M = (int64_t)edge_x * edge_y;
+    const uint32_t *src = plane < D ? num + plane * M : cnt;
+    float *dst = plane < D ? num_blur + plane * M : cnt_blur;
+    const int x0 = blockIdx.x * F::TX, y0 = blockIdx.y * F::TY;
+
+    // taps g[-R .. R] are symmetric: ts[k] = (g[k], g[k]) for k = |d|
+    u64 ts[R + 1];
+#pragma unroll
+    for (int k = 0; k <= R; ++k) ts[k] = pack2(taps.gp[3 + R + k], taps.gp[3 + R + k]);
+
+    // stage the tile and its halo as pairs of rows, zero outside the map
+    for (int item = threadIdx.x; item < F::NRP * F::NC; item += 256) {
+        const int rp = item / F::NC, q = item - rp * F::NC;
+        const int x = x0 - F::RP + 4 * q, y = y0 - R + 2 * rp;
+        uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+        if (x >= 0 && x < edge_x) {
+            if (y >= 0 && y < edge_y)
+                a = __ldcs(reinterpret_cast<const uint4 *>(src + (int64_t)y * edge_x + x));
+            if (y + 1 >= 0 && y + 1 < edge_y)
+                b = __ldcs(reinterpret_cast<const uint4 *>(src + (int64_t)(y + 1) * edge_x + x));
+        }
+        float2 *o = in2 + rp * F::PX + 4 * q;
+        const float2 v[4] = {make_float2((float)a.x, (float)b.x), make_float2((float)a.y, (float)b.y),
+                             make_float2((float)a.z, (float)b.z), make_float2((float)a.w, (float)b.w)};
+        // neighbouring lanes sit 32 bytes apart: lane l stores its four pairs starting with
+        // pair (l / 4) % 4, so that 16 lanes hit 16 different bank pairs at every step
+        const int rot = (threadIdx.x >> 2) & 3;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int kk = (k + rot) & 3;
+            const float2 lo = (kk & 1) ? v[1] : v[0], hi = (kk & 1) ? v[3] : v[2];
+            o[kk] = (kk & 2) ? hi : lo;
+        }
+    }
+    __syncthreads();
+    // row pass: item = (group of four outputs g4, row pair rp), lanes over row pairs
+    for (int item = threadIdx.x; item < F::NRP * (F::TX / 4); item += 256) {
+        const int g4 = item / F::NRP, rp = item - g4 * F::NRP;
+        const u64 *win = reinterpret_cast<const u64 *>(in2 + rp * F::PX + (F::RP - R) + 4 * g4);
+        u64 acc[4] = {0ull, 0ull, 0ull, 0ull};
+#pragma unroll
+        for (int e = 0; e < 4 + 2 * R; ++e) {
+            const u64 v = win[e];
+#pragma unroll
+            for (int o = 0; o < 4; ++o) {
+                const int d = e - o - R;                 // tap offset of input e for output o
+                if (d >= -R && d <= R) fma2(acc[o], ts[d < 0 ? -d : d], v);
+            }
+        }
+        float *m0 = mid + (2 * rp) * F::PM + 4 * g4;
+        *reinterpret_cast<float4 *>(m0) = make_float4(lo_f(acc[0]), lo_f(acc[1]), lo_f(acc[2]), lo_f(acc[3]));
+        *reinterpret_cast<float4 *>(m0 + F::PM) =
+            make_float4(hi_f(acc[0]), hi_f(acc[1]), hi_f(acc[2]), hi_f(acc[3]));
+    }
+    __syncthreads();
+    // column pass: a thread takes two neighbouring columns and eight rows
+    {
+        const int c2 = threadIdx.x & 31, rg = threadIdx.x >> 5;
+        const float *col = mid + (8 * rg) * F::PM + 2 * c2;
+        u64 acc[8] = {0ull, 0ull, 0ull, 0ull, 0ull, 0ull, 0ull, 0ull};
+#pragma unroll
+        for (int e = 0; e < 8 + 2 * R; ++e) {
+            const u64 v = *reinterpret_cast<const u64 *>(col + e * F::PM);
+#pragma unroll
+            for (int o = 0; o < 8; ++o) {
+                const int d = e - o - R;
+                if (d >= -R && d <= R) fma2(acc[o], ts[d < 0 ? -d : d], v);
+            }
+        }
+        const int x = x0 + 2 * c2, y = y0 + 8 * rg;
+        if (x < edge_x) {
+#pragma unroll
+            for (int o = 0; o < 8; ++o)
+                if (y + o < edge_y)
+                    __stcs(reinterpret_cast<float2 *>(dst + (int64_t)(y + o) * edge_x + x),
+                           make_float2(lo_f(acc[o]), hi_f(acc[o])));
+        }
+    }
+}
+
+template <int R>
+static int launch_blur_fast(const uint32_t *num, const uint32_t *cnt, int64_t D, int32_t edge_x,
+                            int32_t edge_y, const BlurTaps &t, float *num_blur, float *cnt_blur,
+                            cudaStream_t s)
+{
+    using F = BlurFast<R>;
+    static bool configured[64];
+    int dev = 0;
+    BMU_CUDA(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        BMU_CUDA(cudaFuncSetAttribute(update_blur_fast_kernel<R>,
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)F::SMEM));
+        configured[dev] = true;
+    }
+    const dim3 grid((unsigned)((edge_x + F::TX - 1) / F::TX), (unsigned)((edge_y + F::TY - 1) / F::TY),
+                    (unsigned)(D + 1));
+    update_blur_fast_kernel<R><<<grid, 256, F::SMEM, s>>>(num, cnt, D, edge_x, edge_y, t, num_blur,
+                                                         cnt_blur);
+    BMU_CUDA(cudaGetLastError());
+    return BMU_OK;
+}
+
 // One row of W per blockIdx.y; float4 pieces when the row pitch allows.
 template <bool VEC>
 __global__ void __launch_bounds__(256)
@@ -227,6 +367,22 @@ int launch_update_blur(const uint32_t *num, const uint32_t *cnt, int64_t D, int3
     for (int d = -t.R; d <= t.R; ++d)
         t.gp[d + t.R + 3] = sigma > 0.f
             ? (float)exp(-(double)(d * d) / (2.0 * (double)sigma * (double)sigma)) : 1.f;
+    // radii 1 .. 8 on maps whose rows are whole, aligned 16-byte pieces: the unrolled kernel
+    const bool aligned = edge_x % 4 == 0 &&
+                         ((reinterpret_cast<uintptr_t>(num) | reinterpret_cast<uintptr_t>(cnt) |
+                           reinterpret_cast<uintptr_t>(num_blur) | reinterpret_cast<uintptr_t>(cnt_blur)) & 15) == 0;
+    if (aligned && t.R >= 1 && t.R <= 8) {
+        switch (t.R) {
+        case 1: return launch_blur_fast<1>(num, cnt, D, edge_x, edge_y, t, num_blur, cnt_blur, s);
+        case 2: return launch_blur_fast<2>(num, cnt, D, edge_x, edge_y, t, num_blur, cnt_blur, s);
+        case 3: return launch_blur_fast<3>(num, cnt, D, edge_x, edge_y, t, num_blur, cnt_blur, s);
+        case 4: return launch_blur_fast<4>(num, cnt, D, edge_x, edge_y, t, num_blur, cnt_blur, s);
+        case 5: return launch_blur_fast<5>(num, cnt, D, edge_x, edge_y, t, num_blur, cnt_blur, s);
+        case 6: return launch_blur_fast<6>(num, cnt, D, edge_x, edge_y, t, num_blur, cnt_blur, s);
+        case 7: return launch_blur_fast<7>(num, cnt, D, edge_x, edge_y, t, num_blur, cnt_blur, s);
+        default: return launch_blur_fast<8>(num, cnt, D, edge_x, edge_y, t, num_blur, cnt_blur, s);
+        }
+    }
     const int span_y = BLUR_TY + 2 * t.R;
     const int pitch = (BLUR_TX + 2 * t.R + 3) / 4 * 4 + 4;
     const size_t smem = (size_t)(span_y * pitch + span_y * BLUR_TX) * sizeof(float);

@@ -63,7 +63,8 @@ def test_scatter_accumulates_batches_and_takes_odd_rows(bmu):
 
 @pytest.mark.parametrize("ex,ey,sigma,D", [(32, 32, 1.0, 5), (64, 64, 2.5, 3), (45, 70, 0.4, 4),
                                           (33, 31, 8.0, 2), (7, 5, 1.5, 6), (128, 16, 0.0, 3),
-                                          (100, 100, 3.3, 2)])
+                                          (100, 100, 3.3, 2), (128, 96, 2.0, 2), (64, 200, 0.3, 2),
+                                          (512, 512, 1.4, 1), (68, 72, 2.6, 3), (4, 4, 1.0, 2)])
 def test_blur_matches_oracle(bmu, ex, ey, sigma, D):
     M = ex * ey
     g = torch.Generator().manual_seed(ex + ey)
