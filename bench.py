@@ -87,6 +87,17 @@ class ClockSampler:
                 self.proc.kill()
         self.tmp.flush()
         self.tmp.seek(0)
+        if not self.tmp.read().strip():
+            # the timed region was shorter than one sampling period: one reading right after it
+            cmd = ["nvidia-smi", "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits"]
+            if self.uuid:
+                cmd += ["-i", self.uuid]
+            try:
+                self.tmp.write(subprocess.run(cmd, capture_output=True, text=True, timeout=20).stdout)
+            except (OSError, subprocess.SubprocessError):
+                pass
+            self.tmp.flush()
+        self.tmp.seek(0)
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.tmp.read().splitlines():
