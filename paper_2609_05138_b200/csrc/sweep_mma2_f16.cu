@@ -478,6 +478,17 @@ int launch_sweep_mma2_f16(const MmaArgs &a, const bmu_opts &o, cudaStream_t s)
     int dev = 0;
     BMU_CUDA(cudaGetDevice(&dev));
     if (dev >= 0 && dev < 64 && !configured[dev]) {
+        // the register hand-over inside the kernel must fit what a block is launched with, or
+        // the increase would wait for ever: refuse to launch a build where it does not
+        cudaFuncAttributes fa, fb;
+        BMU_CUDA(cudaFuncGetAttributes(&fa, sweep_mma2_f16_kernel<false>));
+        BMU_CUDA(cudaFuncGetAttributes(&fb, sweep_mma2_f16_kernel<true>));
+        const int regs = fa.numRegs < fb.numRegs ? fa.numRegs : fb.numRegs;
+        if (M2_THREADS * regs < 128 * 56 + 512 * 104) {
+            set_error("half-precision tensor-core sweep: built with %d registers per thread, the "
+                      "register hand-over needs %d", regs, (128 * 56 + 512 * 104 + M2_THREADS - 1) / M2_THREADS);
+            return BMU_ERR_UNSUPPORTED;
+        }
         BMU_CUDA(cudaFuncSetAttribute(sweep_mma2_f16_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)m2_smem_bytes(HEAD_ROWS_MAX, false)));
         BMU_CUDA(cudaFuncSetAttribute(sweep_mma2_f16_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
