@@ -68,7 +68,7 @@ def test_f16_top2_and_limits(bmu):
                                                      ("cfg1", 900, 512, "dupes", 1024)])
 def test_f16_tensor_core_sweep_matches_oracle(bmu, name, n_docs, M, kind, head):
     """The wide tensor-core sweep on a half-precision codebook: the weights are fp16 already, so
-    the head image has one part and the tail gathers 8-byte pieces."""
+    the head image has one part and the tail gathers 16-byte pieces."""
     cfg = synth.CONFIGS[name]
     rowptr, colidx = synth.make_corpus(cfg, n_docs=n_docs)
     W16 = synth.make_codebook(cfg.D, M, 52, kind=kind).half()
@@ -83,3 +83,71 @@ def test_f16_tensor_core_sweep_matches_oracle(bmu, name, n_docs, M, kind, head):
         assert int((ob % 2).sum()) == 0
     b1, d1, b2, d2 = bmu.bmu_search_f16_ws(W16.cuda(), rowptr.cuda(), colidx.cuda(), opts=o, top2=True)
     assert torch.equal(b1, ob) and torch.equal(d1, od) and bool((b2 != b1).all())
+
+
+def _csr(rows):
+    rowptr = np.zeros(len(rows) + 1, dtype=np.int32)
+    rowptr[1:] = np.cumsum([len(r) for r in rows])
+    colidx = np.concatenate([np.asarray(r, dtype=np.int32) for r in rows]) if rowptr[-1] else \
+        np.zeros(0, dtype=np.int32)
+    return torch.from_numpy(rowptr), torch.from_numpy(colidx)
+
+
+@pytest.mark.parametrize("n_docs", [1, 7, 129, 300])
+def test_f16_tensor_core_sweep_ragged_documents(bmu, n_docs):
+    """Few documents (less than a block, a block and a bit), rows that are empty, only head ids,
+    only gathered ids, one long row, unsorted rows; several chunks of neurons."""
+    D, M = 2048, 1536
+    r = np.random.default_rng(n_docs)
+    rows = []
+    for i in range(n_docs):
+        kind = i % 5
+        if kind == 0:
+            rows.append([])
+        elif kind == 1:
+            rows.append(r.choice(512, size=int(r.integers(1, 40)), replace=False))        # head only
+        elif kind == 2:
+            rows.append(512 + r.choice(D - 512, size=int(r.integers(1, 40)), replace=False))
+        elif kind == 3:
+            rows.append(r.permutation(D)[:400])                                            # long, unsorted
+        else:
+            rows.append(r.choice(D, size=int(r.integers(1, 90)), replace=False))
+    rowptr, colidx = _csr(rows)
+    W16 = (synth.make_codebook(D, M, 53, kind="scaled")).half()
+    o = bmu.Opts()
+    o.kernel = 6
+    o.chunk_neurons = 512
+    ob, od = bmu.bmu_search_f16_ws(W16.cuda(), rowptr.cuda(), colidx.cuda(), opts=o)
+    torch.cuda.synchronize()
+    parity.compare(ob.cpu().numpy(), od.cpu().numpy(), W16.float().numpy(), rowptr.numpy(),
+                   colidx.numpy())
+    # one chunk or three: the same bits
+    o.chunk_neurons = 1536
+    ob1, od1 = bmu.bmu_search_f16_ws(W16.cuda(), rowptr.cuda(), colidx.cuda(), opts=o)
+    assert torch.equal(ob, ob1) and torch.equal(od, od1)
+
+
+def test_f16_tensor_core_sweep_second_best_and_unlabelled_vocabulary(bmu):
+    cfg = synth.CONFIGS["cfg3"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=1200)
+    g = torch.Generator().manual_seed(9)
+    relabel = torch.randperm(cfg.D, generator=g).to(torch.int32)       # frequent ids anywhere
+    colidx = relabel[colidx.long()]
+    W16 = synth.make_codebook(cfg.D, 1024, 54, kind="scaled").half()
+    o = bmu.Opts()
+    o.kernel = 6
+    b1, d1, b2, d2 = bmu.bmu_search_f16_ws(W16.cuda(), rowptr.cuda(), colidx.cuda(), opts=o, top2=True)
+    torch.cuda.synchronize()
+    W32 = W16.float().numpy()
+    parity.compare(b1.cpu().numpy(), d1.cpu().numpy(), W32, rowptr.numpy(), colidx.numpy())
+    e1, f1, e2, f2 = oracle.bmu2(W32, rowptr.numpy(), colidx.numpy())
+    np.testing.assert_allclose(d2.cpu().numpy(), f2, rtol=1e-5)
+    clear = (f2 - f1) > 1e-4 * np.abs(f1)
+    assert np.array_equal(b1.cpu().numpy()[clear], e1[clear])
+    # the second-best index wherever the third-best distance is clearly apart: recompute its
+    # distance with the oracle's pair evaluation
+    sample = np.arange(0, 1200, 37)
+    nrm = oracle.norms(W32)
+    for i in sample:
+        got = oracle.eval_pair(W32, rowptr.numpy(), colidx.numpy(), nrm, int(i), int(b2[i]))
+        assert abs(got - f2[i]) <= 1e-5 * abs(f2[i])
