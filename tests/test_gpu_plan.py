@@ -48,3 +48,39 @@ def test_planned_search_argument_checks(bmu):
         plan.search(W)
     assert e.value.status == 2
     assert bmu.load().bmu_search_planned(None, None, None, None, None, None) == 1
+
+
+def test_search_with_workspace_can_be_captured_in_a_cuda_graph(bmu):
+    """bmu_search_ws allocates nothing and only enqueues work, so a caller can capture it once
+    and replay it; the replay gives the bits of the eager call."""
+    lib = bmu
+    cfg = synth.CONFIGS["cfg1"]
+    dev = torch.device("cuda")
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=3000, device=dev)
+    W = synth.make_codebook(cfg.D, cfg.M, 3, device=dev)
+    N = rowptr.numel() - 1
+    norms = lib.bmu_codebook_norms(W)
+    need = lib.bmu_search_workspace_bytes(cfg.D, cfg.M, N, colidx.numel())
+    ws = torch.empty(need + 256, dtype=torch.uint8, device=dev)
+    ob = torch.empty(N, dtype=torch.int32, device=dev)
+    od = torch.empty(N, dtype=torch.float32, device=dev)
+
+    def call():
+        lib.bmu_search_ws(W, rowptr, colidx, norms=norms, workspace=ws, out_bmu=ob, out_dist=od)
+
+    call()
+    torch.cuda.synchronize()
+    ref_b, ref_d = ob.clone(), od.clone()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):                      # first call on another stream, uncaptured
+        call()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        call()
+    for _ in range(3):
+        ob.zero_()
+        od.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(ob, ref_b) and torch.equal(od, ref_d)
