@@ -156,3 +156,39 @@ def test_mma_kernel_few_documents_and_empty_corpus_rows(bmu, kernel, N):
     empty_rp = torch.zeros(N + 1, dtype=torch.int32)
     res = run_and_check(bmu, W, empty_rp, torch.zeros(0, dtype=torch.int32), opts_of(bmu, kernel))
     assert res["docs"] == N
+
+
+@pytest.mark.parametrize("kernel", [0, 3, 4, 6])
+def test_largest_vocabulary_with_16_bit_ids(bmu, kernel):
+    """D = 65024, the most the 16-bit id lists hold: ids up to 65023 sit next to the 0xffff
+    sentinel of a ragged row."""
+    D, M, N = 65024, 512, 300
+    r = np.random.default_rng(kernel)
+    rows = []
+    for i in range(N):
+        n = int(r.integers(0, 60))
+        low = r.choice(2000, size=n // 2, replace=False)
+        high = D - 1 - r.choice(3000, size=n - n // 2, replace=False)      # 62024 .. 65023
+        rows.append(np.sort(np.concatenate([low, high])))
+    rows[5] = np.array([D - 1])
+    rows[6] = np.arange(D - 40, D)
+    rowptr = np.zeros(N + 1, dtype=np.int32)
+    rowptr[1:] = np.cumsum([len(x) for x in rows])
+    colidx = np.concatenate(rows).astype(np.int32)
+    W = synth.make_codebook(D, M, 60, kind="scaled")
+    run_and_check(bmu, W, torch.from_numpy(rowptr), torch.from_numpy(colidx), opts_of(bmu, kernel))
+
+
+def test_vocabulary_beyond_16_bit_ids_takes_the_generic_kernel(bmu):
+    D, M, N = 70000, 260, 150
+    r = np.random.default_rng(3)
+    rows = [np.sort(r.choice(D, size=int(r.integers(0, 50)), replace=False)) for _ in range(N)]
+    rows[0] = np.array([D - 1, 65535, 65536, 65024])
+    rowptr = np.zeros(N + 1, dtype=np.int32)
+    rowptr[1:] = np.cumsum([len(x) for x in rows])
+    colidx = np.concatenate(rows).astype(np.int32)
+    W = synth.make_codebook(D, M, 61, kind="scaled")
+    run_and_check(bmu, W, torch.from_numpy(rowptr), torch.from_numpy(colidx), opts_of(bmu, 0))
+    with pytest.raises(bmu.BmuError) as e:
+        run_and_check(bmu, W, torch.from_numpy(rowptr), torch.from_numpy(colidx), opts_of(bmu, 6))
+    assert e.value.status == 2
