@@ -98,22 +98,37 @@ __global__ void plan_rank_tables_kernel(const uint32_t *__restrict__ sorted, int
 }
 
 // Sorting key of a document: how many of its ids the gather will visit, i.e. the ids at or
-// above `head` (all of them when head == 0).  One warp per document.
+// above `head` (all of them when head == 0) -- or the whole list if it repeats an id below
+// `head`: such a list keeps multiset semantics by staying out of the dense head altogether
+// (head_of_doc below), so all of it is gathered.  The key must be the gathered length exactly:
+// the room reserved for the tile id matrices counts on documents ordered by it.  One warp per
+// document.
 __global__ void __launch_bounds__(256)
 plan_key_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colidx,
                 const uint16_t *__restrict__ rank, int64_t N, int32_t head,
                 uint32_t *__restrict__ key)
 {
-    const int lane = threadIdx.x & 31;
+    __shared__ uint32_t seen[8][HEAD_ROWS_MAX / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (i >= N) return;
+    for (int w = lane; w < head / 32; w += 32) seen[warp][w] = 0u;
+    __syncwarp();
     const int beg = rowptr[i], end = rowptr[i + 1];
-    int cnt = 0;
-    for (int e = beg + lane; e < end; e += 32)
-        cnt += (rank ? (int32_t)rank[colidx[e]] : colidx[e]) >= head;
+    int cnt = 0, repeat = 0;
+    for (int e = beg + lane; e < end; e += 32) {
+        const int32_t r = rank ? (int32_t)rank[colidx[e]] : colidx[e];
+        if (r >= head) {
+            ++cnt;
+        } else {
+            const uint32_t bit = 1u << (r & 31);
+            repeat |= (atomicOr(&seen[warp][r >> 5], bit) & bit) != 0u;
+        }
+    }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
-    if (lane == 0) key[i] = (uint32_t)cnt;
+    repeat = __any_sync(0xffffffffu, repeat);
+    if (lane == 0) key[i] = repeat ? (uint32_t)(end - beg) : (uint32_t)cnt;
 }
 
 __global__ void plan_hist_kernel(const int32_t *__restrict__ rowptr,

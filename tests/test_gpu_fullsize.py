@@ -164,3 +164,42 @@ def test_cfg2_full_size_update_step_properties(bmu):
     live = cb > 0
     assert float(W1[:, live].min()) >= 0.0 and float(W1[:, live].max()) <= 1.0 + 1e-6
     assert torch.equal(W1[:, ~live], W[:, ~live])
+
+
+@pytest.mark.parametrize("M", [256, 512])           # planned kernel; wide tensor-core sweep
+def test_listing_count_next_to_the_32_bit_limit(bmu, M):
+    """nnz = 2.1e9 of the 2^31 - 1 a CSR batch with int32 offsets can hold (16.5 M documents of
+    120-134 listings, repeats allowed: rows are multisets): offsets, the tiling pass and the
+    kernels must not wrap.  Checked on sampled documents against a plain fp64 recomputation and
+    by agreement of the planned and the generic kernel."""
+    dev = torch.device("cuda")
+    D, N = 4096, 16_500_000
+    g = torch.Generator(device=dev).manual_seed(1)
+    lens = torch.randint(120, 135, (N,), generator=g, device=dev, dtype=torch.int64)
+    rowptr64 = torch.zeros(N + 1, dtype=torch.int64, device=dev)
+    rowptr64[1:] = torch.cumsum(lens, 0)
+    nnz = int(rowptr64[-1])
+    assert 2_000_000_000 < nnz < 2 ** 31
+    rowptr = rowptr64.to(torch.int32)
+    del rowptr64, lens
+    colidx = torch.randint(0, D, (nnz,), generator=g, device=dev, dtype=torch.int32)
+    W = torch.rand((D, M), generator=g, device=dev) * 0.05
+    norms64 = (W.double() ** 2).sum(0)
+    outs = []
+    for kernel in (0, 1):
+        o = bmu.Opts()
+        o.kernel = kernel
+        ob, od = bmu.bmu_search_ws(W, rowptr, colidx, opts=o)
+        torch.cuda.synchronize()
+        assert int(ob.min()) >= 0 and int(ob.max()) < M
+        sample = list(range(0, 50)) + list(range(N - 50, N)) + \
+            torch.randint(0, N, (100,), generator=torch.Generator().manual_seed(2)).tolist()
+        for i in sample:
+            ids = colidx[int(rowptr[i]):int(rowptr[i + 1])].long()
+            d = float(ids.numel()) + norms64 - 2.0 * W[ids].double().sum(0)
+            j = int(torch.argmin(d))
+            assert abs(float(od[i]) - float(d[j])) <= 1e-5 * abs(float(d[j]))
+            assert int(ob[i]) == j or abs(float(d[int(ob[i])]) - float(d[j])) <= 1e-5 * abs(float(d[j]))
+        outs.append((ob, od))
+    assert float((outs[0][0] == outs[1][0]).float().mean()) > 0.9999      # near-ties aside
+    assert float(((outs[0][1] - outs[1][1]).abs() / outs[1][1].abs()).max()) < 1e-6
