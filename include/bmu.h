@@ -21,12 +21,14 @@
  *           colidx[rowptr[i] .. rowptr[i+1])            (CSR of the binary corpus)
  *   colidx  int32 [nnz], feature ids in [0, D); distinct inside a row (a
  *           repeated id is simply added twice and counted twice in |x_i|);
- *           any order inside a row.
+ *           any order inside a row; at most 65535 ids in a row (more is only
+ *           possible with repeats; the planned and tile kernels keep row lengths
+ *           in 16 bits).
  *   norms   float32 [M], ||w_j||^2.
  *   out_bmu int32 [N], out_dist float32 [N], in the caller's document order.
  * Limits: M < 2^30; N, D < 2^31; nnz < 2^31 per call (int32 rowptr).  Ids out of
- * range and non-finite weights are preconditions that the hot path does not
- * check (bmu_validate_csr checks the former).  An empty row is legal: its
+ * range, rows of more than 65535 ids and non-finite weights are preconditions
+ * that the hot path does not check (bmu_validate_csr checks the first two).  An empty row is legal: its
  * distances are the norms.  N == 0 is legal and does nothing.
  *
  * Every call is asynchronous on `stream` (a cudaStream_t passed as void*, NULL =
@@ -282,7 +284,8 @@ BMU_API int bmu_release_scratch(void);
 
 /*
  * Checks the CSR preconditions on the device: rowptr[0] == 0, rowptr
- * non-decreasing, rowptr[N] == nnz, 0 <= colidx < D.  Synchronises the stream.
+ * non-decreasing, rowptr[N] == nnz, 0 <= colidx < D, no row of more than 65535
+ * ids.  Synchronises the stream.
  * Returns BMU_ERR_INVALID_ARG (detail in bmu_last_error) when one fails.
  */
 BMU_API int bmu_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,

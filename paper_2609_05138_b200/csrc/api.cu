@@ -467,8 +467,10 @@ __global__ void validate_kernel(const int32_t *__restrict__ rowptr,
         if (rowptr[0] != 0) atomicOr(flags, 1);
         if ((int64_t)rowptr[N] != nnz) atomicOr(flags, 2);
     }
-    for (int64_t i = t; i < N; i += stride)
+    for (int64_t i = t; i < N; i += stride) {
         if (rowptr[i + 1] < rowptr[i]) atomicOr(flags, 4);
+        if ((int64_t)rowptr[i + 1] - rowptr[i] > 65535) atomicOr(flags, 16);
+    }
     for (int64_t e = t; e < nnz; e += stride) {
         const int32_t f = colidx[e];
         if (f < 0 || (int64_t)f >= D) atomicOr(flags, 8);
@@ -918,9 +920,10 @@ int bmu_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, in
     BMU_CUDA(cudaMemcpyAsync(&h, flags, sizeof(h), cudaMemcpyDeviceToHost, s));
     BMU_CUDA(cudaStreamSynchronize(s));
     if (h) {
-        set_error("invalid CSR:%s%s%s%s", (h & 1) ? " rowptr[0] != 0;" : "",
+        set_error("invalid CSR:%s%s%s%s%s", (h & 1) ? " rowptr[0] != 0;" : "",
                   (h & 2) ? " rowptr[N] != nnz;" : "", (h & 4) ? " rowptr decreases;" : "",
-                  (h & 8) ? " colidx outside [0, D);" : "");
+                  (h & 8) ? " colidx outside [0, D);" : "",
+                  (h & 16) ? " a row lists more than 65535 ids;" : "");
         return BMU_ERR_INVALID_ARG;
     }
     return BMU_OK;

@@ -192,6 +192,11 @@ def test_validate_csr(bmu):
         bmu.bmu_validate_csr(rp, ci, 5)
     with pytest.raises(bmu.BmuError, match="decreases"):
         bmu.bmu_validate_csr(torch.tensor([0, 3, 2, 3], dtype=torch.int32).cuda(), ci, 6)
+    long_rp = torch.tensor([0, 65535, 65535 + 65536], dtype=torch.int32).cuda()
+    long_ci = torch.zeros(65535 + 65536, dtype=torch.int32).cuda()
+    with pytest.raises(bmu.BmuError, match="more than 65535"):
+        bmu.bmu_validate_csr(long_rp, long_ci, 6)
+    bmu.bmu_validate_csr(long_rp[:2], long_ci[:65535], 6)          # exactly 65535 is allowed
 
 
 def test_workspace_errors(bmu):
