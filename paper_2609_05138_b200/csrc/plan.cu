@@ -196,7 +196,7 @@ __global__ void plan_groups_kernel(const int32_t *__restrict__ rowptr,
 }
 
 // One warp per planned document: writes its ascending 16-bit id list.  Rows that
-// are not already ascending are ordered by counting, for each id, the ids that
+// are not already in non-decreasing order are ordered by counting, for each id, the ids that
 // must precede it (quadratic in the row length, rows are short).
 __global__ void __launch_bounds__(256)
 plan_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colidx,
@@ -215,7 +215,7 @@ plan_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__
     const int padded = ((len + 7) / 8 + 1) * 8;
 
     bool sorted = true;
-    for (int e = lane; e + 1 < len; e += 32) sorted &= BMU_PLAN_ID(e) < BMU_PLAN_ID(e + 1);
+    for (int e = lane; e + 1 < len; e += 32) sorted &= BMU_PLAN_ID(e) <= BMU_PLAN_ID(e + 1);
     sorted = __all_sync(0xffffffffu, sorted);
     if (sorted) {
         for (int e = lane; e < padded; e += 32) dst[e] = e < len ? (uint16_t)BMU_PLAN_ID(e) : 0xFFFFu;
