@@ -65,7 +65,9 @@ def test_f16_top2_and_limits(bmu):
 @pytest.mark.parametrize("name,n_docs,M,kind,head", [("cfg1", 4000, 1024, "uniform", 0),
                                                      ("cfg3", 1500, 2048, "scaled", 0),
                                                      ("cfg5", 700, 512, "signed", 256),
-                                                     ("cfg1", 900, 512, "dupes", 1024)])
+                                                     ("cfg1", 900, 512, "dupes", 1024),
+                                                     ("cfg3", 600, 1024, "scaled", 2048),
+                                                     ("cfg2", 500, 512, "uniform", 64)])
 def test_f16_tensor_core_sweep_matches_oracle(bmu, name, n_docs, M, kind, head):
     """The wide tensor-core sweep on a half-precision codebook: the weights are fp16 already, so
     the head image has one part and the tail gathers 16-byte pieces."""

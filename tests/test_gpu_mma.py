@@ -49,7 +49,7 @@ def run_and_check(bmu, W, rowptr, colidx, opts, cancel_floor=False):
 
 @pytest.mark.parametrize("kernel,tile_order,head_rows", [(5, 0, 0), (5, 1, 256), (5, 0, 512),
                                                          (6, 0, 0), (6, 1, 64), (6, 0, 512),
-                                                         (6, 0, 1024), (6, 1, 320), (7, 0, 0),
+                                                         (6, 0, 1024), (6, 1, 320), (6, 0, 2048), (7, 0, 0),
                                                          (7, 1, 64), (7, 0, 768), (7, 0, 2048)])
 @pytest.mark.parametrize("name,n_docs,M,chunk", [("cfg3", 2500, 2048, 1024), ("cfg5", 1203, 1536, 512),
                                                  ("cfg1", 4001, 1024 + 36, 0), ("cfg2", 777, 512, 0)])
