@@ -84,3 +84,33 @@ def test_search_with_workspace_can_be_captured_in_a_cuda_graph(bmu):
         graph.replay()
         torch.cuda.synchronize()
         assert torch.equal(ob, ref_b) and torch.equal(od, ref_d)
+
+
+@pytest.mark.parametrize("kernel", [0, 3, 6])
+def test_calls_on_two_streams_with_their_own_workspaces_do_not_interfere(bmu, kernel):
+    """The library keeps no device-side state outside the caller's workspace (the one-shot and
+    the static entry points aside): two searches in flight at once give what they give alone."""
+    cfg = synth.CONFIGS["cfg3"]
+    dev = torch.device("cuda")
+    jobs = []
+    for k, (n_docs, M) in enumerate(((6000, 2048), (4000, 1536))):
+        rowptr, colidx = synth.make_corpus(cfg, batch=k, n_docs=n_docs, device=dev)
+        W = synth.make_codebook(cfg.D, M, 70 + k, kind="scaled", device=dev)
+        o = bmu.Opts()
+        o.kernel = kernel
+        alone = bmu.bmu_search_ws(W, rowptr, colidx, opts=o)
+        N = rowptr.numel() - 1
+        need = bmu.bmu_search_workspace_bytes(cfg.D, M, N, colidx.numel(), o)
+        jobs.append(dict(W=W, rp=rowptr, ci=colidx, o=o, alone=alone, s=torch.cuda.Stream(),
+                         ws=torch.empty(need + 256, dtype=torch.uint8, device=dev),
+                         ob=torch.empty(N, dtype=torch.int32, device=dev),
+                         od=torch.empty(N, dtype=torch.float32, device=dev)))
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for j in jobs:
+            with torch.cuda.stream(j["s"]):
+                bmu.bmu_search_ws(j["W"], j["rp"], j["ci"], opts=j["o"], workspace=j["ws"],
+                                  out_bmu=j["ob"], out_dist=j["od"])
+    torch.cuda.synchronize()
+    for j in jobs:
+        assert torch.equal(j["ob"], j["alone"][0]) and torch.equal(j["od"], j["alone"][1])
