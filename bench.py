@@ -268,13 +268,14 @@ def run_ours(args, cfg, rank, local_rank, world):
     n_chunks = (cfg.M + chunk - 1) // chunk
     # documents that share one SM's L1 at a time: resident warps x documents per warp
     kernel_name = {3: "sweep_rows_kernel", 1: "sweep_direct_kernel", 2: "sweep_lanes_kernel",
-                   4: "sweep_tiles_kernel", 5: "sweep_mma_kernel", 6: "sweep_mma2_kernel"}[kernel]
+                   4: "sweep_tiles_kernel", 5: "sweep_mma_kernel", 6: "sweep_mma2_kernel",
+                   7: "sweep_mma3_kernel"}[kernel]
     if kernel == 4:
         vec, slab = 4, 128
         chunk = opts.chunk_neurons or max(slab, (l2_bytes // 2) // (cfg.D * 4) // slab * slab)
         chunk = min((chunk + slab - 1) // slab * slab, (cfg.M + slab - 1) // slab * slab)
         n_chunks = (cfg.M + chunk - 1) // chunk
-    if kernel in (5, 6):
+    if kernel in (5, 6, 7):
         vec, slab = 4, 512
         chunk = opts.chunk_neurons or max(slab, int(l2_bytes * 0.55) // (cfg.D * 4) // slab * slab)
         chunk = min((chunk + slab - 1) // slab * slab, cfg.M // slab * slab)
@@ -287,8 +288,8 @@ def run_ours(args, cfg, rank, local_rank, world):
         docs_per_block = 8 * (opts.warps or 4) * 5
     elif kernel == 1:
         docs_per_block = (opts.warps or 16) * (opts.docs_per_warp or 4) * 2
-    elif kernel in (5, 6):
-        docs_per_block = 128
+    elif kernel in (5, 6, 7):
+        docs_per_block = 256 if kernel == 7 else 128
     else:
         docs_per_block = 48
 
@@ -383,16 +384,17 @@ def run_ours(args, cfg, rank, local_rank, world):
                 peaks["hbm_gbs"] * 1e9, "B/s"),
     }
     extra = {}
-    if kernel in (5, 6):
+    if kernel in (5, 6, 7):
         # the frequent features' updates are MMAs, not loads and adds: only the tail's updates
         # pass through L1 and the fp32 pipe.  The L2 figure stays the algorithmic one (each
         # block of 128 documents fetches every distinct row it touches once); what the design
         # really moves is the tail's rows per document plus the head image per block.
-        head = opts.head_rows or (256 if kernel == 5 else min(768, cfg.D // 64 * 64))
+        head = opts.head_rows or (256 if kernel == 5 else
+                                  min(896 if kernel == 7 else 768, cfg.D // 64 * 64))
         tail_share = float((colidx >= head).sum().item()) / max(1, colidx.numel())
         alg["alu"] = (tail_share * adds / launch_s, roofs["fadd2"], "add/s")
         alg["l1"] = (4.0 * tail_share * adds / launch_s, roofs["smem"], "B/s")
-        moved = 4.0 * chunk * (tail_share * nnz + head * (N / 128.0))
+        moved = 4.0 * chunk * (tail_share * nnz + head * (N / float(docs_per_block)))
         mma_flops = 2.0 * 2.0 * head * N * chunk        # hi and lo parts, 2 flops per MAC
         extra = {"tail_share_of_updates": tail_share,
                  "l2_bytes_moved_by_design_GBs": moved / launch_s / 1e9,
@@ -439,8 +441,8 @@ def run_ours(args, cfg, rank, local_rank, world):
                         "with the search of the current one)" % len(batches)) +
                        " (codebook resident in HBM; CSR from pinned host memory; results back "
                        "to host)", "matches_device_path": same},
-        "gpu_launches": args.steps * (1 + len(batches) * ({1: 0, 2: 7, 3: 7, 4: 11, 5: 24, 6: 24}[kernel]
-                                                           + n_chunks * (2 if kernel in (5, 6) and
+        "gpu_launches": args.steps * (1 + len(batches) * ({1: 0, 2: 7, 3: 7, 4: 11, 5: 24, 6: 24, 7: 24}[kernel]
+                                                           + n_chunks * (2 if kernel in (5, 6, 7) and
                                                                          opts.repack != 2 and
                                                                          n_chunks > 1 else 1)
                                                            + 1)),
