@@ -86,7 +86,8 @@ typedef struct bmu_opts {
                                slabs, head of 256 or 512, best unit only); 7 the same split
                                with 256 documents per block (128-neuron slabs; the head image
                                is shared by twice as many documents; head_rows 0 = 896;
-                               best unit only; within 2 % of 6 on the benchmark shapes);
+                               best unit only; 1-2 % faster than 6 on the large benchmark
+                               shapes);
                                2 staged (a lane per
                                document, rows streamed through shared memory by tensor (TMA)
                                box copies; needs M % 4 == 0, M >= 32, 256 <= D <= 65024) */
@@ -107,7 +108,7 @@ typedef struct bmu_opts {
     int32_t head_rows;      /* tensor-core sweeps: how many of the most frequent features (ids
                                below this) are summed by the tensor cores: a multiple of 64
                                up to 2048 (kernel 5: 256 or 512); 0 = 768 (kernel 5: 256,
-                               kernel 7: 896) */
+                               kernel 7: 896, half-precision codebook: 512) */
     int32_t repack;         /* tensor-core sweeps: 0/1 gather from a compact [D][chunk] copy
                                of the chunk's columns, made before each launch, 2 gather
                                from the codebook itself */
