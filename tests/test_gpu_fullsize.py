@@ -3,8 +3,9 @@
 The oracle cannot sweep 2,000,000 documents against 262,144 neurons in test
 time, so the full-size run is checked (a) on a seeded sample of documents the
 oracle computes one by one, (b) by properties that hold for every document,
-and (c), on the 64x64 configuration, against an independent full-N
-computation by a library sparse-dense product (test-only code).
+and (c) against an independent computation by a library sparse-dense product (test-only
+code): every document of the 64x64 and 128x128 configurations, a 150,000-document prefix of
+the 512x512 one.
 """
 import numpy as np
 import pytest
@@ -104,18 +105,22 @@ def test_cfg5_one_streamed_batch_sampled(bmu):
         check_sample(W, rowptr, colidx, ob, od, 1500, seed=5 + batch)
 
 
-def test_cfg2_full_size_against_library_product(bmu):
-    cfg = synth.CONFIGS["cfg2"]
+@pytest.mark.parametrize("name,n_check,step", [("cfg2", 0, 50_000), ("cfg3", 0, 20_000),
+                                               ("cfg4", 150_000, 2_048)])
+def test_full_size_against_library_product(bmu, name, n_check, step):
+    """Every document of configs 2 and 3 (and the first 150,000 of config 4's full search)
+    against an independent computation: a library sparse-dense product per document batch, the
+    distance formula and an arg-min in fp64 (test-only code)."""
+    cfg = synth.CONFIGS[name]
     dev = torch.device("cuda")
     W = synth.make_codebook(cfg.D, cfg.M, synth.codebook_seed(cfg), device=dev)
     rowptr, colidx = synth.make_corpus(cfg, device=dev)
-    N = cfg.N
+    N = n_check or cfg.N
     ob, od = bmu.bmu_search(W, rowptr, colidx)
     torch.cuda.synchronize()
-    check_sample(W, rowptr, colidx, ob, od, 3000, seed=2)
+    check_sample(W, rowptr, colidx, ob, od, 3000 if cfg.M <= 16384 else 200, seed=2)
     norms = (W.double() ** 2).sum(0)
     bad_d = bad_j = 0
-    step = 50_000
     for lo in range(0, N, step):
         hi = min(N, lo + step)
         rp = (rowptr[lo:hi + 1] - rowptr[lo]).to(torch.int64)
@@ -123,7 +128,7 @@ def test_cfg2_full_size_against_library_product(bmu):
         X = torch.sparse_csr_tensor(rp, ci, torch.ones(ci.numel(), device=dev),
                                     size=(hi - lo, cfg.D))
         S = (X @ W).double()                                         # library sparse-dense product
-        d = (rp[1:] - rp[:-1]).double()[:, None] + norms[None, :] - 2.0 * S
+        d = S.mul_(-2.0).add_(norms[None, :]).add_((rp[1:] - rp[:-1]).double()[:, None])
         dmin, jmin = d.min(dim=1)
         got_d = od[lo:hi].double()
         got_j = ob[lo:hi].to(torch.int64)
@@ -131,6 +136,7 @@ def test_cfg2_full_size_against_library_product(bmu):
         bad_d += int(((got_d - dmin).abs() > tol).sum())
         d_at = d.gather(1, got_j[:, None])[:, 0]
         bad_j += int(((got_j != jmin) & (d_at > dmin + tol)).sum())
+        del X, S, d
     assert bad_d == 0 and bad_j == 0
 
 
