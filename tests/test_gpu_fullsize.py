@@ -209,3 +209,40 @@ def test_listing_count_next_to_the_32_bit_limit(bmu, M):
         outs.append((ob, od))
     assert float((outs[0][0] == outs[1][0]).float().mean()) > 0.9999      # near-ties aside
     assert float(((outs[0][1] - outs[1][1]).abs() / outs[1][1].abs()).max()) < 1e-6
+
+
+def test_cfg5_whole_corpus_streamed_in_batches_against_library_product(bmu):
+    """Config 5 as it is meant to run: all 27 batches (26.9 M documents) from host memory through
+    bmu_search_batches_host, every document checked against the library sparse-dense product."""
+    cfg = synth.CONFIGS["cfg5"]
+    dev = torch.device("cuda")
+    W = synth.make_codebook(cfg.D, cfg.M, synth.codebook_seed(cfg), device=dev)
+    n_batches = (cfg.N + synth.batch_size(cfg) - 1) // synth.batch_size(cfg)
+    assert n_batches == 27
+    host = []
+    for k in range(n_batches):
+        rp, ci = synth.make_corpus(cfg, batch=k, device=dev)
+        host.append((rp.cpu(), ci.cpu()))
+    assert sum(rp.numel() - 1 for rp, _ in host) == cfg.N
+    outs = bmu.bmu_search_batches_host(W, host)
+    norms = (W.double() ** 2).sum(0)
+    bad_d = bad_j = 0
+    step = 25_000
+    for (rp_h, ci_h), (ob_h, od_h) in zip(host, outs):
+        rowptr, colidx, ob, od = rp_h.to(dev), ci_h.to(dev), ob_h.to(dev), od_h.to(dev)
+        n = rowptr.numel() - 1
+        for lo in range(0, n, step):
+            hi = min(n, lo + step)
+            rp = (rowptr[lo:hi + 1] - rowptr[lo]).to(torch.int64)
+            ci = colidx[int(rowptr[lo]):int(rowptr[hi])].to(torch.int64)
+            X = torch.sparse_csr_tensor(rp, ci, torch.ones(ci.numel(), device=dev),
+                                        size=(hi - lo, cfg.D))
+            S = (X @ W).double()
+            d = S.mul_(-2.0).add_(norms[None, :]).add_((rp[1:] - rp[:-1]).double()[:, None])
+            dmin, jmin = d.min(dim=1)
+            got_j = ob[lo:hi].to(torch.int64)
+            tol = 1e-5 * dmin.abs()
+            bad_d += int(((od[lo:hi].double() - dmin).abs() > tol).sum())
+            bad_j += int(((got_j != jmin) & (d.gather(1, got_j[:, None])[:, 0] > dmin + tol)).sum())
+            del X, S, d
+    assert bad_d == 0 and bad_j == 0
