@@ -325,9 +325,7 @@ sweep_mma2_kernel(const MmaArgs a)
                 // Tensor-memory lane 32q + lane holds neurons 4i + 2h, 4i + 2h + 1 for all 16
                 // documents; lanes l and l ^ 16 swap halves so that each ends up with four
                 // neurons of its own eight documents.
-#ifndef M2_DEBUG_NOWAIT
                 if (it == 0) mm_wait(tfull0 + 8 * buf, (sl >> 1) & 1, abort_flag, a.status, 8u);
-#endif
                 mm_fence_after();
                 uint32_t h0[16], h1[16];
                 const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 256 + dg * 16);
