@@ -395,7 +395,7 @@ def run_ours(args, cfg, rank, local_rank, world):
         # block of 128 documents fetches every distinct row it touches once); what the design
         # really moves is the tail's rows per document plus the head image per block.
         head = opts.head_rows or (256 if kernel == 5 else
-                                  min(896 if kernel == 7 else 768, cfg.D // 64 * 64))
+                                  min(896 if kernel == 7 else 640, cfg.D // 64 * 64))
         tail_share = float((colidx >= head).sum().item()) / max(1, colidx.numel())
         alg["alu"] = (tail_share * adds / launch_s, roofs["fadd2"], "add/s")
         alg["l1"] = (4.0 * tail_share * adds / launch_s, roofs["smem"], "B/s")
@@ -492,16 +492,19 @@ def f16_codebook(bmu, cfg, W, rowptr, colidx, args):
     n16 = bmu.bmu_codebook_norms_f16(W16)
     n0, nnz = rowptr.numel() - 1, colidx.numel()
     D, M = W16.shape
-    need = int(bmu.load().bmu_search_f16_workspace_bytes(D, M, n0, nnz, None))
+    o16 = bmu.Opts()
+    o16.head_rows = args.f16_head
+    import ctypes
+    need = int(bmu.load().bmu_search_f16_workspace_bytes(D, M, n0, nnz, ctypes.byref(o16)))
     ws = torch.empty(need + 256, dtype=torch.uint8, device=W.device)
     for _ in range(max(1, args.warmup)):
-        bmu.bmu_search_f16_ws(W16, rowptr, colidx, norms=n16, workspace=ws)
+        bmu.bmu_search_f16_ws(W16, rowptr, colidx, norms=n16, opts=o16, workspace=ws)
     torch.cuda.synchronize(W.device)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
         bmu.bmu_codebook_norms_f16(W16)
-        bmu.bmu_search_f16_ws(W16, rowptr, colidx, norms=n16, workspace=ws)
+        bmu.bmu_search_f16_ws(W16, rowptr, colidx, norms=n16, opts=o16, workspace=ws)
     e1.record()
     torch.cuda.synchronize(W.device)
     ms = e0.elapsed_time(e1) / args.steps
@@ -630,6 +633,7 @@ def main():
                     help="also time the materialised-score route (library SpMM + argmin)")
     ap.add_argument("--f16", action="store_true",
                     help="also time the same sweep on the codebook rounded to fp16 (the paper's storage)")
+    ap.add_argument("--f16-head", type=int, default=0, help="head_rows of the --f16 sweep (0 = default)")
     ap.add_argument("--epoch", action="store_true",
                     help="also time one whole epoch (search + scatter + blur + write-back)")
     ap.add_argument("--sigma", type=float, default=2.0, help="neighbourhood width of --epoch")

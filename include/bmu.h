@@ -107,8 +107,8 @@ typedef struct bmu_opts {
                                densely, one load per tile, 1 treat them like all other ids */
     int32_t head_rows;      /* tensor-core sweeps: how many of the most frequent features (ids
                                below this) are summed by the tensor cores: a multiple of 64
-                               up to 2048 (kernel 5: 256 or 512); 0 = 768 (kernel 5: 256,
-                               kernel 7: 896, half-precision codebook: 512) */
+                               up to 2048 (kernel 5: 256 or 512); 0 = 640 (kernel 5: 256,
+                               kernel 7: 896, half-precision codebook: 576) */
     int32_t repack;         /* tensor-core sweeps: 0/1 gather from a compact [D][chunk] copy
                                of the chunk's columns, made before each launch, 2 gather
                                from the codebook itself */
@@ -215,7 +215,7 @@ BMU_API int bmu_search_top2_ws(const float *W, int64_t D, int64_t M, const float
  * planned kernel, 6 the wide tensor-core sweep (needs M % 512 == 0 and D >=
  * head_rows; the weights being fp16 already, its head image has one part), 0
  * the tensor-core sweep for large sweeps, else the planned kernel; head_rows
- * defaults to 512 here.  Workspace: bmu_search_f16_workspace_bytes(...) with the
+ * defaults to 576 here.  Workspace: bmu_search_f16_workspace_bytes(...) with the
  * same sizes and options (enough with or without the second-best outputs).
  */
 BMU_API size_t bmu_search_f16_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,

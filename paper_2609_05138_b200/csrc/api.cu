@@ -92,13 +92,15 @@ repack_chunk_kernel(const char *__restrict__ W, int64_t pitch_bytes, int64_t off
     for (int i = threadIdx.x; i < width_bytes / 16; i += 256) dst[i] = __ldcs(src + i);
 }
 
-// Features summed on the tensor cores: 256 for the first tensor-core sweep; 768 for the wide
-// one (measured best of 512 .. 1024 on configs 2-5), less if the vocabulary is smaller.
+// Features summed on the tensor cores: 256 for the first tensor-core sweep; 640 for the wide
+// one (measured best of 512 .. 1024 on configs 2-5 in full-length runs, where the board sits at
+// its power cap: 768 wins short runs at boost clocks and loses 1-2 % once the cap binds), less
+// if the vocabulary is smaller.
 static int mma_head_rows(const bmu_opts &o, int64_t D)
 {
     if (o.head_rows) return o.head_rows;
     if (o.kernel == 5) return MMA_HEAD;
-    const int64_t cap = D / 64 * 64, want = o.kernel == 7 ? 896 : 768;
+    const int64_t cap = D / 64 * 64, want = o.kernel == 7 ? 896 : 640;
     return (int)(cap < want ? (cap < 64 ? 64 : cap) : want);
 }
 
@@ -576,15 +578,16 @@ int bmu_codebook_norms_f16(const void *W16, int64_t D, int64_t M, float *norms, 
 
 // Which kernel a half-precision search takes: large sweeps the wide tensor-core sweep (whole
 // 512-neuron slabs only), the rest the planned kernel.  `ow` = the options of the wide sweep, its
-// head resolved (512 by default: with 2-byte rows the gathered tail is cheap, so the balance
-// point sits lower than the fp32 sweep's 768).
+// head resolved (576 by default: with 2-byte rows the gathered tail is cheap, so the balance
+// point sits lower than the fp32 sweep's 640; config 4 at full length: 2364 / 2348 / 2331 / 2473
+// ms per step at 448 / 512 / 576 / 704).
 static bool f16_route(const bmu_opts &o, int64_t D, int64_t M, int64_t nnz, bmu_opts &ow, bool &wide)
 {
     ow = o;
     ow.kernel = 6;
     if (!ow.head_rows) {
         const int64_t cap = D / 64 * 64;
-        ow.head_rows = (int32_t)(cap < 512 ? (cap < 64 ? 64 : cap) : 512);
+        ow.head_rows = (int32_t)(cap < 576 ? (cap < 64 ? 64 : cap) : 576);
     }
     const bool wide_ok = M % MMA_SLAB == 0 && D >= ow.head_rows && o.cluster != 2;
     wide = wide_ok && (o.kernel == 6 || (o.kernel == 0 && (double)nnz * (double)M >= 2e10));
