@@ -152,7 +152,7 @@ static int check_sizes(int64_t D, int64_t M, int64_t N, int64_t nnz)
 
 static int check_opts(const bmu_opts &o)
 {
-    if (o.tile_order < 0 || o.tile_order > 1) { set_error("bmu_opts.tile_order must be 0 or 1"); return BMU_ERR_INVALID_ARG; }
+    if (o.tile_order < 0 || o.tile_order > 2) { set_error("bmu_opts.tile_order must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
     if (o.tile_head < 0 || o.tile_head > 1) { set_error("bmu_opts.tile_head must be 0 or 1"); return BMU_ERR_INVALID_ARG; }
     if (o.head_rows < 0 || o.head_rows > HEAD_ROWS_MAX || o.head_rows % 64 != 0 ||
         (o.kernel == 5 && o.head_rows != 0 && o.head_rows != 256 && o.head_rows != 512)) {
@@ -283,7 +283,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
             return rc;
     if (mma) {
         if (phase != 2 &&
-            (rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, relabel, pw, l.plan, s)))
+            (rc = launch_plan_tiles(rowptr, N, o.tile_order == 2, head, relabel, pw, l.plan, s)))
             return rc;
         if (phase == 1) return BMU_OK;
         const int64_t m_full = M / MMA_SLAB * MMA_SLAB;
@@ -659,7 +659,7 @@ int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
         char *pw = base + l.plan_off;
         const int relabel = o.relabel;
         if ((rc = launch_plan(rowptr, colidx, N, nnz, 1, head, relabel, D, pw, l.plan, s))) return rc;
-        if ((rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, relabel, pw, l.plan, s))) return rc;
+        if ((rc = launch_plan_tiles(rowptr, N, o.tile_order == 2, head, relabel, pw, l.plan, s))) return rc;
         unsigned char *img = reinterpret_cast<unsigned char *>(base + l.head_off);
         const uint16_t *feat = (relabel != 2 && l.plan.fsort_tmp_bytes > 0)
                                    ? reinterpret_cast<const uint16_t *>(pw + l.plan.feat_off) : nullptr;

@@ -83,7 +83,7 @@ def draw_opts(bmu, rng, kernel):
         o.relabel = rng.choice([0, 1, 2])
         o.repack = rng.choice([0, 2])
     if kernel in (4, 5, 6, 7):
-        o.tile_order = rng.choice([0, 1])
+        o.tile_order = rng.choice([0, 1, 2])
     return o
 
 
