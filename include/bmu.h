@@ -75,48 +75,39 @@ typedef struct bmu_opts {
                                4 tiled (a warp carries 8 documents; frequent rows loaded once
                                per tile; the warps of a block walk the feature axis in step
                                so that L1 serves the rows they share; needs what 3 needs and
-                               length-ordered documents); 6 wide tensor-core head (the sum over
-                               the head_rows most frequent features -- ids below head_rows:
-                               the paper keeps its vocabulary frequency-ordered, Table 8 --
-                               is a dense contraction on tcgen05 tensor cores with fp32
-                               accumulation into double-buffered tensor memory, the
-                               remaining ids are gathered as in 4; needs what 4 needs,
-                               D >= head_rows and M >= 512; the automatic choice for large
-                               sweeps); 5 first tensor-core sweep (same split, 512-neuron
-                               slabs, head of 256 or 512, best unit only); 7 the same split
-                               with 256 documents per block (128-neuron slabs; the head image
-                               is shared by twice as many documents; head_rows 0 = 896;
-                               best unit only; 1-2 % faster than 6 on the large benchmark
-                               shapes);
-                               2 staged (a lane per
-                               document, rows streamed through shared memory by tensor (TMA)
-                               box copies; needs M % 4 == 0, M >= 32, 256 <= D <= 65024) */
+                               length-ordered documents); 6 tensor-core head (the sum over
+                               the head_rows most frequent features is a dense contraction
+                               on tcgen05 tensor cores with fp32 accumulation into
+                               double-buffered tensor memory, the remaining ids are gathered
+                               as in 4; needs what 4 needs, D >= head_rows and M >= 512; the
+                               automatic choice for large sweeps).  Other values are
+                               refused. */
     int32_t chunk_neurons;  /* neurons per L2-resident chunk of the codebook (Section 4.2,
                                "neuron-axis chunking"); rounded to the slab width */
     int32_t vec;            /* warp-per-document kernels: floats per lane per row, 4 or 8 */
     int32_t docs_per_warp;  /* generic kernel: documents a warp carries through one slab */
     int32_t warps;          /* warp-per-document kernels: warps per thread block */
-    int32_t cluster;        /* staged kernel, tile membership (Section 4.2): 0/1 order the
-                               documents by length before cutting tiles, so that the lanes
-                               of a warp carry similar rows; 2 keep the corpus order */
-    int32_t stage_rows;     /* staged kernel: codebook rows per pipeline stage (256) */
-    int32_t stages;         /* staged kernel: pipeline depth, a power of two (4) */
+    int32_t cluster;        /* tile membership (Section 4.2): 0/1 order the documents by
+                               length before cutting tiles, so that the documents of a tile
+                               finish together; 2 keep the corpus order (generic and planned
+                               kernels only) */
+    int32_t stage_rows;     /* unused, must be 0 */
+    int32_t stages;         /* unused, must be 0 */
     int32_t tile_order;     /* order of the gathered ids inside a tile: 1 ascending; 2 dealt
                                alternately from the frequent and the rare half of each list
                                (so that a warp mixes loads that hit L1 with loads that go to
-                               L2); 0 = 2 for the tiled kernel, 1 for the tensor-core sweeps
-                               (their dense head has taken the frequent ids already; ascending
+                               L2); 0 = 2 for the tiled kernel, 1 for the tensor-core sweep
+                               (its dense head has taken the frequent ids already; ascending
                                measured 0.7 % faster on config 4) */
     int32_t tile_head;      /* tiled kernel: 0 sweep the 32 most frequent features (ids < 32)
                                densely, one load per tile, 1 treat them like all other ids */
-    int32_t head_rows;      /* tensor-core sweeps: how many of the most frequent features (ids
-                               below this) are summed by the tensor cores: a multiple of 64
-                               up to 2048 (kernel 5: 256 or 512); 0 = 640 (kernel 5: 256,
-                               kernel 7: 896, half-precision codebook: 576) */
-    int32_t repack;         /* tensor-core sweeps: 0/1 gather from a compact [D][chunk] copy
+    int32_t head_rows;      /* tensor-core sweep: how many of the most frequent features
+                               are summed by the tensor cores: a multiple of 64 up to 2048;
+                               0 = 640 (half-precision codebook: 576) */
+    int32_t repack;         /* tensor-core sweep: 0/1 gather from a compact [D][chunk] copy
                                of the chunk's columns, made before each launch, 2 gather
                                from the codebook itself */
-    int32_t relabel;        /* tensor-core sweeps: which features form the dense head.
+    int32_t relabel;        /* tensor-core sweep: which features form the dense head.
                                1 the head_rows features listed by the most documents of
                                this corpus (ranked inside the tiling pass; the caller's ids
                                stay as they are); 2 the ids below head_rows (a vocabulary
@@ -143,7 +134,7 @@ BMU_API int bmu_codebook_norms(const float *W, int64_t D, int64_t M, float *norm
  * Scratch bytes bmu_search_ws needs for a problem of this size (norms, the
  * per-document running minimum merged across neuron chunks, the tiling plan,
  * the split image of the frequent rows (4 * head_rows bytes per neuron) and the
- * compact chunk copy of the tensor-core sweeps).  `nnz` is the length of colidx.
+ * compact chunk copy of the tensor-core sweep).  `nnz` is the length of colidx.
  */
 BMU_API size_t bmu_search_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,
                                   const bmu_opts *opts);
@@ -156,9 +147,8 @@ BMU_API size_t bmu_search_workspace_bytes(int64_t D, int64_t M, int64_t N, int64
  * 256-byte aligned device memory of at least bmu_search_workspace_bytes(...)
  * bytes; its contents are undefined afterwards, except that its first 32-bit
  * word is a status word: 0 after a clean run, non-zero if a bounded device-side
- * wait of the staged kernel or of the tensor-core sweep ran out (results are
- * then invalid).  Allocates
- * nothing.  Calls that share a workspace must not overlap on the GPU.
+ * wait of the tensor-core sweep ran out or a size check of the tiling pass
+ * failed (results are then invalid).  Allocates nothing.  Calls that share a workspace must not overlap on the GPU.
  */
 BMU_API int bmu_search_ws(const float *W, int64_t D, int64_t M, const float *norms,
                   const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
@@ -198,8 +188,7 @@ BMU_API void bmu_plan_destroy(bmu_plan *plan);
  * kernel tracks because topographic error -- gated on by its stopping rules --
  * needs it (Table 5, "bmu1-only").  out_bmu2[i] is the lowest index j !=
  * out_bmu[i] attaining the second-smallest distance, out_dist2[i] that distance
- * (-1 and +inf when M == 1).  Same tie rule, same options (the staged kernel
- * does not support it), workspace of bmu_search_top2_workspace_bytes(...).
+ * (-1 and +inf when M == 1).  Same tie rule, same options, workspace of bmu_search_top2_workspace_bytes(...).
  */
 BMU_API size_t bmu_search_top2_workspace_bytes(int64_t D, int64_t M, int64_t N, int64_t nnz,
                                                const bmu_opts *opts);
@@ -274,8 +263,8 @@ BMU_API int bmu_search_batches_host(const float *W, int64_t D, int64_t M, int32_
                                     void *stream);
 
 /*
- * Self-test of the failure path of device-side waits.  The staged kernel's
- * producer and consumers wait on shared-memory barriers; every such wait has an
+ * Self-test of the failure path of device-side waits.  The tensor-core sweep's
+ * producer, MMA issuer and tail warps wait on shared-memory barriers; every such wait has an
  * iteration limit, after which the kernel records a status word and returns
  * instead of trapping or spinning forever.  This call runs a one-block kernel
  * that waits (limit: 4096 polls) on a barrier nothing ever arrives on and hands

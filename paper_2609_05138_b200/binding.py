@@ -119,15 +119,18 @@ EXPORTS = {
 }
 
 
-def load():
-    """Loads libbmu.so (raises if it has not been built)."""
+def load(path: str | None = None):
+    """Loads libbmu.so (raises if it has not been built).  `path` (or the environment
+    variable BMU_LIBRARY) names another build of the same library, e.g. the bounds-checked
+    one; it must be given on the first call, the library is loaded once per process."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
+        path = path or os.environ.get("BMU_LIBRARY") or LIB_PATH
+        if not os.path.exists(path):
             raise ImportError(
-                "libbmu.so is not built: run `python -m paper_2609_05138_b200.build` "
-                "(there is no CPU fallback)")
-        lib = ctypes.CDLL(LIB_PATH)
+                "%s is not built: run `python -m paper_2609_05138_b200.build` "
+                "(there is no CPU fallback)" % path)
+        lib = ctypes.CDLL(path)
         for name, (res, args) in EXPORTS.items():
             fn = getattr(lib, name)
             fn.restype, fn.argtypes = res, args

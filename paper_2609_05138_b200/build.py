@@ -1,19 +1,28 @@
-"""Builds libbmu.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a."""
+"""Builds libbmu.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
+
+Every .cu file is compiled to an object of its own (in parallel, re-compiled
+only when it or a header is newer) and the objects are linked into the shared
+library.  `extra_flags` / `out` / `objdir` give a second build beside the
+default one, e.g. the bounds-checked build (-DBMU_BOUNDS_CHECK).
+"""
 from __future__ import annotations
 
 import glob
 import os
 import subprocess
 import sys
+import zlib
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbmu.so")
+OBJDIR = os.path.join(HERE, "build")
 
-NVCC_FLAGS = [*os.environ.get("BMU_EXTRA_NVCC", "").split(),
+NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--use_fast_math=false",
+    "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",
 ]
 
 
@@ -26,27 +35,44 @@ def headers():
         sorted(glob.glob(os.path.join(ROOT, "include", "*.h")))
 
 
-def up_to_date() -> bool:
-    if not os.path.exists(LIB):
+def up_to_date(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return False
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     return all(os.path.getmtime(p) <= t for p in sources() + headers())
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    if not force and up_to_date():
-        return LIB
+def build_library(force: bool = False, verbose: bool = False, extra_flags=(), out: str = LIB,
+                  objdir: str = OBJDIR) -> str:
+    extra = [*os.environ.get("BMU_EXTRA_NVCC", "").split(), *extra_flags]
+    if not force and not extra and up_to_date(out):
+        return out
     nvcc = os.environ.get("NVCC", "nvcc")
-    flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
+    flags = [*extra, *NVCC_FLAGS]
+    if extra:                             # objects of another flag set live apart
+        objdir = os.path.join(objdir, "x%08x" % (zlib.crc32(" ".join(extra).encode()) & 0xffffffff))
     if verbose:
         flags += ["-Xptxas", "-v"]
-    tmp = LIB + ".tmp%d" % os.getpid()
-    cmd = [nvcc, *flags, "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           *sources(), "-o", tmp]
-    subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
-    return LIB
+    os.makedirs(objdir, exist_ok=True)
+    newest_header = max(os.path.getmtime(p) for p in headers())
+
+    def compile_one(src):
+        obj = os.path.join(objdir, os.path.basename(src)[:-3] + ".o")
+        if (not force and not verbose and os.path.exists(obj)
+                and os.path.getmtime(obj) >= max(os.path.getmtime(src), newest_header)):
+            return obj
+        subprocess.check_call([nvcc, *flags, "-I", os.path.join(ROOT, "include"), "-I", CSRC,
+                               "-c", src, "-o", obj])
+        return obj
+
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+        objs = list(pool.map(compile_one, sources()))
+    tmp = out + ".tmp%d" % os.getpid()
+    subprocess.check_call([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a",
+                           *objs, "-o", tmp])
+    os.replace(tmp, out)
+    return out
 
 
 if __name__ == "__main__":
-    print(build_library(force=True, verbose="-v" in sys.argv))
+    print(build_library(force="-f" in sys.argv or "-v" in sys.argv, verbose="-v" in sys.argv))

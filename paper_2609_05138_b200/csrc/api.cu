@@ -37,14 +37,6 @@ struct Layout {
     PlanLayout plan;
 };
 
-// The staged kernel needs 16-bit feature ids, whole 16-byte row segments and
-// boxes that fit inside the codebook; everything else takes the direct kernel.
-static bool staged_possible(const float *W, int64_t D, int64_t M)
-{
-    return M % 4 == 0 && M >= 32 && D >= 256 && D <= LANES_MAX_D &&
-           (reinterpret_cast<uintptr_t>(W) & 15) == 0;
-}
-
 // Neurons per launch of the tensor-core sweep: whole 512-neuron slabs whose rows take a little
 // over half of L2 (1024 neurons at D = 16384 on a 126 MB L2; measured best there, 512 and 2048
 // within 2 %).
@@ -73,8 +65,7 @@ static int64_t mma_chunk(const bmu_opts &o, int64_t D, int64_t M)
 static size_t mma_repack_bytes(const bmu_opts &o, int64_t D, int64_t M, int64_t N, int64_t nnz,
                                bool top2)
 {
-    if (o.repack == 2 || (top2 && o.kernel == 5) ||
-        (o.kernel != 0 && o.kernel != 5 && o.kernel != 6 && o.kernel != 7)) return 0;
+    if (o.repack == 2 || (o.kernel != 0 && o.kernel != 6)) return 0;
     if (D > LANES_MAX_D || M < MMA_SLAB) return 0;
     const int64_t chunk = mma_chunk(o, D, M);
     if (M <= chunk) return 0;                      // one launch: the codebook is the chunk
@@ -92,20 +83,18 @@ repack_chunk_kernel(const char *__restrict__ W, int64_t pitch_bytes, int64_t off
     for (int i = threadIdx.x; i < width_bytes / 16; i += 256) dst[i] = __ldcs(src + i);
 }
 
-// Features summed on the tensor cores: 256 for the first tensor-core sweep; 640 for the wide
-// one (measured best of 512 .. 1024 on configs 2-5 in full-length runs, where the board sits at
-// its power cap: 768 wins short runs at boost clocks and loses 1-2 % once the cap binds), less
-// if the vocabulary is smaller.
+// Features summed on the tensor cores: 640 (measured best of 512 .. 1024 on configs 2-5 in
+// full-length runs, where the board sits at its power cap: 768 wins short runs at boost clocks
+// and loses 1-2 % once the cap binds), less if the vocabulary is smaller.
 static int mma_head_rows(const bmu_opts &o, int64_t D)
 {
     if (o.head_rows) return o.head_rows;
-    if (o.kernel == 5) return MMA_HEAD;
-    const int64_t cap = D / 64 * 64, want = o.kernel == 7 ? 896 : 640;
+    const int64_t cap = D / 64 * 64, want = 640;
     return (int)(cap < want ? (cap < 64 ? 64 : cap) : want);
 }
 
 static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kernel,
-                         bool top2 = false, int head = MMA_HEAD, size_t repack_bytes = 0)
+                         bool top2 = false, int head = 640, size_t repack_bytes = 0)
 {
     Layout l;
     size_t off = 0;
@@ -116,9 +105,7 @@ static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kerne
     if (top2) off = align_up(off + (size_t)N * sizeof(u64), 256);
     // split image of the frequent rows for the tensor-core sweep (it may be the automatic choice)
     l.head_off = off;
-    if (kernel == 5 && !top2 && D >= head && D <= LANES_MAX_D && M >= MMA_SLAB)
-        off = align_up(off + head_image_bytes(M, head), 256);
-    if ((kernel == 0 || kernel == 6 || kernel == 7) && D >= head && D <= LANES_MAX_D && M >= MMA_SLAB)
+    if ((kernel == 0 || kernel == 6) && D >= head && D <= LANES_MAX_D && M >= MMA_SLAB)
         off = align_up(off + head_image2_bytes(M, head), 256);
     l.repack_off = off;                  // compact copy of the codebook chunk being swept
     off = align_up(off + repack_bytes, 256);
@@ -154,16 +141,22 @@ static int check_opts(const bmu_opts &o)
 {
     if (o.tile_order < 0 || o.tile_order > 2) { set_error("bmu_opts.tile_order must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
     if (o.tile_head < 0 || o.tile_head > 1) { set_error("bmu_opts.tile_head must be 0 or 1"); return BMU_ERR_INVALID_ARG; }
-    if (o.head_rows < 0 || o.head_rows > HEAD_ROWS_MAX || o.head_rows % 64 != 0 ||
-        (o.kernel == 5 && o.head_rows != 0 && o.head_rows != 256 && o.head_rows != 512)) {
-        set_error("bmu_opts.head_rows must be 0 or a multiple of 64 up to %d (kernel 5: 256 or 512)", HEAD_ROWS_MAX);
+    if (o.head_rows < 0 || o.head_rows > HEAD_ROWS_MAX || o.head_rows % 64 != 0) {
+        set_error("bmu_opts.head_rows must be 0 or a multiple of 64 up to %d", HEAD_ROWS_MAX);
         return BMU_ERR_INVALID_ARG;
     }
     if (o.repack < 0 || o.repack > 2) { set_error("bmu_opts.repack must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
     if (o.relabel < 0 || o.relabel > 2) { set_error("bmu_opts.relabel must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
     for (int i = 0; i < 3; ++i)
         if (o.reserved[i] != 0) { set_error("bmu_opts.reserved must be zero"); return BMU_ERR_INVALID_ARG; }
-    if (o.kernel < 0 || o.kernel > 7) { set_error("bmu_opts.kernel must be 0 .. 7"); return BMU_ERR_INVALID_ARG; }
+    if (o.kernel != 0 && o.kernel != 1 && o.kernel != 3 && o.kernel != 4 && o.kernel != 6) {
+        set_error("bmu_opts.kernel must be 0, 1, 3, 4 or 6");
+        return BMU_ERR_INVALID_ARG;
+    }
+    if (o.stage_rows != 0 || o.stages != 0) {
+        set_error("bmu_opts.stage_rows and bmu_opts.stages must be zero");
+        return BMU_ERR_INVALID_ARG;
+    }
     if (o.cluster < 0 || o.cluster > 2) { set_error("bmu_opts.cluster must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
     if (o.chunk_neurons < 0) { set_error("bmu_opts.chunk_neurons < 0"); return BMU_ERR_INVALID_ARG; }
     if (o.vec != 0 && o.vec != 4 && o.vec != 8) { set_error("bmu_opts.vec must be 0, 4 or 8"); return BMU_ERR_INVALID_ARG; }
@@ -235,16 +228,6 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     }
     uint32_t *status = reinterpret_cast<uint32_t *>(base + l.status_off);
     BMU_CUDA(cudaMemsetAsync(status, 0, 256, s));
-    const bool staged = o.kernel == 2;
-    if (staged && top2) {
-        set_error("the staged kernel does not track the second-best unit");
-        return BMU_ERR_UNSUPPORTED;
-    }
-    if (staged && !staged_possible(reinterpret_cast<const float *>(w_addr), D, M)) {
-        set_error("staged kernel needs M %% 4 == 0, M >= 32, 256 <= D <= %d and W 16-byte aligned",
-                  LANES_MAX_D);
-        return BMU_ERR_UNSUPPORTED;
-    }
     // the planned warp-per-document kernel needs 16-bit ids and whole 16-byte row pieces
     const bool planned_ok = D <= LANES_MAX_D && M % 4 == 0 && M >= rows_slab_width(o) &&
                             (w_addr & 15) == 0;
@@ -254,19 +237,17 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         return BMU_ERR_UNSUPPORTED;
     }
     const bool tiled_ok = planned_ok && M >= 128 && o.cluster != 2;
-    // tensor-core head: additionally whole 512-neuron slabs, at least 256 features, best unit only
-    const bool mma_ok = tiled_ok && !(top2 && (o.kernel == 5 || o.kernel == 7)) && D >= head &&
-                        M >= MMA_SLAB;
-    if ((o.kernel == 5 || o.kernel == 6 || o.kernel == 7) && !mma_ok) {
-        set_error("tensor-core sweep needs what the tiled kernel needs, D >= %d and M >= %d "
-                  "(kernel 5: no second-best unit)", head, MMA_SLAB);
+    // tensor-core head: additionally at least one whole 512-neuron slab and `head` features
+    const bool mma_ok = tiled_ok && D >= head && M >= MMA_SLAB;
+    if (o.kernel == 6 && !mma_ok) {
+        set_error("tensor-core sweep needs what the tiled kernel needs, D >= %d and M >= %d",
+                  head, MMA_SLAB);
         return BMU_ERR_UNSUPPORTED;
     }
     // automatic choice for large sweeps: the tensor-core sweep where it applies, else the tiled
     // kernel; both repay their extra preparation only when there is enough to sweep
     const bool big = (double)nnz * (double)M >= 2e10;
-    const bool mma = o.kernel == 5 || o.kernel == 6 || o.kernel == 7 || (o.kernel == 0 && mma_ok && big);
-    const bool wide = o.kernel != 5;
+    const bool mma = o.kernel == 6 || (o.kernel == 0 && mma_ok && big);
     const bool tiled = !mma && (o.kernel == 4 || (o.kernel == 0 && tiled_ok && big));
     if (tiled && !tiled_ok) {
         set_error("tiled kernel needs M %% 4 == 0, M >= 128, D <= %d, W 16-byte aligned and "
@@ -277,7 +258,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     char *pw = base + l.plan_off;
     // dense head = the most frequent features by the corpus's own counts (bmu_opts.relabel)
     const int relabel = mma ? o.relabel : 2;        // 0 decide from the counts, 1 always, 2 never
-    if ((staged || planned || tiled || mma) && phase != 2)
+    if ((planned || tiled || mma) && phase != 2)
         if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, mma ? head : 0, relabel, D, pw,
                               l.plan, s)))
             return rc;
@@ -291,9 +272,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         unsigned char *img = reinterpret_cast<unsigned char *>(base + l.head_off);
         const uint16_t *feat = (relabel != 2 && l.plan.fsort_tmp_bytes > 0)
                                    ? reinterpret_cast<const uint16_t *>(pw + l.plan.feat_off) : nullptr;
-        if ((rc = o.kernel == 7 ? launch_head_split3(W, M, m_full, head, feat, head_max, img, s)
-                  : wide ? launch_head_split2(W, M, m_full, head, feat, head_max, img, s)
-                         : launch_head_split(W, M, m_full, head, feat, head_max, img, s))) return rc;
+        if ((rc = launch_head_split2(W, M, m_full, head, feat, head_max, img, s))) return rc;
         MmaArgs a;
         a.W = W; a.M = M; a.N = N; a.n_tiles = (N + 7) / 8; a.norms = norms;
         a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
@@ -318,10 +297,9 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
                                                       (uintptr_t)j * sizeof(float));
                 a.M = width;
             }
-            // both images take 4 * head bytes per neuron, slab after slab
+            // the image takes 4 * head bytes per neuron, slab after slab
             a.head_img = img + (size_t)j * head * 4;
-            if ((rc = o.kernel == 7 ? launch_sweep_mma3(a, o, s)
-                      : wide ? launch_sweep_mma2(a, o, s) : launch_sweep_mma(a, o, s))) return rc;
+            if ((rc = launch_sweep_mma2(a, o, s))) return rc;
         }
         if (m_full < M) {                      // ragged last slab: generic kernel, merged in
             SweepArgs g;
@@ -395,25 +373,6 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
             if ((rc = launch_sweep_direct(g, go, s))) return rc;
         }
         return launch_finalize(state, state2, rowptr, N, out_bmu, out_dist, out_bmu2, out_dist2, s);
-    }
-    if (staged) {
-        alignas(64) unsigned char tmap[128];
-        if ((rc = make_codebook_tensor_map(W, D, M, o.stage_rows ? o.stage_rows : 256, tmap)))
-            return rc;
-        LanesArgs a;
-        a.norms = norms;
-        a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
-        a.doc_off = reinterpret_cast<const uint32_t *>(pw + l.plan.docoff_off);
-        a.ids = reinterpret_cast<const uint4 *>(pw + l.plan.ids_off);
-        a.N = N; a.M = M; a.D = (int32_t)D; a.state = state; a.status = status;
-        int64_t chunk = o.chunk_neurons ? (o.chunk_neurons + 31) / 32 * 32 : auto_chunk(D, M, 32);
-        for (int64_t j = 0; j < M; j += chunk) {
-            a.j_lo = (int32_t)j;
-            a.j_hi = (int32_t)(j + chunk < M ? j + chunk : M);
-            a.first = j == 0;
-            if ((rc = launch_sweep_lanes(tmap, a, o, s))) return rc;
-        }
-        return launch_finalize(state, nullptr, rowptr, N, out_bmu, out_dist, nullptr, nullptr, s);
     }
     const int V = o.vec ? o.vec : 4;
     const int slab = 32 * V;

@@ -76,16 +76,6 @@ struct Best {
             d2 = d; j2 = j;
         }
     }
-    // any order of j (staged kernel): full lexicographic test
-    __device__ __forceinline__ void push_any(float d, int j)
-    {
-        if (d < d1 || (d == d1 && j < j1)) {
-            if (TOP2) { d2 = d1; j2 = j1; }
-            d1 = d; j1 = j;
-        } else if (TOP2 && (d < d2 || (d == d2 && j < j2))) {
-            d2 = d; j2 = j;
-        }
-    }
     static __device__ __forceinline__ void merge(u64 &a1, u64 &a2, u64 b1, u64 b2)
     {
         const u64 lo = a1 < b1 ? a1 : b1, mid = a1 < b1 ? b1 : a1;
@@ -151,7 +141,7 @@ int launch_sweep_direct(const SweepArgs &a, const bmu_opts &o, cudaStream_t s);
 int launch_finalize(const u64 *state, const u64 *state2, const int32_t *rowptr, int64_t N,
                     int32_t *out_bmu, float *out_dist, int32_t *out_bmu2, float *out_dist2,
                     cudaStream_t s);
-// ---- tiling plan (plan.cu) and staged sweep (sweep_lanes.cu) ---------------
+// ---- tiling plan (plan.cu) ---------------------------------------------------
 struct PlanLayout {
     size_t perm_off, docoff_off, ngroups_off, bins_off, ids_off, scan_off, scan_bytes, total;
     size_t tilelen_off, tilerows_off, tileoff_off, tilehead_off, tileids_off, tile_rows_cap;
@@ -179,15 +169,11 @@ struct TileArgs {
 };
 int launch_sweep_tiles(const TileArgs &a, const bmu_opts &o, cudaStream_t s);
 
-// tensor-core head + gathered tail (sweep_mma.cu): a block carries 128 documents through
-// slabs of 512 neurons
-static const int MMA_HEAD = 256;         // features (ids below this) summed on the tensor cores:
-static const int MMA_HEAD_MAX = 512;     // 256 by default, 512 on request (bmu_opts.head_rows)
-static const int MMA_SLAB = 512;         // neurons per slab
+// tensor-core head + gathered tail (sweep_mma2.cu, sweep_mma2_f16.cu): a block carries 128
+// documents through slabs of 256 neurons; launches cover whole multiples of MMA_SLAB neurons
+static const int MMA_SLAB = 512;         // granularity of a launch's neuron range
 static const int MMA_DOCS = 128;         // documents per block
 static const size_t MMA_STAGE_BYTES = 16384;                  // 128 neurons x 64 features x fp16
-// stages per slab: 4 tiles x (hi, lo) x blocks of 64 features
-static inline int mma_stages_per_slab(int head) { return 4 * 2 * (head / 64); }
 struct MmaArgs {
     const float *W;
     int64_t M, N, n_tiles;
@@ -196,26 +182,21 @@ struct MmaArgs {
     const uint32_t *tile_len;
     const uint32_t *tile_off;
     const uint4 *tile_ids;
-    int32_t head;               // 256 or 512
+    int32_t head;               // features summed on the tensor cores (a multiple of 64)
     const uint32_t *tile_head;  // head / 32 mask words per planned document
-    const unsigned char *head_img;  // split head of slab j_lo / MMA_SLAB onwards (head_image_bytes)
+    const unsigned char *head_img;  // split head of slab j_lo / 256 onwards (head_image2_bytes)
     const uint32_t *head_max;   // bit pattern of max |W[f][j]| over the head rows
     u64 *state;
-    u64 *state2;                // wide-head sweep only: second-best unit (NULL unless wanted)
+    u64 *state2;                // second-best unit (NULL unless wanted)
     uint32_t *status;           // set non-zero if a bounded wait ran out
     int32_t j_lo, j_hi, first;
-    int32_t f16;                // wide-head sweep only: W is an fp16 codebook (row pitch 2 * M bytes)
+    int32_t f16;                // W is an fp16 codebook (row pitch 2 * M bytes)
 };
-size_t head_image_bytes(int64_t M, int head);
-// writes the fp16 (hi, lo) split of rows [0, head) of W, scaled by a power of two, as the
-// shared-memory images the tensor-core sweep copies; whole slabs of [0, m_full) only
 // `feat` (may be NULL = identity): the feature whose row of W is head row r
 int launch_head_absmax(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
                        uint32_t *head_max, cudaStream_t s);
-int launch_head_split(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
-                      uint32_t *head_max, unsigned char *head_img, cudaStream_t s);
-int launch_sweep_mma(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
-// wide-head variant (sweep_mma2.cu): 256-neuron slabs, head of 64 .. HEAD_ROWS_MAX features
+// writes the fp16 (hi, lo) split of the `head` most frequent rows of W, scaled by a power of
+// two, as the shared-memory images the sweep copies; whole slabs of [0, m_full) only
 size_t head_image2_bytes(int64_t M, int head);
 int launch_head_split2(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
                        uint32_t *head_max, unsigned char *head_img, cudaStream_t s);
@@ -223,10 +204,6 @@ int launch_sweep_mma2(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
 int launch_sweep_mma2_f16(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
 int launch_head_split2_f16(const void *W16, int64_t M, int64_t m_full, int head, const uint16_t *feat,
                            unsigned char *head_img, cudaStream_t s);
-// 256-document variant (sweep_mma3.cu): 128-neuron slabs, same image size (4 * head bytes per neuron)
-int launch_head_split3(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
-                       uint32_t *head_max, unsigned char *head_img, cudaStream_t s);
-int launch_sweep_mma3(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
 size_t plan_bytes(int64_t N, int64_t nnz, int head, int64_t D, PlanLayout *l);
 int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                 int order_by_length, int head, int relabel, int64_t D, char *ws, const PlanLayout &l,
@@ -234,22 +211,6 @@ int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t
 
 static const int LANES_MAX_D = 65024;    // 16-bit ids with 0xFFFF as the end marker
 
-struct LanesArgs {
-    const float *norms;
-    const int32_t *perm;       // planned position -> document
-    const uint32_t *doc_off;   // planned position -> first 8-id group of its list (minus one)
-    const uint4 *ids;          // 8 ascending 16-bit ids per uint4, 0xFFFF = end
-    int64_t N, M;
-    int32_t D;
-    u64 *state;
-    uint32_t *status;          // set non-zero if a bounded wait ran out
-    int32_t j_lo, j_hi, first;
-};
-// `tensor_map` is a host copy of the CUtensorMap describing W as a [D][M] fp32 tensor
-int make_codebook_tensor_map(const float *W, int64_t D, int64_t M, int rows_per_stage,
-                             void *tensor_map_out);
-int launch_sweep_lanes(const void *tensor_map, const LanesArgs &a, const bmu_opts &o,
-                       cudaStream_t s);
 int launch_wait_timeout_selftest(uint32_t *status, cudaStream_t s);
 
 // planned warp-per-document sweep (sweep_direct.cu): whole slabs of [j_lo, j_hi) only

@@ -46,6 +46,38 @@ static inline size_t m2_smem_bytes(int head, bool top2)
            16 * 8 + (top2 ? 4 * MMA_DOCS * 16 : 0);
 }
 
+// bit pattern of the largest |weight| among the head rows: sets the power-of-two scale of the
+// fp16 split
+__global__ void head_absmax_kernel(const float *__restrict__ W, int64_t M, int64_t m_full,
+                                   int head, const uint16_t *__restrict__ feat,
+                                   uint32_t *__restrict__ out)
+{
+    const int64_t n4 = m_full / 4, total = n4 * head;
+    uint32_t mx = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t f = i / n4, c = i - f * n4;
+        const int64_t row = feat ? (int64_t)feat[f] : f;
+        const float4 v = __ldg(reinterpret_cast<const float4 *>(W + row * M) + c);
+        mx = max(mx, __float_as_uint(fabsf(v.x)));
+        mx = max(mx, __float_as_uint(fabsf(v.y)));
+        mx = max(mx, __float_as_uint(fabsf(v.z)));
+        mx = max(mx, __float_as_uint(fabsf(v.w)));
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    if ((threadIdx.x & 31) == 0 && mx) atomicMax(out, mx);
+}
+
+int launch_head_absmax(const float *W, int64_t M, int64_t m_full, int head, const uint16_t *feat,
+                       uint32_t *head_max, cudaStream_t s)
+{
+    BMU_CUDA(cudaMemsetAsync(head_max, 0, sizeof(uint32_t), s));
+    head_absmax_kernel<<<592, 256, 0, s>>>(W, M, m_full, head, feat, head_max);
+    BMU_CUDA(cudaGetLastError());
+    return BMU_OK;
+}
+
 // One thread per (slab, group of 8 features, neuron).  Stage order inside a slab: block of
 // 64 features, tile c (neuron % 2), part (hi, lo).
 __global__ void __launch_bounds__(M2_SLAB)
@@ -457,6 +489,29 @@ int launch_sweep_mma2(const MmaArgs &a, const bmu_opts &o, cudaStream_t s)
     const unsigned blocks = (unsigned)((a.N + MMA_DOCS - 1) / MMA_DOCS);
     if (a.state2) sweep_mma2_kernel<true><<<blocks, M2_THREADS, m2_smem_bytes(a.head, true), s>>>(a);
     else sweep_mma2_kernel<false><<<blocks, M2_THREADS, m2_smem_bytes(a.head, false), s>>>(a);
+    BMU_CUDA(cudaGetLastError());
+    return BMU_OK;
+}
+
+// A wait that cannot succeed: one mbarrier that nothing ever arrives on.  It shows
+// that a wait which runs out leaves the kernel through the status word and the
+// context usable (no trap, no endless loop); the limit here is short on purpose.
+__global__ void wait_timeout_selftest_kernel(uint32_t *status)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    if (threadIdx.x == 0) {
+        mm_bar_init(mm_smem(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    bool ok = false;
+    for (uint32_t spin = 0; spin < 4096u && !ok; ++spin) ok = mm_bar_try(mm_smem(&bar), 0u);
+    if (!ok && threadIdx.x == 0) atomicOr(status, 2u);
+}
+
+int launch_wait_timeout_selftest(uint32_t *status, cudaStream_t s)
+{
+    wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(status);
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

@@ -208,94 +208,6 @@ def test_workspace_errors(bmu):
     assert e.value.status == 3
 
 
-# ------------------------------------------------------------------ staged kernel (a lane per document)
-def run_staged(bmu, W, rowptr, colidx, cancel_floor=False, **kw):
-    Wd, rp, ci = dev(W, rowptr, colidx)
-    opts = make_opts(bmu, kernel=2, **kw)
-    need = bmu.bmu_search_workspace_bytes(W.shape[0], W.shape[1], rp.numel() - 1, ci.numel(), opts)
-    ws = torch.empty(need + 256, dtype=torch.uint8, device="cuda")
-    ob, od = bmu.bmu_search_ws(Wd, rp, ci, opts=opts, workspace=ws)
-    torch.cuda.synchronize()
-    off = (-ws.data_ptr()) % 256
-    assert int(ws[off:off + 4].view(torch.int32).item()) == 0, "device-side wait timed out"
-    res = parity.compare(ob.cpu().numpy(), od.cpu().numpy(), W.numpy(), rowptr.numpy(),
-                         colidx.numpy(), cancel_floor=cancel_floor)
-    return ob, od, res
-
-
-@pytest.mark.parametrize("name,n_docs,M", [("cfg1", 10000, 1024), ("cfg2", 2500, 4096),
-                                           ("cfg3", 1100, 16384), ("cfg5", 1300, 2048)])
-def test_staged_benchmark_shapes(bmu, name, n_docs, M):
-    cfg = synth.CONFIGS[name]
-    rowptr, colidx = synth.make_corpus(cfg, n_docs=n_docs)
-    W = synth.make_codebook(cfg.D, M, synth.codebook_seed(cfg))
-    run_staged(bmu, W, rowptr, colidx)
-
-
-@pytest.mark.parametrize("kind,floor", [("scaled", False), ("sparse", False), ("signed", False),
-                                        ("dupes", False), ("const", False), ("prototype", True)])
-def test_staged_codebook_kinds(bmu, kind, floor):
-    cfg = synth.CONFIGS["cfg1"]
-    rowptr, colidx = synth.make_corpus(cfg, n_docs=2100)
-    W = synth.make_codebook(cfg.D, 416, 78, kind=kind, docs=(rowptr, colidx))
-    ob, _, _ = run_staged(bmu, W, rowptr, colidx, cancel_floor=floor)
-    if kind == "dupes":
-        assert int((ob % 2).sum()) == 0
-    if kind == "const":
-        assert int(ob.abs().sum()) == 0
-
-
-@pytest.mark.parametrize("N,D,M,chunk", [
-    (1, 256, 32, 0), (993, 300, 36, 0), (2000, 257, 1000, 0), (31, 1000, 1028, 256),
-    (5000, 700, 100, 64), (1985, 4096, 160, 96),
-])
-def test_staged_ragged_shapes(bmu, N, D, M, chunk):
-    r = np.random.default_rng(N * 11 + M)
-    rows = [np.sort(r.choice(D, size=int(r.integers(0, 60)), replace=False)) for _ in range(N)]
-    rowptr = np.zeros(N + 1, dtype=np.int32)
-    rowptr[1:] = np.cumsum([len(x) for x in rows])
-    colidx = np.concatenate(rows).astype(np.int32) if rowptr[-1] else np.zeros(0, np.int32)
-    W = synth.make_codebook(D, M, 5 + M, kind="scaled")
-    kw = {"chunk_neurons": chunk} if chunk else {}
-    run_staged(bmu, W, torch.from_numpy(rowptr), torch.from_numpy(colidx), **kw)
-
-
-def test_staged_long_empty_and_unsorted_rows(bmu):
-    D, M = 16384, 288
-    nnz = torch.tensor([400, 0, 1, 33, 0, 400, 97, 64, 32, 31, 0, 8, 16, 7, 9, 2000] * 70)
-    rowptr, colidx = synth.draw_corpus(nnz.numel(), D, 1.1, nnz, seed=5)
-    ci = colidx.numpy().copy()
-    rp = rowptr.numpy()
-    r = np.random.default_rng(1)
-    for i in range(0, nnz.numel(), 3):             # every third row in random order
-        r.shuffle(ci[rp[i]:rp[i + 1]])
-    W = synth.make_codebook(D, M, 9, kind="scaled")
-    run_staged(bmu, W, rowptr, torch.from_numpy(ci))
-
-
-@pytest.mark.parametrize("stage_rows,stages", [(256, 4), (128, 8), (256, 2), (128, 4), (64, 16)])
-@pytest.mark.parametrize("cluster", [0, 2])
-def test_staged_options_agree_with_direct(bmu, stage_rows, stages, cluster):
-    cfg = synth.CONFIGS["cfg2"]
-    rowptr, colidx = synth.make_corpus(cfg, n_docs=3100)
-    W = synth.make_codebook(cfg.D, 736, 14, kind="scaled")
-    ob, od, _ = run_staged(bmu, W, rowptr, colidx, stage_rows=stage_rows, stages=stages,
-                           cluster=cluster, chunk_neurons=320)
-    Wd, rp, ci = dev(W, rowptr, colidx)
-    db, dd = bmu.bmu_search_ws(Wd, rp, ci, opts=make_opts(bmu, kernel=1))
-    # both kernels add a row's features in ascending order in fp32: same bits
-    assert torch.equal(ob, db) and torch.equal(od, dd)
-
-
-def test_staged_refuses_what_it_cannot_do(bmu):
-    W = torch.zeros(100, 64, device="cuda")        # D < 256
-    rp = torch.tensor([0, 1], dtype=torch.int32).cuda()
-    ci = torch.tensor([0], dtype=torch.int32).cuda()
-    with pytest.raises(bmu.BmuError) as e:
-        bmu.bmu_search_ws(W, rp, ci, opts=make_opts(bmu, kernel=2))
-    assert e.value.status == 2
-
-
 # ------------------------------------------------------------------ planned warp-per-document kernel
 @pytest.mark.parametrize("vec", [4, 8])
 @pytest.mark.parametrize("warps", [4, 8, 32])
