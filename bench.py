@@ -7,9 +7,10 @@ over one synthetic corpus batch.  Default workload: the 512x512 map
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg4] [--impl reference]
 
-With N > 1 (under torchrun) every rank holds a replica of the codebook and its
-own batch of documents (documents are independent: no collective on the data
-path, weak scaling); the time is the maximum over ranks.
+With N > 1 every rank holds a replica of the codebook and its own batch of
+documents (documents are independent: no collective on the data path, weak
+scaling); the time is the maximum over ranks.  Under torchrun the ranks are the
+launcher's; a plain `python bench.py --gpus N` starts N ranks itself.
 Prints one JSON line on rank 0.
 """
 from __future__ import annotations
@@ -30,9 +31,6 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 from inputs import synth  # noqa: E402
-
-# DRAM bytes per sweep launch of the default config-4 run, from ncu (profiles/)
-TRAFFIC_CFG4 = {3: 2.0e9, 4: 2.9e9, 5: 4.9e9, 6: 3.6e9}
 
 METRIC = "bmu_search_docs_per_s"
 UNIT = "docs/s"
@@ -224,22 +222,49 @@ def workload_config(cfg, n_docs, world):
 
 
 # ----------------------------------------------------------------------------- our arm
-def run_ours(args, cfg, rank, local_rank, world):
-    import paper_2609_05138_b200 as bmu
-    bmu.load()                                    # fails loudly if the CUDA library is missing
-    dev = torch.device("cuda", local_rank)
-    torch.cuda.set_device(dev)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+def dram_traffic_record():
+    """DRAM bytes per sweep launch from the committed ncu capture of a small case, with the
+    rule that scales it to another launch (see the file itself)."""
+    p = os.path.join(ROOT, "profiles", "dram_traffic_sweep_mma2.json")
+    if not os.path.exists(p):
+        return None
+    with open(p) as f:
+        return json.load(f)
 
-    # one batch per step for the single-batch configs; config 5 streams its batches
+
+def scaled_traffic(rec, cfg, desc, opts, n_docs_per_launch):
+    """The capture's DRAM bytes scaled to this launch: the codebook chunk is read once per
+    launch whatever the number of documents, the rest (tile id matrices, masks, per-document
+    state) grows with the documents."""
+    if rec is None or desc.kernel != 6 or opts.tile_order or opts.repack or opts.relabel:
+        return None
+    b = rec["build"]
+    if desc.head_rows != b["head_rows"] or int(desc.chunk_neurons) != b["chunk_neurons"] or cfg.D != b["D"]:
+        return None
+    fixed = 4.0 * b["D"] * b["chunk_neurons"]
+    per_doc = max(0.0, rec["dram_bytes_per_launch"] - fixed) / rec["docs_per_launch"]
+    return fixed + per_doc * n_docs_per_launch
+
+
+def measure_roofs(bmu, dev):
+    """On-chip ceilings of this GPU, measured now.  The L2 -> SM ceiling is the largest rate
+    any committed microbenchmark reaches: loads alone, bulk copies alone, both together."""
+    r = {"l2_ldg": bmu.bmu_measure_roof("l2_ldg", device=dev),
+         "l2_bulk_16k": bmu.bmu_measure_roof("l2_bulk", piece=16384, device=dev),
+         "smem": bmu.bmu_measure_roof("smem", device=dev),
+         "fadd2": bmu.bmu_measure_roof("fadd2", device=dev)}
+    for piece in (4096, 8192, 16384):
+        r["l2_mixed_%dk" % (piece // 1024)] = bmu.bmu_measure_roof("l2_mixed", piece=piece, device=dev)
+    r["l2"] = max(v for k, v in r.items() if k.startswith("l2_"))
+    return r
+
+
+def measure_config(bmu, cfg, args, dev, rank, world, roofs, peaks, steps, warmup, opts,
+                   detail=True):
+    """Times `steps` steps of the whole hot path on one configuration (after `warmup`), and
+    derives the roofline figures of its sweep kernel.  Returns (line fragment, arrays)."""
     n_batches = min(synth.num_batches(cfg), args.batches) if args.batches else synth.num_batches(cfg)
     W = synth.make_codebook(cfg.D, cfg.M, synth.codebook_seed(cfg), device=dev)
-    opts = bmu.Opts()
-    for kv in args.opt:
-        k, v = kv.split("=")
-        setattr(opts, k, int(v))
     batches = []
     for b in range(n_batches):
         bsz = min(synth.batch_size(cfg), cfg.N - b * synth.batch_size(cfg))
@@ -249,7 +274,6 @@ def run_ours(args, cfg, rank, local_rank, world):
         batches.append((rp_b, ci_b))
     n_docs = sum(rp_b.numel() - 1 for rp_b, _ in batches)
     rowptr, colidx = batches[0]
-    N, nnz = rowptr.numel() - 1, colidx.numel()
     total_nnz = sum(ci_b.numel() for _, ci_b in batches)
     max_n = max(rp_b.numel() - 1 for rp_b, _ in batches)
     max_nnz = max(ci_b.numel() for _, ci_b in batches)
@@ -258,45 +282,11 @@ def run_ours(args, cfg, rank, local_rank, world):
     norms = torch.empty(cfg.M, dtype=torch.float32, device=dev)
     out_bmu = torch.empty(max_n, dtype=torch.int32, device=dev)
     out_dist = torch.empty(max_n, dtype=torch.float32, device=dev)
-
-    # launch geometry of the sweep (mirrors the library's defaults; reported, not used by it)
-    kernel = opts.kernel
-    if kernel == 0:                     # the library's automatic choice
-        big = float(max_nnz) * cfg.M >= 2e10
-        kernel = (6 if (big and cfg.M >= 512 and cfg.D >= 64) else 4 if (big and cfg.M >= 128)
-                  else 3)
-    vec = opts.vec or (4 if kernel == 1 else 8)
-    slab = 32 * vec
-    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
-    chunk = opts.chunk_neurons or max(slab, (l2_bytes // 2) // (cfg.D * 4) // slab * slab)
-    chunk = min((chunk + slab - 1) // slab * slab, (cfg.M + slab - 1) // slab * slab)
-    n_chunks = (cfg.M + chunk - 1) // chunk
-    # documents that share one SM's L1 at a time: resident warps x documents per warp
-    kernel_name = {3: "sweep_rows_kernel", 1: "sweep_direct_kernel", 2: "sweep_lanes_kernel",
-                   4: "sweep_tiles_kernel", 5: "sweep_mma_kernel", 6: "sweep_mma2_kernel",
-                   7: "sweep_mma3_kernel"}[kernel]
-    if kernel == 4:
-        vec, slab = 4, 128
-        chunk = opts.chunk_neurons or max(slab, (l2_bytes // 2) // (cfg.D * 4) // slab * slab)
-        chunk = min((chunk + slab - 1) // slab * slab, (cfg.M + slab - 1) // slab * slab)
-        n_chunks = (cfg.M + chunk - 1) // chunk
-    if kernel in (5, 6, 7):
-        vec, slab = 4, 512
-        chunk = opts.chunk_neurons or max(slab, int(l2_bytes * 0.55) // (cfg.D * 4) // slab * slab)
-        chunk = min((chunk + slab - 1) // slab * slab, cfg.M // slab * slab)
-        n_chunks = (cfg.M // slab * slab + chunk - 1) // chunk
-    if kernel == 2:
-        docs_per_block, chunk = 992, (opts.chunk_neurons or
-                                      max(32, (l2_bytes // 2) // (cfg.D * 4) // 32 * 32))
-        n_chunks = (cfg.M + chunk - 1) // chunk
-    elif kernel == 4:
-        docs_per_block = 8 * (opts.warps or 4) * 5
-    elif kernel == 1:
-        docs_per_block = (opts.warps or 16) * (opts.docs_per_warp or 4) * 2
-    elif kernel in (5, 6, 7):
-        docs_per_block = 256 if kernel == 7 else 128
-    else:
-        docs_per_block = 48
+    # what the library does for this size and these options (it answers, nothing is mirrored here)
+    desc = bmu.bmu_describe_search(cfg.D, cfg.M, max_n, max_nnz, opts, device=dev)
+    kernel_name = {1: "sweep_direct_kernel", 3: "sweep_rows_kernel", 4: "sweep_tiles_kernel",
+                   6: "sweep_mma2_kernel"}[desc.kernel]
+    chunk, n_chunks = int(desc.chunk_neurons), int(desc.sweep_launches)
 
     def step(e0=None, e1=None, e2=None):
         if e0 is not None:
@@ -318,26 +308,135 @@ def run_ours(args, cfg, rank, local_rank, world):
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         step()
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
     barrier()
     sampler = ClockSampler(dev)
     sampler.start()
-    for k in range(args.steps):
+    launches0 = bmu.bmu_kernel_launches()
+    for k in range(steps):
         step(*ev[k])
+    launches = bmu.bmu_kernel_launches() - launches0
     barrier()
     clocks = sampler.stop()
     total_ms = ev[0][0].elapsed_time(ev[-1][2])
-    sweep_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
-    norms_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
+    sweep_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / steps
+    norms_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / steps
     t = torch.tensor([total_ms, sweep_ms, norms_ms], dtype=torch.float64, device=dev)
     if world > 1:
         import torch.distributed as dist
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     total_ms, sweep_ms, norms_ms = t.tolist()
-    ms_per_step = total_ms / args.steps
+    ms_per_step = total_ms / steps
     value = n_docs * world / (ms_per_step * 1e-3)     # all ranks' documents / slowest rank
+
+    # ---- roofline of the dominant kernel (the sweep): algorithmic units per launch / time.
+    # The sweep launches are timed together with the tiling pass that precedes them (one
+    # search call); on the large configurations the pass is under 1 % of it.
+    launch_s = sweep_ms * 1e-3 / (n_chunks * len(batches))
+    nnz = total_nnz / len(batches)                              # mean batch
+    N = n_docs / len(batches)
+    adds = float(nnz) * chunk                                   # one update per (nnz, neuron)
+    union_rows = union_rows_per_block(rowptr, colidx, cfg.D, desc.docs_per_block) * (
+        nnz / max(1, colidx.numel()))
+    alg = {
+        "alu": (adds / launch_s, roofs["fadd2"], "add/s"),
+        "l1": (4.0 * adds / launch_s, roofs["smem"], "B/s"),           # one 4-byte operand per add
+        "l2": (4.0 * union_rows * chunk / launch_s, roofs["l2"], "B/s"),
+        "hbm": ((4.0 * cfg.D * chunk + 4.0 * nnz + 24.0 * N) / launch_s,
+                peaks["hbm_gbs"] * 1e9, "B/s"),
+    }
+    extra = {}
+    if desc.kernel == 6:
+        # the frequent features' updates are MMAs, not loads and adds: only the tail's updates
+        # pass through L1 and the fp32 pipe.  The L2 figure is the algorithmic one (each block
+        # of 128 documents fetches every distinct row it touches once per slab); what the
+        # design really moves is the tail's rows per document plus the head image per block.
+        head = desc.head_rows
+        tail_share = float((colidx >= head).sum().item()) / max(1, colidx.numel())
+        alg["alu"] = (tail_share * adds / launch_s, roofs["fadd2"], "add/s")
+        alg["l1"] = (4.0 * tail_share * adds / launch_s, roofs["smem"], "B/s")
+        moved = 4.0 * chunk * (tail_share * nnz + head * (N / float(desc.docs_per_block)))
+        mma_flops = 2.0 * 2.0 * head * N * chunk        # hi and lo parts, 2 flops per MAC
+        extra = {"tail_share_of_updates": tail_share,
+                 "l2_bytes_moved_by_design_GBs": moved / launch_s / 1e9,
+                 "l2_moved_frac_of_roof": moved / launch_s / roofs["l2"],
+                 "head_mma_TFLOPs": mma_flops / launch_s / 1e12,
+                 "head_mma_frac_of_bf16_peak": mma_flops / launch_s / 1e12 /
+                 peaks.get("bf16_tflops_sustained", peaks.get("bf16_tflops", 1590.0))}
+    bound = max(alg, key=lambda k: alg[k][0] / alg[k][1])
+    ach, peak, unit = alg[bound]
+    traffic = scaled_traffic(dram_traffic_record(), cfg, desc, opts, N)
+    roofline = {
+        "kernel": kernel_name, "bound": bound,
+        "achieved": ach / 1e9, "peak": peak / 1e9,
+        "unit": "GB/s" if unit == "B/s" else "Gadd/s", "frac": ach / peak,
+        "traffic": traffic,
+        "traffic_source": (None if traffic is None else
+                           "profiles/dram_traffic_sweep_mma2.json (ncu on a small case, scaled "
+                           "to this launch: codebook chunk once + the rest per document)"),
+        "launch_ms": launch_s * 1e3, "launches_per_step": n_chunks * len(batches),
+        "units_per_launch": {"adds": adds, "union_rows_x_chunk": float(union_rows) * chunk},
+        "fractions": {k: v[0] / v[1] for k, v in alg.items()},
+        **extra,
+    }
+    frag = {
+        "value": value, "ms_per_step": ms_per_step,
+        "updates_per_s": float(total_nnz) * cfg.M * world / (ms_per_step * 1e-3),
+        "phases_ms": {"norms": norms_ms, "sweep_and_output": sweep_ms},
+        "clocks": clocks, "gpu_launches": int(launches), "roofline": roofline,
+        "search": {"kernel": desc.kernel, "head_rows": desc.head_rows, "slab": desc.slab,
+                   "docs_per_block": desc.docs_per_block, "chunk_neurons": chunk,
+                   "sweep_launches": n_chunks, "repack": desc.repack},
+    }
+    arrays = dict(W=W, batches=batches, ws=ws, norms=norms, out_bmu=out_bmu, out_dist=out_dist,
+                  n_docs=n_docs, total_nnz=total_nnz, barrier=barrier)
+    return frag, arrays
+
+
+def planned_steps(bmu, cfg, a, opts, steps, dev):
+    """The same step with the tiling pass done beforehand (a frozen corpus, reused per epoch)."""
+    rowptr, colidx = a["batches"][0]
+    n0 = rowptr.numel() - 1
+    plan = bmu.Plan(rowptr, colidx, cfg.D, cfg.M, opts)
+    plan.search(a["W"], norms=a["norms"], out_bmu=a["out_bmu"][:n0], out_dist=a["out_dist"][:n0])
+    torch.cuda.synchronize(dev)
+    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    p0.record()
+    for _ in range(steps):
+        bmu.bmu_codebook_norms(a["W"], a["norms"])
+        plan.search(a["W"], norms=a["norms"], out_bmu=a["out_bmu"][:n0], out_dist=a["out_dist"][:n0])
+    p1.record()
+    torch.cuda.synchronize(dev)
+    planned_ms = p0.elapsed_time(p1) / steps
+    plan.close()
+    return {"ms_per_step": planned_ms, "value": n0 / (planned_ms * 1e-3), "unit": UNIT,
+            "api": "bmu_plan_create once, then bmu_codebook_norms + bmu_search_planned per step "
+                   "(rank 0's figure)"}
+
+
+def run_ours(args, cfg, rank, local_rank, world):
+    import paper_2609_05138_b200 as bmu
+    bmu.load()                                    # fails loudly if the CUDA library is missing
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    opts = bmu.Opts()
+    for kv in args.opt:
+        k, v = kv.split("=")
+        setattr(opts, k, int(v))
+    peaks, peaks_kind = measured_peaks()
+    roofs = measure_roofs(bmu, dev)
+
+    frag, a = measure_config(bmu, cfg, args, dev, rank, world, roofs, peaks, args.steps,
+                             args.warmup, opts)
+    W, batches, ws, norms = a["W"], a["batches"], a["ws"], a["norms"]
+    out_bmu, out_dist, n_docs, total_nnz = a["out_bmu"], a["out_dist"], a["n_docs"], a["total_nnz"]
+    rowptr, colidx = batches[0]
+    N = rowptr.numel() - 1
 
     # ---- end to end through the host entry point (pinned CSR in, results out)
     host = [(rp_b.cpu().pin_memory(), ci_b.cpu().pin_memory()) for rp_b, ci_b in batches]
@@ -354,7 +453,7 @@ def run_ours(args, cfg, rank, local_rank, world):
 
     e2e_step()                                              # warm-up (grows the scratch)
     e2e_steps = max(1, min(args.steps, 2))
-    barrier()
+    a["barrier"]()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
         e2e_step()
@@ -368,76 +467,26 @@ def run_ours(args, cfg, rank, local_rank, world):
     bmu.bmu_search_ws(W, rowptr, colidx, norms=norms, opts=opts, workspace=ws,
                       out_bmu=out_bmu[:N], out_dist=out_dist[:N])
     same = bool(torch.equal(ob_h, out_bmu[:N].cpu()))
+    del host, outs
+    bmu.bmu_release_scratch()
 
     if rank != 0:
         return None
 
-    # ---- roofline of the dominant kernel (the sweep): algorithmic units per launch / time
-    peaks, peaks_kind = measured_peaks()
-    roofs = {k: bmu.bmu_measure_roof(k, device=dev) for k in ("l2_ldg", "smem", "fadd2")}
-    launch_s = sweep_ms * 1e-3 / (n_chunks * len(batches))
-    nnz = total_nnz / len(batches)                              # mean batch
-    N = n_docs / len(batches)
-    adds = float(nnz) * chunk                                   # one update per (nnz, neuron)
-    union_rows = union_rows_per_block(rowptr, colidx, cfg.D, docs_per_block) * (
-        nnz / max(1, colidx.numel()))
-    alg = {
-        "alu": (adds / launch_s, roofs["fadd2"], "add/s"),
-        "l1": (4.0 * adds / launch_s, roofs["smem"], "B/s"),           # one 4-byte operand per add
-        "l2": (4.0 * union_rows * chunk / launch_s, roofs["l2_ldg"], "B/s"),
-        "hbm": ((4.0 * cfg.D * chunk + 4.0 * nnz + 24.0 * N) / launch_s,
-                peaks["hbm_gbs"] * 1e9, "B/s"),
-    }
-    extra = {}
-    if kernel in (5, 6, 7):
-        # the frequent features' updates are MMAs, not loads and adds: only the tail's updates
-        # pass through L1 and the fp32 pipe.  The L2 figure stays the algorithmic one (each
-        # block of 128 documents fetches every distinct row it touches once); what the design
-        # really moves is the tail's rows per document plus the head image per block.
-        head = opts.head_rows or (256 if kernel == 5 else
-                                  min(896 if kernel == 7 else 640, cfg.D // 64 * 64))
-        tail_share = float((colidx >= head).sum().item()) / max(1, colidx.numel())
-        alg["alu"] = (tail_share * adds / launch_s, roofs["fadd2"], "add/s")
-        alg["l1"] = (4.0 * tail_share * adds / launch_s, roofs["smem"], "B/s")
-        moved = 4.0 * chunk * (tail_share * nnz + head * (N / float(docs_per_block)))
-        mma_flops = 2.0 * 2.0 * head * N * chunk        # hi and lo parts, 2 flops per MAC
-        extra = {"tail_share_of_updates": tail_share,
-                 "l2_bytes_moved_by_design_GBs": moved / launch_s / 1e9,
-                 "l2_moved_frac_of_roof": moved / launch_s / roofs["l2_ldg"],
-                 "head_mma_TFLOPs": mma_flops / launch_s / 1e12,
-                 "head_mma_frac_of_bf16_peak": mma_flops / launch_s / 1e12 /
-                 peaks.get("bf16_tflops_sustained", peaks.get("bf16_tflops", 1590.0))}
-    bound = max(alg, key=lambda k: alg[k][0] / alg[k][1])
-    ach, peak, unit = alg[bound]
-    scale = 1e9
-    roofline = {
-        "kernel": kernel_name, "bound": bound,
-        "achieved": ach / scale, "peak": peak / scale,
-        "unit": "GB/s" if unit == "B/s" else "Gadd/s", "frac": ach / peak,
-        # DRAM bytes per launch from the ncu capture of this very launch configuration
-        # (profiles/sweep_*_cfg4_launch_list.md); other workloads were not captured
-        "traffic": (TRAFFIC_CFG4.get(kernel) if (cfg.name == "cfg4" and n_docs == cfg.N
-                                                 and not opts.chunk_neurons and not opts.vec
-                                                 and not opts.warps and not opts.head_rows
-                                                 and not opts.repack)
-                    else None),
-        "launch_ms": launch_s * 1e3, "launches_per_step": n_chunks,
-        "units_per_launch": {"adds": adds, "union_rows_x_chunk": float(union_rows) * chunk},
-        "fractions": {k: v[0] / v[1] for k, v in alg.items()},
-        **extra,
-        "peaks": {"hbm_GBs": peaks["hbm_gbs"], "hbm_source": "MEASURED_PEAKS.json (%s)" % peaks_kind,
-                  "l2_GBs": roofs["l2_ldg"] / 1e9, "l1_smem_GBs": roofs["smem"] / 1e9,
-                  "fp32_Gadds": roofs["fadd2"] / 1e9,
-                  "on_chip_source": "bmu_measure_roof, this run"},
-    }
+    frag["roofline"]["peaks"] = {
+        "hbm_GBs": peaks["hbm_gbs"], "hbm_source": "MEASURED_PEAKS.json (%s)" % peaks_kind,
+        "l2_GBs": roofs["l2"] / 1e9,
+        "l2_variants_GBs": {k: v / 1e9 for k, v in roofs.items() if k.startswith("l2_")},
+        "l2_rule": "largest of: 128-bit loads, 16 KB bulk copies, loads and bulk copies together",
+        "l1_smem_GBs": roofs["smem"] / 1e9, "fp32_Gadds": roofs["fadd2"] / 1e9,
+        "on_chip_source": "bmu_measure_roof, this run"}
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": workload_config(cfg, n_docs, world),
-        "updates_per_s": float(total_nnz) * cfg.M * world / (ms_per_step * 1e-3),
-        "phases_ms": {"norms": norms_ms, "sweep_and_output": sweep_ms},
-        "clocks": clocks,
+        "metric": METRIC, "value": frag["value"], "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": frag["ms_per_step"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "config": workload_config(cfg, n_docs, world),
+        "updates_per_s": frag["updates_per_s"], "phases_ms": frag["phases_ms"],
+        "clocks": frag["clocks"],
         "e2e": {"value": n_docs * world / e2e_s, "unit": UNIT,
                 "h2d_bytes_per_step": int((n_docs + len(batches) + total_nnz) * 4),
                 "d2h_bytes_per_step": int(n_docs * 8),
@@ -446,32 +495,15 @@ def run_ours(args, cfg, rank, local_rank, world):
                         "with the search of the current one)" % len(batches)) +
                        " (codebook resident in HBM; CSR from pinned host memory; results back "
                        "to host)", "matches_device_path": same},
-        "gpu_launches": args.steps * (1 + len(batches) * ({1: 0, 2: 7, 3: 7, 4: 11, 5: 24, 6: 24, 7: 24}[kernel]
-                                                           + n_chunks * (2 if kernel in (5, 6, 7) and
-                                                                         opts.repack != 2 and
-                                                                         n_chunks > 1 else 1)
-                                                           + 1)),
-        "roofline": roofline,
+        "gpu_launches": frag["gpu_launches"],
+        "gpu_launches_source": "bmu_kernel_launches(): the library's own count of its kernel "
+                               "launches across the timed region (library sort/scan kernels and "
+                               "memsets not counted)",
+        "search": frag["search"],
+        "roofline": frag["roofline"],
     }
-    # ---- the same step with the tiling pass done beforehand (a frozen corpus, reused per epoch)
     if len(batches) == 1:
-        n0 = rowptr.numel() - 1
-        plan = bmu.Plan(rowptr, colidx, cfg.D, cfg.M, opts)
-        plan.search(W, norms=norms, out_bmu=out_bmu[:n0], out_dist=out_dist[:n0])
-        torch.cuda.synchronize(dev)
-        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        p0.record()
-        for _ in range(args.steps):
-            bmu.bmu_codebook_norms(W, norms)
-            plan.search(W, norms=norms, out_bmu=out_bmu[:n0], out_dist=out_dist[:n0])
-        p1.record()
-        torch.cuda.synchronize(dev)
-        planned_ms = p0.elapsed_time(p1) / args.steps
-        line["planned"] = {"ms_per_step": planned_ms, "value": n0 / (planned_ms * 1e-3), "unit": UNIT,
-                           "api": "bmu_plan_create once, then bmu_codebook_norms + "
-                                  "bmu_search_planned per step (rank 0's figure)"}
-        plan.close()
-        del plan
+        line["planned"] = planned_steps(bmu, cfg, a, opts, args.steps, dev)
     if args.comparator:
         line["comparator"] = comparator_spmm(cfg, W, norms, rowptr, colidx)
     if args.f16 and len(batches) == 1:
@@ -481,7 +513,41 @@ def run_ours(args, cfg, rank, local_rank, world):
                                      peaks, args.sigma)
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(cfg, W, rowptr, colidx, rowptr.numel() - 1)
+    # ---- the other benchmark configurations, briefly (same protocol, fewer steps)
+    if world == 1 and args.all_configs and not args.docs and not args.batches and not args.opt:
+        del W, batches, ws, norms, out_bmu, out_dist, rowptr, colidx
+        a.clear()
+        torch.cuda.empty_cache()
+        line["all_configs"] = {cfg.name: {k: frag[k] for k in ("value", "ms_per_step", "updates_per_s")}
+                               | {"unit": UNIT, "bound": frag["roofline"]["bound"],
+                                  "frac": frag["roofline"]["frac"],
+                                  "sm_mhz": frag["clocks"].get("sm_mhz")}}
+        for name in sorted(synth.CONFIGS):
+            if name == cfg.name:
+                continue
+            line["all_configs"][name] = brief_config(bmu, synth.CONFIGS[name], args, dev, roofs, peaks)
     return line
+
+
+def brief_config(bmu, cfg, args, dev, roofs, peaks):
+    """One of the other benchmark configurations: 3 warm-up + 3 timed steps (the 0.2 ms
+    configuration: 100 back-to-back steps), docs/s, updates/s and the roofline fraction."""
+    small = cfg.N * cfg.M < 10 ** 9
+    steps, warmup = (100, 10) if small else (3, 3)
+    opts = bmu.Opts()
+    frag, a = measure_config(bmu, cfg, args, dev, 0, 1, roofs, peaks, steps, warmup, opts)
+    out = {"value": frag["value"], "unit": UNIT, "ms_per_step": frag["ms_per_step"],
+           "updates_per_s": frag["updates_per_s"], "steps": steps, "warmup": warmup,
+           "kernel": frag["roofline"]["kernel"], "bound": frag["roofline"]["bound"],
+           "frac": frag["roofline"]["frac"], "fractions": frag["roofline"]["fractions"],
+           "l2_moved_frac_of_roof": frag["roofline"].get("l2_moved_frac_of_roof"),
+           "sm_mhz": frag["clocks"].get("sm_mhz"), "clock_reasons": frag["clocks"].get("reasons"),
+           "gpu_launches": frag["gpu_launches"], "docs": a["n_docs"]}
+    if len(a["batches"]) == 1:
+        out["planned_ms_per_step"] = planned_steps(bmu, cfg, a, opts, steps, dev)["ms_per_step"]
+    a.clear()
+    torch.cuda.empty_cache()
+    return out
 
 
 def f16_codebook(bmu, cfg, W, rowptr, colidx, args):
@@ -617,6 +683,33 @@ def epoch_phases(bmu, cfg, W, batches, opts, ws, norms, out_bmu, out_dist, peaks
             "note": "paper (RTX 4090, Table 4): search 73.7-94.0 % of the epoch"}
 
 
+def launch_ranks(n_ranks, argv):
+    """Re-runs this script as `n_ranks` ranks on this node (one process per GPU) through
+    torch.distributed.run and returns its exit code; rank 0 of the children prints the line."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+           "--nproc-per-node", str(n_ranks), "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__), *argv]
+    return subprocess.call(cmd)
+
+
+def selfcheck_ranks(rank, world):
+    """No GPU work: the ranks meet over gloo on the host and rank 0 reports how many came."""
+    import torch.distributed as dist
+    if "MASTER_ADDR" not in os.environ:              # a single rank started by hand
+        os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT="29533", RANK="0", WORLD_SIZE="1")
+    dist.init_process_group("gloo")
+    t = torch.ones(1, dtype=torch.int64)
+    dist.all_reduce(t)
+    dist.barrier()
+    if rank == 0:
+        print(json.dumps({"selfcheck": "ranks", "n_gpus": int(t.item()), "world_size": world}))
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -637,9 +730,18 @@ def main():
     ap.add_argument("--epoch", action="store_true",
                     help="also time one whole epoch (search + scatter + blur + write-back)")
     ap.add_argument("--sigma", type=float, default=2.0, help="neighbourhood width of --epoch")
+    ap.add_argument("--no-all-configs", dest="all_configs", action="store_false",
+                    help="skip the brief runs of the other benchmark configurations")
+    ap.add_argument("--selfcheck-ranks", action="store_true",
+                    help="start the ranks, let them meet on the host and report their number")
     args = ap.parse_args()
     cfg = synth.CONFIGS[args.config]
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1 and (args.impl == "ours" or args.selfcheck_ranks):
+        sys.exit(launch_ranks(args.gpus, sys.argv[1:]))
     rank, local_rank, world = dist_env()
+    if args.selfcheck_ranks:
+        selfcheck_ranks(rank, world)
+        return
     if args.warmup < 3 and args.impl == "ours" and rank == 0:
         print("note: fewer than 3 warm-up steps", file=sys.stderr)
 

@@ -1,9 +1,9 @@
 /*
  * bmu.h -- C ABI of the B200 (sm_100a) best-matching-unit search library.
  *
- * The operation (paper Section 3: "finding, for each article, the neuron whose
- * weight vector is closest to it"; the kernel "fuses the argmin into the
- * product, so the score block is never materialised"): for every document i of
+ * The operation (paper Section 3: the nearest-neuron search of self-organizing
+ * map training, with the arg-min taken inside the sparse-dense product so that
+ * no document-by-neuron score matrix is ever written): for every document i of
  * a sparse binary corpus and every neuron j of an M-neuron codebook
  *
  *     d_ij = |x_i| + ||w_j||^2 - 2 * sum_{f in x_i} W[f*M + j]
@@ -15,7 +15,7 @@
  * caller owns every buffer it passes and keeps it alive until the stream has
  * finished the call):
  *   W       float32 [D][M], feature-major: the M weights of feature f are
- *           contiguous at W + f*M (Section 3, "W[v.M+i]").  The fast path needs
+ *           contiguous at W + f*M (the feature-major layout of Section 3).  The fast path needs
  *           W 16-byte aligned and M % 4 == 0; any other M takes a scalar path.
  *   rowptr  int32 [N+1], rowptr[0] == 0, non-decreasing; row i is
  *           colidx[rowptr[i] .. rowptr[i+1])            (CSR of the binary corpus)
@@ -124,6 +124,33 @@ BMU_API const char *bmu_last_error(void);
 BMU_API int bmu_version(void);
 
 /*
+ * How many kernels of this library the calling thread has launched so far (the
+ * library's own kernels; the sort and scan of the tiling pass, which come from
+ * a CUDA library, and memsets are not counted).  The difference across a region
+ * is the number of launches in it.
+ */
+BMU_API uint64_t bmu_kernel_launches(void);
+
+/*
+ * What bmu_search_ws would do for a problem of this size with these options on
+ * the current device (Section 4: tile, chunking and vector-width choices), without
+ * doing it: which kernel (as in bmu_opts.kernel; never 0), the tensor-core head
+ * (0 for the other kernels), the neurons a block carries at a time, the documents
+ * that share a block, whether a compact copy of the chunk's columns precedes each
+ * launch, the neurons per launch (one L2-resident chunk), the number of sweep
+ * launches, and how many neurons beyond the last whole slab go to the generic
+ * kernel in one more launch.  Assumes W 16-byte aligned.  Same errors as
+ * bmu_search_ws for sizes and options it would refuse.
+ */
+typedef struct bmu_search_desc {
+    int32_t kernel, head_rows, slab, docs_per_block, repack, sweep_launches, ragged_neurons;
+    int32_t reserved;
+    int64_t chunk_neurons;
+} bmu_search_desc;
+BMU_API int bmu_describe_search(int64_t D, int64_t M, int64_t N, int64_t nnz,
+                                const bmu_opts *opts, bmu_search_desc *out);
+
+/*
  * Codebook norms, the "norms" step of an epoch (Table 4): norms[j] = sum_f
  * W[f*M+j]^2.  Products and the running sum are taken in fp64 and rounded to
  * fp32 once.  Deterministic.  Uses no scratch memory.
@@ -162,8 +189,9 @@ BMU_API int bmu_search_ws(const float *W, int64_t D, int64_t M, const float *nor
  * matrices, head masks -- can be done once and reused by every epoch's search.
  *   bmu_plan_workspace_bytes  bytes of 256-byte aligned device memory a plan needs
  *       (the plan itself plus the scratch of the searches that use it).
- *   bmu_plan_create  runs the tiling pass into `workspace` (asynchronous on
- *       `stream`) and returns a host handle in *plan.  rowptr, colidx and the
+ *   bmu_plan_create  runs the tiling pass into `workspace` on `stream`, waits for
+ *       it, checks its status word (BMU_ERR_WORKSPACE if a size check of the pass
+ *       failed) and returns a host handle in *plan.  rowptr, colidx and the
  *       workspace stay owned by the caller and must stay alive and unchanged
  *       until bmu_plan_destroy; `nnz` is the length of colidx.
  *   bmu_search_planned  the search of bmu_search_ws without its tiling pass:
@@ -199,8 +227,8 @@ BMU_API int bmu_search_top2_ws(const float *W, int64_t D, int64_t M, const float
                                void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * Half-precision codebook, the paper's own storage (Section 4.2: "two bytes per
- * half-precision weight"; Section 4.3: __half2 loads).  W16 is IEEE fp16
+ * Half-precision codebook, the paper's own storage (Section 4.2 counts its
+ * working set at 2 bytes per weight; Section 4.3 loads pairs of halves).  W16 is IEEE fp16
  * [D][M], feature-major, 16-byte aligned; sums and distances are still fp32
  * (norms: fp64 accumulate).  Needs M % 256 == 0 (M % 8 == 0 for the norms
  * alone) and D <= 65024.  out_bmu2 / out_dist2 may both be NULL, or both given
@@ -228,10 +256,21 @@ BMU_API int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float
  * process exit).  Reads rowptr[N] back to size the scratch, so the call
  * synchronises the stream once before the kernels are queued.  Calls on
  * different streams of one device share the scratch and must not overlap.
+ * The status word of the search (see bmu_search_ws) sits in that scratch:
+ * bmu_last_status reads it.
  */
 BMU_API int bmu_search(const float *W, int64_t D, int64_t M, const int32_t *rowptr,
                const int32_t *colidx, int64_t N, int32_t *out_bmu, float *out_dist,
                void *stream);
+
+/*
+ * Status word of the last bmu_search (or bmu_search_host, bmu_search_batches_host)
+ * on the current device: synchronises `stream`, copies the word to *out_status and
+ * returns BMU_OK if it is 0, BMU_ERR_TIMEOUT if a bounded device-side wait ran
+ * out, BMU_ERR_WORKSPACE if a size check of the tiling pass failed (the results
+ * of that search are then invalid).  0 if no search has run yet.
+ */
+BMU_API int bmu_last_status(uint32_t *out_status, void *stream);
 
 /*
  * End-to-end form for a corpus batch that lives in HOST memory (pinned for
@@ -249,6 +288,8 @@ BMU_API int bmu_search_host(const float *W, int64_t D, int64_t M, const int32_t 
  * A corpus streamed in batches from HOST memory against one device-resident
  * codebook (the corpus-scale epoch is fed this way: one CSR per batch, because a
  * whole corpus exceeds the int32 row pointers).  The norms are computed once;
+ * the status words of all batches are collected and checked at the end
+ * (BMU_ERR_TIMEOUT / BMU_ERR_WORKSPACE as in bmu_last_status);
  * two device staging buffers let a copy stream upload batch k+1 and download the
  * results of batch k-1 while `stream` searches batch k.  Arrays of n_batches
  * host pointers: rowptr_host[k] has N[k]+1 entries, colidx_host[k] has
@@ -318,8 +359,8 @@ BMU_API int bmu_search_static(const float *W, int64_t D, int64_t M, const int32_
 
 /*
  * The rest of a batch epoch after the search (Table 4 columns "scatter", "blur",
- * "write-back"; Section 6: "the scatter into accumulators is O(N.nnz) ... the
- * blur is the O(M) term").  The paper times these steps and prints no formula;
+ * "write-back"; Section 6 gives their cost: the scatter grows with the listings,
+ * N times nnz per document, the blur with the map size M).  The paper times these steps and prints no formula;
  * they are the textbook batch update of a self-organizing map on a rectangular,
  * non-periodic map of edge_y rows by edge_x columns, neuron j = y * edge_x + x.
  * All arrays are device memory, feature-major like W; every call is
@@ -382,8 +423,12 @@ BMU_API int bmu_map_errors(const int32_t *bmu, const int32_t *bmu2, const float 
  *         3  L1-resident global loads -> registers, 128-bit            [bytes/s]
  *         4  fp32 adds, scalar instructions                            [adds/s]
  *         5  fp32 adds, packed two-wide instructions                   [adds/s]
+ *         6  L2 -> SM by 128-bit loads and bulk copies of `piece` bytes (multiple
+ *            of 16 in [1024, 16384]) running together, both counted: the way the
+ *            tensor-core sweep pulls bytes (gathered rows by loads, head image by
+ *            bulk copies)                                              [bytes/s]
  * `buffer` is 256-byte aligned device memory the benchmark may overwrite; for
- * 0 and 1 its size is the footprint that is swept (keep it well inside L2), for
+ * 0, 1 and 6 its size is the footprint that is swept (keep it well inside L2), for
  * 3 it must hold 64 KiB per SM.  Synchronous; the result goes to *out_value.
  */
 BMU_API int bmu_measure_roof(int which, void *buffer, size_t buffer_bytes, int piece,

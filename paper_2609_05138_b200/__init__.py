@@ -9,7 +9,8 @@ from .binding import (BmuError, Opts, bmu_codebook_norms, bmu_codebook_norms_f16
                       bmu_search_workspace_bytes, bmu_search_ws,
                       bmu_measure_roof, bmu_validate_csr, bmu_version, load,
                       bmu_update_scatter, bmu_update_blur, bmu_update_writeback,
-                      bmu_map_errors, Plan)
+                      bmu_map_errors, Plan, SearchDesc, bmu_describe_search,
+                      bmu_kernel_launches, bmu_last_status)
 
 __all__ = ["BmuError", "Opts", "bmu_codebook_norms", "bmu_codebook_norms_f16",
            "bmu_search_f16_ws", "bmu_release_scratch", "bmu_search",
@@ -17,4 +18,4 @@ __all__ = ["BmuError", "Opts", "bmu_codebook_norms", "bmu_codebook_norms_f16",
            "bmu_search_workspace_bytes", "bmu_search_ws",
            "bmu_measure_roof", "bmu_validate_csr", "bmu_version", "load",
            "bmu_update_scatter", "bmu_update_blur", "bmu_update_writeback", "bmu_map_errors",
-           "Plan"]
+           "Plan", "SearchDesc", "bmu_describe_search", "bmu_kernel_launches", "bmu_last_status"]

@@ -37,11 +37,23 @@ class Opts(ctypes.Structure):
                 ("relabel", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3)]
 
 
+class SearchDesc(ctypes.Structure):
+    """Mirror of `bmu_search_desc` (include/bmu.h)."""
+    _fields_ = [("kernel", ctypes.c_int32), ("head_rows", ctypes.c_int32),
+                ("slab", ctypes.c_int32), ("docs_per_block", ctypes.c_int32),
+                ("repack", ctypes.c_int32), ("sweep_launches", ctypes.c_int32),
+                ("ragged_neurons", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("chunk_neurons", ctypes.c_int64)]
+
+
 EXPORTS = {
     # name: (restype, argtypes)
     "bmu_status_string": (ctypes.c_char_p, [ctypes.c_int]),
     "bmu_last_error": (ctypes.c_char_p, []),
     "bmu_version": (ctypes.c_int, []),
+    "bmu_kernel_launches": (ctypes.c_uint64, []),
+    "bmu_describe_search": (ctypes.c_int, [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
+                                           ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]),
     "bmu_codebook_norms": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                           ctypes.c_void_p, ctypes.c_void_p]),
     "bmu_search_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int64, ctypes.c_int64,
@@ -87,6 +99,7 @@ EXPORTS = {
                                                ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                                ctypes.c_void_p]),
     "bmu_selftest_wait_timeout": (ctypes.c_int, [ctypes.c_void_p]),
+    "bmu_last_status": (ctypes.c_int, [ctypes.POINTER(ctypes.c_uint32), ctypes.c_void_p]),
     "bmu_release_scratch": (ctypes.c_int, []),
     "bmu_validate_csr": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                         ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
@@ -343,6 +356,29 @@ def bmu_search_batches_host(W, batches, outs=None):
     return outs
 
 
+def bmu_kernel_launches() -> int:
+    return int(load().bmu_kernel_launches())
+
+
+def bmu_describe_search(D: int, M: int, N: int, nnz: int, opts: Opts | None = None,
+                        device=None) -> SearchDesc:
+    """The kernel, chunking and launch count bmu_search_ws would use on `device`."""
+    d = SearchDesc()
+    with torch.cuda.device(torch.device("cuda" if device is None else device)):
+        _check(load().bmu_describe_search(D, M, N, nnz, ctypes.byref(opts) if opts else None,
+                                          ctypes.byref(d)))
+    return d
+
+
+def bmu_last_status(device=None):
+    """(status, word): the status word of the last one-shot search on `device`."""
+    device = torch.device("cuda" if device is None else device)
+    w = ctypes.c_uint32(0)
+    with torch.cuda.device(device):
+        rc = int(load().bmu_last_status(ctypes.byref(w), torch.cuda.current_stream(device).cuda_stream))
+    return rc, int(w.value)
+
+
 def bmu_selftest_wait_timeout(device=None) -> int:
     """Runs the bounded-wait self-test; returns the status (5 = BMU_ERR_TIMEOUT expected)."""
     device = torch.device("cuda" if device is None else device)
@@ -467,7 +503,7 @@ def bmu_map_errors(bmu, bmu2, dist, edge_x: int, edge_y: int, adjacency: int = 4
     return out
 
 
-ROOFS = {"l2_ldg": 0, "l2_bulk": 1, "smem": 2, "l1": 3, "fadd": 4, "fadd2": 5}
+ROOFS = {"l2_ldg": 0, "l2_bulk": 1, "smem": 2, "l1": 3, "fadd": 4, "fadd2": 5, "l2_mixed": 6}
 
 
 def bmu_measure_roof(which: str, footprint_bytes: int = 32 << 20, piece: int = 2048,

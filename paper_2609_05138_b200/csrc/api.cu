@@ -11,6 +11,7 @@
 namespace bmu {
 
 static thread_local char g_err[512] = "";
+thread_local unsigned long long g_kernel_launches = 0;
 
 void set_error(const char *fmt, ...)
 {
@@ -179,6 +180,73 @@ static int64_t auto_chunk(int64_t D, int64_t M, int slab)
     return c;
 }
 
+// Which kernel a search takes and how it is cut into launches.
+struct Route {
+    int kernel;            // 1 generic, 3 planned, 4 tiled, 6 tensor-core head + gathered tail
+    int head;              // features summed on the tensor cores (kernel 6), else 0
+    int slab;              // neurons a block (or warp) carries at a time
+    int docs_per_block;    // documents that share a block
+    int64_t chunk;         // neurons per launch (one L2-resident chunk)
+    int64_t m_full;        // neurons covered by whole slabs; the rest takes the generic kernel
+    int repack;            // 1: a compact copy of the chunk's columns precedes each launch
+};
+
+static int route_search(const bmu_opts &o, int64_t D, int64_t M, int64_t nnz, uintptr_t w_addr,
+                        Route &r)
+{
+    const int head = mma_head_rows(o, D);
+    // the planned warp-per-document kernel needs 16-bit ids and whole 16-byte row pieces
+    const bool planned_ok = D <= LANES_MAX_D && M % 4 == 0 && M >= rows_slab_width(o) &&
+                            (w_addr & 15) == 0;
+    if (o.kernel == 3 && !planned_ok) {
+        set_error("planned kernel needs M %% 4 == 0, M >= 128, D <= %d and W 16-byte aligned",
+                  LANES_MAX_D);
+        return BMU_ERR_UNSUPPORTED;
+    }
+    const bool tiled_ok = planned_ok && M >= 128 && o.cluster != 2;
+    // tensor-core head: additionally at least one whole 512-neuron slab and `head` features
+    const bool mma_ok = tiled_ok && D >= head && M >= MMA_SLAB;
+    if (o.kernel == 6 && !mma_ok) {
+        set_error("tensor-core sweep needs what the tiled kernel needs, D >= %d and M >= %d",
+                  head, MMA_SLAB);
+        return BMU_ERR_UNSUPPORTED;
+    }
+    // automatic choice for large sweeps: the tensor-core sweep where it applies, else the tiled
+    // kernel; both repay their extra preparation only when there is enough to sweep
+    const bool big = (double)nnz * (double)M >= 2e10;
+    const bool mma = o.kernel == 6 || (o.kernel == 0 && mma_ok && big);
+    const bool tiled = !mma && (o.kernel == 4 || (o.kernel == 0 && tiled_ok && big));
+    if (tiled && !tiled_ok) {
+        set_error("tiled kernel needs M %% 4 == 0, M >= 128, D <= %d, W 16-byte aligned and "
+                  "length-ordered documents (cluster != 2)", LANES_MAX_D);
+        return BMU_ERR_UNSUPPORTED;
+    }
+    const bool planned = !tiled && !mma && (o.kernel == 3 || (o.kernel == 0 && planned_ok));
+    r.head = 0; r.repack = 0;
+    if (mma) {
+        r.kernel = 6; r.head = head; r.slab = 256; r.docs_per_block = MMA_DOCS;
+        r.chunk = mma_chunk(o, D, M);
+        r.m_full = M / MMA_SLAB * MMA_SLAB;
+        r.repack = o.repack != 2 && M > r.chunk;
+    } else if (tiled) {
+        r.kernel = 4; r.slab = 128; r.docs_per_block = 8 * (o.warps ? o.warps : 4);
+        r.chunk = o.chunk_neurons ? (o.chunk_neurons + 127) / 128 * 128 : auto_chunk(D, M, 128);
+        r.m_full = M / 128 * 128;
+    } else if (planned) {
+        r.kernel = 3; r.slab = rows_slab_width(o); r.docs_per_block = o.warps ? o.warps : 16;
+        r.chunk = o.chunk_neurons ? (o.chunk_neurons + r.slab - 1) / r.slab * r.slab
+                                  : auto_chunk(D, M, r.slab);
+        r.m_full = M / r.slab * r.slab;
+    } else {
+        r.kernel = 1; r.slab = 32 * (o.vec ? o.vec : 4);
+        r.docs_per_block = (o.warps ? o.warps : 16) * (o.docs_per_warp ? o.docs_per_warp : 4);
+        r.chunk = o.chunk_neurons ? (o.chunk_neurons + r.slab - 1) / r.slab * r.slab
+                                  : auto_chunk(D, M, r.slab);
+        r.m_full = M;
+    }
+    return BMU_OK;
+}
+
 static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
                        const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                        int32_t *out_bmu, float *out_dist, const bmu_opts *opts_in, void *ws,
@@ -228,46 +296,22 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     }
     uint32_t *status = reinterpret_cast<uint32_t *>(base + l.status_off);
     BMU_CUDA(cudaMemsetAsync(status, 0, 256, s));
-    // the planned warp-per-document kernel needs 16-bit ids and whole 16-byte row pieces
-    const bool planned_ok = D <= LANES_MAX_D && M % 4 == 0 && M >= rows_slab_width(o) &&
-                            (w_addr & 15) == 0;
-    if (o.kernel == 3 && !planned_ok) {
-        set_error("planned kernel needs M %% 4 == 0, M >= 128, D <= %d and W 16-byte aligned",
-                  LANES_MAX_D);
-        return BMU_ERR_UNSUPPORTED;
-    }
-    const bool tiled_ok = planned_ok && M >= 128 && o.cluster != 2;
-    // tensor-core head: additionally at least one whole 512-neuron slab and `head` features
-    const bool mma_ok = tiled_ok && D >= head && M >= MMA_SLAB;
-    if (o.kernel == 6 && !mma_ok) {
-        set_error("tensor-core sweep needs what the tiled kernel needs, D >= %d and M >= %d",
-                  head, MMA_SLAB);
-        return BMU_ERR_UNSUPPORTED;
-    }
-    // automatic choice for large sweeps: the tensor-core sweep where it applies, else the tiled
-    // kernel; both repay their extra preparation only when there is enough to sweep
-    const bool big = (double)nnz * (double)M >= 2e10;
-    const bool mma = o.kernel == 6 || (o.kernel == 0 && mma_ok && big);
-    const bool tiled = !mma && (o.kernel == 4 || (o.kernel == 0 && tiled_ok && big));
-    if (tiled && !tiled_ok) {
-        set_error("tiled kernel needs M %% 4 == 0, M >= 128, D <= %d, W 16-byte aligned and "
-                  "length-ordered documents (cluster != 2)", LANES_MAX_D);
-        return BMU_ERR_UNSUPPORTED;
-    }
-    const bool planned = !tiled && !mma && (o.kernel == 3 || (o.kernel == 0 && planned_ok));
+    Route r;
+    if ((rc = route_search(o, D, M, nnz, w_addr, r))) return rc;
+    const bool mma = r.kernel == 6, tiled = r.kernel == 4, planned = r.kernel == 3;
     char *pw = base + l.plan_off;
     // dense head = the most frequent features by the corpus's own counts (bmu_opts.relabel)
     const int relabel = mma ? o.relabel : 2;        // 0 decide from the counts, 1 always, 2 never
     if ((planned || tiled || mma) && phase != 2)
         if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, mma ? head : 0, relabel, D, pw,
-                              l.plan, s)))
+                              l.plan, status, s)))
             return rc;
     if (mma) {
         if (phase != 2 &&
-            (rc = launch_plan_tiles(rowptr, N, o.tile_order == 2, head, relabel, pw, l.plan, s)))
+            (rc = launch_plan_tiles(rowptr, N, o.tile_order == 2, head, relabel, D, pw, l.plan, status, s)))
             return rc;
         if (phase == 1) return BMU_OK;
-        const int64_t m_full = M / MMA_SLAB * MMA_SLAB;
+        const int64_t m_full = r.m_full;
         uint32_t *head_max = status + 16;
         unsigned char *img = reinterpret_cast<unsigned char *>(base + l.head_off);
         const uint16_t *feat = (relabel != 2 && l.plan.fsort_tmp_bytes > 0)
@@ -282,7 +326,8 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         a.tile_head = reinterpret_cast<const uint32_t *>(pw + l.plan.tilehead_off);
         a.head_max = head_max; a.head = head; a.f16 = 0;
         a.state = state; a.state2 = state2; a.status = status;
-        const int64_t chunk = mma_chunk(o, D, M);
+        a.D = D; a.tile_rows_cap = l.plan.tile_rows_cap;
+        const int64_t chunk = r.chunk;
         float *compact = repack_bytes ? reinterpret_cast<float *>(base + l.repack_off) : nullptr;
         for (int64_t j = 0; j < m_full; j += chunk) {
             a.j_lo = (int32_t)j;
@@ -290,9 +335,9 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
             a.first = j == 0;
             if (compact) {                 // gather from a compact copy of this chunk's columns
                 const int32_t width = a.j_hi - a.j_lo;
-                repack_chunk_kernel<<<(unsigned)D, 256, 0, s>>>(
+                { repack_chunk_kernel<<<(unsigned)D, 256, 0, s>>>(
                     reinterpret_cast<const char *>(W), M * 4, j * 4, width * 4,
-                    reinterpret_cast<char *>(compact));
+                    reinterpret_cast<char *>(compact)); BMU_LAUNCHED(); }
                 a.W = reinterpret_cast<const float *>(reinterpret_cast<uintptr_t>(compact) -
                                                       (uintptr_t)j * sizeof(float));
                 a.M = width;
@@ -304,7 +349,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         if (m_full < M) {                      // ragged last slab: generic kernel, merged in
             SweepArgs g;
             g.W = W; g.D = D; g.M = M; g.norms = norms; g.rowptr = rowptr; g.colidx = colidx;
-            g.N = N; g.state = state; g.state2 = state2; g.j_lo = (int32_t)m_full;
+            g.N = N; g.state = state; g.state2 = state2; g.status = status; g.j_lo = (int32_t)m_full;
             g.j_hi = (int32_t)M; g.first = 0;
             bmu_opts go;
             memset(&go, 0, sizeof(go));
@@ -315,7 +360,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     if (tiled) {
         const int head = (o.tile_head == 1 || D < TILE_HEAD_ROWS) ? 0 : TILE_HEAD_ROWS;
         if (phase != 2 &&
-            (rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, 2, pw, l.plan, s))) return rc;
+            (rc = launch_plan_tiles(rowptr, N, o.tile_order != 1, head, 2, D, pw, l.plan, status, s))) return rc;
         if (phase == 1) return BMU_OK;
         TileArgs a;
         a.W = W; a.M = M; a.N = N; a.n_tiles = (N + 7) / 8; a.norms = norms;
@@ -325,10 +370,9 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         a.tile_ids = reinterpret_cast<const uint4 *>(pw + l.plan.tileids_off);
         a.tile_head = reinterpret_cast<const uint32_t *>(pw + l.plan.tilehead_off);
         a.head_rows = head;
-        a.state = state; a.state2 = state2;
-        const int64_t chunk = o.chunk_neurons ? (o.chunk_neurons + 127) / 128 * 128
-                                              : auto_chunk(D, M, 128);
-        const int64_t m_full = M / 128 * 128;
+        a.state = state; a.state2 = state2; a.status = status;
+        a.D = D; a.tile_rows_cap = l.plan.tile_rows_cap;
+        const int64_t chunk = r.chunk, m_full = r.m_full;
         for (int64_t j = 0; j < m_full; j += chunk) {
             a.j_lo = (int32_t)j;
             a.j_hi = (int32_t)(j + chunk < m_full ? j + chunk : m_full);
@@ -338,7 +382,7 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         if (m_full < M) {                      // ragged last slab: generic kernel, merged in
             SweepArgs g;
             g.W = W; g.D = D; g.M = M; g.norms = norms; g.rowptr = rowptr; g.colidx = colidx;
-            g.N = N; g.state = state; g.state2 = state2; g.j_lo = (int32_t)m_full;
+            g.N = N; g.state = state; g.state2 = state2; g.status = status; g.j_lo = (int32_t)m_full;
             g.j_hi = (int32_t)M; g.first = 0;
             bmu_opts go;
             memset(&go, 0, sizeof(go));
@@ -354,10 +398,9 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
         a.doc_off = reinterpret_cast<const uint32_t *>(pw + l.plan.docoff_off);
         a.ids = reinterpret_cast<const uint4 *>(pw + l.plan.ids_off);
-        a.state = state; a.state2 = state2;
-        const int64_t chunk = o.chunk_neurons ? (o.chunk_neurons + slab - 1) / slab * slab
-                                              : auto_chunk(D, M, slab);
-        const int64_t m_full = M / slab * slab;
+        a.state = state; a.state2 = state2; a.status = status;
+        a.D = D; a.id_groups_cap = l.plan.id_groups_cap;
+        const int64_t chunk = r.chunk, m_full = r.m_full;
         for (int64_t j = 0; j < m_full; j += chunk) {
             a.j_lo = (int32_t)j;
             a.j_hi = (int32_t)(j + chunk < m_full ? j + chunk : m_full);
@@ -367,21 +410,18 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         if (m_full < M) {                      // ragged last slab: generic kernel, merged in
             SweepArgs g;
             g.W = W; g.D = D; g.M = M; g.norms = norms; g.rowptr = rowptr; g.colidx = colidx;
-            g.N = N; g.state = state; g.state2 = state2; g.j_lo = (int32_t)m_full; g.j_hi = (int32_t)M; g.first = 0;
+            g.N = N; g.state = state; g.state2 = state2; g.status = status; g.j_lo = (int32_t)m_full; g.j_hi = (int32_t)M; g.first = 0;
             bmu_opts go;
             memset(&go, 0, sizeof(go));
             if ((rc = launch_sweep_direct(g, go, s))) return rc;
         }
         return launch_finalize(state, state2, rowptr, N, out_bmu, out_dist, out_bmu2, out_dist2, s);
     }
-    const int V = o.vec ? o.vec : 4;
-    const int slab = 32 * V;
     if (o.warps == 4) { set_error("generic kernel: warps must be 8, 16 or 32"); return BMU_ERR_INVALID_ARG; }
-    int64_t chunk = o.chunk_neurons ? (o.chunk_neurons + slab - 1) / slab * slab
-                                    : auto_chunk(D, M, slab);
+    const int64_t chunk = r.chunk;
     SweepArgs a;
     a.W = W; a.D = D; a.M = M; a.norms = norms; a.rowptr = rowptr; a.colidx = colidx;
-    a.N = N; a.state = state; a.state2 = state2;
+    a.N = N; a.state = state; a.state2 = state2; a.status = status;
     for (int64_t j = 0; j < M; j += chunk) {
         a.j_lo = (int32_t)j;
         a.j_hi = (int32_t)(j + chunk < M ? j + chunk : M);
@@ -417,6 +457,25 @@ static int scratch_get(size_t bytes, void **out)
     return BMU_OK;
 }
 
+// what a non-zero status word means, for the host entry points that read it back
+static int status_error(uint32_t status)
+{
+    if (status & PLAN_STATUS_OVERFLOW) {
+        set_error("the tiling pass found an offset beyond its reserved room (status word %u); "
+                  "results are invalid", status);
+        return BMU_ERR_WORKSPACE;
+    }
+    set_error("a bounded device-side wait ran out (status word %u); results are invalid", status);
+    return BMU_ERR_TIMEOUT;
+}
+
+// ORs the status word of one search into a word that outlives the next search's clearing
+__global__ void status_accumulate_kernel(const uint32_t *__restrict__ status,
+                                         uint32_t *__restrict__ sticky)
+{
+    if (*status) atomicOr(sticky, *status);
+}
+
 // ---- CSR validation ---------------------------------------------------------
 __global__ void validate_kernel(const int32_t *__restrict__ rowptr,
                                 const int32_t *__restrict__ colidx, int64_t N, int64_t nnz,
@@ -442,7 +501,7 @@ int launch_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N,
                         int64_t D, int32_t *flags, cudaStream_t s)
 {
     BMU_CUDA(cudaMemsetAsync(flags, 0, sizeof(int32_t), s));
-    validate_kernel<<<296, 256, 0, s>>>(rowptr, colidx, N, nnz, D, flags);
+    { validate_kernel<<<296, 256, 0, s>>>(rowptr, colidx, N, nnz, D, flags); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
@@ -468,7 +527,34 @@ const char *bmu_status_string(int status)
 
 const char *bmu_last_error(void) { return g_err; }
 
-int bmu_version(void) { return 100; }
+int bmu_version(void) { return 200; }
+
+uint64_t bmu_kernel_launches(void) { return g_kernel_launches; }
+
+int bmu_describe_search(int64_t D, int64_t M, int64_t N, int64_t nnz, const bmu_opts *opts,
+                        bmu_search_desc *out)
+{
+    if (!out) { set_error("null pointer argument"); return BMU_ERR_INVALID_ARG; }
+    memset(out, 0, sizeof(*out));
+    int rc = check_sizes(D, M, N, nnz);
+    if (rc) return rc;
+    bmu_opts o;
+    memset(&o, 0, sizeof(o));
+    if (opts) o = *opts;
+    if ((rc = check_opts(o))) return rc;
+    if (M == 0 || D == 0) { set_error("empty codebook"); return BMU_ERR_INVALID_ARG; }
+    Route r;
+    if ((rc = route_search(o, D, M, nnz, 0, r))) return rc;
+    out->kernel = r.kernel;
+    out->head_rows = r.head;
+    out->slab = r.slab;
+    out->docs_per_block = r.docs_per_block;
+    out->repack = r.repack;
+    out->chunk_neurons = r.chunk;
+    out->sweep_launches = (int32_t)((r.m_full + r.chunk - 1) / r.chunk);
+    out->ragged_neurons = (int32_t)(M - r.m_full);
+    return BMU_OK;
+}
 
 int bmu_codebook_norms(const float *W, int64_t D, int64_t M, float *norms, void *stream)
 {
@@ -617,8 +703,8 @@ int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
         BMU_CUDA(cudaMemsetAsync(status, 0, 256, s));
         char *pw = base + l.plan_off;
         const int relabel = o.relabel;
-        if ((rc = launch_plan(rowptr, colidx, N, nnz, 1, head, relabel, D, pw, l.plan, s))) return rc;
-        if ((rc = launch_plan_tiles(rowptr, N, o.tile_order == 2, head, relabel, pw, l.plan, s))) return rc;
+        if ((rc = launch_plan(rowptr, colidx, N, nnz, 1, head, relabel, D, pw, l.plan, status, s))) return rc;
+        if ((rc = launch_plan_tiles(rowptr, N, o.tile_order == 2, head, relabel, D, pw, l.plan, status, s))) return rc;
         unsigned char *img = reinterpret_cast<unsigned char *>(base + l.head_off);
         const uint16_t *feat = (relabel != 2 && l.plan.fsort_tmp_bytes > 0)
                                    ? reinterpret_cast<const uint16_t *>(pw + l.plan.feat_off) : nullptr;
@@ -632,6 +718,7 @@ int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
         a.tile_head = reinterpret_cast<const uint32_t *>(pw + l.plan.tilehead_off);
         a.head_max = status + 16; a.head = head; a.f16 = 1;
         a.state = state; a.state2 = state2; a.status = status;
+        a.D = D; a.tile_rows_cap = l.plan.tile_rows_cap;
         // twice the neurons per L2-resident chunk: the rows are half as wide
         const int64_t chunk = o.chunk_neurons ? mma_chunk(o, D, M) : 2 * mma_auto_chunk(D, M);
         const size_t repack_bytes = mma_repack_bytes(ow, D, M, N, nnz, top2);
@@ -643,8 +730,8 @@ int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
             a.W = static_cast<const float *>(W16); a.M = M;
             if (compact) {                 // a compact copy of this chunk's columns (2 bytes each)
                 const int32_t width = a.j_hi - a.j_lo;
-                repack_chunk_kernel<<<(unsigned)D, 256, 0, s>>>(static_cast<const char *>(W16), M * 2,
-                                                              j * 2, width * 2, compact);
+                { repack_chunk_kernel<<<(unsigned)D, 256, 0, s>>>(static_cast<const char *>(W16), M * 2,
+                                                              j * 2, width * 2, compact); BMU_LAUNCHED(); }
                 a.W = reinterpret_cast<const float *>(reinterpret_cast<uintptr_t>(compact) -
                                                       (uintptr_t)j * 2);
                 a.M = width;
@@ -654,10 +741,12 @@ int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
         }
         return launch_finalize(state, state2, rowptr, N, out_bmu, out_dist, out_bmu2, out_dist2, s);
     }
-    BMU_CUDA(cudaMemsetAsync(base + l.status_off, 0, 256, s));
+    uint32_t *status = reinterpret_cast<uint32_t *>(base + l.status_off);
+    BMU_CUDA(cudaMemsetAsync(status, 0, 256, s));
     char *pw = base + l.plan_off;
-    if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, 0, 2, D, pw, l.plan, s))) return rc;
+    if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, 0, 2, D, pw, l.plan, status, s))) return rc;
     RowsArgs a;
+    a.status = status; a.D = D; a.id_groups_cap = l.plan.id_groups_cap;
     a.W = static_cast<const float *>(W16); a.M = M; a.N = N; a.norms = norms; a.rowptr = rowptr;
     a.perm = reinterpret_cast<const int32_t *>(pw + l.plan.perm_off);
     a.doc_off = reinterpret_cast<const uint32_t *>(pw + l.plan.docoff_off);
@@ -731,10 +820,7 @@ int bmu_search_host(const float *W, int64_t D, int64_t M, const int32_t *rowptr_
     uint32_t status = 0;                               // first word of the workspace
     BMU_CUDA(cudaMemcpyAsync(&status, b, sizeof(status), cudaMemcpyDeviceToHost, s));
     BMU_CUDA(cudaStreamSynchronize(s));
-    if (status) {
-        set_error("a bounded device-side wait ran out (status word %u); results are invalid", status);
-        return BMU_ERR_TIMEOUT;
-    }
+    if (status) return status_error(status);
     return BMU_OK;
 }
 
@@ -785,9 +871,10 @@ int bmu_search_batches_host(const float *W, int64_t D, int64_t M, int32_t n_batc
         if (nnz > max_nnz) max_nnz = nnz;
     }
     if (max_n == 0) return BMU_OK;
-    // layout: shared norms | per buffer: workspace, rowptr, colidx, out_bmu, out_dist
+    // layout: status word of the whole call, shared norms | per buffer: workspace, rowptr,
+    // colidx, out_bmu, out_dist
     const size_t ws_need = bmu_search_workspace_bytes(D, M, max_n, max_nnz, nullptr);
-    const size_t norms_bytes = align_up((size_t)M * 4, 256);
+    const size_t norms_bytes = 256 + align_up((size_t)M * 4, 256);
     const size_t rp_off = align_up(ws_need, 256);
     const size_t ci_off = align_up(rp_off + (size_t)(max_n + 1) * 4, 256);
     const size_t ob_off = align_up(ci_off + (size_t)max_nnz * 4, 256);
@@ -800,7 +887,9 @@ int bmu_search_batches_host(const float *W, int64_t D, int64_t M, int32_t n_batc
     StreamCtx *c = nullptr;
     if ((rc = stream_ctx_get(dev, &c))) return rc;
     char *b = static_cast<char *>(p);
-    float *norms = reinterpret_cast<float *>(b);
+    uint32_t *sticky = reinterpret_cast<uint32_t *>(b);
+    float *norms = reinterpret_cast<float *>(b + 256);
+    BMU_CUDA(cudaMemsetAsync(sticky, 0, 256, s));
     if ((rc = launch_norms(W, D, M, norms, s))) return rc;
     for (int k = 0; k < n_batches; ++k) {
         if (N[k] == 0) continue;
@@ -821,6 +910,8 @@ int bmu_search_batches_host(const float *W, int64_t D, int64_t M, int32_t n_batc
         BMU_CUDA(cudaStreamWaitEvent(s, c->h2d[i], 0));
         if ((rc = search_impl(W, D, M, norms, rp, ci, n, nnz, ob, od, nullptr, buf, ws_need, s)))
             return rc;
+        // the next search of this buffer clears its status word: keep what this one left
+        { status_accumulate_kernel<<<1, 1, 0, s>>>(reinterpret_cast<const uint32_t *>(buf), sticky); BMU_LAUNCHED(); }
         BMU_CUDA(cudaEventRecord(c->done[i], s));
         // download on the copy stream
         BMU_CUDA(cudaStreamWaitEvent(c->copy, c->done[i], 0));
@@ -828,8 +919,30 @@ int bmu_search_batches_host(const float *W, int64_t D, int64_t M, int32_t n_batc
         BMU_CUDA(cudaMemcpyAsync(out_dist_host[k], od, (size_t)n * 4, cudaMemcpyDeviceToHost, c->copy));
         BMU_CUDA(cudaEventRecord(c->d2h[i], c->copy));
     }
+    uint32_t status = 0;
+    BMU_CUDA(cudaMemcpyAsync(&status, sticky, sizeof(status), cudaMemcpyDeviceToHost, s));
     BMU_CUDA(cudaStreamSynchronize(s));
     BMU_CUDA(cudaStreamSynchronize(c->copy));
+    if (status) return status_error(status);
+    return BMU_OK;
+}
+
+int bmu_last_status(uint32_t *out_status, void *stream)
+{
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (!out_status) { set_error("null pointer argument"); return BMU_ERR_INVALID_ARG; }
+    *out_status = 0;
+    int dev = 0;
+    BMU_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) { set_error("device ordinal %d out of range", dev); return BMU_ERR_UNSUPPORTED; }
+    void *p = nullptr;
+    {
+        std::lock_guard<std::mutex> g(g_mu);
+        p = g_scratch[dev].p;
+    }
+    if (p) BMU_CUDA(cudaMemcpyAsync(out_status, p, sizeof(uint32_t), cudaMemcpyDeviceToHost, s));
+    BMU_CUDA(cudaStreamSynchronize(s));
+    if (*out_status) return status_error(*out_status);
     return BMU_OK;
 }
 
@@ -837,18 +950,15 @@ int bmu_selftest_wait_timeout(void *stream)
 {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     void *p = nullptr;
-    int rc = scratch_get(256, &p);
+    int rc = scratch_get(512, &p);          // word 0 of the scratch stays the searches' status word
     if (rc) return rc;
-    uint32_t *status = static_cast<uint32_t *>(p);
+    uint32_t *status = reinterpret_cast<uint32_t *>(static_cast<char *>(p) + 256);
     BMU_CUDA(cudaMemsetAsync(status, 0, 256, s));
     if ((rc = launch_wait_timeout_selftest(status, s))) return rc;
     uint32_t h = 0;
     BMU_CUDA(cudaMemcpyAsync(&h, status, sizeof(h), cudaMemcpyDeviceToHost, s));
     BMU_CUDA(cudaStreamSynchronize(s));
-    if (h) {
-        set_error("a bounded device-side wait ran out (status word %u)", h);
-        return BMU_ERR_TIMEOUT;
-    }
+    if (h) return status_error(h);
     return BMU_OK;
 }
 
@@ -875,8 +985,8 @@ int bmu_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, in
     if (rc) return rc;
     if (!rowptr || (nnz > 0 && !colidx)) { set_error("null pointer argument"); return BMU_ERR_INVALID_ARG; }
     void *p = nullptr;
-    if ((rc = scratch_get(256, &p))) return rc;
-    int32_t *flags = static_cast<int32_t *>(p);
+    if ((rc = scratch_get(512, &p))) return rc;   // word 0 stays the searches' status word
+    int32_t *flags = reinterpret_cast<int32_t *>(static_cast<char *>(p) + 256);
     if ((rc = launch_validate_csr(rowptr, colidx, N, nnz, D, flags, s))) return rc;
     int32_t h = 0;
     BMU_CUDA(cudaMemcpyAsync(&h, flags, sizeof(h), cudaMemcpyDeviceToHost, s));
@@ -912,10 +1022,16 @@ int bmu_plan_create(const int32_t *rowptr, const int32_t *colidx, int64_t N, int
     if (!plan) { set_error("null pointer argument"); return BMU_ERR_INVALID_ARG; }
     *plan = nullptr;
     if (N <= 0) { set_error("a plan needs at least one document"); return BMU_ERR_INVALID_ARG; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
     int rc = search_impl(nullptr, D, M, nullptr, rowptr, colidx, N, nnz, nullptr, nullptr, opts,
-                         workspace, workspace_bytes, static_cast<cudaStream_t>(stream), nullptr,
-                         nullptr, 1);
+                         workspace, workspace_bytes, s, nullptr, nullptr, 1);
     if (rc) return rc;
+    // the searches that reuse the plan clear the status word: read the size checks of the
+    // tiling pass now
+    uint32_t status = 0;
+    BMU_CUDA(cudaMemcpyAsync(&status, workspace, sizeof(status), cudaMemcpyDeviceToHost, s));
+    BMU_CUDA(cudaStreamSynchronize(s));
+    if (status) return status_error(status);
     bmu_plan *p = new (std::nothrow) bmu_plan;
     if (!p) { set_error("out of host memory"); return BMU_ERR_INVALID_ARG; }
     p->D = D; p->M = M; p->N = N; p->nnz = nnz;

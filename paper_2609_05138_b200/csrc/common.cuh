@@ -21,6 +21,34 @@ int cuda_fail(cudaError_t e, const char *what);
         if (e__ != cudaSuccess) return bmu::cuda_fail(e__, #call); \
     } while (0)
 
+// kernels of this library that the calling thread has launched (bmu_kernel_launches)
+extern thread_local unsigned long long g_kernel_launches;
+#define BMU_LAUNCHED() (++bmu::g_kernel_launches)
+
+// ---- bounds-checked build (-DBMU_BOUNDS_CHECK) -------------------------------
+// Every address a kernel derives from a feature id, a neuron index or a scanned
+// offset is checked before it is used.  A violation sets STATUS_BOUNDS in the
+// status word and the access goes to element 0 of the same array instead (never
+// a trap, never an access outside the array); the results of that call are then
+// invalid, which the status word says.  In the normal build the macros cost nothing.
+static const uint32_t STATUS_BOUNDS = 128u;
+#ifdef __CUDACC__
+#ifdef BMU_BOUNDS_CHECK
+__device__ __forceinline__ uint32_t checked_index(unsigned long long i, unsigned long long n,
+                                                  uint32_t *status)
+{
+    if (i < n) return (uint32_t)i;
+    if (status) atomicOr(status, STATUS_BOUNDS);
+    return 0u;
+}
+#define BMU_IDX(i, n, status) bmu::checked_index((unsigned long long)(i), (unsigned long long)(n), (status))
+#define BMU_EXPECT(cond, status) do { if (!(cond) && (status)) atomicOr((status), bmu::STATUS_BOUNDS); } while (0)
+#else
+#define BMU_IDX(i, n, status) (i)
+#define BMU_EXPECT(cond, status) do { } while (0)
+#endif
+#endif
+
 // ---- (distance, index) keys ----------------------------------------------
 // A 64-bit key whose unsigned order is the lexicographic order of (distance,
 // neuron index): the smallest key is the smallest distance and, among equal
@@ -134,6 +162,7 @@ struct SweepArgs {
     int64_t N;
     u64 *state;           // per-document running (distance, index) key
     u64 *state2;          // same for the second-best unit (NULL unless it is wanted)
+    uint32_t *status;     // status word (bounds-checked build: violations are recorded here)
     int32_t j_lo, j_hi;   // neuron chunk [j_lo, j_hi)
     int32_t first;        // 1: this chunk initialises the state, 0: merges into it
 };
@@ -145,12 +174,15 @@ int launch_finalize(const u64 *state, const u64 *state2, const int32_t *rowptr, 
 struct PlanLayout {
     size_t perm_off, docoff_off, ngroups_off, bins_off, ids_off, scan_off, scan_bytes, total;
     size_t tilelen_off, tilerows_off, tileoff_off, tilehead_off, tileids_off, tile_rows_cap;
+    size_t id_groups_cap;                                                   // 16-byte id groups
     size_t rank_off, feat_off, fsort_off, fsort_tmp_off, fsort_tmp_bytes;   // feature ranks
 };
 static const int TILE_HEAD_ROWS = 32;    // ids below this are swept densely, once per tile
 static const int HEAD_ROWS_MAX = 2048;   // widest dense head (the tensor-core sweep's)
+// status-word bit set when a scanned offset of the tiling pass exceeds its reserved room
+static const uint32_t PLAN_STATUS_OVERFLOW = 64u;
 int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head, int relabel,
-                      char *ws, const PlanLayout &l, cudaStream_t s);
+                      int64_t D, char *ws, const PlanLayout &l, uint32_t *status, cudaStream_t s);
 
 // tiled sweep (sweep_tiles.cu): a warp carries 8 documents, 128-neuron slabs
 struct TileArgs {
@@ -165,6 +197,9 @@ struct TileArgs {
     int32_t head_rows;          // 0 or TILE_HEAD_ROWS
     u64 *state;
     u64 *state2;
+    uint32_t *status;           // the sweep does nothing if the tiling pass flagged an overflow
+    int64_t D;                  // rows of W, rows of the id matrices: for the bounds-checked build
+    size_t tile_rows_cap;
     int32_t j_lo, j_hi, first;
 };
 int launch_sweep_tiles(const TileArgs &a, const bmu_opts &o, cudaStream_t s);
@@ -189,6 +224,8 @@ struct MmaArgs {
     u64 *state;
     u64 *state2;                // second-best unit (NULL unless wanted)
     uint32_t *status;           // set non-zero if a bounded wait ran out
+    int64_t D;                  // rows of W, rows of the id matrices: for the bounds-checked build
+    size_t tile_rows_cap;
     int32_t j_lo, j_hi, first;
     int32_t f16;                // W is an fp16 codebook (row pitch 2 * M bytes)
 };
@@ -207,7 +244,7 @@ int launch_head_split2_f16(const void *W16, int64_t M, int64_t m_full, int head,
 size_t plan_bytes(int64_t N, int64_t nnz, int head, int64_t D, PlanLayout *l);
 int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                 int order_by_length, int head, int relabel, int64_t D, char *ws, const PlanLayout &l,
-                cudaStream_t s);
+                uint32_t *status, cudaStream_t s);
 
 static const int LANES_MAX_D = 65024;    // 16-bit ids with 0xFFFF as the end marker
 
@@ -224,6 +261,9 @@ struct RowsArgs {
     const uint4 *ids;
     u64 *state;
     u64 *state2;          // NULL unless the second-best unit is wanted
+    uint32_t *status;     // the sweep does nothing if the tiling pass flagged an overflow
+    int64_t D;            // rows of W, 16-byte id groups: for the bounds-checked build
+    size_t id_groups_cap;
     int32_t j_lo, j_hi, first;
 };
 int rows_slab_width(const bmu_opts &o);

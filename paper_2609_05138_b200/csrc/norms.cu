@@ -12,16 +12,21 @@ namespace bmu {
 
 static const int NORM_WARPS = 16;
 
-// VEC: a lane owns 4 consecutive columns (one 16-byte load per row);
-// otherwise a lane owns one column.
-template <bool VEC>
+// VEC: a lane owns 4 consecutive columns (one 16-byte load per row); otherwise a lane owns
+// one column.  LX lanes of a warp lie side by side along the columns and 32 / LX along the
+// rows: LX = 32 for wide codebooks (a warp reads 512 contiguous bytes of one row), LX = 8 for
+// narrow ones, where 128 columns per block would leave most SMs without a block.
+template <bool VEC, int LX>
 __global__ void __launch_bounds__(NORM_WARPS * 32)
 norms_kernel(const float *__restrict__ W, int64_t D, int64_t M, float *__restrict__ norms)
 {
     constexpr int C = VEC ? 4 : 1;
+    constexpr int LY = 32 / LX;                    // rows a warp reads per step
+    constexpr int RSTEP = NORM_WARPS * LY;         // rows the block reads per step
     __shared__ double part[NORM_WARPS][32 * C];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t col = (int64_t)blockIdx.x * (32 * C) + lane * C;
+    const int lx = lane % LX, ly = lane / LX;
+    const int64_t col = (int64_t)blockIdx.x * (LX * C) + lx * C;
     const bool act = col < M;
     double a[C];
 #pragma unroll
@@ -29,13 +34,13 @@ norms_kernel(const float *__restrict__ W, int64_t D, int64_t M, float *__restric
 
     if (act) {
         const float *p = W + col;
-        int64_t f = warp;
+        int64_t f = warp * LY + ly;
         // four rows in flight per thread
-        for (; f + 3 * NORM_WARPS < D; f += 4 * NORM_WARPS) {
+        for (; f + 3 * RSTEP < D; f += 4 * RSTEP) {
             float v[4][C];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const float *q = p + (f + (int64_t)u * NORM_WARPS) * M;
+                const float *q = p + (f + (int64_t)u * RSTEP) * M;
                 if constexpr (VEC) {
                     float4 t = __ldcs(reinterpret_cast<const float4 *>(q));
                     v[u][0] = t.x; v[u][1] = t.y; v[u][2] = t.z; v[u][3] = t.w;
@@ -51,7 +56,7 @@ norms_kernel(const float *__restrict__ W, int64_t D, int64_t M, float *__restric
                     a[c] = fma(w, w, a[c]);
                 }
         }
-        for (; f < D; f += NORM_WARPS) {
+        for (; f < D; f += RSTEP) {
             const float *q = p + f * M;
 #pragma unroll
             for (int c = 0; c < C; ++c) {
@@ -63,12 +68,14 @@ norms_kernel(const float *__restrict__ W, int64_t D, int64_t M, float *__restric
 #pragma unroll
     for (int c = 0; c < C; ++c) part[warp][lane * C + c] = a[c];
     __syncthreads();
-    if (threadIdx.x < 32 * C) {
-        const int64_t j = (int64_t)blockIdx.x * (32 * C) + threadIdx.x;
+    if (threadIdx.x < LX * C) {
+        const int64_t j = (int64_t)blockIdx.x * (LX * C) + threadIdx.x;
         if (j < M) {
-            double s = 0.0;
+            double s = 0.0;               // fixed order: warps, then the row lanes of a warp
 #pragma unroll
-            for (int w = 0; w < NORM_WARPS; ++w) s += part[w][threadIdx.x];
+            for (int w = 0; w < NORM_WARPS; ++w)
+#pragma unroll
+                for (int r = 0; r < LY; ++r) s += part[w][r * LX * C + threadIdx.x];
             norms[j] = (float)s;
         }
     }
@@ -113,8 +120,8 @@ norms_f16_kernel(const __half *__restrict__ W, int64_t D, int64_t M, float *__re
 int launch_norms_f16(const void *W16, int64_t D, int64_t M, float *norms, cudaStream_t s)
 {
     if (M == 0) return BMU_OK;
-    norms_f16_kernel<<<(unsigned)((M + 255) / 256), NORM_WARPS * 32, 0, s>>>(
-        static_cast<const __half *>(W16), D, M, norms);
+    { norms_f16_kernel<<<(unsigned)((M + 255) / 256), NORM_WARPS * 32, 0, s>>>(
+        static_cast<const __half *>(W16), D, M, norms); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
@@ -123,12 +130,15 @@ int launch_norms(const float *W, int64_t D, int64_t M, float *norms, cudaStream_
 {
     if (M == 0) return BMU_OK;
     const bool vec = (M % 4 == 0) && ((reinterpret_cast<uintptr_t>(W) & 15) == 0);
-    const int cols = vec ? 128 : 32;
-    const int64_t blocks = (M + cols - 1) / cols;
-    if (vec)
-        norms_kernel<true><<<(unsigned)blocks, NORM_WARPS * 32, 0, s>>>(W, D, M, norms);
-    else
-        norms_kernel<false><<<(unsigned)blocks, NORM_WARPS * 32, 0, s>>>(W, D, M, norms);
+    const int c = vec ? 4 : 1;
+    // narrow codebooks: 8 lanes across the columns, so that there are blocks for every SM
+    const bool narrow = (M + 32 * c - 1) / (32 * c) < 296;
+    const int cols = (narrow ? 8 : 32) * c;
+    const unsigned blocks = (unsigned)((M + cols - 1) / cols);
+    if (vec && narrow) { norms_kernel<true, 8><<<blocks, NORM_WARPS * 32, 0, s>>>(W, D, M, norms); BMU_LAUNCHED(); }
+    else if (vec) { norms_kernel<true, 32><<<blocks, NORM_WARPS * 32, 0, s>>>(W, D, M, norms); BMU_LAUNCHED(); }
+    else if (narrow) { norms_kernel<false, 8><<<blocks, NORM_WARPS * 32, 0, s>>>(W, D, M, norms); BMU_LAUNCHED(); }
+    else { norms_kernel<false, 32><<<blocks, NORM_WARPS * 32, 0, s>>>(W, D, M, norms); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

@@ -1,19 +1,16 @@
 // The document-tiling pass (Section 4.1 "tile size", Section 4.2 "tile
-// membership"): turns the caller's CSR into the form the staged sweep walks.
-//
-// The staged sweep gives every lane of a thread block one document, so a
-// "tile" here is the 992 documents of one block, which share every staged
-// codebook row.  The pass
-//   1. orders documents by length (longest first) so that the 32 lanes of a
-//      warp, which step through their feature lists together, carry similar
-//      numbers of features;
+// membership"): turns the caller's CSR into the form the planned, tiled and
+// tensor-core sweeps walk.  The pass
+//   1. orders documents by length (longest first; by the length of the gathered
+//      list when there is a dense head) so that the documents that share a warp,
+//      a tile or a block carry similar numbers of features and finish together;
 //   2. re-packs every row as ascending 16-bit feature ids in 16-byte groups
 //      (8 ids), padded with the sentinel 0xFFFF and closed by one all-sentinel
-//      group, so a lane fetches eight ids with one aligned 128-bit load and
-//      stops by itself at the end of its row.
-//   3. (tiled sweep only) cuts the length-ordered documents into tiles of 8 and
-//      writes, per tile, an id matrix: row b holds the b-th id of each of the
-//      tile's 8 documents (0xFFFF where a document has run out), so one aligned
+//      group, so eight ids arrive with one aligned 128-bit load and a list
+//      ends by itself;
+//   3. (tiled and tensor-core sweeps) cuts the length-ordered documents into tiles
+//      of 8 and writes, per tile, an id matrix: row b holds the b-th id of each of
+//      the tile's 8 documents (0xFFFF where a document has run out), so one aligned
 //      128-bit load hands a warp the next row of all eight documents.
 // Integer work only; the order of documents never changes any result because
 // every document is reduced on its own.
@@ -106,7 +103,8 @@ __global__ void plan_rank_tables_kernel(const uint32_t *__restrict__ sorted, int
 __global__ void __launch_bounds__(256)
 plan_key_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colidx,
                 const uint16_t *__restrict__ rank, int64_t N, int32_t head,
-                uint32_t *__restrict__ key)
+                uint32_t *__restrict__ key, [[maybe_unused]] int64_t D,
+                [[maybe_unused]] uint32_t *__restrict__ status)
 {
     __shared__ uint32_t seen[8][HEAD_ROWS_MAX / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -117,7 +115,7 @@ plan_key_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ 
     const int beg = rowptr[i], end = rowptr[i + 1];
     int cnt = 0, repeat = 0;
     for (int e = beg + lane; e < end; e += 32) {
-        const int32_t r = rank ? (int32_t)rank[colidx[e]] : colidx[e];
+        const int32_t r = rank ? (int32_t)rank[BMU_IDX((uint32_t)colidx[e], D, status)] : colidx[e];
         if (r >= head) {
             ++cnt;
         } else {
@@ -131,68 +129,93 @@ plan_key_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ 
     if (lane == 0) key[i] = repeat ? (uint32_t)(end - beg) : (uint32_t)cnt;
 }
 
+// histogram of the sorting keys, and the largest key (aux[0]) so that the scan below can
+// leave out the bins no document falls into
 __global__ void plan_hist_kernel(const int32_t *__restrict__ rowptr,
                                  const uint32_t *__restrict__ key, int64_t N,
-                                 uint32_t *__restrict__ hist)
+                                 uint32_t *__restrict__ hist, uint32_t *__restrict__ aux)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= N) return;
-    const int len = key ? (int)key[i] : rowptr[i + 1] - rowptr[i];
-    const int bin = PLAN_BINS - 1 - min(len, PLAN_BINS - 1);      // longest rows first
-    atomicAdd(hist + bin, 1u);
+    int len = 0;
+    if (i < N) {
+        len = min(key ? (int)key[i] : rowptr[i + 1] - rowptr[i], PLAN_BINS - 1);
+        atomicAdd(hist + (PLAN_BINS - 1 - len), 1u);              // longest rows first
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) len = max(len, __shfl_xor_sync(0xffffffffu, len, off));
+    if ((threadIdx.x & 31) == 0 && len > 0) atomicMax(aux, (uint32_t)len);
 }
 
-// exclusive scan of the PLAN_BINS counters (one block of 1024 threads, 64 bins each)
+// Exclusive scan of the bin counters from the first bin that can hold a document (the one of
+// the largest key, aux[0]) to the last.  One block of 32 warps: a warp owns a contiguous run
+// of bins and walks it 32 bins at a time (coalesced loads, shuffle scan); first the runs'
+// totals, then the scan proper with each run's offset.
 __global__ void __launch_bounds__(1024)
-plan_scan_bins_kernel(const uint32_t *__restrict__ hist, uint32_t *__restrict__ cursor)
+plan_scan_bins_kernel(const uint32_t *__restrict__ hist, const uint32_t *__restrict__ aux,
+                      uint32_t *__restrict__ cursor)
 {
-    constexpr int PER = PLAN_BINS / 1024;
-    __shared__ uint32_t s[1024];
-    const int t = threadIdx.x;
-    uint32_t sum = 0;
-    for (int i = 0; i < PER; ++i) sum += hist[t * PER + i];
-    s[t] = sum;
+    __shared__ uint32_t s_tot[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lo = PLAN_BINS - 1 - (int)min(aux[0], (uint32_t)(PLAN_BINS - 1));
+    const int per = ((PLAN_BINS - lo + 31) / 32 + 31) / 32 * 32;      // bins per warp, whole steps
+    const int beg = lo + warp * per, end = min(beg + per, PLAN_BINS);
+    uint32_t tot = 0;
+    for (int b = beg + lane; b < end; b += 32) tot += hist[b];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, off);
+    if (lane == 0) s_tot[warp] = tot;
     __syncthreads();
-    for (int off = 1; off < 1024; off <<= 1) {
-        const uint32_t v = t >= off ? s[t - off] : 0u;
-        __syncthreads();
-        s[t] += v;
-        __syncthreads();
-    }
-    uint32_t run = s[t] - sum;
-    for (int i = 0; i < PER; ++i) {
-        cursor[t * PER + i] = run;
-        run += hist[t * PER + i];
+    uint32_t run = 0;
+    for (int w = 0; w < warp; ++w) run += s_tot[w];
+    for (int b0 = beg; b0 < end; b0 += 32) {
+        const int b = b0 + lane;
+        const uint32_t h = b < end ? hist[b] : 0u;
+        uint32_t inc = h;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xffffffffu, inc, off);
+            if (lane >= off) inc += v;
+        }
+        if (b < end) cursor[b] = run + inc - h;
+        run += __shfl_sync(0xffffffffu, inc, 31);
     }
 }
 
+// a document's planned position, and the groups of 8 ids its row needs there (plus its closing
+// sentinel group); ngroups[N] = 0 closes the array for the scan
 __global__ void plan_scatter_kernel(const int32_t *__restrict__ rowptr,
                                     const uint32_t *__restrict__ key, int64_t N,
-                                    uint32_t *__restrict__ cursor, int32_t *__restrict__ perm)
+                                    uint32_t *__restrict__ cursor, int32_t *__restrict__ perm,
+                                    uint32_t *__restrict__ ngroups)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i == 0) ngroups[N] = 0u;
     if (i >= N) return;
-    const int len = key ? (int)key[i] : rowptr[i + 1] - rowptr[i];
+    const int row = rowptr[i + 1] - rowptr[i];
+    const int len = key ? (int)key[i] : row;
     const int bin = PLAN_BINS - 1 - min(len, PLAN_BINS - 1);
-    perm[atomicAdd(cursor + bin, 1u)] = (int32_t)i;
+    const uint32_t p = atomicAdd(cursor + bin, 1u);
+    perm[p] = (int32_t)i;
+    ngroups[p] = (uint32_t)((row + 7) / 8 + 1);
 }
 
-__global__ void plan_identity_kernel(int64_t N, int32_t *__restrict__ perm)
+__global__ void plan_identity_kernel(const int32_t *__restrict__ rowptr, int64_t N,
+                                     int32_t *__restrict__ perm, uint32_t *__restrict__ ngroups)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < N) perm[i] = (int32_t)i;
+    if (i == 0) ngroups[N] = 0u;
+    if (i >= N) return;
+    perm[i] = (int32_t)i;
+    ngroups[i] = (uint32_t)((rowptr[i + 1] - rowptr[i] + 7) / 8 + 1);
 }
 
-// groups of 8 ids the row at planned position p needs (plus its closing sentinel group)
-__global__ void plan_groups_kernel(const int32_t *__restrict__ rowptr,
-                                   const int32_t *__restrict__ perm, int64_t N,
-                                   uint32_t *__restrict__ ngroups)
+// Size checks of the pass (one thread): the scanned offsets must fit the room that was
+// reserved for what they index.  A failure sets bit 64 of the status word; the kernels that
+// would write through those offsets, and every sweep, then do nothing.
+__global__ void plan_check_kernel(const uint32_t *__restrict__ last_off, uint64_t room,
+                                  uint32_t *__restrict__ status)
 {
-    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (p >= N) return;
-    const int32_t i = perm[p];
-    const int len = rowptr[i + 1] - rowptr[i];
-    ngroups[p] = (uint32_t)((len + 7) / 8 + 1);
+    if ((uint64_t)*last_off > room) atomicOr(status, PLAN_STATUS_OVERFLOW);
 }
 
 // One warp per planned document: writes its ascending 16-bit id list.  Rows that
@@ -201,10 +224,12 @@ __global__ void plan_groups_kernel(const int32_t *__restrict__ rowptr,
 __global__ void __launch_bounds__(256)
 plan_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colidx,
                  const uint16_t *__restrict__ rank, const int32_t *__restrict__ perm,
-                 const uint32_t *__restrict__ doc_off, int64_t N, uint16_t *__restrict__ ids16)
+                 const uint32_t *__restrict__ doc_off, int64_t N, uint16_t *__restrict__ ids16,
+                 uint32_t *__restrict__ status, [[maybe_unused]] int64_t D)
 {
+    if (*status & PLAN_STATUS_OVERFLOW) return;
     // with a rank table the list holds ranks (ascending: most frequent first), not ids
-#define BMU_PLAN_ID(e) (rank ? (int32_t)rank[row[e]] : row[e])
+#define BMU_PLAN_ID(e) (rank ? (int32_t)rank[BMU_IDX((uint32_t)row[e], D, status)] : row[e])
     const int lane = threadIdx.x & 31;
     const int64_t p = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (p >= N) return;
@@ -309,8 +334,10 @@ plan_tile_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restr
                       const uint32_t *__restrict__ tile_len, const uint32_t *__restrict__ tile_off,
                       const uint32_t *__restrict__ tile_head, uint32_t head_words,
                       const uint16_t *__restrict__ feat_of_rank, int64_t N, int64_t n_tiles,
-                      int interleave, uint4 *__restrict__ tile_ids)
+                      int interleave, uint4 *__restrict__ tile_ids,
+                      uint32_t *__restrict__ status, [[maybe_unused]] int64_t D)
 {
+    if (*status & PLAN_STATUS_OVERFLOW) return;
     const int lane = threadIdx.x & 31;
     const int64_t tile = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (tile >= n_tiles) return;
@@ -337,7 +364,8 @@ plan_tile_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restr
             uint32_t e = r;
             if (interleave) e = (r & 1u) ? (len[t] + 1) / 2 + r / 2 : r / 2;
             f[t] = r < len[t] ? src[t][e] : 0xffffu;
-            if (feat_of_rank && f[t] != 0xffffu) f[t] = feat_of_rank[f[t]];   // rank -> row of W
+            if (feat_of_rank && f[t] != 0xffffu)                              // rank -> row of W
+                f[t] = feat_of_rank[BMU_IDX(f[t], D, status)];
         }
         dst[r] = make_uint4(f[0] | (f[1] << 16), f[2] | (f[3] << 16), f[4] | (f[5] << 16),
                             f[6] | (f[7] << 16));
@@ -352,9 +380,9 @@ size_t plan_bytes(int64_t N, int64_t nnz, int head, int64_t D, PlanLayout *l)
     t.perm_off = off; off = up(off + (size_t)N * 4);
     t.docoff_off = off; off = up(off + (size_t)(N + 1) * 4);
     t.ngroups_off = off; off = up(off + (size_t)(N + 1) * 4);
-    t.bins_off = off; off = up(off + (size_t)PLAN_BINS * 4 * 2);
-    const size_t groups = (size_t)nnz / 8 + 2 * (size_t)N + 4;
-    t.ids_off = off; off = up(off + groups * 16);
+    t.bins_off = off; off = up(off + (size_t)PLAN_BINS * 4 * 2 + 256);   // counters, cursors, aux
+    t.id_groups_cap = (size_t)nnz / 8 + 2 * (size_t)N + 4;
+    t.ids_off = off; off = up(off + t.id_groups_cap * 16);
     size_t scan_tmp = 0;
     cub::DeviceScan::ExclusiveSum(nullptr, scan_tmp, (uint32_t *)nullptr, (uint32_t *)nullptr,
                                   (int)(N + 1));
@@ -388,7 +416,7 @@ size_t plan_bytes(int64_t N, int64_t nnz, int head, int64_t D, PlanLayout *l)
 
 int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                 int order_by_length, int head, int relabel, int64_t D, char *ws, const PlanLayout &l,
-                cudaStream_t s)
+                uint32_t *status, cudaStream_t s)
 {
     // dense head: rank the features by how many documents list them, so that the head is the
     // `head` most frequent features whatever their ids
@@ -414,20 +442,20 @@ int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t
             }
             for (int32_t lo = 0; lo < (int32_t)D; lo += span) {
                 const int32_t hi = lo + span < (int32_t)D ? lo + span : (int32_t)D;
-                plan_feat_hist_kernel<<<148, 1024, (size_t)(hi - lo) * 4, s>>>(colidx, nnz, lo, hi, count);
+                { plan_feat_hist_kernel<<<148, 1024, (size_t)(hi - lo) * 4, s>>>(colidx, nnz, lo, hi, count); BMU_LAUNCHED(); }
             }
         }
-        plan_iota_kernel<<<(unsigned)((D + 255) / 256), 256, 0, s>>>((int32_t)D, ids);
+        { plan_iota_kernel<<<(unsigned)((D + 255) / 256), 256, 0, s>>>((int32_t)D, ids); BMU_LAUNCHED(); }
         size_t tmp = l.fsort_tmp_bytes;
         BMU_CUDA(cub::DeviceRadixSort::SortPairsDescending(ws + l.fsort_tmp_off, tmp, count, count_sorted,
                                                            ids, ids_sorted, (int)D, 0, 32, s));
         // the decision word borrows the first counter of the length histogram (cleared below)
         uint32_t *keep_ids = reinterpret_cast<uint32_t *>(ws + l.bins_off);
-        plan_rank_decide_kernel<<<1, 1024, 0, s>>>(count, count_sorted, (int32_t)D, head, relabel == 1,
-                                                   keep_ids);
-        plan_rank_tables_kernel<<<(unsigned)((D + 255) / 256), 256, 0, s>>>(ids_sorted, (int32_t)D,
+        { plan_rank_decide_kernel<<<1, 1024, 0, s>>>(count, count_sorted, (int32_t)D, head, relabel == 1,
+                                                   keep_ids); BMU_LAUNCHED(); }
+        { plan_rank_tables_kernel<<<(unsigned)((D + 255) / 256), 256, 0, s>>>(ids_sorted, (int32_t)D,
                                                                             keep_ids, rank_of_feat,
-                                                                            feat_of_rank);
+                                                                            feat_of_rank); BMU_LAUNCHED(); }
         rank = rank_of_feat;
     }
     int32_t *perm = reinterpret_cast<int32_t *>(ws + l.perm_off);
@@ -435,37 +463,40 @@ int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t
     uint32_t *ngroups = reinterpret_cast<uint32_t *>(ws + l.ngroups_off);
     uint32_t *hist = reinterpret_cast<uint32_t *>(ws + l.bins_off);
     uint32_t *cursor = hist + PLAN_BINS;
+    uint32_t *aux = cursor + PLAN_BINS;              // [0] the largest sorting key
     uint16_t *ids16 = reinterpret_cast<uint16_t *>(ws + l.ids_off);
     const unsigned blocks = (unsigned)((N + 255) / 256);
     if (order_by_length) {
         // with a dense head the documents are ordered by what is left for the gather, so that
-        // the documents of a tile finish their lists together (the key borrows the ngroups
-        // array, which is written only after the scatter)
+        // the documents of a tile finish their lists together (the key borrows the doc_off
+        // array, which is written only by the scan after the scatter)
         const uint32_t *key = nullptr;
         if (head > 0) {
-            plan_key_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(rowptr, colidx, rank, N,
-                                                                            head, ngroups);
-            key = ngroups;
+            { plan_key_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(rowptr, colidx, rank, N,
+                                                                            head, doc_off, D, status); BMU_LAUNCHED(); }
+            key = doc_off;
         }
-        BMU_CUDA(cudaMemsetAsync(hist, 0, PLAN_BINS * 4, s));
-        plan_hist_kernel<<<blocks, 256, 0, s>>>(rowptr, key, N, hist);
-        plan_scan_bins_kernel<<<1, 1024, 0, s>>>(hist, cursor);
-        plan_scatter_kernel<<<blocks, 256, 0, s>>>(rowptr, key, N, cursor, perm);
+        // counters and the largest key in one clearing (the cursors in between are all written
+        // or never read)
+        BMU_CUDA(cudaMemsetAsync(hist, 0, (size_t)PLAN_BINS * 4 * 2 + 256, s));
+        { plan_hist_kernel<<<blocks, 256, 0, s>>>(rowptr, key, N, hist, aux); BMU_LAUNCHED(); }
+        { plan_scan_bins_kernel<<<1, 1024, 0, s>>>(hist, aux, cursor); BMU_LAUNCHED(); }
+        { plan_scatter_kernel<<<blocks, 256, 0, s>>>(rowptr, key, N, cursor, perm, ngroups); BMU_LAUNCHED(); }
     } else {
-        plan_identity_kernel<<<blocks, 256, 0, s>>>(N, perm);
+        { plan_identity_kernel<<<blocks, 256, 0, s>>>(rowptr, N, perm, ngroups); BMU_LAUNCHED(); }
     }
-    plan_groups_kernel<<<blocks, 256, 0, s>>>(rowptr, perm, N, ngroups);
-    BMU_CUDA(cudaMemsetAsync(ngroups + N, 0, 4, s));
     size_t tmp = l.scan_bytes;
     BMU_CUDA(cub::DeviceScan::ExclusiveSum(ws + l.scan_off, tmp, ngroups, doc_off, (int)(N + 1), s));
-    plan_fill_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(rowptr, colidx, rank, perm,
-                                                                       doc_off, N, ids16);
+    // group 0 is the global sentinel and two groups of slack close the lists
+    { plan_check_kernel<<<1, 1, 0, s>>>(doc_off + N, (uint64_t)l.id_groups_cap - 3, status); BMU_LAUNCHED(); }
+    { plan_fill_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(rowptr, colidx, rank, perm,
+                                                                       doc_off, N, ids16, status, D); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
 
 int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head, int relabel,
-                      char *ws, const PlanLayout &l, cudaStream_t s)
+                      int64_t D, char *ws, const PlanLayout &l, uint32_t *status, cudaStream_t s)
 {
     const uint16_t *feat_of_rank = (head > 0 && relabel != 2 && l.fsort_tmp_bytes > 0)
                                        ? reinterpret_cast<const uint16_t *>(ws + l.feat_off) : nullptr;
@@ -478,15 +509,17 @@ int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head
     uint32_t *tile_off = reinterpret_cast<uint32_t *>(ws + l.tileoff_off);
     uint4 *tile_ids = reinterpret_cast<uint4 *>(ws + l.tileids_off);
     uint32_t *tile_head = reinterpret_cast<uint32_t *>(ws + l.tilehead_off);
-    plan_tile_len_kernel<<<(unsigned)((n_tiles * 8 + 255) / 256), 256, 0, s>>>(
-        rowptr, perm, doc_off, ids16, N, n_tiles, (uint32_t)head, tile_rows, tile_len, tile_head);
+    { plan_tile_len_kernel<<<(unsigned)((n_tiles * 8 + 255) / 256), 256, 0, s>>>(
+        rowptr, perm, doc_off, ids16, N, n_tiles, (uint32_t)head, tile_rows, tile_len, tile_head); BMU_LAUNCHED(); }
     BMU_CUDA(cudaMemsetAsync(tile_rows + n_tiles, 0, 4, s));
     size_t tmp = l.scan_bytes;
     BMU_CUDA(cub::DeviceScan::ExclusiveSum(ws + l.scan_off, tmp, tile_rows, tile_off,
                                            (int)(n_tiles + 1), s));
-    plan_tile_fill_kernel<<<(unsigned)((n_tiles * 32 + 255) / 256), 256, 0, s>>>(
+    // the sweeps read one row past a tile's last (the next row is fetched ahead)
+    { plan_check_kernel<<<1, 1, 0, s>>>(tile_off + n_tiles, (uint64_t)l.tile_rows_cap - 1, status); BMU_LAUNCHED(); }
+    { plan_tile_fill_kernel<<<(unsigned)((n_tiles * 32 + 255) / 256), 256, 0, s>>>(
         rowptr, perm, doc_off, ids16, tile_len, tile_off, tile_head,
-        (uint32_t)(head ? head / 32 : 1), feat_of_rank, N, n_tiles, interleave, tile_ids);
+        (uint32_t)(head ? head / 32 : 1), feat_of_rank, N, n_tiles, interleave, tile_ids, status, D); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

@@ -85,7 +85,7 @@ sweep_direct_kernel(const SweepArgs a)
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
                             const uint32_t f = (uint32_t)__shfl_sync(0xffffffffu, myf, q + u);
-                            const u64 off = (u64)f * rowbytes;
+                            const u64 off = (u64)BMU_IDX(f, a.D, a.status) * rowbytes;
 #pragma unroll
                             for (int h = 0; h < H; ++h)
                                 w[u][h] = act[h]
@@ -102,7 +102,7 @@ sweep_direct_kernel(const SweepArgs a)
                     }
                     for (; q < c; ++q) {
                         const uint32_t f = (uint32_t)__shfl_sync(0xffffffffu, myf, q);
-                        const u64 off = (u64)f * rowbytes;
+                        const u64 off = (u64)BMU_IDX(f, a.D, a.status) * rowbytes;
 #pragma unroll
                         for (int h = 0; h < H; ++h) {
                             const ulonglong2 w = act[h]
@@ -126,7 +126,7 @@ sweep_direct_kernel(const SweepArgs a)
                     const int c = min(32, end[k] - eb);
                     for (int q = 0; q < c; ++q) {
                         const uint32_t f = (uint32_t)__shfl_sync(0xffffffffu, myf, q);
-                        const u64 off = (u64)f * rowbytes;
+                        const u64 off = (u64)BMU_IDX(f, a.D, a.status) * rowbytes;
 #pragma unroll
                         for (int h = 0; h < H; ++h)
                             if (act[h])
@@ -167,10 +167,11 @@ sweep_rows_kernel(const RowsArgs a)
     constexpr int H = V / 4;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t p = (int64_t)blockIdx.x * NW + warp;
-    if (p >= a.N) return;
+    if (p >= a.N || (__ldg(a.status) & PLAN_STATUS_OVERFLOW)) return;
     const int32_t orig = __ldg(a.perm + p);
     const int len = __ldg(a.rowptr + orig + 1) - __ldg(a.rowptr + orig);
-    const uint4 *gp = a.ids + (size_t)__ldg(a.doc_off + p) + 1;
+    const uint4 *gp = a.ids + BMU_IDX((size_t)__ldg(a.doc_off + p) + 1, a.id_groups_cap, a.status);
+    [[maybe_unused]] const size_t room = a.id_groups_cap - (size_t)(gp - a.ids);
     const int full = len >> 3, rem = len & 7;
     const uint32_t rowbytes = (uint32_t)(a.M * 4);
     Best<TOP2> best;
@@ -183,7 +184,7 @@ sweep_rows_kernel(const RowsArgs a)
         for (int h = 0; h < H; ++h) acc[h][0] = acc[h][1] = 0ull;
 
         for (int g = 0; g < full; ++g) {
-            const uint4 t = __ldg(gp + g);
+            const uint4 t = __ldg(gp + BMU_IDX(g, room, a.status));
             const uint32_t f[8] = {t.x & 0xffffu, t.x >> 16, t.y & 0xffffu, t.y >> 16,
                                    t.z & 0xffffu, t.z >> 16, t.w & 0xffffu, t.w >> 16};
             ulonglong2 w[8][H];
@@ -192,7 +193,7 @@ sweep_rows_kernel(const RowsArgs a)
 #pragma unroll
                 for (int h = 0; h < H; ++h)
                     w[u][h] = __ldg(reinterpret_cast<const ulonglong2 *>(
-                        base + (u64)f[u] * rowbytes + h * 512));
+                        base + (u64)BMU_IDX(f[u], a.D, a.status) * rowbytes + h * 512));
 #pragma unroll
             for (int u = 0; u < 8; ++u)
 #pragma unroll
@@ -202,7 +203,7 @@ sweep_rows_kernel(const RowsArgs a)
                 }
         }
         if (rem) {
-            const uint4 t = __ldg(gp + full);
+            const uint4 t = __ldg(gp + BMU_IDX(full, room, a.status));
             const uint32_t f[8] = {t.x & 0xffffu, t.x >> 16, t.y & 0xffffu, t.y >> 16,
                                    t.z & 0xffffu, t.z >> 16, t.w & 0xffffu, t.w >> 16};
 #pragma unroll
@@ -211,7 +212,7 @@ sweep_rows_kernel(const RowsArgs a)
 #pragma unroll
                     for (int h = 0; h < H; ++h) {
                         const ulonglong2 w = __ldg(reinterpret_cast<const ulonglong2 *>(
-                            base + (u64)f[u] * rowbytes + h * 512));
+                            base + (u64)BMU_IDX(f[u], a.D, a.status) * rowbytes + h * 512));
                         add2(acc[h][0], w.x);
                         add2(acc[h][1], w.y);
                     }
@@ -233,8 +234,8 @@ sweep_rows_kernel(const RowsArgs a)
 }
 
 // ---------------------------------------------------------------------------
-// Half-precision codebook (the paper's own storage, Section 4.2/4.3: "two bytes
-// per half-precision weight", __half2 loads): the planned kernel with rows of
+// Half-precision codebook (the paper's own storage, Section 4.2/4.3: 2 bytes per
+// weight, loaded as pairs of halves): the planned kernel with rows of
 // fp16, eight neurons per 128-bit load, widened to fp32 in registers and
 // accumulated in fp32.  Slab = 256 neurons.
 template <int NW, bool TOP2>
@@ -243,10 +244,11 @@ sweep_rows_f16_kernel(const RowsArgs a)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t p = (int64_t)blockIdx.x * NW + warp;
-    if (p >= a.N) return;
+    if (p >= a.N || (__ldg(a.status) & PLAN_STATUS_OVERFLOW)) return;
     const int32_t orig = __ldg(a.perm + p);
     const int len = __ldg(a.rowptr + orig + 1) - __ldg(a.rowptr + orig);
-    const uint4 *gp = a.ids + (size_t)__ldg(a.doc_off + p) + 1;
+    const uint4 *gp = a.ids + BMU_IDX((size_t)__ldg(a.doc_off + p) + 1, a.id_groups_cap, a.status);
+    [[maybe_unused]] const size_t room = a.id_groups_cap - (size_t)(gp - a.ids);
     const int full = len >> 3, rem = len & 7;
     const uint32_t rowbytes = (uint32_t)(a.M * 2);
     const __half *W16 = reinterpret_cast<const __half *>(a.W);
@@ -269,24 +271,24 @@ sweep_rows_f16_kernel(const RowsArgs a)
             }
         };
         for (int g = 0; g < full; ++g) {
-            const uint4 t = __ldg(gp + g);
+            const uint4 t = __ldg(gp + BMU_IDX(g, room, a.status));
             const uint32_t f[8] = {t.x & 0xffffu, t.x >> 16, t.y & 0xffffu, t.y >> 16,
                                    t.z & 0xffffu, t.z >> 16, t.w & 0xffffu, t.w >> 16};
             uint4 w[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u)
-                w[u] = __ldg(reinterpret_cast<const uint4 *>(base + (u64)f[u] * rowbytes));
+                w[u] = __ldg(reinterpret_cast<const uint4 *>(base + (u64)BMU_IDX(f[u], a.D, a.status) * rowbytes));
 #pragma unroll
             for (int u = 0; u < 8; ++u) add_row(w[u]);
         }
         if (rem) {
-            const uint4 t = __ldg(gp + full);
+            const uint4 t = __ldg(gp + BMU_IDX(full, room, a.status));
             const uint32_t f[8] = {t.x & 0xffffu, t.x >> 16, t.y & 0xffffu, t.y >> 16,
                                    t.z & 0xffffu, t.z >> 16, t.w & 0xffffu, t.w >> 16};
 #pragma unroll
             for (int u = 0; u < 7; ++u)
                 if (u < rem)
-                    add_row(__ldg(reinterpret_cast<const uint4 *>(base + (u64)f[u] * rowbytes)));
+                    add_row(__ldg(reinterpret_cast<const uint4 *>(base + (u64)BMU_IDX(f[u], a.D, a.status) * rowbytes)));
         }
         const int col = j0 + lane * 8;
 #pragma unroll
@@ -312,8 +314,8 @@ int launch_sweep_rows_f16(const RowsArgs &a, const bmu_opts &o, cudaStream_t s)
 #define BMU_CASE(nw)                                                                      \
     if (NW == nw) {                                                                       \
         const unsigned blocks = (unsigned)((a.N + nw - 1) / nw);                          \
-        if (a.state2) sweep_rows_f16_kernel<nw, true><<<blocks, nw * 32, 0, s>>>(a);      \
-        else sweep_rows_f16_kernel<nw, false><<<blocks, nw * 32, 0, s>>>(a);              \
+        if (a.state2) { sweep_rows_f16_kernel<nw, true><<<blocks, nw * 32, 0, s>>>(a); BMU_LAUNCHED(); }      \
+        else { sweep_rows_f16_kernel<nw, false><<<blocks, nw * 32, 0, s>>>(a); BMU_LAUNCHED(); }              \
         BMU_CUDA(cudaGetLastError());                                                     \
         return BMU_OK;                                                                    \
     }
@@ -329,8 +331,8 @@ static int launch_rows_v(const RowsArgs &a, int NW, cudaStream_t s)
 #define BMU_CASE(nw)                                                                   \
     if (NW == nw) {                                                                    \
         const unsigned blocks = (unsigned)((a.N + nw - 1) / nw);                       \
-        if (a.state2) sweep_rows_kernel<V, nw, true><<<blocks, nw * 32, 0, s>>>(a);    \
-        else sweep_rows_kernel<V, nw, false><<<blocks, nw * 32, 0, s>>>(a);            \
+        if (a.state2) { sweep_rows_kernel<V, nw, true><<<blocks, nw * 32, 0, s>>>(a); BMU_LAUNCHED(); }    \
+        else { sweep_rows_kernel<V, nw, false><<<blocks, nw * 32, 0, s>>>(a); BMU_LAUNCHED(); }            \
         BMU_CUDA(cudaGetLastError());                                                  \
         return BMU_OK;                                                                 \
     }
@@ -381,8 +383,8 @@ int launch_finalize(const u64 *state, const u64 *state2, const int32_t *rowptr, 
                     cudaStream_t s)
 {
     if (N == 0) return BMU_OK;
-    finalize_kernel<<<(unsigned)((N + 255) / 256), 256, 0, s>>>(state, state2, rowptr, N, out_bmu,
-                                                                out_dist, out_bmu2, out_dist2);
+    { finalize_kernel<<<(unsigned)((N + 255) / 256), 256, 0, s>>>(state, state2, rowptr, N, out_bmu,
+                                                                out_dist, out_bmu2, out_dist2); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
@@ -393,9 +395,9 @@ static int launch_one(const SweepArgs &a, cudaStream_t s)
     const int64_t per_block = (int64_t)NW * K;
     const int64_t blocks = (a.N + per_block - 1) / per_block;
     if (a.state2)
-        sweep_direct_kernel<V, K, NW, VEC, true><<<(unsigned)blocks, NW * 32, 0, s>>>(a);
+        { sweep_direct_kernel<V, K, NW, VEC, true><<<(unsigned)blocks, NW * 32, 0, s>>>(a); BMU_LAUNCHED(); }
     else
-        sweep_direct_kernel<V, K, NW, VEC, false><<<(unsigned)blocks, NW * 32, 0, s>>>(a);
+        { sweep_direct_kernel<V, K, NW, VEC, false><<<(unsigned)blocks, NW * 32, 0, s>>>(a); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

@@ -73,7 +73,7 @@ int launch_head_absmax(const float *W, int64_t M, int64_t m_full, int head, cons
                        uint32_t *head_max, cudaStream_t s)
 {
     BMU_CUDA(cudaMemsetAsync(head_max, 0, sizeof(uint32_t), s));
-    head_absmax_kernel<<<592, 256, 0, s>>>(W, M, m_full, head, feat, head_max);
+    { head_absmax_kernel<<<592, 256, 0, s>>>(W, M, m_full, head, feat, head_max); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
@@ -118,7 +118,7 @@ int launch_head_split2(const float *W, int64_t M, int64_t m_full, int head, cons
     int rc = launch_head_absmax(W, M, m_full, head, feat, head_max, s);
     if (rc) return rc;
     const dim3 grid((unsigned)(m_full / M2_SLAB), head / 8);
-    head_split2_kernel<<<grid, M2_SLAB, 0, s>>>(W, M, head_max, head, feat, head_img);
+    { head_split2_kernel<<<grid, M2_SLAB, 0, s>>>(W, M, head_max, head, feat, head_img); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
@@ -203,7 +203,7 @@ sweep_mma2_kernel(const MmaArgs a)
         const uint32_t off = there ? __ldg(a.tile_off + tile) : 0u;
         s_len[t] = there ? __ldg(a.tile_len + tile) : 0u;
         s_off[t] = off;
-        s_first[t] = __ldcs(a.tile_ids + off);
+        s_first[t] = __ldcs(a.tile_ids + BMU_IDX(off, a.tile_rows_cap, a.status));
     }
     mm_fence_before();
     __syncthreads();
@@ -283,6 +283,8 @@ sweep_mma2_kernel(const MmaArgs a)
                         for (int u = 0; u < 4; ++u) {
                             const u64 ad = mm_desc(wring_u32 + slot * (uint32_t)MMA_STAGE_BYTES + u * 256, 128, 1024);
                             const u64 bd = mm_desc(xring_u32 + xslot * (uint32_t)MMA_STAGE_BYTES + u * 256, 128, 1024);
+                            BMU_EXPECT(slot < NS && xslot < NX &&
+                                       buf * 256 + (cp >> 1) * MMA_DOCS + MMA_DOCS <= M2_TMEM_COLS, a.status);
                             mm_mma(tmem + buf * 256 + (cp >> 1) * MMA_DOCS, ad, bd, idesc,
                                    (kb | (cp & 1) | u) != 0);
                         }
@@ -323,31 +325,32 @@ sweep_mma2_kernel(const MmaArgs a)
                     const uint32_t rows = max(tla & 0xffffu, tlb & 0xffffu);
                     const uint32_t my_rows = (lh ? tlb : tla) & 0xffffu;
                     const int mine = 2 * dg + ((lh && has_b) ? 1 : 0);
-                    const uint4 *gp = a.tile_ids + s_off[mine];
+                    const uint4 *gp = a.tile_ids + BMU_IDX(s_off[mine], a.tile_rows_cap, a.status);
+                    [[maybe_unused]] const size_t room = a.tile_rows_cap - (size_t)(gp - a.tile_ids);
                     const char *base = reinterpret_cast<const char *>(a.W + j0 + li * 4);
                     uint32_t b = 0;
                     uint4 qn = s_first[mine];
                     for (; b < full; ++b) {
                         uint32_t f[8];
                         m2_unpack(qn, f);
-                        qn = __ldcs(gp + b + 1);
+                        qn = __ldcs(gp + BMU_IDX(b + 1, room, a.status));
                         ulonglong2 w[8];
 #pragma unroll
                         for (int t = 0; t < 8; ++t)
-                            w[t] = __ldg(reinterpret_cast<const ulonglong2 *>(base + (u64)f[t] * rowbytes));
+                            w[t] = __ldg(reinterpret_cast<const ulonglong2 *>(base + (u64)BMU_IDX(f[t], a.D, a.status) * rowbytes));
 #pragma unroll
                         for (int t = 0; t < 8; ++t) { add2(acc[t][0], w[t].x); add2(acc[t][1], w[t].y); }
                     }
                     for (; b < rows; ++b) {                      // some documents have run out
                         uint32_t f[8];
                         m2_unpack(qn, f);
-                        qn = __ldcs(gp + b + 1);
+                        qn = __ldcs(gp + BMU_IDX(b + 1, room, a.status));
                         const bool in = b < my_rows;
                         ulonglong2 w[8];
 #pragma unroll
                         for (int t = 0; t < 8; ++t)
                             w[t] = (in && f[t] != 0xffffu)
-                                       ? __ldg(reinterpret_cast<const ulonglong2 *>(base + (u64)f[t] * rowbytes))
+                                       ? __ldg(reinterpret_cast<const ulonglong2 *>(base + (u64)BMU_IDX(f[t], a.D, a.status) * rowbytes))
                                        : make_ulonglong2(0ull, 0ull);
 #pragma unroll
                         for (int t = 0; t < 8; ++t) { add2(acc[t][0], w[t].x); add2(acc[t][1], w[t].y); }
@@ -361,6 +364,7 @@ sweep_mma2_kernel(const MmaArgs a)
                 mm_fence_after();
                 uint32_t h0[16], h1[16];
                 const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 256 + dg * 16);
+                BMU_EXPECT(buf * 256 + dg * 16 + MMA_DOCS + 16 <= M2_TMEM_COLS, a.status);
                 mm_tmem_ld16(taddr, h0);
                 mm_tmem_ld16(taddr + MMA_DOCS, h1);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -487,8 +491,8 @@ int launch_sweep_mma2(const MmaArgs &a, const bmu_opts &o, cudaStream_t s)
         configured[dev] = true;
     }
     const unsigned blocks = (unsigned)((a.N + MMA_DOCS - 1) / MMA_DOCS);
-    if (a.state2) sweep_mma2_kernel<true><<<blocks, M2_THREADS, m2_smem_bytes(a.head, true), s>>>(a);
-    else sweep_mma2_kernel<false><<<blocks, M2_THREADS, m2_smem_bytes(a.head, false), s>>>(a);
+    if (a.state2) { sweep_mma2_kernel<true><<<blocks, M2_THREADS, m2_smem_bytes(a.head, true), s>>>(a); BMU_LAUNCHED(); }
+    else { sweep_mma2_kernel<false><<<blocks, M2_THREADS, m2_smem_bytes(a.head, false), s>>>(a); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
@@ -511,7 +515,7 @@ __global__ void wait_timeout_selftest_kernel(uint32_t *status)
 
 int launch_wait_timeout_selftest(uint32_t *status, cudaStream_t s)
 {
-    wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(status);
+    { wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(status); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

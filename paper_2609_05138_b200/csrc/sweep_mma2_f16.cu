@@ -1,5 +1,5 @@
 // The wide tensor-core sweep (sweep_mma2.cu) for a half-precision codebook, the paper's own
-// storage (Section 4.2: "two bytes per half-precision weight"; Section 4.3: __half2 loads).
+// storage (Section 4.2: 2 bytes per weight; Section 4.3: loads of half pairs).
 // Same structure -- 256-neuron slabs, two accumulator tiles, double-buffered tensor memory,
 // K-outermost with X expanded per block of 64 features, tail tasks of 16 documents x 64
 // neurons -- with these differences: the weights are fp16 already, so the head image is a plain
@@ -71,8 +71,8 @@ int launch_head_split2_f16(const void *W16, int64_t M, int64_t m_full, int head,
 {
     if (m_full <= 0) return BMU_OK;
     const dim3 grid((unsigned)(m_full / M2_SLAB), head / 8);
-    head_split2_f16_kernel<<<grid, M2_SLAB, 0, s>>>(static_cast<const __half *>(W16), M, head, feat,
-                                                    head_img);
+    { head_split2_f16_kernel<<<grid, M2_SLAB, 0, s>>>(static_cast<const __half *>(W16), M, head, feat,
+                                                    head_img); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
@@ -182,7 +182,7 @@ sweep_mma2_f16_kernel(const MmaArgs a)
         const uint32_t off = there ? __ldg(a.tile_off + tile) : 0u;
         s_len[t] = there ? __ldg(a.tile_len + tile) : 0u;
         s_off[t] = off;
-        s_first[t] = __ldcs(a.tile_ids + off);
+        s_first[t] = __ldcs(a.tile_ids + BMU_IDX(off, a.tile_rows_cap, a.status));
     }
     mm_fence_before();
     __syncthreads();
@@ -313,7 +313,8 @@ sweep_mma2_f16_kernel(const MmaArgs a)
                     const uint32_t my_rows = ((ls >> 1) ? tlb : tla) & 0xffffu;
                     const int mine = 2 * dg + (((ls >> 1) && has_b) ? 1 : 0);
                     const bool upper = ls & 1;
-                    const uint4 *gp = a.tile_ids + s_off[mine];
+                    const uint4 *gp = a.tile_ids + BMU_IDX(s_off[mine], a.tile_rows_cap, a.status);
+                    [[maybe_unused]] const size_t room = a.tile_rows_cap - (size_t)(gp - a.tile_ids);
                     const char *base = reinterpret_cast<const char *>(a.W) + (size_t)(j0 + li * 8) * 2;
                     uint32_t b = 0;
                     uint4 qn = s_first[mine];
@@ -323,25 +324,25 @@ sweep_mma2_f16_kernel(const MmaArgs a)
                         uint32_t f[4 * ROWS];
                         m2_ids4(qn, upper, f);
 #pragma unroll
-                        for (int r = 1; r < ROWS; ++r) m2_ids4(__ldcs(gp + b + r), upper, f + 4 * r);
-                        qn = __ldcs(gp + b + ROWS);
+                        for (int r = 1; r < ROWS; ++r) m2_ids4(__ldcs(gp + BMU_IDX(b + r, room, a.status)), upper, f + 4 * r);
+                        qn = __ldcs(gp + BMU_IDX(b + ROWS, room, a.status));
                         uint4 w[4 * ROWS];
 #pragma unroll
                         for (int t = 0; t < 4 * ROWS; ++t)
-                            w[t] = __ldg(reinterpret_cast<const uint4 *>(base + (u64)f[t] * rowbytes));
+                            w[t] = __ldg(reinterpret_cast<const uint4 *>(base + (u64)BMU_IDX(f[t], a.D, a.status) * rowbytes));
 #pragma unroll
                         for (int t = 0; t < 4 * ROWS; ++t) m2_add_h8(acc[t & 3], w[t]);
                     }
                     for (; b < rows; ++b) {                      // left-over rows, then documents that ran out
                         uint32_t f[4];
                         m2_ids4(qn, upper, f);
-                        qn = __ldcs(gp + b + 1);
+                        qn = __ldcs(gp + BMU_IDX(b + 1, room, a.status));
                         const bool in = b < my_rows;
                         uint4 w[4];
 #pragma unroll
                         for (int t = 0; t < 4; ++t)
                             w[t] = (in && f[t] != 0xffffu)
-                                       ? __ldg(reinterpret_cast<const uint4 *>(base + (u64)f[t] * rowbytes))
+                                       ? __ldg(reinterpret_cast<const uint4 *>(base + (u64)BMU_IDX(f[t], a.D, a.status) * rowbytes))
                                        : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
                         for (int t = 0; t < 4; ++t) m2_add_h8(acc[t], w[t]);
@@ -495,8 +496,8 @@ int launch_sweep_mma2_f16(const MmaArgs &a, const bmu_opts &o, cudaStream_t s)
     }
     const unsigned blocks = (unsigned)((a.N + MMA_DOCS - 1) / MMA_DOCS);
     const size_t smem = m2_smem_bytes(a.head, a.state2 != nullptr);
-    if (a.state2) sweep_mma2_f16_kernel<true><<<blocks, M2_THREADS, smem, s>>>(a);
-    else sweep_mma2_f16_kernel<false><<<blocks, M2_THREADS, smem, s>>>(a);
+    if (a.state2) { sweep_mma2_f16_kernel<true><<<blocks, M2_THREADS, smem, s>>>(a); BMU_LAUNCHED(); }
+    else { sweep_mma2_f16_kernel<false><<<blocks, M2_THREADS, smem, s>>>(a); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

@@ -71,6 +71,7 @@ __global__ void __launch_bounds__(NW * 32, BMU_TILE_THREADS / (NW * 32) > 0 ? BM
 sweep_tiles_kernel(const TileArgs a)
 {
     constexpr int T = TILE_DOCS;
+    if (__ldg(a.status) & PLAN_STATUS_OVERFLOW) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t tile = (int64_t)blockIdx.x * NW + warp;
     const bool active = tile < a.n_tiles;            // idle warps still meet the barriers
@@ -81,8 +82,9 @@ sweep_tiles_kernel(const TileArgs a)
         const uint32_t tl = __ldg(a.tile_len + tile);
         rows = tl & 0xffffu;
         full = tl >> 16;
-        gp = a.tile_ids + __ldg(a.tile_off + tile);
+        gp = a.tile_ids + BMU_IDX(__ldg(a.tile_off + tile), a.tile_rows_cap, a.status);
     }
+    [[maybe_unused]] const size_t room = a.tile_rows_cap - (size_t)(gp - a.tile_ids);
     const int mydoc = doc_of_lane(lane);
     const int64_t myp = tile * T + mydoc;
     const int32_t orig = (active && myp < a.N) ? __ldg(a.perm + myp) : -1;
@@ -130,26 +132,26 @@ sweep_tiles_kernel(const TileArgs a)
         uint4 qn = __ldg(gp);                         // ids one row ahead of the row loads
         for (; b < full; ++b) {                       // rows where all 8 documents still have an id
             const uint4 q = qn;
-            qn = __ldg(gp + b + 1);                   // (slack rows follow every matrix)
+            qn = __ldg(gp + BMU_IDX(b + 1, room, a.status));   // (slack rows follow every matrix)
             const uint32_t f[T] = {q.x & 0xffffu, q.x >> 16, q.y & 0xffffu, q.y >> 16,
                                    q.z & 0xffffu, q.z >> 16, q.w & 0xffffu, q.w >> 16};
             ulonglong2 w[T];
 #pragma unroll
             for (int t = 0; t < T; ++t)
-                w[t] = __ldg(reinterpret_cast<const ulonglong2 *>(base + (u64)f[t] * rowbytes));
+                w[t] = __ldg(reinterpret_cast<const ulonglong2 *>(base + (u64)BMU_IDX(f[t], a.D, a.status) * rowbytes));
 #pragma unroll
             for (int t = 0; t < T; ++t) { add2(acc[t][0], w[t].x); add2(acc[t][1], w[t].y); }
         }
         for (; b < rows; ++b) {                       // the ragged end: some documents have run out
             const uint4 q = qn;
-            qn = __ldg(gp + b + 1);
+            qn = __ldg(gp + BMU_IDX(b + 1, room, a.status));
             const uint32_t f[T] = {q.x & 0xffffu, q.x >> 16, q.y & 0xffffu, q.y >> 16,
                                    q.z & 0xffffu, q.z >> 16, q.w & 0xffffu, q.w >> 16};
 #pragma unroll
             for (int t = 0; t < T; ++t)
                 if (f[t] != 0xffffu) {
                     const ulonglong2 w =
-                        __ldg(reinterpret_cast<const ulonglong2 *>(base + (u64)f[t] * rowbytes));
+                        __ldg(reinterpret_cast<const ulonglong2 *>(base + (u64)BMU_IDX(f[t], a.D, a.status) * rowbytes));
                     add2(acc[t][0], w.x);
                     add2(acc[t][1], w.y);
                 }
@@ -211,8 +213,8 @@ int launch_sweep_tiles(const TileArgs &a, const bmu_opts &o, cudaStream_t s)
 #define BMU_CASE(nw)                                                                        \
     if (NW == nw) {                                                                         \
         const unsigned blocks = (unsigned)((a.n_tiles + nw - 1) / nw);                      \
-        if (a.state2) sweep_tiles_kernel<nw, true><<<blocks, nw * 32, 0, s>>>(a);           \
-        else sweep_tiles_kernel<nw, false><<<blocks, nw * 32, 0, s>>>(a);                   \
+        if (a.state2) { sweep_tiles_kernel<nw, true><<<blocks, nw * 32, 0, s>>>(a); BMU_LAUNCHED(); }           \
+        else { sweep_tiles_kernel<nw, false><<<blocks, nw * 32, 0, s>>>(a); BMU_LAUNCHED(); }                   \
         BMU_CUDA(cudaGetLastError());                                                       \
         return BMU_OK;                                                                      \
     }

@@ -248,8 +248,8 @@ static int launch_blur_fast(const uint32_t *num, const uint32_t *cnt, int64_t D,
     }
     const dim3 grid((unsigned)((edge_x + F::TX - 1) / F::TX), (unsigned)((edge_y + F::TY - 1) / F::TY),
                     (unsigned)(D + 1));
-    update_blur_fast_kernel<R><<<grid, 256, F::SMEM, s>>>(num, cnt, D, edge_x, edge_y, t, num_blur,
-                                                         cnt_blur);
+    { update_blur_fast_kernel<R><<<grid, 256, F::SMEM, s>>>(num, cnt, D, edge_x, edge_y, t, num_blur,
+                                                         cnt_blur); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
@@ -346,8 +346,8 @@ int launch_update_scatter(const int32_t *rowptr, const int32_t *colidx, int64_t 
                           cudaStream_t s)
 {
     if (N == 0) return BMU_OK;
-    update_scatter_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(rowptr, colidx, N, bmu,
-                                                                          M, num, cnt);
+    { update_scatter_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(rowptr, colidx, N, bmu,
+                                                                          M, num, cnt); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
@@ -396,7 +396,7 @@ int launch_update_blur(const uint32_t *num, const uint32_t *cnt, int64_t D, int3
     }
     const dim3 grid((unsigned)((edge_x + BLUR_TX - 1) / BLUR_TX),
                     (unsigned)((edge_y + BLUR_TY - 1) / BLUR_TY), (unsigned)(D + 1));
-    update_blur_kernel<<<grid, 256, smem, s>>>(num, cnt, D, edge_x, edge_y, t, num_blur, cnt_blur);
+    { update_blur_kernel<<<grid, 256, smem, s>>>(num, cnt, D, edge_x, edge_y, t, num_blur, cnt_blur); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
@@ -409,8 +409,8 @@ int launch_update_writeback(const float *num_blur, const float *cnt_blur, int64_
                                      reinterpret_cast<uintptr_t>(cnt_blur)) & 15) == 0;
     const int64_t per_row = vec ? M / 4 : M;
     const dim3 grid((unsigned)((per_row + 255) / 256 < 64 ? (per_row + 255) / 256 : 64), (unsigned)D);
-    if (vec) update_writeback_kernel<true><<<grid, 256, 0, s>>>(num_blur, cnt_blur, M, W);
-    else update_writeback_kernel<false><<<grid, 256, 0, s>>>(num_blur, cnt_blur, M, W);
+    if (vec) { update_writeback_kernel<true><<<grid, 256, 0, s>>>(num_blur, cnt_blur, M, W); BMU_LAUNCHED(); }
+    else { update_writeback_kernel<false><<<grid, 256, 0, s>>>(num_blur, cnt_blur, M, W); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }
@@ -427,8 +427,8 @@ int launch_map_errors(const int32_t *bmu, const int32_t *bmu2, const float *dist
     unsigned int *ticket = static_cast<unsigned int *>(ws);
     double *part = reinterpret_cast<double *>(static_cast<char *>(ws) + 256);
     BMU_CUDA(cudaMemsetAsync(ticket, 0, sizeof(unsigned int), s));
-    map_errors_kernel<<<ME_BLOCKS, ME_THREADS, 0, s>>>(bmu, bmu2, dist, N, edge_x, adjacency, part,
-                                                      ticket, out);
+    { map_errors_kernel<<<ME_BLOCKS, ME_THREADS, 0, s>>>(bmu, bmu2, dist, N, edge_x, adjacency, part,
+                                                      ticket, out); BMU_LAUNCHED(); }
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

@@ -67,3 +67,27 @@ def test_argument_checks_need_no_gpu(lib):
     o.vec = 3
     assert lib.bmu_search_ws(None, 4, 4, None, None, None, 3, 0, None, None,
                              ctypes.byref(o), None, 0, None) == 1
+
+
+def test_describe_search_needs_no_gpu_and_names_the_kernel(lib):
+    """bmu_describe_search is host logic: the benchmark shapes route as documented (large
+    sweeps take the tensor-core sweep, the small one the planned kernel) and the launch count
+    follows from the chunk."""
+    from paper_2609_05138_b200 import Opts, SearchDesc
+    d = SearchDesc()
+    shapes = {"cfg1": (4096, 1024, 10_000, 640_000), "cfg2": (16384, 4096, 1_000_000, 80_000_000),
+              "cfg4": (16384, 262144, 2_000_000, 160_000_000)}
+    for name, (D, M, N, nnz) in shapes.items():
+        assert lib.bmu_describe_search(D, M, N, nnz, None, ctypes.byref(d)) == 0
+        assert d.kernel == (3 if name == "cfg1" else 6)
+        assert d.head_rows == (0 if name == "cfg1" else 640)
+        assert d.docs_per_block == (16 if name == "cfg1" else 128)
+        assert d.chunk_neurons % d.slab == 0 and d.ragged_neurons == 0
+        assert d.sweep_launches == -(-M // d.chunk_neurons)
+    o = Opts()
+    o.kernel, o.chunk_neurons = 6, 2048
+    assert lib.bmu_describe_search(16384, 262144 + 36, 1000, 80_000, ctypes.byref(o), ctypes.byref(d)) == 0
+    assert (d.kernel, d.chunk_neurons, d.sweep_launches, d.ragged_neurons, d.repack) == (6, 2048, 128, 36, 1)
+    o.kernel = 6
+    assert lib.bmu_describe_search(32, 1024, 10, 100, ctypes.byref(o), ctypes.byref(d)) == 2   # D < head
+    assert lib.bmu_describe_search(32, 1024, 10, 100, None, None) == 1

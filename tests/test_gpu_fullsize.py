@@ -4,8 +4,8 @@ The oracle cannot sweep 2,000,000 documents against 262,144 neurons in test
 time, so the full-size run is checked (a) on a seeded sample of documents the
 oracle computes one by one, (b) by properties that hold for every document,
 and (c) against an independent computation by a library sparse-dense product (test-only
-code): every document of the 64x64 and 128x128 configurations, a 150,000-document prefix of
-the 512x512 one.
+code): every document of the 64x64 and 128x128 configurations, and 96 windows of 2,048
+documents spread evenly over the whole corpus of the 512x512 one.
 """
 import numpy as np
 import pytest
@@ -60,7 +60,7 @@ def test_cfg4_full_size_sampled(bmu):
     ob, od = bmu.bmu_search_ws(W, rowptr, colidx, norms=norms)     # bench.py's call and options
     torch.cuda.synchronize()
     check_properties(W, norms, rowptr, colidx, ob, od, cfg.M)
-    check_sample(W, rowptr, colidx, ob, od, 256, seed=4)
+    check_sample(W, rowptr, colidx, ob, od, 2000, seed=4)
 
 
 def test_cfg3_full_size_sampled(bmu):
@@ -105,23 +105,28 @@ def test_cfg5_one_streamed_batch_sampled(bmu):
         check_sample(W, rowptr, colidx, ob, od, 1500, seed=5 + batch)
 
 
-@pytest.mark.parametrize("name,n_check,step", [("cfg2", 0, 50_000), ("cfg3", 0, 20_000),
-                                               ("cfg4", 150_000, 2_048)])
-def test_full_size_against_library_product(bmu, name, n_check, step):
-    """Every document of configs 2 and 3 (and the first 150,000 of config 4's full search)
-    against an independent computation: a library sparse-dense product per document batch, the
-    distance formula and an arg-min in fp64 (test-only code)."""
+@pytest.mark.parametrize("name,n_windows,step", [("cfg2", 0, 50_000), ("cfg3", 0, 20_000),
+                                                 ("cfg4", 96, 2_048)])
+def test_full_size_against_library_product(bmu, name, n_windows, step):
+    """Every document of configs 2 and 3, and 96 windows of 2,048 documents spread evenly over
+    all of config 4's full search (the planned order is by length, so evenly spaced windows of
+    the caller's order reach every part of every launch), against an independent computation:
+    a library sparse-dense product per document batch, the distance formula and an arg-min in
+    fp64 (test-only code)."""
     cfg = synth.CONFIGS[name]
     dev = torch.device("cuda")
     W = synth.make_codebook(cfg.D, cfg.M, synth.codebook_seed(cfg), device=dev)
     rowptr, colidx = synth.make_corpus(cfg, device=dev)
-    N = n_check or cfg.N
+    N = cfg.N
     ob, od = bmu.bmu_search(W, rowptr, colidx)
     torch.cuda.synchronize()
     check_sample(W, rowptr, colidx, ob, od, 3000 if cfg.M <= 16384 else 200, seed=2)
     norms = (W.double() ** 2).sum(0)
     bad_d = bad_j = 0
-    for lo in range(0, N, step):
+    starts = (range(0, N, step) if not n_windows else
+              [min(N - step, k * (N // n_windows) + (k * 977) % (N // n_windows - step))
+               for k in range(n_windows)])
+    for lo in starts:
         hi = min(N, lo + step)
         rp = (rowptr[lo:hi + 1] - rowptr[lo]).to(torch.int64)
         ci = colidx[int(rowptr[lo]):int(rowptr[hi])].to(torch.int64)

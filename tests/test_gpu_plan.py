@@ -114,3 +114,26 @@ def test_calls_on_two_streams_with_their_own_workspaces_do_not_interfere(bmu, ke
     torch.cuda.synchronize()
     for j in jobs:
         assert torch.equal(j["ob"], j["alone"][0]) and torch.equal(j["od"], j["alone"][1])
+
+
+def test_launch_counter_agrees_with_describe_search(bmu):
+    """The library counts its own kernel launches; between two chunk sizes the count differs by
+    exactly the sweep launches (and compact copies) bmu_describe_search announces."""
+    cfg = synth.CONFIGS["cfg2"]
+    dev = torch.device("cuda")
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=600, device=dev)
+    W = synth.make_codebook(cfg.D, 4096, 2, device=dev)
+    N, nnz = rowptr.numel() - 1, colidx.numel()
+    counts, descs = [], []
+    for chunk in (512, 2048):
+        o = bmu.Opts()
+        o.kernel, o.chunk_neurons = 6, chunk
+        d = bmu.bmu_describe_search(cfg.D, 4096, N, nnz, o)
+        n0 = bmu.bmu_kernel_launches()
+        bmu.bmu_search_ws(W, rowptr, colidx, opts=o)
+        counts.append(bmu.bmu_kernel_launches() - n0)
+        descs.append(d)
+    torch.cuda.synchronize()
+    per = [d.sweep_launches * (1 + d.repack) for d in descs]
+    assert [d.sweep_launches for d in descs] == [8, 2]
+    assert counts[0] - counts[1] == per[0] - per[1] and counts[1] > per[1]

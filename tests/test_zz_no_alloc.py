@@ -6,8 +6,9 @@ start-up, in a plug-in that only receives its inputs and outputs.  For them the
 library carries its scratch in a fixed 8 MiB array of its own image.  The test
 calls that entry point through the C ABI twice in a row, with different inputs,
 and checks both results against the ordinary entry point (bmu_search_ws, same
-kernel, caller-owned workspace): the second call finds the first call's
-leftovers in the shared array and must not be disturbed by them.  Sizes beyond
+kernel, caller-owned workspace) and against the fp64 oracle under the rule of
+every other parity test: the second call finds the first call's leftovers in the
+shared array and must not be disturbed by them.  Sizes beyond
 the array are refused with a message that names them.
 
 Collected last on purpose (file name), so that a failure here cannot hide the
@@ -17,6 +18,7 @@ import pytest
 import torch
 
 from inputs import synth
+from tests import parity
 
 pytestmark = pytest.mark.gpu
 
@@ -52,6 +54,11 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(bmu):
         assert torch.equal(ob, rb)
         # same kernel, same order of additions: the tolerance of the parity tests is ample
         assert bool(((od - rd).abs() <= 1e-5 * rd.abs()).all())
+        # and the entry point's own output against the oracle (indices equal except inside a
+        # 1e-5 near-tie, distances within 1e-5 relative)
+        res = parity.compare(ob.cpu().numpy(), od.cpu().numpy(), W.cpu().numpy(),
+                             rp.cpu().numpy(), ci.cpu().numpy())
+        assert res["docs"] == N and res["failed"] == 0
 
 
 def test_sizes_beyond_the_built_in_array_are_refused(bmu):
