@@ -505,7 +505,7 @@ def run_ours(args, cfg, rank, local_rank, world):
     if len(batches) == 1:
         line["planned"] = planned_steps(bmu, cfg, a, opts, args.steps, dev)
     if args.comparator:
-        line["comparator"] = comparator_spmm(cfg, W, norms, rowptr, colidx)
+        line["comparator"] = comparator_spmm(cfg, W, norms, rowptr, colidx, peaks)
     if args.f16 and len(batches) == 1:
         line["f16_codebook"] = f16_codebook(bmu, cfg, W, rowptr, colidx, args)
     if args.epoch:
@@ -579,44 +579,88 @@ def f16_codebook(bmu, cfg, W, rowptr, colidx, args):
             "api": "bmu_codebook_norms_f16 + bmu_search_f16_ws per step (rank 0's figure)"}
 
 
-def comparator_spmm(cfg, W, norms, rowptr, colidx, budget_docs=200_000):
+def comparator_spmm(cfg, W, norms, rowptr, colidx, peaks, budget_docs=0):
     """The other side of the paper's comparison (Section 3: a library sparse-dense product that
-    materialises the score block, then a separate arg-min), on this GPU and these arrays:
-    torch.sparse CSR x dense fp32 (cuSPARSE SpMM) per document batch, then n_j - 2 s_ij and
-    torch.argmin.  A comparator only: nothing of it is part of the library.  Timed on a bounded
-    prefix of the workload (documents are independent, so docs/s extrapolates)."""
+    materialises the score block, then a separate arg-min read-back), tuned the way the paper
+    tunes it (Section 4.4): score block in fp32 and in fp16, batch size swept, and the read-back
+    done by a warp-per-row kernel with 128-bit loads that forms n_j - 2 s_ij on the fly
+    (bmu_score_block_argmin) -- next to the untuned torch.argmin read-back for contrast.  The
+    product is torch.sparse CSR x dense (cuSPARSE SpMM): the library stays the library.  Timed on
+    a bounded prefix of the workload (documents are independent, so docs/s extrapolates)."""
+    import warnings
+    import paper_2609_05138_b200 as bmu
     dev = W.device
+    if not budget_docs:
+        budget_docs = 100_000 if cfg.M > 100_000 else 400_000
     n_docs = min(rowptr.numel() - 1, budget_docs)
-    batch = int(max(1024, min(n_docs, (2 << 30) // (cfg.M * 4))))      # score block <= 2 GiB
-    rp64 = rowptr[: n_docs + 1].to(torch.int64)
+    rp32 = rowptr[: n_docs + 1].contiguous()
+    rp64 = rp32.to(torch.int64)
     ci64 = colidx[: int(rp64[-1])].to(torch.int64)
-    ones = torch.ones(ci64.numel(), device=dev)
+    W16 = None
+    cells = []
 
-    def one_pass():
-        out = torch.empty(n_docs, dtype=torch.int64, device=dev)
+    def one_pass(dtype, batch, tuned):
+        Wd = W if dtype == torch.float32 else W16
+        ones = torch.ones(ci64.numel(), device=dev, dtype=dtype)
+        ob = torch.empty(n_docs, dtype=torch.int32, device=dev)
+        od = torch.empty(n_docs, dtype=torch.float32, device=dev)
+        t_rb = 0.0
         for lo in range(0, n_docs, batch):
             hi = min(n_docs, lo + batch)
             a, b = int(rp64[lo]), int(rp64[hi])
             X = torch.sparse_csr_tensor(rp64[lo:hi + 1] - a, ci64[a:b], ones[a:b],
                                         size=(hi - lo, cfg.D))
-            S = X @ W
-            out[lo:hi] = torch.argmin(torch.addcmul(norms[None, :], S, S.new_full((), -2.0)), dim=1)
-        return out
+            S = X @ Wd                                      # the materialised score block
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            if tuned:
+                bmu.bmu_score_block_argmin(S, norms, rp32[lo:hi + 1], ob[lo:hi], od[lo:hi])
+            else:
+                d = torch.addcmul(norms[None, :], S.float(), S.new_full((), -2.0, dtype=torch.float32))
+                ob[lo:hi] = torch.argmin(d, dim=1).to(torch.int32)
+            e1.record()
+            torch.cuda.synchronize(dev)
+            t_rb += e0.elapsed_time(e1)
+            del X, S
+        return ob, t_rb
 
-    import warnings
     with warnings.catch_warnings():
         warnings.simplefilter("ignore")
-        one_pass()
-        torch.cuda.synchronize(dev)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        one_pass()
-        e1.record()
-        torch.cuda.synchronize(dev)
-    ms = e0.elapsed_time(e1)
-    return {"kind": "materialised score block: torch.sparse CSR x dense fp32 (cuSPARSE SpMM) + "
-                    "torch.argmin, batches of %d documents" % batch,
-            "value": n_docs / (ms * 1e-3), "unit": UNIT, "sample_docs": n_docs, "ms": ms}
+        for dtype in (torch.float32, torch.float16):
+            esize = 4 if dtype == torch.float32 else 2
+            if dtype == torch.float16:
+                W16 = W.half()
+            for batch in (1024, 4096, 16384, 65536):
+                if batch * cfg.M * esize > (4 << 30) or batch > 4 * n_docs:
+                    continue
+                for tuned in (True, False):
+                    if not tuned and (dtype == torch.float16 or batch != 4096):
+                        continue                      # the untuned read-back once, for contrast
+                    try:
+                        one_pass(dtype, batch, tuned)             # warm-up
+                        torch.cuda.synchronize(dev)
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record()
+                        _, t_rb = one_pass(dtype, batch, tuned)
+                        e1.record()
+                        torch.cuda.synchronize(dev)
+                    except RuntimeError as ex:        # e.g. no half-precision SpMM in this library build
+                        cells.append({"score_dtype": str(dtype).replace("torch.", ""), "batch": batch,
+                                      "tuned_readback": tuned, "unavailable": str(ex)[:120]})
+                        continue
+                    ms = e0.elapsed_time(e1)
+                    cells.append({"score_dtype": str(dtype).replace("torch.", ""), "batch": batch,
+                                  "tuned_readback": tuned, "ms": ms, "value": n_docs / (ms * 1e-3),
+                                  "readback_ms": t_rb,
+                                  "readback_frac_of_hbm": (n_docs * cfg.M * esize / (t_rb * 1e-3) /
+                                                           (peaks["hbm_gbs"] * 1e9)) if tuned else None})
+        del W16
+    ok = [c for c in cells if "value" in c and c["tuned_readback"]]
+    best = max(ok, key=lambda c: c["value"]) if ok else None
+    return {"kind": "materialised score block: torch.sparse CSR x dense (cuSPARSE SpMM) into an fp32 "
+                    "or fp16 block, then a warp-per-row 128-bit arg-min read-back "
+                    "(bmu_score_block_argmin); batch size and score dtype swept",
+            "sample_docs": n_docs, "unit": UNIT, "best": best, "cells": cells}
 
 
 def epoch_phases(bmu, cfg, W, batches, opts, ws, norms, out_bmu, out_dist, peaks, sigma):

@@ -413,6 +413,22 @@ BMU_API int bmu_map_errors(const int32_t *bmu, const int32_t *bmu2, const float 
                            void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Arg-min read-back over a MATERIALISED score block: the second half of the other
+ * route to the same search (Section 3: a sparse-dense product writes all
+ * n_rows x M scores s_ij = sum_{f in x_i} W[f][j], a separate pass reads them
+ * back; Section 4.4 tunes that pass to a warp per row with vector loads).  Not
+ * used by bmu_search; it is here so that the fused search can be compared with a
+ * tuned version of that route.  scores: n_rows x M, row-major, fp32 (half == 0)
+ * or IEEE fp16 (half != 0), 16-byte aligned, M % 4 == 0 (fp16: M % 8 == 0);
+ * rowptr: the n_rows + 1 row pointers of these documents (only differences are
+ * used, for |x_i|).  out_bmu[i] = lowest j attaining min_j (norms[j] - 2 s_ij),
+ * out_dist[i] = |x_i| + that minimum.  Reads the block once; no scratch.
+ */
+BMU_API int bmu_score_block_argmin(const void *scores, int32_t half, int64_t n_rows, int64_t M,
+                                   const float *norms, const int32_t *rowptr, int32_t *out_bmu,
+                                   float *out_dist, void *stream);
+
+/*
  * Measures one on-chip ceiling of the current device with a microbenchmark, so
  * that achieved throughput can be quoted against the roof that binds (the paper
  * quotes its kernel against the L2 roof of its card, Section 6 / Table 3).

@@ -10,7 +10,7 @@ from .binding import (BmuError, Opts, bmu_codebook_norms, bmu_codebook_norms_f16
                       bmu_measure_roof, bmu_validate_csr, bmu_version, load,
                       bmu_update_scatter, bmu_update_blur, bmu_update_writeback,
                       bmu_map_errors, Plan, SearchDesc, bmu_describe_search,
-                      bmu_kernel_launches, bmu_last_status)
+                      bmu_kernel_launches, bmu_last_status, bmu_score_block_argmin)
 
 __all__ = ["BmuError", "Opts", "bmu_codebook_norms", "bmu_codebook_norms_f16",
            "bmu_search_f16_ws", "bmu_release_scratch", "bmu_search",
@@ -18,4 +18,5 @@ __all__ = ["BmuError", "Opts", "bmu_codebook_norms", "bmu_codebook_norms_f16",
            "bmu_search_workspace_bytes", "bmu_search_ws",
            "bmu_measure_roof", "bmu_validate_csr", "bmu_version", "load",
            "bmu_update_scatter", "bmu_update_blur", "bmu_update_writeback", "bmu_map_errors",
-           "Plan", "SearchDesc", "bmu_describe_search", "bmu_kernel_launches", "bmu_last_status"]
+           "Plan", "SearchDesc", "bmu_describe_search", "bmu_kernel_launches", "bmu_last_status",
+           "bmu_score_block_argmin"]

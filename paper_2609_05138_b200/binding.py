@@ -126,6 +126,9 @@ EXPORTS = {
                                       ctypes.c_int64, ctypes.c_int32, ctypes.c_int32,
                                       ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
                                       ctypes.c_size_t, ctypes.c_void_p]),
+    "bmu_score_block_argmin": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64,
+                                              ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
+                                              ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "bmu_measure_roof": (ctypes.c_int, [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t,
                                         ctypes.c_int, ctypes.POINTER(ctypes.c_double),
                                         ctypes.c_void_p]),
@@ -225,7 +228,7 @@ def bmu_search_ws(W, rowptr, colidx, norms=None, opts: Opts | None = None, works
     return out_bmu, out_dist
 
 
-def bmu_search_top2_ws(W, rowptr, colidx, norms=None, opts: Opts | None = None):
+def bmu_search_top2_ws(W, rowptr, colidx, norms=None, opts: Opts | None = None, workspace=None):
     """Best and second-best unit.  Returns (out_bmu, out_dist, out_bmu2, out_dist2)."""
     wp, D, M = _codebook(W)
     N = rowptr.numel() - 1
@@ -236,8 +239,11 @@ def bmu_search_top2_ws(W, rowptr, colidx, norms=None, opts: Opts | None = None):
     od2 = torch.empty(N, dtype=torch.float32, device=W.device)
     need = int(load().bmu_search_top2_workspace_bytes(D, M, N, nnz,
                                                       ctypes.byref(opts) if opts else None))
-    ws = torch.empty(need + 256, dtype=torch.uint8, device=W.device)
+    ws = workspace if workspace is not None else torch.empty(need + 256, dtype=torch.uint8,
+                                                             device=W.device)
     ws_ptr = (ws.data_ptr() + 255) // 256 * 256
+    if ws_ptr + need > ws.data_ptr() + ws.numel():
+        raise ValueError("workspace too small: need %d bytes after alignment" % need)
     with torch.cuda.device(W.device):
         _check(load().bmu_search_top2_ws(
             wp, D, M, _dev(norms, torch.float32, "norms") if norms is not None else None,
@@ -501,6 +507,27 @@ def bmu_map_errors(bmu, bmu2, dist, edge_x: int, edge_y: int, adjacency: int = 4
                                      int(edge_x), int(edge_y), int(adjacency), out.data_ptr(),
                                      ws_ptr, need, _stream(dist)))
     return out
+
+
+def bmu_score_block_argmin(scores, norms, rowptr, out_bmu=None, out_dist=None):
+    """Arg-min read-back over a materialised [n_rows, M] score block (fp32 or fp16)."""
+    if scores.dim() != 2 or scores.dtype not in (torch.float32, torch.float16):
+        raise TypeError("scores must be [n_rows, M] fp32 or fp16")
+    n, M = scores.shape
+    _dev(scores, scores.dtype, "scores")
+    if rowptr.numel() != n + 1:
+        raise ValueError("rowptr must have n_rows + 1 entries")
+    if out_bmu is None:
+        out_bmu = torch.empty(n, dtype=torch.int32, device=scores.device)
+    if out_dist is None:
+        out_dist = torch.empty(n, dtype=torch.float32, device=scores.device)
+    with torch.cuda.device(scores.device):
+        _check(load().bmu_score_block_argmin(
+            scores.data_ptr(), int(scores.dtype == torch.float16), n, M,
+            _dev(norms, torch.float32, "norms"), _dev(rowptr, torch.int32, "rowptr"),
+            _dev(out_bmu, torch.int32, "out_bmu"), _dev(out_dist, torch.float32, "out_dist"),
+            _stream(scores)))
+    return out_bmu, out_dist
 
 
 ROOFS = {"l2_ldg": 0, "l2_bulk": 1, "smem": 2, "l1": 3, "fadd": 4, "fadd2": 5, "l2_mixed": 6}

@@ -18,6 +18,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbmu.so")
+# the same library with every id- and offset-derived address checked (-DBMU_BOUNDS_CHECK)
+LIB_CHECKED = os.path.join(HERE, "libbmu_checked.so")
 OBJDIR = os.path.join(HERE, "build")
 
 NVCC_FLAGS = [
@@ -44,8 +46,9 @@ def up_to_date(lib: str = LIB) -> bool:
 
 def build_library(force: bool = False, verbose: bool = False, extra_flags=(), out: str = LIB,
                   objdir: str = OBJDIR) -> str:
-    extra = [*os.environ.get("BMU_EXTRA_NVCC", "").split(), *extra_flags]
-    if not force and not extra and up_to_date(out):
+    env_extra = os.environ.get("BMU_EXTRA_NVCC", "").split()
+    extra = [*env_extra, *extra_flags]
+    if not force and not env_extra and up_to_date(out):   # `out` names its own flag set
         return out
     nvcc = os.environ.get("NVCC", "nvcc")
     flags = [*extra, *NVCC_FLAGS]
@@ -74,5 +77,11 @@ def build_library(force: bool = False, verbose: bool = False, extra_flags=(), ou
     return out
 
 
+def build_checked_library(force: bool = False) -> str:
+    return build_library(force=force, extra_flags=["-DBMU_BOUNDS_CHECK"], out=LIB_CHECKED)
+
+
 if __name__ == "__main__":
     print(build_library(force="-f" in sys.argv or "-v" in sys.argv, verbose="-v" in sys.argv))
+    if "--checked" in sys.argv:
+        print(build_checked_library(force="-f" in sys.argv))

@@ -1098,6 +1098,28 @@ int bmu_update_writeback(const float *num_blur, const float *cnt_blur, int64_t D
     return launch_update_writeback(num_blur, cnt_blur, D, M, W, static_cast<cudaStream_t>(stream));
 }
 
+int bmu_score_block_argmin(const void *scores, int32_t half, int64_t n_rows, int64_t M,
+                           const float *norms, const int32_t *rowptr, int32_t *out_bmu,
+                           float *out_dist, void *stream)
+{
+    int rc = check_sizes(0, M, n_rows, 0);
+    if (rc) return rc;
+    if (n_rows == 0) return BMU_OK;
+    if (!scores || !norms || !rowptr || !out_bmu || !out_dist) {
+        set_error("null pointer argument");
+        return BMU_ERR_INVALID_ARG;
+    }
+    if (M == 0) { set_error("empty score rows: no neuron to return"); return BMU_ERR_INVALID_ARG; }
+    if (M % (half ? 8 : 4) != 0 || (reinterpret_cast<uintptr_t>(scores) & 15) != 0 ||
+        (reinterpret_cast<uintptr_t>(norms) & 15) != 0) {
+        set_error("score read-back needs M %% %d == 0 and 16-byte aligned scores and norms",
+                  half ? 8 : 4);
+        return BMU_ERR_UNSUPPORTED;
+    }
+    return launch_readback_argmin(scores, half != 0, n_rows, M, norms, rowptr, out_bmu, out_dist,
+                                  static_cast<cudaStream_t>(stream));
+}
+
 size_t bmu_map_errors_workspace_bytes(void) { return map_errors_workspace_bytes(); }
 
 int bmu_map_errors(const int32_t *bmu, const int32_t *bmu2, const float *dist, int64_t N,

@@ -284,6 +284,11 @@ int launch_map_errors(const int32_t *bmu, const int32_t *bmu2, const float *dist
 int launch_update_writeback(const float *num_blur, const float *cnt_blur, int64_t D, int64_t M,
                             float *W, cudaStream_t s);
 
+// arg-min read-back over a materialised score block (readback.cu)
+int launch_readback_argmin(const void *scores, int half, int64_t n_rows, int64_t M,
+                           const float *norms, const int32_t *rowptr, int32_t *out_bmu,
+                           float *out_dist, cudaStream_t s);
+
 int launch_validate_csr(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                         int64_t D, int32_t *flags, cudaStream_t s);
 
