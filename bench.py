@@ -123,13 +123,18 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def union_rows_per_block(rowptr, colidx, D, docs_per_block):
-    """Sum over blocks of consecutive documents of the number of distinct features the
-    block touches: the rows an SM has to fetch at least once per slab when `docs_per_block`
-    documents share its L1 (the design's own grouping)."""
+def union_rows_per_block(rowptr, colidx, D, docs_per_block, order=None):
+    """Sum over blocks of `docs_per_block` documents, consecutive in the planned order
+    (`order[p]` = the document at position p; None = the corpus order), of the number of
+    distinct features the block touches: the rows an SM has to fetch at least once per slab
+    when those documents share it (the design's own grouping)."""
     N = rowptr.numel() - 1
     lens = (rowptr[1:] - rowptr[:-1]).to(torch.int64)
     doc = torch.repeat_interleave(torch.arange(N, device=rowptr.device), lens)
+    if order is not None:
+        pos = torch.empty(N, dtype=torch.int64, device=rowptr.device)
+        pos[order.to(torch.int64)] = torch.arange(N, device=rowptr.device)
+        doc = pos[doc]
     key = (doc // docs_per_block) * D + colidx.to(torch.int64)
     del doc
     key = torch.sort(key).values
@@ -206,7 +211,7 @@ def cpu_baseline(cfg, W_dev, rowptr, colidx, n_docs, budget_s=15.0):
                       % (t_norm, sample, t_bmu, cores, n_docs)}
 
 
-def workload_config(cfg, n_docs, world):
+def workload_config(cfg, n_docs, world, corpus="zipf"):
     return {
         "workload": "%s: %dx%d map (M=%d), D=%d, fp32 feature-major codebook U[0,1), "
                     "N=%d docs per GPU, nnz/doc %s, Zipf(s=%.1f) ids without replacement"
@@ -214,7 +219,7 @@ def workload_config(cfg, n_docs, world):
                        "Poisson(%g)>=1" % cfg.nnz_param if cfg.nnz_kind == "poisson"
                        else "lognormal(median %g, sigma 0.5) in [1,400]" % cfg.nnz_param,
                        cfg.zipf_s),
-        "docs_per_gpu": n_docs, "global_docs": n_docs * world,
+        "docs_per_gpu": n_docs, "global_docs": n_docs * world, "corpus": corpus,
         "parallelism": "docs sharded over %d GPU(s), codebook replicated, no collective" % world,
         "l2_policy": "inputs larger than L2 (codebook %.1f GB); no flush between steps"
                      % (cfg.D * cfg.M * 4 / 1e9),
@@ -268,9 +273,14 @@ def measure_config(bmu, cfg, args, dev, rank, world, roofs, peaks, steps, warmup
     batches = []
     for b in range(n_batches):
         bsz = min(synth.batch_size(cfg), cfg.N - b * synth.batch_size(cfg))
-        rp_b, ci_b = synth.make_corpus(cfg, batch=b, device=dev,
-                                       n_docs=min(bsz, args.docs) if args.docs else bsz,
-                                       seed=synth.corpus_seed(cfg, b) + 1000 * rank)
+        if args.corpus == "topical":               # an extra input with co-occurrence structure
+            rp_b, ci_b = synth.make_topical_corpus(cfg, device=dev,
+                                                   n_docs=min(bsz, args.docs) if args.docs else bsz,
+                                                   seed=synth.corpus_seed(cfg, 50 + b) + 1000 * rank)
+        else:
+            rp_b, ci_b = synth.make_corpus(cfg, batch=b, device=dev,
+                                           n_docs=min(bsz, args.docs) if args.docs else bsz,
+                                           seed=synth.corpus_seed(cfg, b) + 1000 * rank)
         batches.append((rp_b, ci_b))
     n_docs = sum(rp_b.numel() - 1 for rp_b, _ in batches)
     rowptr, colidx = batches[0]
@@ -286,7 +296,9 @@ def measure_config(bmu, cfg, args, dev, rank, world, roofs, peaks, steps, warmup
     desc = bmu.bmu_describe_search(cfg.D, cfg.M, max_n, max_nnz, opts, device=dev)
     kernel_name = {1: "sweep_direct_kernel", 3: "sweep_rows_kernel", 4: "sweep_tiles_kernel",
                    6: "sweep_mma2_kernel"}[desc.kernel]
-    chunk, n_chunks = int(desc.chunk_neurons), int(desc.sweep_launches)
+    n_chunks = int(desc.sweep_launches)
+    # neurons per launch, averaged over the launches of one search (the last one may be shorter)
+    chunk = (cfg.M - desc.ragged_neurons) / float(n_chunks)
 
     def step(e0=None, e1=None, e2=None):
         if e0 is not None:
@@ -338,8 +350,18 @@ def measure_config(bmu, cfg, args, dev, rank, world, roofs, peaks, steps, warmup
     nnz = total_nnz / len(batches)                              # mean batch
     N = n_docs / len(batches)
     adds = float(nnz) * chunk                                   # one update per (nnz, neuron)
-    union_rows = union_rows_per_block(rowptr, colidx, cfg.D, desc.docs_per_block) * (
+    order = None
+    if desc.kernel != 1:                        # the order the tiling pass gives the documents
+        plan = bmu.Plan(rowptr, colidx, cfg.D, cfg.M, opts)
+        order = plan.order()
+        plan.close()
+        del plan
+    union_rows = union_rows_per_block(rowptr, colidx, cfg.D, desc.docs_per_block, order) * (
         nnz / max(1, colidx.numel()))
+    # listings per distinct row among the documents that share a block / an 8-document tile
+    reuse = {"per_block_of_%d" % desc.docs_per_block: nnz / max(1.0, union_rows),
+             "per_tile_of_8": colidx.numel() / max(1, union_rows_per_block(rowptr, colidx, cfg.D, 8, order))}
+    del order
     alg = {
         "alu": (adds / launch_s, roofs["fadd2"], "add/s"),
         "l1": (4.0 * adds / launch_s, roofs["smem"], "B/s"),           # one 4-byte operand per add
@@ -378,6 +400,7 @@ def measure_config(bmu, cfg, args, dev, rank, world, roofs, peaks, steps, warmup
                            "to this launch: codebook chunk once + the rest per document)"),
         "launch_ms": launch_s * 1e3, "launches_per_step": n_chunks * len(batches),
         "units_per_launch": {"adds": adds, "union_rows_x_chunk": float(union_rows) * chunk},
+        "tile_reuse": reuse,
         "fractions": {k: v[0] / v[1] for k, v in alg.items()},
         **extra,
     }
@@ -387,7 +410,7 @@ def measure_config(bmu, cfg, args, dev, rank, world, roofs, peaks, steps, warmup
         "phases_ms": {"norms": norms_ms, "sweep_and_output": sweep_ms},
         "clocks": clocks, "gpu_launches": int(launches), "roofline": roofline,
         "search": {"kernel": desc.kernel, "head_rows": desc.head_rows, "slab": desc.slab,
-                   "docs_per_block": desc.docs_per_block, "chunk_neurons": chunk,
+                   "docs_per_block": desc.docs_per_block, "chunk_neurons": int(desc.chunk_neurons),
                    "sweep_launches": n_chunks, "repack": desc.repack},
     }
     arrays = dict(W=W, batches=batches, ws=ws, norms=norms, out_bmu=out_bmu, out_dist=out_dist,
@@ -484,7 +507,7 @@ def run_ours(args, cfg, rank, local_rank, world):
         "metric": METRIC, "value": frag["value"], "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": frag["ms_per_step"],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic", "config": workload_config(cfg, n_docs, world),
+        "data": "synthetic", "config": workload_config(cfg, n_docs, world, args.corpus),
         "updates_per_s": frag["updates_per_s"], "phases_ms": frag["phases_ms"],
         "clocks": frag["clocks"],
         "e2e": {"value": n_docs * world / e2e_s, "unit": UNIT,
@@ -514,7 +537,8 @@ def run_ours(args, cfg, rank, local_rank, world):
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(cfg, W, rowptr, colidx, rowptr.numel() - 1)
     # ---- the other benchmark configurations, briefly (same protocol, fewer steps)
-    if world == 1 and args.all_configs and not args.docs and not args.batches and not args.opt:
+    if (world == 1 and args.all_configs and not args.docs and not args.batches and not args.opt
+            and args.corpus == "zipf"):
         del W, batches, ws, norms, out_bmu, out_dist, rowptr, colidx
         a.clear()
         torch.cuda.empty_cache()
@@ -774,6 +798,9 @@ def main():
     ap.add_argument("--epoch", action="store_true",
                     help="also time one whole epoch (search + scatter + blur + write-back)")
     ap.add_argument("--sigma", type=float, default=2.0, help="neighbourhood width of --epoch")
+    ap.add_argument("--corpus", default="zipf", choices=["zipf", "topical"],
+                    help="zipf: the configuration's own recipe (ids drawn independently); topical: "
+                         "the same sizes with topics, i.e. documents that share rare features")
     ap.add_argument("--no-all-configs", dest="all_configs", action="store_false",
                     help="skip the brief runs of the other benchmark configurations")
     ap.add_argument("--selfcheck-ranks", action="store_true",

@@ -79,7 +79,7 @@ typedef struct bmu_opts {
                                the head_rows most frequent features is a dense contraction
                                on tcgen05 tensor cores with fp32 accumulation into
                                double-buffered tensor memory, the remaining ids are gathered
-                               as in 4; needs what 4 needs, D >= head_rows and M >= 512; the
+                               as in 4; needs what 4 needs, D >= head_rows and M >= 256; the
                                automatic choice for large sweeps).  Other values are
                                refused. */
     int32_t chunk_neurons;  /* neurons per L2-resident chunk of the codebook (Section 4.2,
@@ -87,10 +87,16 @@ typedef struct bmu_opts {
     int32_t vec;            /* warp-per-document kernels: floats per lane per row, 4 or 8 */
     int32_t docs_per_warp;  /* generic kernel: documents a warp carries through one slab */
     int32_t warps;          /* warp-per-document kernels: warps per thread block */
-    int32_t cluster;        /* tile membership (Section 4.2): 0/1 order the documents by
+    int32_t cluster;        /* tile membership (Section 4.2): 1 order the documents by
                                length before cutting tiles, so that the documents of a tile
-                               finish together; 2 keep the corpus order (generic and planned
-                               kernels only) */
+                               finish together (0 = 3 for the tensor-core sweep, 1 for the
+                               other kernels); 3 by length, and among equally long
+                               documents by their two rarest features and their most frequent
+                               gathered one, so that documents sharing features fall in the
+                               same tile; 4 the same with the three most frequent gathered
+                               features as the key (3 and 4: fp32 codebook, and the tensor-core
+                               sweep of the half-precision one); 2 keep the corpus order
+                               (generic and planned kernels only) */
     int32_t stage_rows;     /* unused, must be 0 */
     int32_t stages;         /* unused, must be 0 */
     int32_t tile_order;     /* order of the gathered ids inside a tile: 1 ascending; 2 dealt
@@ -199,6 +205,12 @@ BMU_API int bmu_search_ws(const float *W, int64_t D, int64_t M, const float *nor
  *       Allocates nothing, asynchronous on `stream`; searches that share a plan
  *       must not overlap on the GPU.  Results equal bmu_search_ws with the same
  *       options bit for bit.
+ *   bmu_plan_order  copies the order the tiling pass put the documents in
+ *       (Section 4.2, tile membership) to out_order[N], device memory: the
+ *       document at planned position p is out_order[p]; consecutive positions
+ *       form the tiles (8) and blocks (128) of the tiled and tensor-core sweeps.
+ *       For inspection and measurement (tile reuse); the searches do not need it.
+ *       BMU_ERR_UNSUPPORTED for the generic kernel, which plans nothing.
  *   bmu_plan_destroy  frees the host handle (not the workspace).
  */
 typedef struct bmu_plan bmu_plan;
@@ -209,6 +221,7 @@ BMU_API int bmu_plan_create(const int32_t *rowptr, const int32_t *colidx, int64_
                             size_t workspace_bytes, bmu_plan **plan, void *stream);
 BMU_API int bmu_search_planned(const bmu_plan *plan, const float *W, const float *norms,
                                int32_t *out_bmu, float *out_dist, void *stream);
+BMU_API int bmu_plan_order(const bmu_plan *plan, int32_t *out_order, void *stream);
 BMU_API void bmu_plan_destroy(bmu_plan *plan);
 
 /*
@@ -233,7 +246,7 @@ BMU_API int bmu_search_top2_ws(const float *W, int64_t D, int64_t M, const float
  * (norms: fp64 accumulate).  Needs M % 256 == 0 (M % 8 == 0 for the norms
  * alone) and D <= 65024.  out_bmu2 / out_dist2 may both be NULL, or both given
  * to get the second-best unit as in bmu_search_top2_ws.  bmu_opts.kernel: 3 the
- * planned kernel, 6 the wide tensor-core sweep (needs M % 512 == 0 and D >=
+ * planned kernel, 6 the wide tensor-core sweep (needs D >=
  * head_rows; the weights being fp16 already, its head image has one part), 0
  * the tensor-core sweep for large sweeps, else the planned kernel; head_rows
  * defaults to 576 here.  Workspace: bmu_search_f16_workspace_bytes(...) with the

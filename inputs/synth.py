@@ -36,6 +36,7 @@ import torch
 __all__ = [
     "Config", "CONFIGS", "zipf_cdf", "draw_nnz", "draw_corpus", "make_corpus",
     "make_codebook", "codebook_seed", "corpus_seed", "num_batches", "batch_size",
+    "make_topical_corpus",
 ]
 
 
@@ -210,6 +211,52 @@ def make_corpus(cfg: Config, batch: int = 0, device="cpu", n_docs: int | None = 
     g = _gen(seed ^ 0x5A5A5A5A, device)
     nnz = draw_nnz(cfg.nnz_kind, cfg.nnz_param, n, g, device)
     return draw_corpus(n, cfg.D, cfg.zipf_s, nnz, seed, device)
+
+
+def make_topical_corpus(cfg: Config, device="cpu", n_docs: int | None = None,
+                        seed: int | None = None, n_topics: int = 4096, topic_size: int = 96,
+                        topic_share: float = 0.35, first_rare: int = 640):
+    """A corpus WITH co-occurrence structure, as an extra test input beside the five
+    configurations (whose ids are drawn independently, so that documents share rare features
+    only by chance; a real collection has topics).  Every document belongs to one of `n_topics`
+    topics; a topic owns `topic_size` rare features (ids >= first_rare, a seeded random set).
+    A document takes about `topic_share` of its ids from its topic's features (a uniform sample
+    without replacement) and the rest by the configuration's own Zipf recipe; ids that come up
+    twice are kept once, so rows are a little shorter than the configuration's.  Same layout as
+    make_corpus: (rowptr int32 [N+1], colidx int32 [nnz]), ids ascending in a row."""
+    n = cfg.N if n_docs is None else min(cfg.N, int(n_docs))
+    seed = corpus_seed(cfg, 50) if seed is None else seed
+    device = torch.device(device)
+    g = _gen(seed ^ 0x70B1C5, device)
+    nnz = draw_nnz(cfg.nnz_kind, cfg.nnz_param, n, g, device)
+    k_topic = (nnz.to(torch.float64) * topic_share).round().to(torch.int64).clamp(max=topic_size)
+    base_rp, base_ci = draw_corpus(n, cfg.D, cfg.zipf_s, (nnz - k_topic).clamp(min=0), seed, device)
+    rare = cfg.D - first_rare
+    if rare < topic_size:
+        raise ValueError("vocabulary too small for topics of %d rare features" % topic_size)
+    # topic t owns the first `topic_size` entries of a random permutation of the rare ids
+    feats = torch.rand((n_topics, rare), generator=g, device=device).argsort(dim=1)[:, :topic_size]
+    feats = feats + first_rare
+    topic = torch.randint(0, n_topics, (n,), generator=g, device=device)
+    doc_parts, id_parts = [], []
+    for b0 in range(0, n, 1 << 18):                      # bounded scratch
+        b1 = min(n, b0 + (1 << 18))
+        pick = torch.rand((b1 - b0, topic_size), generator=g, device=device).argsort(dim=1)
+        keep = torch.arange(topic_size, device=device)[None, :] < k_topic[b0:b1, None]
+        ids = feats[topic[b0:b1]].gather(1, pick)[keep]
+        docs = torch.arange(b0, b1, device=device)[:, None].expand(-1, topic_size)[keep]
+        doc_parts.append(docs)
+        id_parts.append(ids)
+    lens = (base_rp[1:] - base_rp[:-1]).to(torch.int64)
+    doc_parts.append(torch.repeat_interleave(torch.arange(n, device=device), lens))
+    id_parts.append(base_ci.to(torch.int64))
+    key = torch.unique(torch.cat(doc_parts) * cfg.D + torch.cat(id_parts))     # sorted, no repeats
+    doc = key // cfg.D
+    counts = torch.zeros(n, dtype=torch.int64, device=device).index_add_(
+        0, doc, torch.ones_like(doc))
+    rowptr = torch.zeros(n + 1, dtype=torch.int32, device=device)
+    rowptr[1:] = torch.cumsum(counts, 0).to(torch.int32)
+    return rowptr, (key - doc * cfg.D).to(torch.int32)
 
 
 def make_codebook(D: int, M: int, seed: int, device="cpu", kind: str = "uniform",

@@ -111,6 +111,7 @@ EXPORTS = {
                                        ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p]),
     "bmu_search_planned": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "bmu_plan_order": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "bmu_plan_destroy": (None, [ctypes.c_void_p]),
     "bmu_update_scatter": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                           ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64,
@@ -439,6 +440,13 @@ class Plan:
                 _dev(out_bmu, torch.int32, "out_bmu"), _dev(out_dist, torch.float32, "out_dist"),
                 _stream(W)))
         return out_bmu, out_dist
+
+    def order(self):
+        """The planned order: int32 [N], the document at each planned position."""
+        out = torch.empty(self.N, dtype=torch.int32, device=self.rowptr.device)
+        with torch.cuda.device(self.rowptr.device):
+            _check(load().bmu_plan_order(self.handle, out.data_ptr(), _stream(self.rowptr)))
+        return out
 
     def close(self):
         if self.handle:

@@ -8,6 +8,7 @@ default one, e.g. the bounds-checked build (-DBMU_BOUNDS_CHECK).
 from __future__ import annotations
 
 import glob
+import hashlib
 import os
 import subprocess
 import sys
@@ -37,18 +38,31 @@ def headers():
         sorted(glob.glob(os.path.join(ROOT, "include", "*.h")))
 
 
-def up_to_date(lib: str = LIB) -> bool:
-    if not os.path.exists(lib):
+def fingerprint(extra=()) -> str:
+    """Hash of everything a build depends on: sources, headers, flags."""
+    h = hashlib.sha256(" ".join([*NVCC_FLAGS, *extra]).encode())
+    for p in sources() + headers():
+        h.update(os.path.basename(p).encode())
+        with open(p, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def up_to_date(lib: str = LIB, extra=()) -> bool:
+    """True if `lib` was built from exactly these sources and flags (a stamp file beside the
+    library holds the fingerprint; file times do not survive a copy of the tree)."""
+    try:
+        with open(lib + ".stamp") as f:
+            return os.path.exists(lib) and f.read().strip() == fingerprint(extra)
+    except OSError:
         return False
-    t = os.path.getmtime(lib)
-    return all(os.path.getmtime(p) <= t for p in sources() + headers())
 
 
 def build_library(force: bool = False, verbose: bool = False, extra_flags=(), out: str = LIB,
                   objdir: str = OBJDIR) -> str:
     env_extra = os.environ.get("BMU_EXTRA_NVCC", "").split()
     extra = [*env_extra, *extra_flags]
-    if not force and not env_extra and up_to_date(out):   # `out` names its own flag set
+    if not force and up_to_date(out, extra):
         return out
     nvcc = os.environ.get("NVCC", "nvcc")
     flags = [*extra, *NVCC_FLAGS]
@@ -74,6 +88,8 @@ def build_library(force: bool = False, verbose: bool = False, extra_flags=(), ou
     subprocess.check_call([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a",
                            *objs, "-o", tmp])
     os.replace(tmp, out)
+    with open(out + ".stamp", "w") as f:
+        f.write(fingerprint(extra) + "\n")
     return out
 
 

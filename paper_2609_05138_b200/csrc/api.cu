@@ -38,16 +38,17 @@ struct Layout {
     PlanLayout plan;
 };
 
-// Neurons per launch of the tensor-core sweep: whole 512-neuron slabs whose rows take a little
-// over half of L2 (1024 neurons at D = 16384 on a 126 MB L2; measured best there, 512 and 2048
-// within 2 %).
+// Neurons per launch of the tensor-core sweep: whole 256-neuron slabs whose rows take about
+// 0.4 of L2 (768 neurons at D = 16384 on a 126 MB L2).  Measured on config 4: 768 beats 1024 by
+// 2 % and 512 by 3 %; at 1024 the chunk (67 MB) no longer stays resident in the two-part L2 and
+// its rows are fetched from DRAM five times over.
 static int64_t mma_auto_chunk(int64_t D, int64_t M)
 {
     int dev = 0, l2 = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess || l2 <= 0)
         l2 = 64 << 20;
-    int64_t c = (int64_t)((double)l2 * 0.55) / (D * 4) / MMA_SLAB * MMA_SLAB;
+    int64_t c = (int64_t)((double)l2 * 0.42) / (D * 4) / MMA_SLAB * MMA_SLAB;
     if (c < MMA_SLAB) c = MMA_SLAB;
     if (c > M) c = M / MMA_SLAB * MMA_SLAB;
     return c;
@@ -95,7 +96,7 @@ static int mma_head_rows(const bmu_opts &o, int64_t D)
 }
 
 static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kernel,
-                         bool top2 = false, int head = 640, size_t repack_bytes = 0)
+                         bool top2 = false, int head = 640, size_t repack_bytes = 0, int cluster = 0)
 {
     Layout l;
     size_t off = 0;
@@ -112,16 +113,26 @@ static Layout layout_for(int64_t D, int64_t M, int64_t N, int64_t nnz, int kerne
     off = align_up(off + repack_bytes, 256);
     l.plan_off = off;
     memset(&l.plan, 0, sizeof(l.plan));
-    if (kernel != 1 && D <= LANES_MAX_D) off += plan_bytes(N, nnz, head, D, &l.plan);
+    if (kernel != 1 && D <= LANES_MAX_D) off += plan_bytes(N, nnz, head, D, cluster, &l.plan);
     l.total = off;
     return l;
+}
+
+// How the tiling pass orders the documents: 0 corpus order, 1 by length, 3 / 4 by length and
+// content.  The tensor-core sweep takes 3 unless told otherwise (measured on configs 2-4: 0.5,
+// 2.8 and 2.5 % faster than by length alone, the extra sort included; 4 gains less).
+static int plan_order(const bmu_opts &o, bool tensor_core_sweep)
+{
+    if (o.cluster == 2) return 0;
+    if (o.cluster >= 3) return o.cluster;
+    return (o.cluster == 0 && tensor_core_sweep) ? 3 : 1;
 }
 
 // the layout search_impl uses for these options (the workspace-size queries must agree with it)
 static Layout layout_of(const bmu_opts &o, int64_t D, int64_t M, int64_t N, int64_t nnz, bool top2)
 {
     return layout_for(D, M, N, nnz, o.kernel, top2, mma_head_rows(o, D),
-                      mma_repack_bytes(o, D, M, N, nnz, top2));
+                      mma_repack_bytes(o, D, M, N, nnz, top2), plan_order(o, true));
 }
 
 static int check_sizes(int64_t D, int64_t M, int64_t N, int64_t nnz)
@@ -158,7 +169,7 @@ static int check_opts(const bmu_opts &o)
         set_error("bmu_opts.stage_rows and bmu_opts.stages must be zero");
         return BMU_ERR_INVALID_ARG;
     }
-    if (o.cluster < 0 || o.cluster > 2) { set_error("bmu_opts.cluster must be 0, 1 or 2"); return BMU_ERR_INVALID_ARG; }
+    if (o.cluster < 0 || o.cluster > 4) { set_error("bmu_opts.cluster must be 0 .. 4"); return BMU_ERR_INVALID_ARG; }
     if (o.chunk_neurons < 0) { set_error("bmu_opts.chunk_neurons < 0"); return BMU_ERR_INVALID_ARG; }
     if (o.vec != 0 && o.vec != 4 && o.vec != 8) { set_error("bmu_opts.vec must be 0, 4 or 8"); return BMU_ERR_INVALID_ARG; }
     return BMU_OK;
@@ -204,7 +215,7 @@ static int route_search(const bmu_opts &o, int64_t D, int64_t M, int64_t nnz, ui
         return BMU_ERR_UNSUPPORTED;
     }
     const bool tiled_ok = planned_ok && M >= 128 && o.cluster != 2;
-    // tensor-core head: additionally at least one whole 512-neuron slab and `head` features
+    // tensor-core head: additionally at least one whole 256-neuron slab and `head` features
     const bool mma_ok = tiled_ok && D >= head && M >= MMA_SLAB;
     if (o.kernel == 6 && !mma_ok) {
         set_error("tensor-core sweep needs what the tiled kernel needs, D >= %d and M >= %d",
@@ -303,8 +314,8 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
     // dense head = the most frequent features by the corpus's own counts (bmu_opts.relabel)
     const int relabel = mma ? o.relabel : 2;        // 0 decide from the counts, 1 always, 2 never
     if ((planned || tiled || mma) && phase != 2)
-        if ((rc = launch_plan(rowptr, colidx, N, nnz, o.cluster != 2, mma ? head : 0, relabel, D, pw,
-                              l.plan, status, s)))
+        if ((rc = launch_plan(rowptr, colidx, N, nnz, plan_order(o, mma),
+                              mma ? head : 0, relabel, D, pw, l.plan, status, s)))
             return rc;
     if (mma) {
         if (phase != 2 &&
@@ -622,7 +633,7 @@ int bmu_codebook_norms_f16(const void *W16, int64_t D, int64_t M, float *norms, 
 }
 
 // Which kernel a half-precision search takes: large sweeps the wide tensor-core sweep (whole
-// 512-neuron slabs only), the rest the planned kernel.  `ow` = the options of the wide sweep, its
+// 256-neuron slabs only), the rest the planned kernel.  `ow` = the options of the wide sweep, its
 // head resolved (576 by default: with 2-byte rows the gathered tail is cheap, so the balance
 // point sits lower than the fp32 sweep's 640; config 4 at full length: 2364 / 2348 / 2331 / 2473
 // ms per step at 448 / 512 / 576 / 704).
@@ -703,7 +714,8 @@ int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
         BMU_CUDA(cudaMemsetAsync(status, 0, 256, s));
         char *pw = base + l.plan_off;
         const int relabel = o.relabel;
-        if ((rc = launch_plan(rowptr, colidx, N, nnz, 1, head, relabel, D, pw, l.plan, status, s))) return rc;
+        if ((rc = launch_plan(rowptr, colidx, N, nnz, plan_order(o, true), head, relabel, D, pw, l.plan,
+                              status, s))) return rc;
         if ((rc = launch_plan_tiles(rowptr, N, o.tile_order == 2, head, relabel, D, pw, l.plan, status, s))) return rc;
         unsigned char *img = reinterpret_cast<unsigned char *>(base + l.head_off);
         const uint16_t *feat = (relabel != 2 && l.plan.fsort_tmp_bytes > 0)
@@ -1049,6 +1061,23 @@ int bmu_search_planned(const bmu_plan *plan, const float *W, const float *norms,
     return search_impl(W, plan->D, plan->M, norms, plan->rowptr, plan->colidx, plan->N, plan->nnz,
                        out_bmu, out_dist, &plan->opts, plan->ws, plan->ws_bytes,
                        static_cast<cudaStream_t>(stream), nullptr, nullptr, 2);
+}
+
+int bmu_plan_order(const bmu_plan *plan, int32_t *out_order, void *stream)
+{
+    if (!plan || !out_order) { set_error("null pointer argument"); return BMU_ERR_INVALID_ARG; }
+    Route r;
+    int rc = route_search(plan->opts, plan->D, plan->M, plan->nnz, 0, r);
+    if (rc) return rc;
+    if (r.kernel == 1) {
+        set_error("the generic kernel makes no plan: documents keep the corpus order");
+        return BMU_ERR_UNSUPPORTED;
+    }
+    const Layout l = layout_of(plan->opts, plan->D, plan->M, plan->N, plan->nnz, false);
+    const char *perm = static_cast<const char *>(plan->ws) + l.plan_off + l.plan.perm_off;
+    BMU_CUDA(cudaMemcpyAsync(out_order, perm, (size_t)plan->N * sizeof(int32_t),
+                             cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)));
+    return BMU_OK;
 }
 
 void bmu_plan_destroy(bmu_plan *plan) { delete plan; }

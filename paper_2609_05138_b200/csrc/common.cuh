@@ -175,6 +175,7 @@ struct PlanLayout {
     size_t perm_off, docoff_off, ngroups_off, bins_off, ids_off, scan_off, scan_bytes, total;
     size_t tilelen_off, tilerows_off, tileoff_off, tilehead_off, tileids_off, tile_rows_cap;
     size_t id_groups_cap;                                                   // 16-byte id groups
+    size_t cluster_off, cluster_tmp_off, cluster_tmp_bytes;                 // ordering by content
     size_t rank_off, feat_off, fsort_off, fsort_tmp_off, fsort_tmp_bytes;   // feature ranks
 };
 static const int TILE_HEAD_ROWS = 32;    // ids below this are swept densely, once per tile
@@ -206,7 +207,7 @@ int launch_sweep_tiles(const TileArgs &a, const bmu_opts &o, cudaStream_t s);
 
 // tensor-core head + gathered tail (sweep_mma2.cu, sweep_mma2_f16.cu): a block carries 128
 // documents through slabs of 256 neurons; launches cover whole multiples of MMA_SLAB neurons
-static const int MMA_SLAB = 512;         // granularity of a launch's neuron range
+static const int MMA_SLAB = 256;         // granularity of a launch's neuron range (the kernel's slab)
 static const int MMA_DOCS = 128;         // documents per block
 static const size_t MMA_STAGE_BYTES = 16384;                  // 128 neurons x 64 features x fp16
 struct MmaArgs {
@@ -241,7 +242,7 @@ int launch_sweep_mma2(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
 int launch_sweep_mma2_f16(const MmaArgs &a, const bmu_opts &o, cudaStream_t s);
 int launch_head_split2_f16(const void *W16, int64_t M, int64_t m_full, int head, const uint16_t *feat,
                            unsigned char *head_img, cudaStream_t s);
-size_t plan_bytes(int64_t N, int64_t nnz, int head, int64_t D, PlanLayout *l);
+size_t plan_bytes(int64_t N, int64_t nnz, int head, int64_t D, int cluster, PlanLayout *l);
 int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                 int order_by_length, int head, int relabel, int64_t D, char *ws, const PlanLayout &l,
                 uint32_t *status, cudaStream_t s);

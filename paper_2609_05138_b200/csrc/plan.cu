@@ -199,6 +199,75 @@ __global__ void plan_scatter_kernel(const int32_t *__restrict__ rowptr,
     ngroups[p] = (uint32_t)((row + 7) / 8 + 1);
 }
 
+// Tile membership by content (Section 4.2: documents that share features are put in the same
+// tile).  Sorting key of a document: its length key first -- tiles must stay exactly
+// length-ordered -- then a few of its features, so that inside a run of equally long documents
+// those with the same features lie next to each other.  Which features (ranks, or ids on a
+// vocabulary labelled by frequency):
+//   mode 3  the two rarest of the list, then the most frequent one at or above `head`;
+//   mode 4  the three most frequent ones at or above `head` (the first three the gather visits).
+// Either way the shared features sit at the same step of the lists of a tile (the front, or the
+// back of equally long lists), so the loads of one step ask for the same row.  One warp per
+// document.
+__device__ __forceinline__ void plan_min3(uint32_t &a, uint32_t &b, uint32_t &c, uint32_t v)
+{
+    if (v < a) { c = b; b = a; a = v; } else if (v < b) { c = b; b = v; } else if (v < c) { c = v; }
+}
+
+__global__ void __launch_bounds__(256)
+plan_cluster_key_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colidx,
+                        const uint16_t *__restrict__ rank, const uint32_t *__restrict__ len_key,
+                        int64_t N, int32_t head, int mode, [[maybe_unused]] int64_t D,
+                        [[maybe_unused]] uint32_t *status, u64 *__restrict__ keys,
+                        uint32_t *__restrict__ vals)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (i >= N) return;
+    const int beg = rowptr[i], end = rowptr[i + 1];
+    uint32_t m1 = 0, m2 = 0;                         // largest and second largest rank
+    uint32_t s1 = 0xffffu, s2 = 0xffffu, s3 = 0xffffu;   // three smallest ranks >= head
+    for (int e = beg + lane; e < end; e += 32) {
+        const uint32_t f = (uint32_t)colidx[e];
+        const uint32_t r = rank ? (uint32_t)rank[BMU_IDX(f, D, status)] : min(f, 0xfffeu);
+        if (r > m1) { m2 = m1; m1 = r; } else if (r > m2) { m2 = r; }
+        if (r >= (uint32_t)head) plan_min3(s1, s2, s3, r);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const uint32_t o1 = __shfl_xor_sync(0xffffffffu, m1, off);
+        const uint32_t o2 = __shfl_xor_sync(0xffffffffu, m2, off);
+        const uint32_t hi = max(m1, o1), lo = min(m1, o1);
+        m2 = max(lo, max(m2, o2));
+        m1 = hi;
+        const uint32_t t1 = __shfl_xor_sync(0xffffffffu, s1, off);
+        const uint32_t t2 = __shfl_xor_sync(0xffffffffu, s2, off);
+        const uint32_t t3 = __shfl_xor_sync(0xffffffffu, s3, off);
+        plan_min3(s1, s2, s3, t1);
+        plan_min3(s1, s2, s3, t2);
+        plan_min3(s1, s2, s3, t3);
+    }
+    if (lane == 0) {
+        const int len = min(len_key ? (int)len_key[i] : end - beg, PLAN_BINS - 1);
+        const u64 top = (u64)(uint32_t)(PLAN_BINS - 1 - len) << 48;
+        keys[i] = mode == 4 ? top | ((u64)s1 << 32) | ((u64)s2 << 16) | (u64)s3
+                            : top | ((u64)m1 << 32) | ((u64)m2 << 16) | (u64)s1;
+        vals[i] = (uint32_t)i;
+    }
+}
+
+// groups of 8 ids the row at planned position p needs (plus its closing sentinel group)
+__global__ void plan_groups_kernel(const int32_t *__restrict__ rowptr,
+                                   const int32_t *__restrict__ perm, int64_t N,
+                                   uint32_t *__restrict__ ngroups)
+{
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p == 0) ngroups[N] = 0u;
+    if (p >= N) return;
+    const int32_t i = perm[p];
+    ngroups[p] = (uint32_t)((rowptr[i + 1] - rowptr[i] + 7) / 8 + 1);
+}
+
 __global__ void plan_identity_kernel(const int32_t *__restrict__ rowptr, int64_t N,
                                      int32_t *__restrict__ perm, uint32_t *__restrict__ ngroups)
 {
@@ -372,7 +441,7 @@ plan_tile_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restr
     }
 }
 
-size_t plan_bytes(int64_t N, int64_t nnz, int head, int64_t D, PlanLayout *l)
+size_t plan_bytes(int64_t N, int64_t nnz, int head, int64_t D, int cluster, PlanLayout *l)
 {
     auto up = [](size_t x) { return (x + 255) / 256 * 256; };
     size_t off = 0;
@@ -408,6 +477,16 @@ size_t plan_bytes(int64_t N, int64_t nnz, int head, int64_t D, PlanLayout *l)
         cub::DeviceRadixSort::SortPairsDescending(nullptr, tmp, (uint32_t *)nullptr, (uint32_t *)nullptr,
                                                   (uint32_t *)nullptr, (uint32_t *)nullptr, (int)D);
         t.fsort_tmp_off = off; t.fsort_tmp_bytes = tmp; off = up(off + tmp);
+    }
+    // ordering by content: 64-bit keys and document numbers, in and out, and the sort's scratch
+    t.cluster_off = t.cluster_tmp_off = off;
+    t.cluster_tmp_bytes = 0;
+    if (cluster >= 3 && N > 0) {
+        t.cluster_off = off; off = up(off + (size_t)N * 8 * 2 + (size_t)N * 4);
+        size_t tmp = 0;
+        cub::DeviceRadixSort::SortPairs(nullptr, tmp, (u64 *)nullptr, (u64 *)nullptr,
+                                        (uint32_t *)nullptr, (uint32_t *)nullptr, (int)N);
+        t.cluster_tmp_off = off; t.cluster_tmp_bytes = tmp; off = up(off + tmp);
     }
     t.total = off;
     if (l) *l = t;
@@ -479,9 +558,23 @@ int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t
         // counters and the largest key in one clearing (the cursors in between are all written
         // or never read)
         BMU_CUDA(cudaMemsetAsync(hist, 0, (size_t)PLAN_BINS * 4 * 2 + 256, s));
-        { plan_hist_kernel<<<blocks, 256, 0, s>>>(rowptr, key, N, hist, aux); BMU_LAUNCHED(); }
-        { plan_scan_bins_kernel<<<1, 1024, 0, s>>>(hist, aux, cursor); BMU_LAUNCHED(); }
-        { plan_scatter_kernel<<<blocks, 256, 0, s>>>(rowptr, key, N, cursor, perm, ngroups); BMU_LAUNCHED(); }
+        if (order_by_length >= 3 && l.cluster_tmp_bytes > 0) {
+            // by length, then by the rarest features: one radix sort of (key, document) pairs
+            u64 *keys_in = reinterpret_cast<u64 *>(ws + l.cluster_off);
+            u64 *keys_out = keys_in + N;
+            uint32_t *vals_in = reinterpret_cast<uint32_t *>(keys_out + N);
+            { plan_cluster_key_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(
+                rowptr, colidx, rank, key, N, head, order_by_length, D, status, keys_in, vals_in); BMU_LAUNCHED(); }
+            size_t ctmp = l.cluster_tmp_bytes;
+            BMU_CUDA(cub::DeviceRadixSort::SortPairs(ws + l.cluster_tmp_off, ctmp, keys_in, keys_out,
+                                                     vals_in, reinterpret_cast<uint32_t *>(perm),
+                                                     (int)N, 0, 64, s));
+            { plan_groups_kernel<<<blocks, 256, 0, s>>>(rowptr, perm, N, ngroups); BMU_LAUNCHED(); }
+        } else {
+            { plan_hist_kernel<<<blocks, 256, 0, s>>>(rowptr, key, N, hist, aux); BMU_LAUNCHED(); }
+            { plan_scan_bins_kernel<<<1, 1024, 0, s>>>(hist, aux, cursor); BMU_LAUNCHED(); }
+            { plan_scatter_kernel<<<blocks, 256, 0, s>>>(rowptr, key, N, cursor, perm, ngroups); BMU_LAUNCHED(); }
+        }
     } else {
         { plan_identity_kernel<<<blocks, 256, 0, s>>>(rowptr, N, perm, ngroups); BMU_LAUNCHED(); }
     }

@@ -38,13 +38,12 @@ static const int M2_NX = BMU_M2_XSTAGES;             // X ring stages
 static const int M2_TAIL_WARPS = 16;
 static const int M2_THREADS = (M2_TAIL_WARPS + 3) * 32;
 static const int M2_TMEM_COLS = 512;                 // 2 buffers x 2 tiles x 128 documents
-static const int M2_IDS_ROWS = 1024;                 // id-matrix rows of a block kept in shared memory
 
 static inline size_t m2_smem_bytes(int head, bool top2)
 {
     return (size_t)MMA_DOCS * (head / 8) + (M2_NS + M2_NX) * MMA_STAGE_BYTES +
            (2 * M2_NS + 2 * M2_NX + 6) * 8 + MMA_DOCS * 8 + 16 + 16 * 16 + 2 * 16 * 4 +
-           16 * 8 + (top2 ? 4 * MMA_DOCS * 16 : 0) + 16 + (size_t)M2_IDS_ROWS * 16;
+           16 * 8 + (top2 ? 4 * MMA_DOCS * 16 : 0);
 }
 
 // bit pattern of the largest |weight| among the head rows: sets the power-of-two scale of the
@@ -154,10 +153,6 @@ sweep_mma2_kernel(const MmaArgs a)
     // document is the same in every slab, so it merges without atomics
     uint2 *lut = reinterpret_cast<uint2 *>(s_off + 16);          // 4 mask bits -> 4 fp16 zeros and ones
     u64 *kq = reinterpret_cast<u64 *>(lut + 16);
-    // the id matrices of the block's tiles (they lie one after the other), fetched once per
-    // launch instead of once per slab when they fit
-    uint4 *ids_s = reinterpret_cast<uint4 *>(
-        (reinterpret_cast<uintptr_t>(kq + (TOP2 ? 4 * MMA_DOCS * 2 : 0)) + 15) & ~(uintptr_t)15);
     const uint32_t wfull0 = mm_smem(bars), wempty0 = mm_smem(bars + NS);
     const uint32_t xfull0 = mm_smem(bars + 2 * NS), xempty0 = mm_smem(bars + 2 * NS + NX);
     const uint32_t tfull0 = mm_smem(bars + 2 * NS + 2 * NX), tempty0 = tfull0 + 16;
@@ -214,25 +209,6 @@ sweep_mma2_kernel(const MmaArgs a)
     __syncthreads();
     mm_fence_after();
     const uint32_t tmem = *tmem_slot;
-    // rows of the block's id matrices.  A pair of tiles is walked to the longer one's end and
-    // one row is fetched ahead, so the walk over the last tile may run past its own rows by as
-    // much as the block's longest tile: those rows are taken along.
-    uint32_t ids_rows = 0;
-    {
-        const int64_t left = a.n_tiles - group * (MMA_DOCS / 8);
-        const int nt = (int)(left < MMA_DOCS / 8 ? left : MMA_DOCS / 8);
-        uint32_t longest = 0;
-        for (int t = 0; t < nt; ++t) longest = max(longest, s_len[t] & 0xffffu);
-        ids_rows = s_off[nt - 1] + longest + 1u - s_off[0];
-    }
-    const bool ids_in_smem = ids_rows <= (uint32_t)M2_IDS_ROWS;
-    if (ids_in_smem) {
-        const uint4 *src = a.tile_ids + BMU_IDX(s_off[0], a.tile_rows_cap, a.status);
-        for (uint32_t r = threadIdx.x; r < ids_rows; r += M2_THREADS)
-            ids_s[r] = __ldcs(src + BMU_IDX(r, a.tile_rows_cap - s_off[0], a.status));
-        __syncthreads();
-    }
-
     if (warp == NTW) {
         // ---------------- producer: W stages of every slab, in order
         if (lane == 0) {
@@ -348,19 +324,15 @@ sweep_mma2_kernel(const MmaArgs a)
                     const uint32_t rows = max(tla & 0xffffu, tlb & 0xffffu);
                     const uint32_t my_rows = (lh ? tlb : tla) & 0xffffu;
                     const int mine = 2 * dg + ((lh && has_b) ? 1 : 0);
-                    const uint4 *gp = ids_in_smem
-                        ? ids_s + (s_off[mine] - s_off[0])
-                        : a.tile_ids + BMU_IDX(s_off[mine], a.tile_rows_cap, a.status);
-                    [[maybe_unused]] const size_t room =
-                        ids_in_smem ? (size_t)(ids_rows - (s_off[mine] - s_off[0]))
-                                    : a.tile_rows_cap - (size_t)(gp - a.tile_ids);
+                    const uint4 *gp = a.tile_ids + BMU_IDX(s_off[mine], a.tile_rows_cap, a.status);
+                    [[maybe_unused]] const size_t room = a.tile_rows_cap - (size_t)(gp - a.tile_ids);
                     const char *base = reinterpret_cast<const char *>(a.W + j0 + li * 4);
                     uint32_t b = 0;
                     uint4 qn = s_first[mine];
                     for (; b < full; ++b) {
                         uint32_t f[8];
                         m2_unpack(qn, f);
-                        qn = gp[BMU_IDX(b + 1, room, a.status)];
+                        qn = __ldcs(gp + BMU_IDX(b + 1, room, a.status));
                         ulonglong2 w[8];
 #pragma unroll
                         for (int t = 0; t < 8; ++t)
@@ -371,7 +343,7 @@ sweep_mma2_kernel(const MmaArgs a)
                     for (; b < rows; ++b) {                      // some documents have run out
                         uint32_t f[8];
                         m2_unpack(qn, f);
-                        qn = gp[BMU_IDX(b + 1, room, a.status)];
+                        qn = __ldcs(gp + BMU_IDX(b + 1, room, a.status));
                         const bool in = b < my_rows;
                         ulonglong2 w[8];
 #pragma unroll

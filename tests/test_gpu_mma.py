@@ -134,7 +134,7 @@ def test_mma_kernel_relabel_off_matches_on_for_ordered_ids(bmu):
 def test_mma_kernel_refuses_what_it_cannot_do(bmu):
     rp = torch.tensor([0, 1], dtype=torch.int32).cuda()
     ci = torch.tensor([0], dtype=torch.int32).cuda()
-    for kernel, D, M in ((6, 32, 1024), (6, 2048, 256)):
+    for kernel, D, M in ((6, 32, 1024), (6, 2048, 128)):
         with pytest.raises(bmu.BmuError) as e:
             bmu.bmu_search_ws(torch.zeros(D, M, device="cuda"), rp, ci, opts=opts_of(bmu, kernel))
         assert e.value.status == 2
@@ -196,3 +196,32 @@ def test_unknown_kernel_numbers_are_refused(bmu, kernel):
     with pytest.raises(bmu.BmuError) as e:
         bmu.bmu_search_ws(torch.zeros(2048, 1024, device="cuda"), rp, ci, opts=opts_of(bmu, kernel))
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("cluster", [3, 4])
+@pytest.mark.parametrize("kernel", [3, 4, 6])
+@pytest.mark.parametrize("corpus", ["iid", "topical"])
+def test_content_clustering_changes_no_result(bmu, cluster, kernel, corpus):
+    """Tile membership by content (bmu_opts.cluster = 3, 4) only reorders documents: every
+    document is reduced on its own, so any order is valid and the outputs still match the oracle
+    -- also on a corpus with topics, where the ordering actually groups documents."""
+    cfg = synth.CONFIGS["cfg3"]
+    if corpus == "iid":
+        rowptr, colidx = synth.make_corpus(cfg, n_docs=2300)
+    else:
+        rowptr, colidx = synth.make_topical_corpus(cfg, n_docs=2300, n_topics=40)
+    W = synth.make_codebook(cfg.D, 768, 17, kind="scaled")
+    res = run_and_check(bmu, W, rowptr, colidx, opts_of(bmu, kernel, cluster=cluster, chunk_neurons=512))
+    assert res["docs"] == 2300 and res["failed"] == 0
+    if kernel == 6:                                        # and with the features ranked by the pass
+        run_and_check(bmu, W, rowptr, colidx, opts_of(bmu, 6, cluster=cluster, relabel=1, head_rows=256))
+
+
+def test_single_slab_codebook(bmu):
+    """M = 256: one 256-neuron slab, the smallest codebook the tensor-core sweep takes."""
+    cfg = synth.CONFIGS["cfg1"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=700)
+    W = synth.make_codebook(cfg.D, 256, 5, kind="scaled")
+    run_and_check(bmu, W, rowptr, colidx, opts_of(bmu, 6))
+    W = synth.make_codebook(cfg.D, 256 * 3 + 20, 6, kind="scaled")      # three slabs and a ragged rest
+    run_and_check(bmu, W, rowptr, colidx, opts_of(bmu, 6, chunk_neurons=256))

@@ -137,3 +137,34 @@ def test_launch_counter_agrees_with_describe_search(bmu):
     per = [d.sweep_launches * (1 + d.repack) for d in descs]
     assert [d.sweep_launches for d in descs] == [8, 2]
     assert counts[0] - counts[1] == per[0] - per[1] and counts[1] > per[1]
+
+
+@pytest.mark.parametrize("kernel,cluster", [(3, 1), (6, 1), (6, 0), (6, 3), (6, 4), (4, 3), (3, 2)])
+def test_planned_order_is_a_length_ordered_permutation(bmu, kernel, cluster):
+    """bmu_plan_order: every document appears once; unless the corpus order is kept, the lists
+    the sweep walks (behind the dense head for the tensor-core sweep) never get longer along
+    the planned order -- with or without ordering by content among equally long documents."""
+    cfg = synth.CONFIGS["cfg3"]
+    dev = torch.device("cuda")
+    rowptr, colidx = synth.make_topical_corpus(cfg, n_docs=5000, device=dev, n_topics=64)
+    o = bmu.Opts()
+    o.kernel, o.cluster, o.relabel = kernel, cluster, 2
+    plan = bmu.Plan(rowptr, colidx, cfg.D, 1024, o)
+    order = plan.order().to(torch.int64)
+    plan.close()
+    N = rowptr.numel() - 1
+    assert torch.equal(torch.sort(order).values, torch.arange(N, device=dev))
+    if cluster == 2:
+        assert torch.equal(order, torch.arange(N, device=dev))
+        return
+    lens = (rowptr[1:] - rowptr[:-1]).to(torch.int64)
+    if kernel == 6:                                   # ids below the head (640) are not gathered
+        doc = torch.repeat_interleave(torch.arange(N, device=dev), lens)
+        lens = torch.zeros(N, dtype=torch.int64, device=dev).index_add_(0, doc, (colidx >= 640).to(torch.int64))
+    walked = lens[order]
+    assert bool((walked[1:] <= walked[:-1]).all())
+    if cluster in (0, 3) and kernel == 6:
+        # among equally long documents: ordered by the rarest feature (ids are frequency ranks)
+        last = colidx[(rowptr[1:] - 1).to(torch.int64)].to(torch.int64)[order]
+        same = walked[1:] == walked[:-1]
+        assert bool((last[1:][same] >= last[:-1][same]).all())
