@@ -277,6 +277,15 @@ BMU_API int bmu_search(const float *W, int64_t D, int64_t M, const int32_t *rowp
                void *stream);
 
 /*
+ * What a status word (the first 32-bit word of a search workspace, read back by the
+ * caller after the stream has finished) means: BMU_OK for 0, BMU_ERR_WORKSPACE if
+ * a size check of the tiling pass failed (bit 64), BMU_ERR_TIMEOUT if a bounded
+ * device-side wait ran out (any other bit; bit 128 is set by the bounds-checked
+ * build for an address it refused).  The detail string names the word.  Host-side only.
+ */
+BMU_API int bmu_status_of_word(uint32_t status_word);
+
+/*
  * Status word of the last bmu_search (or bmu_search_host, bmu_search_batches_host)
  * on the current device: synchronises `stream`, copies the word to *out_status and
  * returns BMU_OK if it is 0, BMU_ERR_TIMEOUT if a bounded device-side wait ran

@@ -99,6 +99,7 @@ EXPORTS = {
                                                ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                                ctypes.c_void_p]),
     "bmu_selftest_wait_timeout": (ctypes.c_int, [ctypes.c_void_p]),
+    "bmu_status_of_word": (ctypes.c_int, [ctypes.c_uint32]),
     "bmu_last_status": (ctypes.c_int, [ctypes.POINTER(ctypes.c_uint32), ctypes.c_void_p]),
     "bmu_release_scratch": (ctypes.c_int, []),
     "bmu_validate_csr": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,

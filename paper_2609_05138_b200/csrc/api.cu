@@ -939,6 +939,11 @@ int bmu_search_batches_host(const float *W, int64_t D, int64_t M, int32_t n_batc
     return BMU_OK;
 }
 
+int bmu_status_of_word(uint32_t status_word)
+{
+    return status_word ? status_error(status_word) : BMU_OK;
+}
+
 int bmu_last_status(uint32_t *out_status, void *stream)
 {
     cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -91,3 +91,17 @@ def test_describe_search_needs_no_gpu_and_names_the_kernel(lib):
     o.kernel = 6
     assert lib.bmu_describe_search(32, 1024, 10, 100, ctypes.byref(o), ctypes.byref(d)) == 2   # D < head
     assert lib.bmu_describe_search(32, 1024, 10, 100, None, None) == 1
+
+
+def test_status_words_map_to_errors_without_a_gpu(lib):
+    """The host entry points that read a search's status word back (bmu_search_host,
+    bmu_search_batches_host, bmu_plan_create, bmu_last_status) turn it into an error through
+    this mapping: a clean word is no error, a failed size check of the tiling pass is a
+    workspace error, a wait that ran out a timeout."""
+    assert lib.bmu_status_of_word(0) == 0
+    assert lib.bmu_status_of_word(64) == 3 and b"tiling pass" in lib.bmu_last_error()
+    assert lib.bmu_status_of_word(64 | 8) == 3
+    for word in (1, 2, 4, 8, 16, 32):
+        assert lib.bmu_status_of_word(word) == 5
+        assert b"wait ran out" in lib.bmu_last_error() and str(word).encode() in lib.bmu_last_error()
+    assert lib.bmu_status_of_word(128) == 5

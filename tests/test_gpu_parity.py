@@ -253,6 +253,21 @@ def test_streamed_batches_match_single_calls(bmu):
         assert torch.equal(rb.cpu(), ob) and torch.equal(rd.cpu(), od)
 
 
+def test_status_word_of_the_one_shot_search_is_readable(bmu):
+    """bmu_search keeps its status word in library-owned scratch; bmu_last_status hands it back
+    (clean run: 0), also after the streamed-batches form, which collects every batch's word."""
+    cfg = synth.CONFIGS["cfg2"]
+    rowptr, colidx = synth.make_corpus(cfg, n_docs=700)
+    W = synth.make_codebook(cfg.D, 1024, 5).cuda()
+    bmu.bmu_search(W, rowptr.cuda(), colidx.cuda())
+    assert bmu.bmu_last_status() == (0, 0)
+    batches = [(rowptr.pin_memory(), colidx.pin_memory())] * 3
+    bmu.bmu_search_batches_host(W, batches)
+    assert bmu.bmu_last_status() == (0, 0)
+    bmu.bmu_selftest_wait_timeout()                       # leaves the searches' word alone
+    assert bmu.bmu_last_status() == (0, 0)
+
+
 def test_bounded_wait_reports_timeout_and_context_survives(bmu):
     """A device-side wait that cannot succeed ends through the status word, not a hang."""
     assert bmu.bmu_selftest_wait_timeout() == 5            # BMU_ERR_TIMEOUT
