@@ -258,6 +258,21 @@ static int route_search(const bmu_opts &o, int64_t D, int64_t M, int64_t nnz, ui
     return BMU_OK;
 }
 
+// Cuts [0, m_full) into the launches of the tensor-core sweep: as many as chunks of `chunk`
+// neurons need, the 256-neuron slabs dealt evenly among them (so that the last launch is not a
+// single slab whose MMAs nothing overlaps).  Launch k covers [cut(k), cut(k + 1)).
+struct LaunchCuts {
+    int64_t slabs, n, base, rem;
+    LaunchCuts(int64_t m_full, int64_t chunk)
+    {
+        slabs = m_full / MMA_SLAB;
+        n = (m_full + chunk - 1) / chunk;
+        base = n ? slabs / n : 0;
+        rem = n ? slabs % n : 0;
+    }
+    int64_t cut(int64_t k) const { return (k * base + (k < rem ? k : rem)) * MMA_SLAB; }
+};
+
 static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
                        const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t nnz,
                        int32_t *out_bmu, float *out_dist, const bmu_opts *opts_in, void *ws,
@@ -340,10 +355,13 @@ static int search_impl(const float *W, int64_t D, int64_t M, const float *norms,
         a.D = D; a.tile_rows_cap = l.plan.tile_rows_cap;
         const int64_t chunk = r.chunk;
         float *compact = repack_bytes ? reinterpret_cast<float *>(base + l.repack_off) : nullptr;
-        for (int64_t j = 0; j < m_full; j += chunk) {
+        const LaunchCuts cuts(m_full, chunk);
+        for (int64_t k = 0; k < cuts.n; ++k) {
+            const int64_t j = cuts.cut(k);
             a.j_lo = (int32_t)j;
-            a.j_hi = (int32_t)(j + chunk < m_full ? j + chunk : m_full);
+            a.j_hi = (int32_t)cuts.cut(k + 1);
             a.first = j == 0;
+            a.W = W; a.M = M;
             if (compact) {                 // gather from a compact copy of this chunk's columns
                 const int32_t width = a.j_hi - a.j_lo;
                 { repack_chunk_kernel<<<(unsigned)D, 256, 0, s>>>(
@@ -735,9 +753,11 @@ int bmu_search_f16_ws(const void *W16, int64_t D, int64_t M, const float *norms,
         const int64_t chunk = o.chunk_neurons ? mma_chunk(o, D, M) : 2 * mma_auto_chunk(D, M);
         const size_t repack_bytes = mma_repack_bytes(ow, D, M, N, nnz, top2);
         char *compact = (repack_bytes && M > chunk) ? base + l.repack_off : nullptr;
-        for (int64_t j = 0; j < M; j += chunk) {
+        const LaunchCuts cuts(M, chunk);
+        for (int64_t k = 0; k < cuts.n; ++k) {
+            const int64_t j = cuts.cut(k);
             a.j_lo = (int32_t)j;
-            a.j_hi = (int32_t)(j + chunk < M ? j + chunk : M);
+            a.j_hi = (int32_t)cuts.cut(k + 1);
             a.first = j == 0;
             a.W = static_cast<const float *>(W16); a.M = M;
             if (compact) {                 // a compact copy of this chunk's columns (2 bytes each)

@@ -97,14 +97,21 @@ __global__ void plan_rank_tables_kernel(const uint32_t *__restrict__ sorted, int
 // Sorting key of a document: how many of its ids the gather will visit, i.e. the ids at or
 // above `head` (all of them when head == 0) -- or the whole list if it repeats an id below
 // `head`: such a list keeps multiset semantics by staying out of the dense head altogether
-// (head_of_doc below), so all of it is gathered.  The key must be the gathered length exactly:
-// the room reserved for the tile id matrices counts on documents ordered by it.  One warp per
-// document.
+// (plan_tile_len_kernel below), so all of it is gathered.  The key must be the gathered length exactly:
+// the room reserved for the tile id matrices counts on documents ordered by it.  With `ckeys`
+// the same pass over the row also forms the 64-bit content key (plan_cluster_key_kernel below
+// says what it holds).  One warp per document.
+__device__ __forceinline__ void plan_min3(uint32_t &a, uint32_t &b, uint32_t &c, uint32_t v)
+{
+    if (v < a) { c = b; b = a; a = v; } else if (v < b) { c = b; b = v; } else if (v < c) { c = v; }
+}
+
 __global__ void __launch_bounds__(256)
 plan_key_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colidx,
                 const uint16_t *__restrict__ rank, int64_t N, int32_t head,
                 uint32_t *__restrict__ key, [[maybe_unused]] int64_t D,
-                [[maybe_unused]] uint32_t *__restrict__ status)
+                [[maybe_unused]] uint32_t *__restrict__ status, int mode,
+                u64 *__restrict__ ckeys, uint32_t *__restrict__ cvals)
 {
     __shared__ uint32_t seen[8][HEAD_ROWS_MAX / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -114,6 +121,8 @@ plan_key_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ 
     __syncwarp();
     const int beg = rowptr[i], end = rowptr[i + 1];
     int cnt = 0, repeat = 0;
+    uint32_t m1 = 0, m2 = 0;                             // largest and second largest rank
+    uint32_t s1 = 0xffffu, s2 = 0xffffu, s3 = 0xffffu;   // three smallest ranks >= head
     for (int e = beg + lane; e < end; e += 32) {
         const int32_t r = rank ? (int32_t)rank[BMU_IDX((uint32_t)colidx[e], D, status)] : colidx[e];
         if (r >= head) {
@@ -122,11 +131,39 @@ plan_key_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ 
             const uint32_t bit = 1u << (r & 31);
             repeat |= (atomicOr(&seen[warp][r >> 5], bit) & bit) != 0u;
         }
+        if (ckeys) {
+            const uint32_t rr = min((uint32_t)r, 0xfffeu);
+            if (rr > m1) { m2 = m1; m1 = rr; } else if (rr > m2) { m2 = rr; }
+            if (r >= head) plan_min3(s1, s2, s3, rr);
+        }
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
     repeat = __any_sync(0xffffffffu, repeat);
-    if (lane == 0) key[i] = repeat ? (uint32_t)(end - beg) : (uint32_t)cnt;
+    const uint32_t len = repeat ? (uint32_t)(end - beg) : (uint32_t)cnt;
+    if (lane == 0) key[i] = len;
+    if (ckeys) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const uint32_t o1 = __shfl_xor_sync(0xffffffffu, m1, off);
+            const uint32_t o2 = __shfl_xor_sync(0xffffffffu, m2, off);
+            const uint32_t hi = max(m1, o1), lo = min(m1, o1);
+            m2 = max(lo, max(m2, o2));
+            m1 = hi;
+            const uint32_t t1 = __shfl_xor_sync(0xffffffffu, s1, off);
+            const uint32_t t2 = __shfl_xor_sync(0xffffffffu, s2, off);
+            const uint32_t t3 = __shfl_xor_sync(0xffffffffu, s3, off);
+            plan_min3(s1, s2, s3, t1);
+            plan_min3(s1, s2, s3, t2);
+            plan_min3(s1, s2, s3, t3);
+        }
+        if (lane == 0) {
+            const u64 top = (u64)(uint32_t)(PLAN_BINS - 1 - min(len, (uint32_t)(PLAN_BINS - 1))) << 48;
+            ckeys[i] = mode == 4 ? top | ((u64)s1 << 32) | ((u64)s2 << 16) | (u64)s3
+                                 : top | ((u64)m1 << 32) | ((u64)m2 << 16) | (u64)s1;
+            cvals[i] = (uint32_t)i;
+        }
+    }
 }
 
 // histogram of the sorting keys, and the largest key (aux[0]) so that the scan below can
@@ -209,11 +246,6 @@ __global__ void plan_scatter_kernel(const int32_t *__restrict__ rowptr,
 // Either way the shared features sit at the same step of the lists of a tile (the front, or the
 // back of equally long lists), so the loads of one step ask for the same row.  One warp per
 // document.
-__device__ __forceinline__ void plan_min3(uint32_t &a, uint32_t &b, uint32_t &c, uint32_t v)
-{
-    if (v < a) { c = b; b = a; a = v; } else if (v < b) { c = b; b = v; } else if (v < c) { c = v; }
-}
-
 __global__ void __launch_bounds__(256)
 plan_cluster_key_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colidx,
                         const uint16_t *__restrict__ rank, const uint32_t *__restrict__ len_key,
@@ -333,60 +365,63 @@ plan_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__
 
 // ---- tiles of 8 documents -------------------------------------------------
 // The ids below `head` (a multiple of 32, at most HEAD_ROWS_MAX) at the front of a document's
-// ascending list, as a bit mask of head / 32 words written to `mask`, and how many list
-// entries that covers.  A list that repeats one of them keeps multiset semantics by opting
-// out (mask 0, nothing skipped): its ids all stay in the list.
-__device__ __forceinline__ uint32_t head_of_doc(const uint16_t *ids, uint32_t len, uint32_t head,
-                                                uint32_t *mask)
-{
-    const uint32_t words = head / 32;
-    for (uint32_t w = 0; w < words; ++w) mask[w] = 0;
-    uint32_t skip = 0, bits = 0;
-    for (uint32_t e = 0; e < len && e <= head; ++e) {
-        const uint32_t f = ids[e];
-        if (f >= head) break;
-        const uint32_t old = mask[f >> 5], now = old | (1u << (f & 31u));
-        bits += now != old;
-        mask[f >> 5] = now;
-        ++skip;
-    }
-    if (skip != bits) {
-        for (uint32_t w = 0; w < words; ++w) mask[w] = 0;
-        skip = 0;
-    }
-    return skip;
-}
-
+// ascending list become a bit mask of head / 32 words, and the list the sweep walks starts
+// behind them.  A list that repeats one of them keeps multiset semantics by opting out (mask
+// 0, nothing skipped): its ids all stay in the list.
 // per tile: longest and shortest list behind the head (max | min << 16), and the head masks
-// (head / 32 words per document, document-major).  One thread per planned document; the eight
-// threads of a tile combine their lengths with shuffles.
+// (head / 32 words per document, document-major).  One block per tile, one warp per document:
+// the lanes read the front of the document's ascending list 32 ids at a time and set the mask
+// bits in shared memory; a list that repeats a head id opts out (mask 0, nothing skipped).
 __global__ void __launch_bounds__(256)
 plan_tile_len_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ perm,
                      const uint32_t *__restrict__ doc_off, const uint16_t *__restrict__ ids16,
                      int64_t N, int64_t n_tiles, uint32_t head, uint32_t *__restrict__ tile_rows,
                      uint32_t *__restrict__ tile_len, uint32_t *__restrict__ tile_head)
 {
-    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;     // planned position
-    const int64_t tile = p >> 3;
-    const bool there = tile < n_tiles;
+    __shared__ uint32_t s_mask[8][HEAD_ROWS_MAX / 32];
+    __shared__ uint32_t s_left[8];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t tile = blockIdx.x;
+    const int64_t p = tile * 8 + warp;                                    // planned position
     const uint32_t words = head ? head / 32 : 1;
+    for (uint32_t w = lane; w < words; w += 32) s_mask[warp][w] = 0u;
+    __syncwarp();
     uint32_t len = 0, skip = 0;
-    if (there) {
-        uint32_t *mask = tile_head + (size_t)p * words;
-        for (uint32_t w = 0; w < words; ++w) mask[w] = 0;
-        if (p < N) {
-            const int32_t i = perm[p];
-            len = (uint32_t)min(rowptr[i + 1] - rowptr[i], 65535);
-            if (head) skip = head_of_doc(ids16 + ((size_t)doc_off[p] + 1) * 8, len, head, mask);
+    if (p < N) {
+        const int32_t i = perm[p];
+        len = (uint32_t)min(rowptr[i + 1] - rowptr[i], 65535);
+        if (head) {
+            const uint16_t *ids = ids16 + ((size_t)doc_off[p] + 1) * 8;
+            bool repeat = false;
+            for (uint32_t e0 = 0; e0 < len && e0 <= head; e0 += 32) {
+                const uint32_t e = e0 + lane;
+                const uint32_t f = (e < len && e <= head) ? ids[e] : 0xffffu;
+                const bool in = f < head;
+                if (in) {
+                    const uint32_t bit = 1u << (f & 31u);
+                    repeat |= (atomicOr(&s_mask[warp][f >> 5], bit) & bit) != 0u;
+                }
+                const uint32_t got = __ballot_sync(0xffffffffu, in);
+                skip += (uint32_t)__popc(got);
+                if (got != 0xffffffffu) break;                            // the list left the head
+            }
+            if (__any_sync(0xffffffffu, repeat)) {
+                __syncwarp();
+                for (uint32_t w = lane; w < words; w += 32) s_mask[warp][w] = 0u;
+                skip = 0;
+            }
         }
     }
-    uint32_t mx = len - skip, mn = len - skip;
-#pragma unroll
-    for (int off = 1; off < 8; off <<= 1) {
-        mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-        mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, off));
+    __syncwarp();
+    {
+        uint32_t *mask = tile_head + (size_t)p * words;
+        for (uint32_t w = lane; w < words; w += 32) mask[w] = s_mask[warp][w];
     }
-    if (there && (threadIdx.x & 7) == 0) {
+    if (lane == 0) s_left[warp] = len - skip;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t mx = 0, mn = 0xffffffffu;
+        for (int t = 0; t < 8; ++t) { mx = max(mx, s_left[t]); mn = min(mn, s_left[t]); }
         tile_rows[tile] = mx;
         tile_len[tile] = mx | (mn << 16);
     }
@@ -550,21 +585,25 @@ int launch_plan(const int32_t *rowptr, const int32_t *colidx, int64_t N, int64_t
         // the documents of a tile finish their lists together (the key borrows the doc_off
         // array, which is written only by the scan after the scatter)
         const uint32_t *key = nullptr;
+        const bool by_content = order_by_length >= 3 && l.cluster_tmp_bytes > 0;
+        u64 *keys_in = reinterpret_cast<u64 *>(ws + l.cluster_off);
+        u64 *keys_out = keys_in + N;
+        uint32_t *vals_in = reinterpret_cast<uint32_t *>(keys_out + N);
         if (head > 0) {
-            { plan_key_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(rowptr, colidx, rank, N,
-                                                                            head, doc_off, D, status); BMU_LAUNCHED(); }
+            // length key and, if wanted, the content key in one pass over the rows
+            { plan_key_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(
+                rowptr, colidx, rank, N, head, doc_off, D, status, order_by_length,
+                by_content ? keys_in : nullptr, vals_in); BMU_LAUNCHED(); }
             key = doc_off;
         }
         // counters and the largest key in one clearing (the cursors in between are all written
         // or never read)
         BMU_CUDA(cudaMemsetAsync(hist, 0, (size_t)PLAN_BINS * 4 * 2 + 256, s));
-        if (order_by_length >= 3 && l.cluster_tmp_bytes > 0) {
+        if (by_content) {
             // by length, then by the rarest features: one radix sort of (key, document) pairs
-            u64 *keys_in = reinterpret_cast<u64 *>(ws + l.cluster_off);
-            u64 *keys_out = keys_in + N;
-            uint32_t *vals_in = reinterpret_cast<uint32_t *>(keys_out + N);
-            { plan_cluster_key_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(
-                rowptr, colidx, rank, key, N, head, order_by_length, D, status, keys_in, vals_in); BMU_LAUNCHED(); }
+            if (head == 0)
+                { plan_cluster_key_kernel<<<(unsigned)((N * 32 + 255) / 256), 256, 0, s>>>(
+                    rowptr, colidx, rank, key, N, head, order_by_length, D, status, keys_in, vals_in); BMU_LAUNCHED(); }
             size_t ctmp = l.cluster_tmp_bytes;
             BMU_CUDA(cub::DeviceRadixSort::SortPairs(ws + l.cluster_tmp_off, ctmp, keys_in, keys_out,
                                                      vals_in, reinterpret_cast<uint32_t *>(perm),
@@ -602,7 +641,7 @@ int launch_plan_tiles(const int32_t *rowptr, int64_t N, int interleave, int head
     uint32_t *tile_off = reinterpret_cast<uint32_t *>(ws + l.tileoff_off);
     uint4 *tile_ids = reinterpret_cast<uint4 *>(ws + l.tileids_off);
     uint32_t *tile_head = reinterpret_cast<uint32_t *>(ws + l.tilehead_off);
-    { plan_tile_len_kernel<<<(unsigned)((n_tiles * 8 + 255) / 256), 256, 0, s>>>(
+    { plan_tile_len_kernel<<<(unsigned)n_tiles, 256, 0, s>>>(
         rowptr, perm, doc_off, ids16, N, n_tiles, (uint32_t)head, tile_rows, tile_len, tile_head); BMU_LAUNCHED(); }
     BMU_CUDA(cudaMemsetAsync(tile_rows + n_tiles, 0, 4, s));
     size_t tmp = l.scan_bytes;
