@@ -526,7 +526,7 @@ def run_ours(args, cfg, rank, local_rank, world):
         "roofline": frag["roofline"],
     }
     if len(batches) == 1:
-        line["planned"] = planned_steps(bmu, cfg, a, opts, args.steps, dev)
+        line["planned"] = planned_steps(bmu, cfg, a, opts, min(args.steps, 5), dev)
     if args.comparator:
         line["comparator"] = comparator_spmm(cfg, W, norms, rowptr, colidx, peaks)
     if args.f16 and len(batches) == 1:
