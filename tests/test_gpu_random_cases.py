@@ -82,6 +82,8 @@ def draw_opts(bmu, rng, kernel):
         o.repack = rng.choice([0, 2])
     if kernel in (4, 6):
         o.tile_order = rng.choice([0, 1, 2])
+    if kernel in (3, 4, 6):
+        o.cluster = rng.choice([0, 1, 3, 4])        # document order: by length / and content
     return o
 
 
