@@ -462,7 +462,8 @@ BMU_API int bmu_score_block_argmin(const void *scores, int32_t half, int64_t n_r
  *         4  fp32 adds, scalar instructions                            [adds/s]
  *         5  fp32 adds, packed two-wide instructions                   [adds/s]
  *         6  L2 -> SM by 128-bit loads and bulk copies of `piece` bytes (multiple
- *            of 16 in [1024, 16384]) running together, both counted: the way the
+ *            of 16 in [256, 16384]; up to sixteen issuing threads per block, as many
+ *            as 64 KB of buffers allow) running together, both counted: the way the
  *            tensor-core sweep pulls bytes (gathered rows by loads, head image by
  *            bulk copies)                                              [bytes/s]
  * `buffer` is 256-byte aligned device memory the benchmark may overwrite; for

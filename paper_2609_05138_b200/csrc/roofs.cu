@@ -82,9 +82,9 @@ roof_l2_bulk_kernel(const char *__restrict__ buf, size_t bytes, int piece, int r
 }
 
 // Loads and bulk copies at once, the way the tensor-core sweep pulls bytes into an SM: fifteen
-// warps of a block sweep the buffer with 128-bit loads (as above) while up to four threads of
-// the sixteenth warp each keep MIX_DEPTH bulk copies of `piece` bytes in flight, until the
-// loading warps are done.  Bytes delivered by loads are known beforehand; the bytes the bulk
+// warps of a block sweep the buffer with 128-bit loads (as above) while up to sixteen threads
+// of the sixteenth warp each keep MIX_DEPTH bulk copies of `piece` bytes in flight (as many
+// threads as 64 KB of shared memory give buffers to), until the loading warps are done.  Bytes delivered by loads are known beforehand; the bytes the bulk
 // copies delivered are counted in *bulk_bytes.  Waits are bounded (sink[1] on timeout).
 static const int MIX_DEPTH = 4;
 static const int MIX_SMEM = 65536;
@@ -93,11 +93,11 @@ roof_l2_mixed_kernel(const char *__restrict__ buf, size_t bytes, int piece, int 
                      unsigned long long *bulk_bytes, uint32_t *sink)
 {
     extern __shared__ __align__(128) char smem[];
-    __shared__ __align__(8) unsigned long long bar[4 * MIX_DEPTH];
+    __shared__ __align__(8) unsigned long long bar[16 * MIX_DEPTH];
     __shared__ uint32_t loaders_done;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int d = 0; d < 4 * MIX_DEPTH; ++d)
+        for (int d = 0; d < 16 * MIX_DEPTH; ++d)
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bar[d])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         loaders_done = 0u;
@@ -296,13 +296,13 @@ extern "C" BMU_API int bmu_measure_roof(int which, void *buffer, size_t buffer_b
     c.bulk_bytes = reinterpret_cast<unsigned long long *>(static_cast<char *>(buffer) + 64);
     double work = 0;
     if (which == 6) {
-        if (piece < 1024 || piece % 16 || piece > MIX_SMEM / MIX_DEPTH) {
-            set_error("piece must be a multiple of 16 in [1024, %d]", MIX_SMEM / MIX_DEPTH);
+        if (piece < 256 || piece % 16 || piece > MIX_SMEM / MIX_DEPTH) {
+            set_error("piece must be a multiple of 16 in [256, %d]", MIX_SMEM / MIX_DEPTH);
             return BMU_ERR_INVALID_ARG;
         }
         size_t usable = (buffer_bytes - 256) / 65536 * 65536 / piece * piece / 16 * 16;
         c.bytes = usable; c.piece = piece;
-        c.issuers = MIX_SMEM / (MIX_DEPTH * piece) < 4 ? MIX_SMEM / (MIX_DEPTH * piece) : 4;
+        c.issuers = MIX_SMEM / (MIX_DEPTH * piece) < 16 ? MIX_SMEM / (MIX_DEPTH * piece) : 16;
         c.rounds = (int)(((size_t)2 << 30) / usable) / 2 + 1;   // about 1 GiB of loads per block
         work = (double)(usable / 16 * 16) * c.rounds * sms * 2;
         BMU_CUDA(cudaFuncSetAttribute(roof_l2_mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MIX_SMEM));
