@@ -9,16 +9,14 @@
 // its fp32 sum with the mixed-precision add of sm_100; the head sums leave tensor memory through
 // a per-warp transposing buffer in shared memory; and the control warpgroup hands registers to
 // the tail warpgroups.  Kept as its own kernel so that the fp32 sweep's code generation is not
-// disturbed.
-#include "common.cuh"
-#include "mma_ptx.cuh"
+// disturbed; the control roles are the shared ones of sweep_mma2_common.cuh.
+#include "sweep_mma2_common.cuh"
 
 #include <cuda_fp16.h>
 #include <math_constants.h>
 
 namespace bmu {
 
-static const int M2_SLAB = 256;
 #ifndef BMU_M2F_WSTAGES
 #define BMU_M2F_WSTAGES 4
 #endif
@@ -27,12 +25,10 @@ static const int M2_SLAB = 256;
 #endif
 static const int M2_NS = BMU_M2F_WSTAGES;             // W ring stages
 static const int M2_NX = BMU_M2F_XSTAGES;             // X ring stages
-static const int M2_TAIL_WARPS = 16;
 static const int M2_THREADS = (M2_TAIL_WARPS + 4) * 32;      // 4 tail warpgroups + 1 control warpgroup
 #ifndef BMU_M2F_ROWS
 #define BMU_M2F_ROWS 3                               // id rows per turn: 4 x ROWS loads in flight per lane
 #endif
-static const int M2_TMEM_COLS = 512;                 // 2 buffers x 2 tiles x 128 documents
 static const int M2_XCH_BYTES = 16 * 64 * 4;         // a tail warp's 16 documents x 64 head sums
 
 static inline size_t m2_smem_bytes(int head, bool top2)
@@ -132,21 +128,15 @@ sweep_mma2_f16_kernel(const MmaArgs a)
     uint2 *lut = reinterpret_cast<uint2 *>(s_off + 16);          // 4 mask bits -> 4 fp16 zeros and ones
     u64 *kq = reinterpret_cast<u64 *>(lut + 16);
     float *xch0 = reinterpret_cast<float *>(kq + (TOP2 ? 4 * MMA_DOCS * 2 : 0));   // per tail warp
-    const uint32_t wfull0 = mm_smem(bars), wempty0 = mm_smem(bars + NS);
-    const uint32_t xfull0 = mm_smem(bars + 2 * NS), xempty0 = mm_smem(bars + 2 * NS + NX);
-    const uint32_t tfull0 = mm_smem(bars + 2 * NS + 2 * NX), tempty0 = tfull0 + 16;
-    const uint32_t drain = tfull0 + 32;
+    const M2Bars<NS, NX> bar(bars);
+    const uint32_t tfull0 = bar.tfull0, tempty0 = bar.tempty0;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t group = blockIdx.x;
     const int n_slabs = (a.j_hi - a.j_lo) / M2_SLAB;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < NS; ++i) { mm_bar_init(wfull0 + 8 * i, 1); mm_bar_init(wempty0 + 8 * i, 1); }
-        for (int i = 0; i < NX; ++i) { mm_bar_init(xfull0 + 8 * i, 1); mm_bar_init(xempty0 + 8 * i, 1); }
-        for (int i = 0; i < 2; ++i) { mm_bar_init(tfull0 + 8 * i, 1); mm_bar_init(tempty0 + 8 * i, NTW); }
-        mm_bar_init(drain, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        bar.init();
         *abort_flag = 0u;
         *skip_flag = *reinterpret_cast<volatile uint32_t *>(a.status);
     }
@@ -158,32 +148,7 @@ sweep_mma2_f16_kernel(const MmaArgs a)
                      ::"r"(mm_smem(tmem_slot)), "r"((uint32_t)M2_TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    {   // the block's head masks into shared memory (document-major, H / 8 bytes each)
-        const int words = H / 32;
-        uint32_t *mw = reinterpret_cast<uint32_t *>(masks);
-        for (int idx = threadIdx.x; idx < MMA_DOCS * words; idx += M2_THREADS) {
-            const int n = idx / words;
-            const int64_t tile = group * (MMA_DOCS / 8) + (n >> 3);
-            mw[idx] = tile < a.n_tiles ? __ldcs(a.tile_head + (size_t)group * MMA_DOCS * words + idx) : 0u;
-        }
-    }
-    if (threadIdx.x < MMA_DOCS) keys[threadIdx.x] = KEY_WORST;
-    if (threadIdx.x < 16) {
-        const uint32_t b = threadIdx.x;
-        lut[b] = make_uint2((b & 1u) * 0x3c00u + (b & 2u) * 0x1e000000u,
-                            ((b >> 2) & 1u) * 0x3c00u + ((b >> 2) & 2u) * 0x1e000000u);
-    }
-    if (TOP2)
-        for (int idx = threadIdx.x; idx < 4 * MMA_DOCS * 2; idx += M2_THREADS) kq[idx] = KEY_WORST;
-    if (threadIdx.x >= M2_THREADS - 16) {            // 16 threads of the last control warp
-        const int t = threadIdx.x - (M2_THREADS - 16);
-        const int64_t tile = group * (MMA_DOCS / 8) + t;
-        const bool there = tile < a.n_tiles;
-        const uint32_t off = there ? __ldg(a.tile_off + tile) : 0u;
-        s_len[t] = there ? __ldg(a.tile_len + tile) : 0u;
-        s_off[t] = off;
-        s_first[t] = __ldcs(a.tile_ids + BMU_IDX(off, a.tile_rows_cap, a.status));
-    }
+    m2_block_setup<M2_THREADS, TOP2>(a, group, H, masks, keys, lut, kq, s_first, s_len, s_off);
     mm_fence_before();
     __syncthreads();
     mm_fence_after();
@@ -196,91 +161,15 @@ sweep_mma2_f16_kernel(const MmaArgs a)
     if (warp >= NTW) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (warp == NTW) {
-        // ---------------- producer: W stages of every slab, in order
-        if (lane == 0) {
-            const unsigned char *src = a.head_img;
-            const int total = n_slabs * 2 * PARTS * KB;
-            int issued = 0;
-            for (int c = 0; c < total; ++c) {
-                const int slot = c % NS;
-                if (c >= NS && !mm_wait(wempty0 + 8 * slot, ((c / NS) - 1) & 1, abort_flag, a.status, 1u))
-                    break;
-                mm_bar_expect_tx(wfull0 + 8 * slot, (uint32_t)MMA_STAGE_BYTES);
-                mm_bulk_load(mm_smem(wring + (size_t)slot * MMA_STAGE_BYTES),
-                             src + (size_t)c * MMA_STAGE_BYTES, (uint32_t)MMA_STAGE_BYTES,
-                             wfull0 + 8 * slot);
-                issued = c + 1;
-            }
-            if (*abort_flag)         // gave up: let the copies in flight land before leaving
-                for (int c = issued > NS ? issued - NS : 0; c < issued; ++c)
-                    for (uint32_t spin = 0; spin < MMA_WAIT_LIMIT; ++spin)
-                        if (mm_bar_try(wfull0 + 8 * (c % NS), (c / NS) & 1)) break;
-        }
+        // ---------------- producer: W stages of every slab (2 tiles x one part per 64 features)
+        if (lane == 0) m2_producer<NS, NX, 2 * PARTS>(a, n_slabs, KB, wring, bar, abort_flag);
         __syncwarp();
     } else if (warp == NTW + 1) {
         // ---------------- expander: X_head, one block of 64 features per stage
-        const int total = n_slabs * KB;
-        for (int x = 0; x < total; ++x) {
-            const int slot = x % NX, kb = x % KB;
-            if (x >= NX && !mm_wait(xempty0 + 8 * slot, ((x / NX) - 1) & 1, abort_flag, a.status, 16u))
-                break;
-            unsigned char *dst = xring + (size_t)slot * MMA_STAGE_BYTES;
-            // a lane takes documents lane, lane + 32, ..: its 8 mask bytes of this block of 64
-            // features in one load, then eight 16-byte stores of fp16 zeros and ones (bit e of
-            // a byte -> half e; 0x3c00 is 1.0), four bits at a time through a 16-entry table
-#pragma unroll
-            for (int j = 0; j < MMA_DOCS / 32; ++j) {
-                const int n = lane + 32 * j;
-                const uint2 mb = *reinterpret_cast<const uint2 *>(masks + (size_t)n * (H / 8) + kb * 8);
-                unsigned char *row = dst + (size_t)(n >> 3) * 1024 + (n & 7) * 16;
-#pragma unroll
-                for (int kc = 0; kc < 8; ++kc) {
-                    const uint32_t b = (kc < 4 ? mb.x : mb.y) >> ((kc & 3) * 8);
-                    const uint2 lo4 = lut[b & 15u], hi4 = lut[(b >> 4) & 15u];
-                    *reinterpret_cast<uint4 *>(row + kc * 128) = make_uint4(lo4.x, lo4.y, hi4.x, hi4.y);
-                }
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mm_bar_arrive(xfull0 + 8 * slot);
-        }
-        __syncwarp();
+        m2_expander<NS, NX>(a, n_slabs, KB, H, masks, xring, lut, bar, abort_flag, lane);
     } else if (warp == NTW + 2) {
         // ---------------- one thread issues every MMA
-        if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | ((uint32_t)(MMA_DOCS >> 3) << 17) | (8u << 24);
-            const uint32_t wring_u32 = mm_smem(wring), xring_u32 = mm_smem(xring);
-            bool ok = true;
-            int wc = 0, xc = 0;
-            for (int sl = 0; sl < n_slabs && ok; ++sl) {
-                const int buf = sl & 1;
-                if (sl >= 2) ok = mm_wait(tempty0 + 8 * buf, ((sl >> 1) - 1) & 1, abort_flag, a.status, 2u);
-                if (!ok) break;
-                mm_fence_after();
-                for (int kb = 0; kb < KB && ok; ++kb, ++xc) {
-                    const int xslot = xc % NX;
-                    if (!mm_wait(xfull0 + 8 * xslot, (xc / NX) & 1, abort_flag, a.status, 32u)) { ok = false; break; }
-                    for (int cp = 0; cp < 2 * PARTS; ++cp, ++wc) {   // cp = tile * PARTS + part
-                        const int slot = wc % NS;
-                        if (!mm_wait(wfull0 + 8 * slot, (wc / NS) & 1, abort_flag, a.status, 4u)) { ok = false; break; }
-                        mm_fence_after();
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const u64 ad = mm_desc(wring_u32 + slot * (uint32_t)MMA_STAGE_BYTES + u * 256, 128, 1024);
-                            const u64 bd = mm_desc(xring_u32 + xslot * (uint32_t)MMA_STAGE_BYTES + u * 256, 128, 1024);
-                            mm_mma(tmem + buf * 256 + (cp / PARTS) * MMA_DOCS, ad, bd, idesc,
-                                   (kb | (cp % PARTS) | u) != 0);
-                        }
-                        mm_commit(wempty0 + 8 * slot);
-                    }
-                    if (ok) mm_commit(xempty0 + 8 * xslot);
-                }
-                if (ok) mm_commit(tfull0 + 8 * buf);
-            }
-            mm_commit(drain);
-            for (uint32_t spin = 0; spin < MMA_WAIT_LIMIT; ++spin)
-                if (mm_bar_try(drain, 0)) break;
-        }
+        if (lane == 0) m2_issuer<NS, NX, PARTS>(a, n_slabs, KB, tmem, wring, xring, bar, abort_flag);
         __syncwarp();
     }   // (the fourth warp only completes the control warpgroup)
     } else {
@@ -439,23 +328,7 @@ sweep_mma2_f16_kernel(const MmaArgs a)
     mm_fence_before();
     __syncthreads();
     mm_fence_after();
-    if (threadIdx.x < MMA_DOCS) {
-        const int64_t p = group * MMA_DOCS + threadIdx.x;
-        if (p < a.N) {
-            const int32_t orig = __ldg(a.perm + p);
-            if (TOP2) {
-                u64 b1 = KEY_WORST, b2 = KEY_WORST;
-#pragma unroll
-                for (int qq = 0; qq < 4; ++qq) {
-                    const u64 *slot = kq + ((size_t)qq * MMA_DOCS + threadIdx.x) * 2;
-                    Best<true>::merge(b1, b2, slot[0], slot[1]);
-                }
-                Best<true>::commit(b1, b2, a.state, a.state2, orig, a.first);
-            } else {
-                Best<false>::commit(keys[threadIdx.x], KEY_WORST, a.state, nullptr, orig, a.first);
-            }
-        }
-    }
+    m2_commit<TOP2>(a, group, keys, kq);
     if (warp == NTW)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
                      ::"r"(tmem), "r"((uint32_t)M2_TMEM_COLS) : "memory");
