@@ -14,8 +14,8 @@ static const int NORM_WARPS = 16;
 
 // VEC: a lane owns 4 consecutive columns (one 16-byte load per row); otherwise a lane owns
 // one column.  LX lanes of a warp lie side by side along the columns and 32 / LX along the
-// rows: LX = 32 for wide codebooks (a warp reads 512 contiguous bytes of one row), LX = 8 for
-// narrow ones, where 128 columns per block would leave most SMs without a block.
+// rows: LX = 32 for wide codebooks (a warp reads 512 contiguous bytes of one row), LX = 8 or 2
+// for narrow ones, where 128 columns per block would leave most SMs without a block.
 template <bool VEC, int LX>
 __global__ void __launch_bounds__(NORM_WARPS * 32)
 norms_kernel(const float *__restrict__ W, int64_t D, int64_t M, float *__restrict__ norms)
@@ -131,14 +131,19 @@ int launch_norms(const float *W, int64_t D, int64_t M, float *norms, cudaStream_
     if (M == 0) return BMU_OK;
     const bool vec = (M % 4 == 0) && ((reinterpret_cast<uintptr_t>(W) & 15) == 0);
     const int c = vec ? 4 : 1;
-    // narrow codebooks: 8 lanes across the columns, so that there are blocks for every SM
-    const bool narrow = (M + 32 * c - 1) / (32 * c) < 296;
-    const int cols = (narrow ? 8 : 32) * c;
+    // narrow codebooks: 8 or 2 lanes across the columns instead of 32, so that there are blocks
+    // for every SM (M = 1024: 128 blocks of 8 columns instead of 8 blocks of 128)
+    const int64_t wide_blocks = (M + 32 * c - 1) / (32 * c);
+    const int lx = wide_blocks >= 296 ? 32 : wide_blocks >= 16 ? 8 : 2;
+    const int cols = lx * c;
     const unsigned blocks = (unsigned)((M + cols - 1) / cols);
-    if (vec && narrow) { norms_kernel<true, 8><<<blocks, NORM_WARPS * 32, 0, s>>>(W, D, M, norms); BMU_LAUNCHED(); }
-    else if (vec) { norms_kernel<true, 32><<<blocks, NORM_WARPS * 32, 0, s>>>(W, D, M, norms); BMU_LAUNCHED(); }
-    else if (narrow) { norms_kernel<false, 8><<<blocks, NORM_WARPS * 32, 0, s>>>(W, D, M, norms); BMU_LAUNCHED(); }
-    else { norms_kernel<false, 32><<<blocks, NORM_WARPS * 32, 0, s>>>(W, D, M, norms); BMU_LAUNCHED(); }
+#define BMU_NORMS(V, L) { norms_kernel<V, L><<<blocks, NORM_WARPS * 32, 0, s>>>(W, D, M, norms); BMU_LAUNCHED(); }
+    if (vec) {
+        if (lx == 32) BMU_NORMS(true, 32) else if (lx == 8) BMU_NORMS(true, 8) else BMU_NORMS(true, 2)
+    } else {
+        if (lx == 32) BMU_NORMS(false, 32) else if (lx == 8) BMU_NORMS(false, 8) else BMU_NORMS(false, 2)
+    }
+#undef BMU_NORMS
     BMU_CUDA(cudaGetLastError());
     return BMU_OK;
 }

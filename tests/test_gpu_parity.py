@@ -48,7 +48,11 @@ def make_opts(bmu, **kw):
 # ------------------------------------------------------------------ norms
 @pytest.mark.parametrize("D,M,kind", [(4096, 1024, "uniform"), (16384, 4096, "uniform"),
                                       (513, 1000, "signed"), (77, 37, "uniform"),
-                                      (1, 5, "uniform"), (300, 130, "scaled")])
+                                      (1, 5, "uniform"), (300, 130, "scaled"),
+                                      # every column layout of the kernel: 2, 8 and 32 lanes
+                                      # across, rows of 16-byte pieces and ragged rows
+                                      (64, 8192, "uniform"), (8, 65536, "signed"),
+                                      (33, 1301, "uniform"), (5, 9999, "scaled")])
 def test_norms_match_oracle(bmu, D, M, kind):
     import oracle
     W = synth.make_codebook(D, M, 5, kind=kind)
